@@ -1,0 +1,167 @@
+/* fdg -- one training iteration of a network split into K modules under fully decoupled parallel
+ * backpropagation, combined with N data-parallel workers whose stale gradients are averaged
+ * before an SGD update.  C ABI of the sm_100a library (libfdg.so).
+ *
+ * What one call of fdg_step computes (paper Sec. 3.2, Sec. 3.3, Eq. "dl_update", Algorithm 1),
+ * with k = 1..K the module, t = 0,1,... the iteration, M = n_workers * per_worker_batch:
+ *   - module k runs its layers forward on the batch sampled at  tau_f = t - k + 1  (if >= 0)
+ *     with its current weights w_k(t), reading what module k-1 produced in iteration t-1;
+ *   - module k back-propagates the batch  tau_b = t - 2K + k + 1  (if >= 0) using the error
+ *     gradient module k+1 produced in iteration t-1, the activations it stashed when it
+ *     forwarded that batch, and the weights it had then, w_k(t - 2K + 2k);
+ *   - every worker's gradient is the sum over its per_worker_batch samples scaled by
+ *     1/per_worker_batch; the workers are mixed by P = (1/N) 1 1^T, i.e. averaged, so that
+ *     w_k(t+1) = w_k(t) - lr * mean over all M samples of dphi/dw_k; the average is taken inside
+ *     the weight-gradient contraction, which reduces over the worker x batch axis;
+ *   - while tau_b < 0 the gradient is zero and w_k(t+1) = w_k(t).
+ * phi is softmax cross-entropy (natural logarithm).  Batch-norm uses the statistics of each
+ * worker's own per_worker_batch * H * W values (biased variance, eps = 1e-5).
+ *
+ * Conventions
+ *   - Every function returns an fdg_status; nothing aborts or throws; on error, outputs are
+ *     left untouched and fdg_last_error() describes the failure.
+ *   - "device" pointers are CUDA device pointers on the context's device, "host" pointers are
+ *     ordinary host memory.  The caller owns every buffer it passes; the context owns all
+ *     device memory it obtained through the allocator and releases it in fdg_destroy.
+ *   - Activations are NHWC, worker-major: rows s*B .. (s+1)*B-1 belong to worker s.
+ *   - Canonical parameter order: layers in list order; per layer W then b (linear W[out][in];
+ *     conv W[c_out][kh][kw][c_in]); batch-norm gamma then beta; a projecting FDG_RES_ADD
+ *     carries Wp[c_out][c_in], gamma_p, beta_p.
+ *   - The library needs an sm_100 device; there is no CPU path.
+ */
+#ifndef FDG_H
+#define FDG_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define FDG_API __attribute__((visibility("default")))
+#else
+#define FDG_API
+#endif
+
+typedef struct fdg_ctx fdg_ctx;          /* opaque; owns all device state */
+
+typedef enum {
+    FDG_OK = 0,
+    FDG_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, unknown enum value          */
+    FDG_ERR_BAD_SPLIT = 2,     /* split points not strictly increasing / cut a residual block  */
+    FDG_ERR_UNSUPPORTED = 3,   /* a shape the kernels do not cover (e.g. odd size before pool) */
+    FDG_ERR_ARCH = 4,          /* no CUDA device of compute capability 10.x                    */
+    FDG_ERR_OOM = 5,           /* the allocator returned NULL                                  */
+    FDG_ERR_CUDA = 6,          /* a CUDA runtime call failed (message in fdg_last_error)       */
+    FDG_ERR_TIMEOUT = 7,       /* a bounded device-side wait gave up                           */
+    FDG_ERR_STATE = 8          /* call order violated (e.g. step before set_params)            */
+} fdg_status;
+
+typedef enum {
+    FDG_LINEAR = 0,            /* y = x W^T + b over the flattened sample                       */
+    FDG_CONV3X3 = 1,           /* padding 1, stride 1 or 2                                      */
+    FDG_CONV1X1 = 2,           /* padding 0, stride 1 or 2                                      */
+    FDG_RELU = 3,
+    FDG_MAXPOOL2 = 4,          /* 2x2 window, stride 2; ties: first maximum in row-major order  */
+    FDG_GLOBAL_AVGPOOL = 5,
+    FDG_BATCHNORM = 6,         /* per-worker batch statistics                                   */
+    FDG_RES_BEGIN = 7,         /* remember the current tensor as the shortcut                   */
+    FDG_RES_ADD = 8            /* add the shortcut (flags & 1: through conv1x1(stride) + BN)    */
+} fdg_layer_kind;
+
+/* flags: bit 0 = has bias (LINEAR / CONV*), or "projection shortcut" (RES_ADD). */
+typedef struct { int32_t kind, c_in, c_out, stride, flags; } fdg_layer;
+
+/* Device-memory allocator of the caller (e.g. PyTorch's caching allocator).  alloc returns a
+ * device pointer aligned to at least 256 bytes or NULL; free receives what alloc returned. */
+typedef struct {
+    void* (*alloc)(size_t bytes, void* user);
+    void  (*free)(void* ptr, void* user);
+    void* user;
+} fdg_allocator;
+
+typedef struct {
+    int32_t dtype;             /* 0: fp32 everywhere.  1: bf16 activations / weight copies /
+                                  error gradients, fp32 accumulation, fp32 master weights       */
+    int32_t in_h, in_w, in_c;  /* sample shape; 1,1,3072 for an MLP on flattened 32x32x3 inputs */
+    int32_t num_classes;       /* must equal the last layer's c_out                             */
+    int32_t serial;            /* 1: run every module on one stream (results are bit-identical
+                                  to the concurrent mode; used to test the event wiring)        */
+    int32_t kernel_path;       /* 0: tensor-core kernels where shapes allow (bf16 only);
+                                  1: plain FMA kernels only                                      */
+    void* const* streams;      /* K cudaStream_t of the caller, or NULL: the library creates K  */
+} fdg_options;
+
+/* Build a context.  Paper: the split of layers 1..L into groups g(1)..g(K) (Sec. 3.2) and the
+ * S x K agents of Sec. 3.3, all placed on the current CUDA device.
+ *   layers/n_layers : the network, host array.
+ *   split_points    : host array of K-1 layer indices (0-based): first layer of modules 2..K.
+ *   n_workers, per_worker_batch : N and B; every step consumes M = N*B samples.
+ *   lr              : step size eta (changeable later with fdg_set_lr).
+ *   alloc           : NULL selects cudaMalloc/cudaFree.
+ * Fails with BAD_SPLIT / UNSUPPORTED / ARCH / OOM before any kernel is launched. */
+FDG_API fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers,
+                      const int32_t* split_points, int32_t K,
+                      int32_t n_workers, int32_t per_worker_batch, float lr,
+                      const fdg_options* opt, const fdg_allocator* alloc, fdg_ctx** out);
+
+/* Number of parameters (length of the canonical parameter vector). */
+FDG_API fdg_status fdg_param_count(const fdg_ctx* ctx, size_t* count);
+
+/* Load version-0 weights from a host fp32 array in canonical order (the library draws no random
+ * numbers).  Resets the iteration counter to 0 and empties every FIFO. */
+FDG_API fdg_status fdg_set_params(fdg_ctx* ctx, const float* host_params, size_t count);
+
+/* One iteration t of Algorithm 1 for all modules and workers (steps listed at the top).
+ *   dev_inputs : device, [M, in_h, in_w, in_c] in the context's dtype (fp32 or bf16), the
+ *                batch sampled at iteration t; must be complete before the call (the library
+ *                copies it into its own FIFO on module 1's stream and does not keep the pointer).
+ *   dev_labels : device, int32 [M].
+ *   host_loss_or_null : if non-NULL the call waits for the last module and stores the mean
+ *                loss of the batch it processed in this iteration (tau = t-K+1; NaN while
+ *                tau < 0).  If NULL the call only enqueues work and returns. */
+FDG_API fdg_status fdg_step(fdg_ctx* ctx, const void* dev_inputs, const int32_t* dev_labels,
+                    float* host_loss_or_null);
+
+/* Same as fdg_step with HOST input buffers (pinned memory makes the copies asynchronous); the
+ * host-to-device copies go straight into the FIFO slot, ordered on module 1's stream. */
+FDG_API fdg_status fdg_step_host(fdg_ctx* ctx, const void* host_inputs, const int32_t* host_labels,
+                         float* host_loss_or_null);
+
+/* Wait for all modules, then copy the fp32 master weights w(t) (t = number of steps done) to a
+ * host array in canonical order.  count receives the number of floats written. */
+FDG_API fdg_status fdg_params(fdg_ctx* ctx, float* host_out, size_t capacity, size_t* count);
+
+/* Debug twin of fdg_params: the averaged gradients that entered the last step's update
+ * (zeros for modules that had no backward batch yet). */
+FDG_API fdg_status fdg_grads(fdg_ctx* ctx, float* host_out, size_t capacity, size_t* count);
+
+/* The delay schedule as observed on the device in the last step: every FIFO slot carries a tag
+ * (batch id, weight version) written on the producer's stream; each module's step copies the
+ * tags of the slots it is about to read into a trace.  Arrays of K int64 (host):
+ *   fwd_batch[k]          batch id found in the activation slot module k forwarded (-1 idle)
+ *   bwd_batch[k]          batch id found in the stash slot module k back-propagated (-1 idle);
+ *                         -2 if the error-gradient slot carried a different batch id
+ *   bwd_weight_version[k] version tag of the weight slot the backward pass read (-1 idle) */
+FDG_API fdg_status fdg_trace(fdg_ctx* ctx, int64_t* fwd_batch, int64_t* bwd_batch,
+                     int64_t* bwd_weight_version, int32_t K);
+
+/* Change the step size used by the following steps (a sequence eta_t, Algorithm 1's input). */
+FDG_API fdg_status fdg_set_lr(fdg_ctx* ctx, float lr);
+
+/* Bytes of device memory the context holds, and how many kernels it has launched so far. */
+FDG_API fdg_status fdg_stats(const fdg_ctx* ctx, size_t* device_bytes, uint64_t* kernel_launches);
+
+/* Device time of the last completed step of every module (ms, CUDA events on the module's
+ * stream; array of K floats) -- waits for the modules. */
+FDG_API fdg_status fdg_module_times(fdg_ctx* ctx, float* ms, int32_t K);
+
+FDG_API const char* fdg_last_error(const fdg_ctx* ctx);   /* ctx may be NULL: last create error */
+FDG_API void        fdg_destroy(fdg_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FDG_H */

@@ -1,0 +1,2 @@
+"""fdg: stale-gradient decoupled training step for sm_100a (see include/fdg.h)."""
+from . import synth  # noqa: F401

@@ -1,0 +1,667 @@
+// Step executor behind the C ABI of include/fdg.h: compiles the layer list into per-module op
+// programs, lays the staleness FIFOs out in device memory, and enqueues one iteration of
+// Algorithm 1 on one CUDA stream per module.
+//
+// FIFO layout per module k (0-based kk = k-1), D = 2(K-k)+1 (a batch forwarded at iteration
+// tau+k-1 is back-propagated at iteration tau+2K-k-1, Sec. 3.2):
+//   in_ring  : D+2 slots of the module's input activation.  Module k-1 writes its boundary output
+//              straight into slot (tau mod (D+2)); module k reads it one iteration later for its
+//              forward pass and 2(K-k) iterations after that for its backward pass.  The two extra
+//              slots keep the producer's next write away from both readers without ordering the
+//              forward and backward passes of an iteration.
+//   stash    : D slots holding every intermediate activation (and batch-norm statistics) of the module.
+//   wring    : D slots of weight versions (storage-dtype copies of the matrices + fp32 copies of the
+//              vectors); version v lives in slot v mod D.
+//   d2       : 2 slots of the error gradient w.r.t. the module's input; written in iteration t to
+//              slot t&1, read by module k-1 in iteration t+1.
+// Streams: module k's work of iteration t+1 waits only for the events modules k-1 and k+1 recorded
+// at the end of iteration t.
+#include "../../include/fdg.h"
+#include "kernels.h"
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+using namespace fdg;
+
+namespace {
+
+thread_local std::string g_create_error;
+
+enum OpType { OP_CONV, OP_BN, OP_RELU, OP_POOL, OP_GAP, OP_ADD };
+enum Loc { LOC_IN, LOC_STASH, LOC_NEXT, LOC_LOGITS };
+
+struct TensorDesc {
+    int h, w, c;
+    Loc loc;
+    size_t off;        // byte offset inside a stash slot (LOC_STASH)
+    size_t goff;       // byte offset of its gradient inside the module's gradient pool
+    bool own_grad;     // gradient lives in the pool (false: d2 slot / dlogits / none)
+    size_t elems() const { return (size_t)h * w * c; }
+};
+
+struct Op {
+    OpType type;
+    int in, in2, out;
+    ConvGeom g;                    // OP_CONV
+    bool bias, relu, has_res;
+    size_t w_off, b_off;           // element offsets: w_off in the big segment, b_off/gamma/beta in the small segment
+    size_t gamma_off, beta_off;
+    size_t stats_off;              // byte offset of saved (mean, invstd) inside the stash slot (OP_BN)
+    bool acc_in, acc_in2;          // backward accumulates into an already written gradient
+    bool need_dgrad;
+};
+
+struct Segment { size_t canon, internal, count; bool big; };
+
+struct Module {
+    int p, q, D, in_depth;
+    std::vector<TensorDesc> t;
+    std::vector<Op> ops;
+    std::vector<Segment> segs;
+    size_t n_big, n_small;         // padded element counts of the two parameter segments
+    size_t in_elems;               // per-sample elements of the input / output tensor
+    size_t stash_slot_bytes, wslot_bytes, grad_pool_bytes, in_slot_bytes;
+    size_t ws_elems, scratch_elems, red_elems;
+    char *in_ring, *stash, *gradpool, *d2, *wring;
+    float *master, *grad, *ws, *scratch, *red;
+    int64_t *tag_in, *tag_stash, *tag_d2, *tag_w, *trace;
+    cudaStream_t stream;
+    cudaEvent_t done, ev0, ev1;
+    bool had_bwd;
+};
+
+}  // namespace
+
+struct fdg_ctx {
+    int K, n_workers, B, M, dt, esz, classes, serial, kernel_path;
+    int in_h, in_w, in_c;
+    float lr;
+    int64_t t;
+    bool have_params;
+    std::vector<fdg_layer> layers;
+    std::vector<Module> mod;
+    std::vector<void*> blocks;
+    fdg_allocator alloc;
+    bool own_streams;
+    std::vector<cudaStream_t> owned;
+    size_t n_params, device_bytes;
+    int label_depth;
+    int32_t* labels;
+    float* logits;
+    char* dlogits;
+    float* loss_ring;
+    int64_t* tags;
+    std::string err;
+};
+
+namespace {
+
+fdg_status fail(fdg_ctx* c, fdg_status s, const char* fmt, ...) {
+    char buf[512];
+    va_list ap; va_start(ap, fmt); vsnprintf(buf, sizeof buf, fmt, ap); va_end(ap);
+    if (c) c->err = buf; else g_create_error = buf;
+    return s;
+}
+#define CK(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return fail(ctx, FDG_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); } while (0)
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+void* default_alloc(size_t bytes, void*) { void* p = nullptr; return cudaMalloc(&p, bytes) == cudaSuccess ? p : nullptr; }
+void default_free(void* p, void*) { cudaFree(p); }
+
+// ---- compile layers [p,q) into ops; returns "" or an error text
+std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool last, size_t& canon_off) {
+    const auto& L = ctx->layers;
+    auto add_tensor = [&](int th, int tw, int tc) { TensorDesc d{}; d.h = th; d.w = tw; d.c = tc; d.loc = LOC_STASH; d.own_grad = true; m.t.push_back(d); return (int)m.t.size() - 1; };
+    int cur = add_tensor(h, w, c);
+    m.t[0].loc = LOC_IN;
+    m.in_elems = m.t[0].elems();
+    std::vector<int> stack;
+    size_t big = 0, small = 0;
+    auto seg = [&](size_t count, bool is_big) {
+        size_t& pos = is_big ? big : small;
+        m.segs.push_back({canon_off, pos, count, is_big});
+        size_t at = pos; canon_off += count; pos += is_big ? align_up(count, 8) : align_up(count, 4);
+        return at;
+    };
+    auto emit_conv = [&](int in, int kind, int cin, int cout, int stride, bool bias, bool relu) -> std::string {
+        const TensorDesc& ti = m.t[in];
+        Op o{}; o.type = OP_CONV; o.in = in; o.in2 = -1; o.bias = bias; o.relu = relu;
+        ConvGeom g{};
+        g.N = ctx->M;
+        if (kind == FDG_LINEAR) {
+            if ((size_t)cin != ti.elems()) return "linear c_in does not match the flattened input";
+            g.H = g.W = 1; g.C = cin; g.R = 1; g.stride = 1; g.pad = 0;
+        } else {
+            if (cin != ti.c) return "conv c_in does not match the input channels";
+            if (stride != 1 && stride != 2) return "stride must be 1 or 2";
+            if (stride == 2 && ((ti.h | ti.w) & 1)) return "stride-2 conv needs even height and width";
+            g.H = ti.h; g.W = ti.w; g.C = cin; g.R = kind == FDG_CONV3X3 ? 3 : 1; g.stride = stride; g.pad = kind == FDG_CONV3X3 ? 1 : 0;
+        }
+        g.Co = cout; g.Ho = (g.H + 2 * g.pad - g.R) / g.stride + 1; g.Wo = (g.W + 2 * g.pad - g.R) / g.stride + 1;
+        o.g = g;
+        o.w_off = seg((size_t)g.R * g.R * g.C * g.Co, true);
+        if (bias) o.b_off = seg(cout, false);
+        o.out = add_tensor(g.Ho, g.Wo, cout);
+        m.ops.push_back(o);
+        return "";
+    };
+    auto emit_bn = [&](int in, int in2, bool relu) {
+        Op o{}; o.type = OP_BN; o.in = in; o.in2 = in2; o.has_res = in2 >= 0; o.relu = relu;
+        const TensorDesc ti = m.t[in];
+        o.g = ConvGeom{}; o.g.C = ti.c;
+        o.gamma_off = seg(ti.c, false); o.beta_off = seg(ti.c, false);
+        o.out = add_tensor(ti.h, ti.w, ti.c);
+        m.ops.push_back(o);
+        return o.out;
+    };
+    // a projecting shortcut: conv1x1(stride) + batch-norm of the saved block input
+    auto emit_shortcut = [&](const fdg_layer& Y, int sc, std::string& err) -> int {
+        if (!(Y.flags & 1)) return sc;
+        err = emit_conv(sc, FDG_CONV1X1, Y.c_in, Y.c_out, Y.stride, false, false);
+        if (!err.empty()) return -1;
+        return emit_bn(m.ops.back().out, -1, false);
+    };
+
+    for (int l = m.p; l < m.q; ++l) {
+        const fdg_layer& Y = L[l];
+        const TensorDesc tc = m.t[cur];
+        auto next_is = [&](int kind) { return l + 1 < m.q && L[l + 1].kind == kind; };
+        switch (Y.kind) {
+            case FDG_LINEAR: case FDG_CONV3X3: case FDG_CONV1X1: {
+                bool relu = next_is(FDG_RELU);
+                std::string e = emit_conv(cur, Y.kind, Y.c_in, Y.c_out, Y.stride, Y.flags & 1, relu);
+                if (!e.empty()) return e;
+                cur = m.ops.back().out;
+                if (relu) ++l;
+                break; }
+            case FDG_BATCHNORM: {
+                if (Y.c_in != tc.c) return "batch-norm channel count does not match";
+                if (next_is(FDG_RES_ADD)) {
+                    // canonical order: the batch-norm's gamma/beta come before the shortcut's parameters
+                    const fdg_layer& A = L[l + 1];
+                    if (stack.empty()) return "RES_ADD without RES_BEGIN";
+                    int sc = stack.back(); stack.pop_back();
+                    size_t gcan = canon_off; canon_off += 2 * (size_t)tc.c;         // reserve gamma, beta
+                    std::string e; int s2 = emit_shortcut(A, sc, e);
+                    if (!e.empty()) return e;
+                    const TensorDesc ts = m.t[s2];
+                    if (ts.h != tc.h || ts.w != tc.w || ts.c != tc.c) return "shortcut shape does not match the block output";
+                    l += 1;
+                    bool relu = next_is(FDG_RELU);
+                    size_t after = canon_off; canon_off = gcan;
+                    cur = emit_bn(cur, s2, relu);
+                    canon_off = after;
+                    if (relu) ++l;
+                } else {
+                    bool relu = next_is(FDG_RELU);
+                    cur = emit_bn(cur, -1, relu);
+                    if (relu) ++l;
+                }
+                break; }
+            case FDG_RELU: { Op o{}; o.type = OP_RELU; o.in = cur; o.in2 = -1; o.out = add_tensor(tc.h, tc.w, tc.c); m.ops.push_back(o); cur = o.out; break; }
+            case FDG_MAXPOOL2: {
+                if ((tc.h | tc.w) & 1) return "max-pool needs even height and width";
+                Op o{}; o.type = OP_POOL; o.in = cur; o.in2 = -1; o.out = add_tensor(tc.h / 2, tc.w / 2, tc.c); m.ops.push_back(o); cur = o.out; break; }
+            case FDG_GLOBAL_AVGPOOL: { Op o{}; o.type = OP_GAP; o.in = cur; o.in2 = -1; o.out = add_tensor(1, 1, tc.c); m.ops.push_back(o); cur = o.out; break; }
+            case FDG_RES_BEGIN: stack.push_back(cur); break;
+            case FDG_RES_ADD: {
+                if (stack.empty()) return "RES_ADD without RES_BEGIN";
+                int sc = stack.back(); stack.pop_back();
+                std::string e; int s2 = emit_shortcut(Y, sc, e);
+                if (!e.empty()) return e;
+                const TensorDesc ts = m.t[s2];
+                if (ts.h != tc.h || ts.w != tc.w || ts.c != tc.c) return "shortcut shape does not match the block output";
+                Op o{}; o.type = OP_ADD; o.in = cur; o.in2 = s2; o.out = add_tensor(tc.h, tc.w, tc.c); m.ops.push_back(o); cur = o.out; break; }
+            default: return "unknown layer kind";
+        }
+    }
+    if (!stack.empty()) return "BAD_SPLIT: a split point cuts a residual block";
+    if (m.ops.empty()) return "a module has no computing layer";
+    if (m.ops.back().out != cur) return "internal: dangling tensor";
+    h = m.t[cur].h; w = m.t[cur].w; c = m.t[cur].c;
+    if (last) {
+        const Op& o = m.ops.back();
+        if (o.type != OP_CONV || o.relu || o.g.Ho * o.g.Wo != 1) return "the network must end with a linear layer";
+        m.t[cur].loc = LOC_LOGITS;
+    } else {
+        m.t[cur].loc = LOC_NEXT;
+    }
+    m.t[cur].own_grad = false;
+    m.t[0].own_grad = false;
+    m.n_big = big; m.n_small = small;
+
+    // stash layout, gradient pool layout, scratch sizes
+    size_t soff = 0, goff = 0;
+    for (size_t i = 0; i < m.t.size(); ++i) {
+        TensorDesc& d = m.t[i];
+        if (d.loc == LOC_STASH) { d.off = soff; soff += align_up(d.elems() * ctx->M * ctx->esz, 256); }
+        if (d.own_grad) { d.goff = goff; goff += align_up(d.elems() * ctx->M * ctx->esz, 256); }
+    }
+    m.ws_elems = 0; m.scratch_elems = 64; m.red_elems = 4;
+    for (Op& o : m.ops) {
+        if (o.type == OP_BN) {
+            o.stats_off = soff; soff += align_up((size_t)ctx->n_workers * o.g.C * 2 * sizeof(float), 256);
+            m.scratch_elems = std::max(m.scratch_elems, (size_t)64 * ctx->n_workers * o.g.C * 2);
+            m.red_elems = std::max(m.red_elems, (size_t)ctx->n_workers * o.g.C * 2);
+        }
+        if (o.type == OP_CONV) {
+            m.ws_elems = std::max(m.ws_elems, wgrad_workspace_elems(o.g));
+            m.scratch_elems = std::max(m.scratch_elems, (size_t)64 * o.g.Co);
+        }
+    }
+    m.stash_slot_bytes = align_up(soff, 256);
+    m.grad_pool_bytes = align_up(goff, 256);
+    // backward write/accumulate analysis: walking the ops in reverse, the first op that touches a
+    // tensor's gradient writes it, later ones add to it
+    std::vector<char> written(m.t.size(), 0);
+    for (int i = (int)m.ops.size() - 1; i >= 0; --i) {
+        Op& o = m.ops[i];
+        o.acc_in = written[o.in]; written[o.in] = 1;
+        if (o.in2 >= 0) { o.acc_in2 = written[o.in2]; written[o.in2] = 1; }
+        o.need_dgrad = true;
+    }
+    return "";
+}
+
+struct StepPtrs {            // resolved addresses for one (module, batch)
+    fdg_ctx* c; Module* m; int kk;
+    int64_t batch;
+    char* tensor(int id) const {
+        const TensorDesc& d = m->t[id];
+        switch (d.loc) {
+            case LOC_IN: return m->in_ring + (size_t)(batch % m->in_depth) * m->in_slot_bytes;
+            case LOC_STASH: return m->stash + (size_t)(batch % m->D) * m->stash_slot_bytes + d.off;
+            case LOC_NEXT: { Module& n = c->mod[kk + 1]; return n.in_ring + (size_t)(batch % n.in_depth) * n.in_slot_bytes; }
+            case LOC_LOGITS: return (char*)c->logits;
+        }
+        return nullptr;
+    }
+    float* stats(const Op& o) const { return (float*)(m->stash + (size_t)(batch % m->D) * m->stash_slot_bytes + o.stats_off); }
+};
+
+char* wslot(fdg_ctx* c, Module& m, int64_t version) { return m.wring + (size_t)(version % m.D) * m.wslot_bytes; }
+char* wbig(fdg_ctx* c, Module& m, int64_t version, size_t off) { return wslot(c, m, version) + off * c->esz; }
+float* wsmall(fdg_ctx* c, Module& m, int64_t version, size_t off) { return (float*)(wslot(c, m, version) + m.n_big * c->esz) + off; }
+
+void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version) {
+    Module& m = c->mod[kk];
+    StepPtrs P{c, &m, kk, batch};
+    cudaStream_t s = m.stream;
+    const int dt = c->dt;
+    for (const Op& o : m.ops) {
+        const TensorDesc& ti = m.t[o.in];
+        const TensorDesc& to = m.t[o.out];
+        size_t n_out = to.elems() * c->M;
+        switch (o.type) {
+            case OP_CONV: {
+                int epi = (o.relu ? EPI_RELU : 0) | (to.loc == LOC_LOGITS ? EPI_OUT_F32 : 0);
+                conv_forward(dt, P.tensor(o.in), wbig(c, m, version, o.w_off), o.bias ? wsmall(c, m, version, o.b_off) : nullptr,
+                             P.tensor(o.out), o.g, epi, s);
+                break; }
+            case OP_BN:
+                bn_forward(dt, P.tensor(o.in), wsmall(c, m, version, o.gamma_off), wsmall(c, m, version, o.beta_off),
+                           o.has_res ? P.tensor(o.in2) : nullptr, P.tensor(o.out), P.stats(o), m.scratch, c->n_workers,
+                           (long)c->B * ti.h * ti.w, ti.c, o.relu, s);
+                break;
+            case OP_RELU: relu_forward(dt, P.tensor(o.in), P.tensor(o.out), n_out, s); break;
+            case OP_POOL: maxpool_forward(dt, P.tensor(o.in), P.tensor(o.out), c->M, ti.h, ti.w, ti.c, s); break;
+            case OP_GAP: gap_forward(dt, P.tensor(o.in), P.tensor(o.out), c->M, ti.h * ti.w, ti.c, s); break;
+            case OP_ADD: add_forward(dt, P.tensor(o.in), P.tensor(o.in2), P.tensor(o.out), n_out, s); break;
+        }
+    }
+}
+
+// gradient buffer of a tensor during iteration t
+char* grad_ptr(fdg_ctx* c, int kk, int id, int64_t t) {
+    Module& m = c->mod[kk];
+    const TensorDesc& d = m.t[id];
+    if (d.own_grad) return m.gradpool + d.goff;
+    if (id == 0) return kk > 0 ? m.d2 + (size_t)(t & 1) * m.in_slot_bytes : nullptr;          // sent to module k-1
+    if (d.loc == LOC_LOGITS) return c->dlogits;
+    Module& n = c->mod[kk + 1];                                                                // received from module k+1
+    return n.d2 + (size_t)((t - 1) & 1) * n.in_slot_bytes;
+}
+
+void backward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int64_t t) {
+    Module& m = c->mod[kk];
+    StepPtrs P{c, &m, kk, batch};
+    cudaStream_t s = m.stream;
+    const int dt = c->dt;
+    for (int i = (int)m.ops.size() - 1; i >= 0; --i) {
+        const Op& o = m.ops[i];
+        const TensorDesc& ti = m.t[o.in];
+        const TensorDesc& to = m.t[o.out];
+        size_t n_out = to.elems() * c->M, n_in = ti.elems() * c->M;
+        char* gout = grad_ptr(c, kk, o.out, t);
+        char* gin = grad_ptr(c, kk, o.in, t);
+        switch (o.type) {
+            case OP_CONV: {
+                if (o.relu) relu_backward(dt, P.tensor(o.out), gout, gout, n_out, false, s);       // in place: dZ = dA * (A > 0)
+                conv_wgrad(dt, P.tensor(o.in), gout, m.grad + o.w_off, m.ws, o.g, s);
+                if (o.bias) bias_grad(dt, gout, m.grad + m.n_big + o.b_off, m.scratch, (long)o.g.N * o.g.Ho * o.g.Wo, o.g.Co, s);
+                if (gin) conv_dgrad(dt, gout, wbig(c, m, version, o.w_off), gin, o.g, o.acc_in ? EPI_ACCUM : 0, s);
+                break; }
+            case OP_BN: {
+                char* gres = o.has_res ? grad_ptr(c, kk, o.in2, t) : nullptr;
+                bn_backward(dt, P.tensor(o.in), P.tensor(o.out), gout, wsmall(c, m, version, o.gamma_off), P.stats(o),
+                            gin, o.acc_in, gres, o.acc_in2, m.grad + m.n_big + o.gamma_off, m.grad + m.n_big + o.beta_off,
+                            m.red, m.scratch, c->n_workers, (long)c->B * ti.h * ti.w, ti.c, o.relu, s);
+                break; }
+            case OP_RELU: if (gin) relu_backward(dt, P.tensor(o.out), gout, gin, n_out, o.acc_in, s); break;
+            case OP_POOL: if (gin) maxpool_backward(dt, P.tensor(o.in), gout, gin, c->M, ti.h, ti.w, ti.c, o.acc_in, s); break;
+            case OP_GAP: if (gin) gap_backward(dt, gout, gin, c->M, ti.h * ti.w, ti.c, o.acc_in, s); break;
+            case OP_ADD: {
+                if (gin) copy_or_accumulate(dt, gout, gin, n_in, o.acc_in, s);
+                char* g2 = grad_ptr(c, kk, o.in2, t);
+                if (g2) copy_or_accumulate(dt, gout, g2, n_in, o.acc_in2, s);
+                break; }
+        }
+    }
+}
+
+fdg_status reset_state(fdg_ctx* ctx) {
+    // tags: everything -1 (empty); weight slot 0 carries version 0
+    size_t n_tags = 0;
+    for (Module& m : ctx->mod) n_tags += 2 * (size_t)(m.in_depth + m.D + 2 + m.D) + 4;
+    std::vector<int64_t> h(n_tags, -1);
+    size_t pos = 0;
+    for (Module& m : ctx->mod) {
+        pos += 2 * (size_t)(m.in_depth + m.D + 2);
+        h[pos + 1] = 0;                      // weight slot 0: version 0
+        pos += 2 * (size_t)m.D + 4;
+    }
+    CK(cudaMemcpy(ctx->tags, h.data(), n_tags * sizeof(int64_t), cudaMemcpyHostToDevice));
+    ctx->t = 0;
+    for (Module& m : ctx->mod) m.had_bwd = false;
+    return FDG_OK;
+}
+
+fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, bool host_src, float* host_loss) {
+    if (!ctx) return FDG_ERR_INVALID_ARG;
+    if (!inputs || !labels) return fail(ctx, FDG_ERR_INVALID_ARG, "inputs and labels must not be NULL");
+    if (!ctx->have_params) return fail(ctx, FDG_ERR_STATE, "fdg_set_params must be called before fdg_step");
+    const int K = ctx->K;
+    const int64_t t = ctx->t;
+    // 1. dependencies on the neighbours' previous iteration (all waits first, so that no wait sees an
+    //    event recorded for THIS iteration)
+    if (!ctx->serial && t > 0)
+        for (int kk = 0; kk < K; ++kk) {
+            if (kk > 0) CK(cudaStreamWaitEvent(ctx->mod[kk].stream, ctx->mod[kk - 1].done, 0));
+            if (kk + 1 < K) CK(cudaStreamWaitEvent(ctx->mod[kk].stream, ctx->mod[kk + 1].done, 0));
+        }
+    // 2. module 1 "samples" the batch of iteration t: copy into its FIFO slot; labels into the label FIFO
+    {
+        Module& m0 = ctx->mod[0];
+        cudaMemcpyKind kind = host_src ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
+        CK(cudaMemcpyAsync(m0.in_ring + (size_t)(t % m0.in_depth) * m0.in_slot_bytes, inputs,
+                           (size_t)ctx->M * m0.in_elems * ctx->esz, kind, m0.stream));
+        CK(cudaMemcpyAsync(ctx->labels + (size_t)(t % ctx->label_depth) * ctx->M, labels, (size_t)ctx->M * sizeof(int32_t), kind, m0.stream));
+    }
+    // 3. every module: forward on tau_f, backward on tau_b, update
+    for (int kk = 0; kk < K; ++kk) {
+        Module& m = ctx->mod[kk];
+        const int64_t tau_f = t - kk;                         // t - k + 1
+        const int64_t tau_b = t - 2 * (int64_t)K + kk + 2;    // t - 2K + k + 1
+        const int64_t v_b = tau_b + kk;                       // t - 2K + 2k: the version the forward of tau_b used
+        const bool lastm = kk == K - 1;
+        CK(cudaEventRecord(m.ev0, m.stream));
+        TagOps tg{};
+        if (tau_f >= 0) {
+            tg.rd_act = m.tag_in + 2 * (tau_f % m.in_depth);
+            tg.rd_wfwd = m.tag_w + 2 * (t % m.D);
+            tg.wr_stash = m.tag_stash + 2 * (tau_f % m.D);
+            if (!lastm) { Module& n = ctx->mod[kk + 1]; tg.wr_out = n.tag_in + 2 * (tau_f % n.in_depth); }
+        }
+        if (kk == 0) tg.wr_in = m.tag_in + 2 * (t % m.in_depth);   // the ingest above filled this slot with batch t
+        if (tau_b >= 0) {
+            tg.rd_stash = m.tag_stash + 2 * (tau_b % m.D);
+            tg.rd_wbwd = m.tag_w + 2 * (v_b % m.D);
+            if (!lastm) tg.rd_grad = ctx->mod[kk + 1].tag_d2 + 2 * ((t - 1) & 1);
+            if (kk > 0) tg.wr_grad = m.tag_d2 + 2 * (t & 1);
+        }
+        tg.wr_wnext = m.tag_w + 2 * ((t + 1) % m.D);
+        tg.fwd_batch = tau_f >= 0 ? tau_f : -1; tg.bwd_batch = tau_b >= 0 ? tau_b : -1; tg.version_now = t;
+        tg.trace = m.trace;
+        tags_step(tg, m.stream);
+
+        if (tau_f >= 0) forward_module(ctx, kk, tau_f, t);
+        if (lastm) {
+            float* loss_slot = ctx->loss_ring + (t % 64);
+            if (tau_f >= 0) softmax_ce(ctx->dt, ctx->logits, ctx->labels + (size_t)(tau_f % ctx->label_depth) * ctx->M, ctx->dlogits,
+                                       loss_slot, ctx->M, ctx->classes, m.stream);
+            else fill_f32(loss_slot, NAN, 1, m.stream);
+        }
+        if (tau_b >= 0) backward_module(ctx, kk, tau_b, v_b, t);
+        // Eq. dl_update with P = 11^T/N: w(t+1) = w(t) - lr * averaged gradient; also emits version t+1
+        sgd_update(ctx->dt, m.master, tau_b >= 0 ? m.grad : nullptr, wslot(ctx, m, t + 1), m.n_big, ctx->lr, m.stream);
+        if (m.n_small)
+            sgd_update(0, m.master + m.n_big, tau_b >= 0 ? m.grad + m.n_big : nullptr,
+                       wsmall(ctx, m, t + 1, 0), m.n_small, ctx->lr, m.stream);
+        m.had_bwd = tau_b >= 0;
+        CK(cudaEventRecord(m.ev1, m.stream));
+        CK(cudaEventRecord(m.done, m.stream));
+    }
+    CK(cudaGetLastError());
+    ctx->t = t + 1;
+    if (host_loss) {
+        CK(cudaStreamSynchronize(ctx->mod[K - 1].stream));
+        CK(cudaMemcpy(host_loss, ctx->loss_ring + (t % 64), sizeof(float), cudaMemcpyDeviceToHost));
+    }
+    return FDG_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* fdg_last_error(const fdg_ctx* ctx) { return ctx ? ctx->err.c_str() : g_create_error.c_str(); }
+
+void fdg_destroy(fdg_ctx* ctx) {
+    if (!ctx) return;
+    cudaDeviceSynchronize();
+    for (Module& m : ctx->mod) {
+        if (m.done) cudaEventDestroy(m.done);
+        if (m.ev0) cudaEventDestroy(m.ev0);
+        if (m.ev1) cudaEventDestroy(m.ev1);
+    }
+    for (cudaStream_t s : ctx->owned) cudaStreamDestroy(s);
+    for (void* p : ctx->blocks) ctx->alloc.free(p, ctx->alloc.user);
+    delete ctx;
+}
+
+fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* split_points, int32_t K,
+                      int32_t n_workers, int32_t per_worker_batch, float lr, const fdg_options* opt,
+                      const fdg_allocator* alloc, fdg_ctx** out) {
+    fdg_ctx* ctx = nullptr;     // errors before the context exists go to the thread-local message
+    if (!layers || n_layers <= 0 || K < 1 || (K > 1 && !split_points) || n_workers < 1 || per_worker_batch < 1 || !opt || !out)
+        return fail(nullptr, FDG_ERR_INVALID_ARG, "null pointer or non-positive size");
+    if (opt->dtype != 0 && opt->dtype != 1) return fail(nullptr, FDG_ERR_INVALID_ARG, "dtype must be 0 (fp32) or 1 (bf16)");
+    if (opt->in_h < 1 || opt->in_w < 1 || opt->in_c < 1 || opt->num_classes < 2) return fail(nullptr, FDG_ERR_INVALID_ARG, "bad input shape or class count");
+    if (K > 64) return fail(nullptr, FDG_ERR_INVALID_ARG, "K > 64");
+    for (int k = 0; k + 1 < K; ++k) {
+        int prev = k ? split_points[k - 1] : 0;
+        if (split_points[k] <= prev || split_points[k] >= n_layers) return fail(nullptr, FDG_ERR_BAD_SPLIT, "split points must be strictly increasing inside 1..n_layers-1");
+    }
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) { cudaGetLastError(); return fail(nullptr, FDG_ERR_ARCH, "no CUDA device"); }
+    int dev = 0; cudaDeviceProp prop;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return fail(nullptr, FDG_ERR_CUDA, "cannot query the device");
+    if (prop.major != 10) return fail(nullptr, FDG_ERR_ARCH, "device is sm_%d%d; this library is built for sm_100a only", prop.major, prop.minor);
+
+    ctx = new fdg_ctx();
+    ctx->K = K; ctx->n_workers = n_workers; ctx->B = per_worker_batch; ctx->M = n_workers * per_worker_batch;
+    ctx->dt = opt->dtype; ctx->esz = opt->dtype ? 2 : 4; ctx->classes = opt->num_classes; ctx->serial = opt->serial;
+    ctx->kernel_path = opt->kernel_path;
+    ctx->in_h = opt->in_h; ctx->in_w = opt->in_w; ctx->in_c = opt->in_c; ctx->lr = lr; ctx->t = 0; ctx->have_params = false;
+    ctx->layers.assign(layers, layers + n_layers);
+    ctx->alloc = alloc ? *alloc : fdg_allocator{default_alloc, default_free, nullptr};
+    ctx->own_streams = opt->streams == nullptr;
+    ctx->device_bytes = 0;
+    ctx->mod.resize(K);
+    auto bail = [&](fdg_status s, const std::string& msg) { g_create_error = msg; fdg_destroy(ctx); return s; };
+
+    int h = opt->in_h, w = opt->in_w, c = opt->in_c;
+    size_t canon = 0;
+    for (int kk = 0; kk < K; ++kk) {
+        Module& m = ctx->mod[kk];
+        m = Module{};
+        m.p = kk ? split_points[kk - 1] : 0; m.q = kk + 1 < K ? split_points[kk] : n_layers;
+        m.D = 2 * (K - kk - 1) + 1; m.in_depth = m.D + 2;
+        std::string e = compile_module(ctx, m, h, w, c, kk == K - 1, canon);
+        if (!e.empty()) {
+            fdg_status s = e.rfind("BAD_SPLIT", 0) == 0 ? FDG_ERR_BAD_SPLIT : FDG_ERR_UNSUPPORTED;
+            char buf[256]; snprintf(buf, sizeof buf, "module %d: %s", kk + 1, e.c_str());
+            return bail(s, buf);
+        }
+        m.in_slot_bytes = align_up((size_t)ctx->M * m.in_elems * ctx->esz, 256);
+        m.wslot_bytes = align_up(m.n_big * ctx->esz + m.n_small * sizeof(float), 256);
+    }
+    if (h * w * c != opt->num_classes) return bail(FDG_ERR_INVALID_ARG, "the last layer's width differs from num_classes");
+    ctx->n_params = canon;
+    ctx->label_depth = 2 * K;
+
+    // ---- device memory
+    bool oom = false;
+    auto get = [&](size_t bytes) -> char* {
+        if (oom) return nullptr;
+        bytes = align_up(bytes ? bytes : 256, 256);
+        void* p = ctx->alloc.alloc(bytes, ctx->alloc.user);
+        if (!p) { oom = true; return nullptr; }
+        ctx->blocks.push_back(p); ctx->device_bytes += bytes;
+        return (char*)p;
+    };
+    size_t n_tags = 0;
+    for (Module& m : ctx->mod) n_tags += 2 * (size_t)(m.in_depth + m.D + 2 + m.D) + 4;
+    ctx->tags = (int64_t*)get(n_tags * sizeof(int64_t));
+    ctx->labels = (int32_t*)get((size_t)ctx->label_depth * ctx->M * sizeof(int32_t));
+    ctx->logits = (float*)get((size_t)ctx->M * ctx->classes * sizeof(float));
+    ctx->dlogits = get((size_t)ctx->M * ctx->classes * ctx->esz);
+    ctx->loss_ring = (float*)get(64 * sizeof(float));
+    size_t tpos = 0;
+    for (int kk = 0; kk < K && !oom; ++kk) {
+        Module& m = ctx->mod[kk];
+        m.in_ring = get((size_t)m.in_depth * m.in_slot_bytes);
+        m.stash = get((size_t)m.D * m.stash_slot_bytes);
+        m.gradpool = get(m.grad_pool_bytes);
+        m.d2 = kk > 0 ? get(2 * m.in_slot_bytes) : nullptr;
+        m.wring = get((size_t)m.D * m.wslot_bytes);
+        m.master = (float*)get((m.n_big + m.n_small) * sizeof(float));
+        m.grad = (float*)get((m.n_big + m.n_small) * sizeof(float));
+        m.ws = (float*)get(m.ws_elems * sizeof(float));
+        m.scratch = (float*)get(m.scratch_elems * sizeof(float));
+        m.red = (float*)get(m.red_elems * sizeof(float));
+        if (oom) break;
+        m.tag_in = ctx->tags + tpos; tpos += 2 * (size_t)m.in_depth;
+        m.tag_stash = ctx->tags + tpos; tpos += 2 * (size_t)m.D;
+        m.tag_d2 = ctx->tags + tpos; tpos += 4;
+        m.tag_w = ctx->tags + tpos; tpos += 2 * (size_t)m.D;
+        m.trace = ctx->tags + tpos; tpos += 4;
+    }
+    if (oom) return bail(FDG_ERR_OOM, "the allocator returned NULL");
+    for (int kk = 0; kk < K; ++kk) {
+        Module& m = ctx->mod[kk];
+        cudaError_t e = cudaSuccess;
+        if (opt->streams) m.stream = (cudaStream_t)opt->streams[ctx->serial ? 0 : kk];
+        else if (ctx->serial && kk > 0) m.stream = ctx->mod[0].stream;
+        else { e = cudaStreamCreateWithFlags(&m.stream, cudaStreamNonBlocking); if (e == cudaSuccess) ctx->owned.push_back(m.stream); }
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.done, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreate(&m.ev0);
+        if (e == cudaSuccess) e = cudaEventCreate(&m.ev1);
+        if (e == cudaSuccess) e = cudaMemset(m.grad, 0, (m.n_big + m.n_small) * sizeof(float));
+        if (e == cudaSuccess) e = cudaMemset(m.master, 0, (m.n_big + m.n_small) * sizeof(float));
+        if (e != cudaSuccess) return bail(FDG_ERR_CUDA, cudaGetErrorString(e));
+    }
+    *out = ctx;
+    return FDG_OK;
+}
+
+fdg_status fdg_param_count(const fdg_ctx* ctx, size_t* count) {
+    if (!ctx || !count) return FDG_ERR_INVALID_ARG;
+    *count = ctx->n_params;
+    return FDG_OK;
+}
+
+fdg_status fdg_set_params(fdg_ctx* ctx, const float* host_params, size_t count) {
+    if (!ctx || !host_params) return FDG_ERR_INVALID_ARG;
+    if (count != ctx->n_params) return fail(ctx, FDG_ERR_INVALID_ARG, "expected %zu parameters, got %zu", ctx->n_params, count);
+    CK(cudaDeviceSynchronize());
+    for (Module& m : ctx->mod) {
+        std::vector<float> h(m.n_big + m.n_small, 0.f);
+        for (const Segment& s : m.segs)
+            std::memcpy(h.data() + (s.big ? 0 : m.n_big) + s.internal, host_params + s.canon, s.count * sizeof(float));
+        CK(cudaMemcpy(m.master, h.data(), h.size() * sizeof(float), cudaMemcpyHostToDevice));
+        // version 0 into weight slot 0
+        sgd_update(ctx->dt, m.master, nullptr, wslot(ctx, m, 0), m.n_big, 0.f, m.stream);
+        if (m.n_small) sgd_update(0, m.master + m.n_big, nullptr, wsmall(ctx, m, 0, 0), m.n_small, 0.f, m.stream);
+        CK(cudaMemsetAsync(m.grad, 0, (m.n_big + m.n_small) * sizeof(float), m.stream));
+    }
+    fdg_status s = reset_state(ctx);
+    if (s != FDG_OK) return s;
+    CK(cudaDeviceSynchronize());
+    ctx->have_params = true;
+    return FDG_OK;
+}
+
+fdg_status fdg_step(fdg_ctx* ctx, const void* dev_inputs, const int32_t* dev_labels, float* host_loss_or_null) {
+    return run_step(ctx, dev_inputs, dev_labels, false, host_loss_or_null);
+}
+fdg_status fdg_step_host(fdg_ctx* ctx, const void* host_inputs, const int32_t* host_labels, float* host_loss_or_null) {
+    return run_step(ctx, host_inputs, host_labels, true, host_loss_or_null);
+}
+
+static fdg_status gather(fdg_ctx* ctx, bool grads, float* host_out, size_t capacity, size_t* count) {
+    if (!ctx || !host_out) return FDG_ERR_INVALID_ARG;
+    if (capacity < ctx->n_params) return fail(ctx, FDG_ERR_INVALID_ARG, "capacity %zu < %zu parameters", capacity, ctx->n_params);
+    CK(cudaDeviceSynchronize());
+    for (Module& m : ctx->mod) {
+        std::vector<float> h(m.n_big + m.n_small, 0.f);
+        if (!grads || m.had_bwd) CK(cudaMemcpy(h.data(), grads ? m.grad : m.master, h.size() * sizeof(float), cudaMemcpyDeviceToHost));
+        for (const Segment& s : m.segs)
+            std::memcpy(host_out + s.canon, h.data() + (s.big ? 0 : m.n_big) + s.internal, s.count * sizeof(float));
+    }
+    if (count) *count = ctx->n_params;
+    return FDG_OK;
+}
+fdg_status fdg_params(fdg_ctx* ctx, float* host_out, size_t capacity, size_t* count) { return gather(ctx, false, host_out, capacity, count); }
+fdg_status fdg_grads(fdg_ctx* ctx, float* host_out, size_t capacity, size_t* count) { return gather(ctx, true, host_out, capacity, count); }
+
+fdg_status fdg_trace(fdg_ctx* ctx, int64_t* fwd_batch, int64_t* bwd_batch, int64_t* bwd_weight_version, int32_t K) {
+    if (!ctx || !fwd_batch || !bwd_batch || !bwd_weight_version || K != ctx->K) return FDG_ERR_INVALID_ARG;
+    CK(cudaDeviceSynchronize());
+    for (int kk = 0; kk < K; ++kk) {
+        int64_t tr[4];
+        CK(cudaMemcpy(tr, ctx->mod[kk].trace, sizeof tr, cudaMemcpyDeviceToHost));
+        fwd_batch[kk] = tr[0];
+        bwd_batch[kk] = tr[1]; bwd_weight_version[kk] = tr[2];
+    }
+    return FDG_OK;
+}
+
+fdg_status fdg_set_lr(fdg_ctx* ctx, float lr) {
+    if (!ctx || !(lr >= 0.f)) return FDG_ERR_INVALID_ARG;
+    ctx->lr = lr;
+    return FDG_OK;
+}
+
+fdg_status fdg_stats(const fdg_ctx* ctx, size_t* device_bytes, uint64_t* kernel_launches) {
+    if (!ctx) return FDG_ERR_INVALID_ARG;
+    if (device_bytes) *device_bytes = ctx->device_bytes;
+    if (kernel_launches) *kernel_launches = launches();
+    return FDG_OK;
+}
+
+fdg_status fdg_module_times(fdg_ctx* ctx, float* ms, int32_t K) {
+    if (!ctx || !ms || K != ctx->K) return FDG_ERR_INVALID_ARG;
+    if (ctx->t == 0) return fail(ctx, FDG_ERR_STATE, "no step has run yet");
+    CK(cudaDeviceSynchronize());
+    for (int kk = 0; kk < K; ++kk) CK(cudaEventElapsedTime(&ms[kk], ctx->mod[kk].ev0, ctx->mod[kk].ev1));
+    return FDG_OK;
+}
+
+}  // extern "C"

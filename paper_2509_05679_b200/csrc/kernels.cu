@@ -1,0 +1,580 @@
+// Plain-FMA (CUDA-core) kernels: every layer kind in fp32 or bf16 storage with fp32 arithmetic.
+// They are the whole fp32 path (true fp32 FMAs: TF32 would break the 1e-5 parameter tolerance)
+// and, on the bf16 path, serve the shapes the tensor-core kernels do not take (3-channel stem,
+// strided convs, 10-class head) plus all memory-bound elementwise / reduction work.
+#include "kernels.h"
+
+#include <cuda_bf16.h>
+#include <atomic>
+
+namespace fdg {
+
+static std::atomic<uint64_t> g_launches{0};
+uint64_t launches() { return g_launches.load(); }
+#define COUNT_LAUNCH() g_launches.fetch_add(1, std::memory_order_relaxed)
+
+typedef __nv_bfloat16 bf16;
+
+__device__ __forceinline__ float ld(const float* p) { return *p; }
+__device__ __forceinline__ float ld(const bf16* p) { return __bfloat162float(*p); }
+__device__ __forceinline__ void st(float* p, float v) { *p = v; }
+__device__ __forceinline__ void st(bf16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+static inline unsigned cdiv(size_t a, size_t b) { return (unsigned)((a + b - 1) / b); }
+
+// ------------------------------------------------------------------------------------------
+// Implicit GEMM  C[m][n] = sum_k A(m,k) * B(k,n)  with the operands gathered on the fly.
+//   FWD  : m = output pixel, n = c_out, k = (r,s,c_in)
+//   DGRAD: m = input pixel,  n = c_in,  k = (r,s,c_out)
+//   WGRAD: m = c_out,        n = (r,s,c_in), k = output pixel   (split over blockIdx.z)
+// 64x64 tile, 16-deep k slices, 256 threads, 4x4 outputs per thread.
+// ------------------------------------------------------------------------------------------
+enum { M_FWD = 0, M_DGRAD = 1, M_WGRAD = 2 };
+constexpr int BM = 64, BN = 64, BK = 16;
+
+template <typename T, int MODE>
+__global__ void __launch_bounds__(256) igemm_simt(const T* __restrict__ P0, const T* __restrict__ P1,
+                                                  void* __restrict__ out, const float* __restrict__ bias,
+                                                  float* __restrict__ partial, ConvGeom g, int Mg, int Ng, int Kg,
+                                                  int k_per_split, int epi) {
+    __shared__ float As[BK][BM + 4];
+    __shared__ float Bs[BK][BN + 4];
+    const int tid = threadIdx.x;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int kbeg = blockIdx.z * k_per_split;
+    const int kend = min(Kg, kbeg + k_per_split);
+
+    // which element of the A / B tile this thread fetches: one row (column) and 4 consecutive k
+    int a_row, a_kq, b_col, b_kq;
+    if (MODE == M_WGRAD) { a_row = tid & 63; a_kq = tid >> 6; b_col = tid & 63; b_kq = tid >> 6; }
+    else if (MODE == M_DGRAD) { a_row = tid >> 2; a_kq = tid & 3; b_col = tid & 63; b_kq = tid >> 6; }
+    else { a_row = tid >> 2; a_kq = tid & 3; b_col = tid >> 2; b_kq = tid & 3; }
+
+    const int HoWo = g.Ho * g.Wo, HW = g.H * g.W, RC = g.R * g.C, RCo = g.R * g.Co;
+    const int am = m0 + a_row, bn = n0 + b_col;
+    // per-thread decode of the fixed index
+    int a_n = 0, a_y = 0, a_x = 0;       // FWD: (n, oy*st-pad, ox*st-pad); DGRAD: (n, iy+pad, ix+pad)
+    if (MODE == M_FWD && am < Mg) { a_n = am / HoWo; int p = am - a_n * HoWo; int oy = p / g.Wo; a_y = oy * g.stride - g.pad; a_x = (p - oy * g.Wo) * g.stride - g.pad; }
+    if (MODE == M_DGRAD && am < Mg) { a_n = am / HW; int p = am - a_n * HW; int iy = p / g.W; a_y = iy + g.pad; a_x = (p - iy * g.W) + g.pad; }
+    int b_r = 0, b_s = 0, b_c = 0;       // WGRAD: n -> (r, s, ci)
+    if (MODE == M_WGRAD && bn < Ng) { b_r = bn / RC; int q = bn - b_r * RC; b_s = q / g.C; b_c = q - b_s * g.C; }
+
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    const int tx = tid & 15, ty = tid >> 4;
+
+    for (int k0 = kbeg; k0 < kend; k0 += BK) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            // ---- A element
+            int k = k0 + a_kq * 4 + j;
+            float v = 0.f;
+            if (am < Mg && k < kend) {
+                if (MODE == M_FWD) {
+                    int rs = k / g.C, ci = k - rs * g.C; int r = rs / g.R, s = rs - r * g.R;
+                    int iy = a_y + r, ix = a_x + s;
+                    if (iy >= 0 && iy < g.H && ix >= 0 && ix < g.W) v = ld(P0 + (((size_t)a_n * g.H + iy) * g.W + ix) * g.C + ci);
+                } else if (MODE == M_DGRAD) {
+                    int rs = k / g.Co, co = k - rs * g.Co; int r = rs / g.R, s = rs - r * g.R;
+                    int ty_ = a_y - r, tx_ = a_x - s;
+                    if (ty_ >= 0 && tx_ >= 0) {
+                        int oy = ty_ / g.stride, ox = tx_ / g.stride;
+                        if (oy * g.stride == ty_ && ox * g.stride == tx_ && oy < g.Ho && ox < g.Wo)
+                            v = ld(P0 + (((size_t)a_n * g.Ho + oy) * g.Wo + ox) * g.Co + co);
+                    }
+                } else {
+                    v = ld(P0 + (size_t)k * g.Co + am);
+                }
+            }
+            As[a_kq * 4 + j][a_row] = v;
+            // ---- B element
+            k = k0 + b_kq * 4 + j;
+            v = 0.f;
+            if (bn < Ng && k < kend) {
+                if (MODE == M_FWD) {
+                    v = ld(P1 + (size_t)bn * Kg + k);
+                } else if (MODE == M_DGRAD) {
+                    int rs = k / g.Co, co = k - rs * g.Co;
+                    v = ld(P1 + ((size_t)co * g.R * g.R + rs) * g.C + bn);
+                } else {
+                    int n = k / HoWo; int p = k - n * HoWo; int oy = p / g.Wo, ox = p - oy * g.Wo;
+                    int iy = oy * g.stride - g.pad + b_r, ix = ox * g.stride - g.pad + b_s;
+                    if (iy >= 0 && iy < g.H && ix >= 0 && ix < g.W) v = ld(P1 + (((size_t)n * g.H + iy) * g.W + ix) * g.C + b_c);
+                }
+            }
+            Bs[b_kq * 4 + j][b_col] = v;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < BK; ++kk) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) b[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    (void)RCo;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int m = m0 + ty * 4 + i;
+        if (m >= Mg) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            int n = n0 + tx * 4 + j;
+            if (n >= Ng) continue;
+            size_t o = (size_t)m * Ng + n;
+            float v = acc[i][j];
+            if (partial) { partial[(size_t)blockIdx.z * Mg * Ng + o] = v; continue; }
+            if (bias) v += bias[n];
+            if (epi & EPI_RELU) v = fmaxf(v, 0.f);
+            if (epi & EPI_OUT_F32) {
+                float* c = (float*)out;
+                c[o] = (epi & EPI_ACCUM) ? c[o] + v : v;
+            } else {
+                T* c = (T*)out;
+                if (epi & EPI_ACCUM) v += ld(c + o);
+                st(c + o, v);
+            }
+        }
+    }
+}
+
+// out[i] = sum_z partial[z][i], z ascending (fixed order => run-to-run identical results)
+__global__ void splitk_reduce(const float* __restrict__ partial, float* __restrict__ out, size_t n, int splits) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    float s = 0.f;
+    for (int z = 0; z < splits; ++z) s += partial[(size_t)z * n + i];
+    out[i] = s;
+}
+
+int wgrad_splits(const ConvGeom& g) {
+    long Kg = (long)g.N * g.Ho * g.Wo;
+    int tiles = (int)(cdiv(g.Co, BM) * cdiv((size_t)g.R * g.R * g.C, BN));
+    int want = (148 * 4 + tiles - 1) / tiles;               // about four waves of CTAs
+    int maxs = (int)((Kg + 255) / 256);                     // at least 256 contraction rows per split
+    int s = want < maxs ? want : maxs;
+    if (s < 1) s = 1;
+    if (s > 256) s = 256;
+    return s;
+}
+size_t wgrad_workspace_elems(const ConvGeom& g) {
+    int s = wgrad_splits(g);
+    return s > 1 ? (size_t)s * g.Co * g.R * g.R * g.C : 0;
+}
+
+template <typename T>
+static void conv_forward_t(const void* x, const void* w, const float* bias, void* y, const ConvGeom& g, int epi, cudaStream_t s) {
+    int Mg = g.N * g.Ho * g.Wo, Ng = g.Co, Kg = g.R * g.R * g.C;
+    dim3 grid(cdiv(Ng, BN), cdiv(Mg, BM), 1);
+    igemm_simt<T, M_FWD><<<grid, 256, 0, s>>>((const T*)x, (const T*)w, y, bias, nullptr, g, Mg, Ng, Kg, Kg, epi);
+    COUNT_LAUNCH();
+}
+void conv_forward(int dt, const void* x, const void* w, const float* bias, void* y, const ConvGeom& g, int epi, cudaStream_t s) {
+    if (dt) conv_forward_t<bf16>(x, w, bias, y, g, epi, s); else conv_forward_t<float>(x, w, bias, y, g, epi, s);
+}
+
+template <typename T>
+static void conv_dgrad_t(const void* dy, const void* w, void* dx, const ConvGeom& g, int epi, cudaStream_t s) {
+    int Mg = g.N * g.H * g.W, Ng = g.C, Kg = g.R * g.R * g.Co;
+    dim3 grid(cdiv(Ng, BN), cdiv(Mg, BM), 1);
+    igemm_simt<T, M_DGRAD><<<grid, 256, 0, s>>>((const T*)dy, (const T*)w, dx, nullptr, nullptr, g, Mg, Ng, Kg, Kg, epi);
+    COUNT_LAUNCH();
+}
+void conv_dgrad(int dt, const void* dy, const void* w, void* dx, const ConvGeom& g, int epi, cudaStream_t s) {
+    if (dt) conv_dgrad_t<bf16>(dy, w, dx, g, epi, s); else conv_dgrad_t<float>(dy, w, dx, g, epi, s);
+}
+
+template <typename T>
+static void conv_wgrad_t(const void* x, const void* dy, float* dw, float* ws, const ConvGeom& g, cudaStream_t s) {
+    int Mg = g.Co, Ng = g.R * g.R * g.C, Kg = g.N * g.Ho * g.Wo;
+    int splits = wgrad_splits(g);
+    int kps = ((Kg + splits - 1) / splits + BK - 1) / BK * BK;
+    splits = (Kg + kps - 1) / kps;
+    dim3 grid(cdiv(Ng, BN), cdiv(Mg, BM), splits);
+    if (splits == 1) {
+        igemm_simt<T, M_WGRAD><<<grid, 256, 0, s>>>((const T*)dy, (const T*)x, dw, nullptr, nullptr, g, Mg, Ng, Kg, kps, EPI_OUT_F32);
+        COUNT_LAUNCH();
+    } else {
+        igemm_simt<T, M_WGRAD><<<grid, 256, 0, s>>>((const T*)dy, (const T*)x, dw, nullptr, ws, g, Mg, Ng, Kg, kps, EPI_OUT_F32);
+        COUNT_LAUNCH();
+        size_t n = (size_t)Mg * Ng;
+        splitk_reduce<<<cdiv(n, 256), 256, 0, s>>>(ws, dw, n, splits);
+        COUNT_LAUNCH();
+    }
+}
+void conv_wgrad(int dt, const void* x, const void* dy, float* dw, float* ws, const ConvGeom& g, cudaStream_t s) {
+    if (dt) conv_wgrad_t<bf16>(x, dy, dw, ws, g, s); else conv_wgrad_t<float>(x, dy, dw, ws, g, s);
+}
+
+// ------------------------------------------------------------------------------------------
+// column sums (bias gradient): two stages, fixed order
+// ------------------------------------------------------------------------------------------
+constexpr int RED_CHUNKS = 64;
+
+template <typename T>
+__global__ void colsum_partial(const T* __restrict__ dy, float* __restrict__ part, long rows, int C) {
+    int c = blockIdx.x * 32 + threadIdx.x;
+    long per = (rows + gridDim.y - 1) / gridDim.y;
+    long r0 = (long)blockIdx.y * per, r1 = min(rows, r0 + per);
+    float s = 0.f;
+    if (c < C) for (long r = r0 + threadIdx.y; r < r1; r += blockDim.y) s += ld(dy + r * C + c);
+    __shared__ float sh[8][33];
+    sh[threadIdx.y][threadIdx.x] = s;
+    __syncthreads();
+    if (threadIdx.y == 0 && c < C) {
+        float t = 0.f;
+        for (int i = 0; i < 8; ++i) t += sh[i][threadIdx.x];
+        part[(size_t)blockIdx.y * C + c] = t;
+    }
+}
+__global__ void colsum_final(const float* __restrict__ part, float* __restrict__ out, int chunks, int C) {
+    int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    float s = 0.f;
+    for (int i = 0; i < chunks; ++i) s += part[(size_t)i * C + c];
+    out[c] = s;
+}
+void bias_grad(int dt, const void* dy, float* db, float* scratch, long rows, int C, cudaStream_t s) {
+    int chunks = (int)(rows < RED_CHUNKS ? rows : RED_CHUNKS);
+    dim3 grid(cdiv(C, 32), chunks), blk(32, 8);
+    if (dt) colsum_partial<bf16><<<grid, blk, 0, s>>>((const bf16*)dy, scratch, rows, C);
+    else colsum_partial<float><<<grid, blk, 0, s>>>((const float*)dy, scratch, rows, C);
+    COUNT_LAUNCH();
+    colsum_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, db, chunks, C);
+    COUNT_LAUNCH();
+}
+
+// ------------------------------------------------------------------------------------------
+// elementwise layers
+// ------------------------------------------------------------------------------------------
+template <typename T> __global__ void relu_fwd_k(const T* x, T* y, size_t n) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; if (i < n) st(y + i, fmaxf(ld(x + i), 0.f)); }
+template <typename T> __global__ void relu_bwd_k(const T* y, const T* dy, T* dx, size_t n, bool accum) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) { float v = ld(y + i) > 0.f ? ld(dy + i) : 0.f; if (accum) v += ld(dx + i); st(dx + i, v); } }
+template <typename T> __global__ void add_k(const T* a, const T* b, T* y, size_t n) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; if (i < n) st(y + i, ld(a + i) + ld(b + i)); }
+template <typename T> __global__ void copy_acc_k(const T* src, T* dst, size_t n, bool accum) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) { float v = ld(src + i); if (accum) v += ld(dst + i); st(dst + i, v); } }
+
+void relu_forward(int dt, const void* x, void* y, size_t n, cudaStream_t s) {
+    if (dt) relu_fwd_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)x, (bf16*)y, n);
+    else relu_fwd_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)x, (float*)y, n);
+    COUNT_LAUNCH();
+}
+void relu_backward(int dt, const void* y, const void* dy, void* dx, size_t n, bool accum, cudaStream_t s) {
+    if (dt) relu_bwd_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)y, (const bf16*)dy, (bf16*)dx, n, accum);
+    else relu_bwd_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)y, (const float*)dy, (float*)dx, n, accum);
+    COUNT_LAUNCH();
+}
+void add_forward(int dt, const void* a, const void* b, void* y, size_t n, cudaStream_t s) {
+    if (dt) add_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)a, (const bf16*)b, (bf16*)y, n);
+    else add_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)a, (const float*)b, (float*)y, n);
+    COUNT_LAUNCH();
+}
+void copy_or_accumulate(int dt, const void* src, void* dst, size_t n, bool accum, cudaStream_t s) {
+    if (dt) copy_acc_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)src, (bf16*)dst, n, accum);
+    else copy_acc_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)src, (float*)dst, n, accum);
+    COUNT_LAUNCH();
+}
+
+template <typename T>
+__global__ void maxpool_fwd_k(const T* x, T* y, int N, int H, int W, int C) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    int Ho = H / 2, Wo = W / 2;
+    size_t total = (size_t)N * Ho * Wo * C;
+    if (i >= total) return;
+    int c = i % C; size_t p = i / C; int ox = p % Wo; p /= Wo; int oy = p % Ho; int n = p / Ho;
+    const T* b = x + (((size_t)n * H + 2 * oy) * W + 2 * ox) * C + c;
+    float m = ld(b);
+    m = fmaxf(m, ld(b + C)); m = fmaxf(m, ld(b + (size_t)W * C)); m = fmaxf(m, ld(b + (size_t)W * C + C));
+    st(y + i, m);
+}
+template <typename T>
+__global__ void maxpool_bwd_k(const T* x, const T* dy, T* dx, int N, int H, int W, int C, bool accum) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    int Ho = H / 2, Wo = W / 2;
+    size_t total = (size_t)N * Ho * Wo * C;
+    if (i >= total) return;
+    int c = i % C; size_t p = i / C; int ox = p % Wo; p /= Wo; int oy = p % Ho; int n = p / Ho;
+    size_t base = (((size_t)n * H + 2 * oy) * W + 2 * ox) * C + c;
+    size_t o[4] = {base, base + (size_t)C, base + (size_t)W * C, base + (size_t)W * C + C};
+    int best = 0; float m = ld(x + o[0]);
+#pragma unroll
+    for (int j = 1; j < 4; ++j) { float v = ld(x + o[j]); if (v > m) { m = v; best = j; } }   // first maximum wins
+    float g = ld(dy + i);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { float v = (j == best) ? g : 0.f; if (accum) v += ld(dx + o[j]); st(dx + o[j], v); }
+}
+void maxpool_forward(int dt, const void* x, void* y, int N, int H, int W, int C, cudaStream_t s) {
+    size_t n = (size_t)N * (H / 2) * (W / 2) * C;
+    if (dt) maxpool_fwd_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)x, (bf16*)y, N, H, W, C);
+    else maxpool_fwd_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)x, (float*)y, N, H, W, C);
+    COUNT_LAUNCH();
+}
+void maxpool_backward(int dt, const void* x, const void* dy, void* dx, int N, int H, int W, int C, bool accum, cudaStream_t s) {
+    size_t n = (size_t)N * (H / 2) * (W / 2) * C;
+    if (dt) maxpool_bwd_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)x, (const bf16*)dy, (bf16*)dx, N, H, W, C, accum);
+    else maxpool_bwd_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)x, (const float*)dy, (float*)dx, N, H, W, C, accum);
+    COUNT_LAUNCH();
+}
+
+template <typename T>
+__global__ void gap_fwd_k(const T* x, T* y, int N, int HW, int C) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)N * C) return;
+    int c = i % C; size_t n = i / C;
+    float s = 0.f;
+    for (int p = 0; p < HW; ++p) s += ld(x + (n * HW + p) * C + c);
+    st(y + i, s / (float)HW);
+}
+template <typename T>
+__global__ void gap_bwd_k(const T* dy, T* dx, int N, int HW, int C, bool accum) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)N * HW * C) return;
+    int c = i % C; size_t n = i / ((size_t)HW * C);
+    float v = ld(dy + n * C + c) / (float)HW;
+    if (accum) v += ld(dx + i);
+    st(dx + i, v);
+}
+void gap_forward(int dt, const void* x, void* y, int N, int HW, int C, cudaStream_t s) {
+    size_t n = (size_t)N * C;
+    if (dt) gap_fwd_k<bf16><<<cdiv(n, 128), 128, 0, s>>>((const bf16*)x, (bf16*)y, N, HW, C);
+    else gap_fwd_k<float><<<cdiv(n, 128), 128, 0, s>>>((const float*)x, (float*)y, N, HW, C);
+    COUNT_LAUNCH();
+}
+void gap_backward(int dt, const void* dy, void* dx, int N, int HW, int C, bool accum, cudaStream_t s) {
+    size_t n = (size_t)N * HW * C;
+    if (dt) gap_bwd_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)dy, (bf16*)dx, N, HW, C, accum);
+    else gap_bwd_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)dy, (float*)dx, N, HW, C, accum);
+    COUNT_LAUNCH();
+}
+
+// ------------------------------------------------------------------------------------------
+// batch-norm, statistics per worker
+// ------------------------------------------------------------------------------------------
+// grid (C/32, chunks, workers), block (32, 8).  part: [chunk][worker][C][2]
+template <typename T, bool BWD>
+__global__ void bn_reduce_partial(const T* __restrict__ x, const T* __restrict__ out, const T* __restrict__ dout,
+                                  const float* __restrict__ stats, float* __restrict__ part, long rpw, int C, bool relu) {
+    int c = blockIdx.x * 32 + threadIdx.x;
+    int w = blockIdx.z, nw = gridDim.z;
+    long per = (rpw + gridDim.y - 1) / gridDim.y;
+    long r0 = (long)blockIdx.y * per, r1 = min(rpw, r0 + per);
+    float s1 = 0.f, s2 = 0.f;
+    if (c < C) {
+        float mean = 0.f, istd = 0.f;
+        if (BWD) { mean = stats[((size_t)w * C + c) * 2]; istd = stats[((size_t)w * C + c) * 2 + 1]; }
+        for (long r = r0 + threadIdx.y; r < r1; r += blockDim.y) {
+            size_t o = ((size_t)w * rpw + r) * C + c;
+            if (BWD) {
+                float dy = ld(dout + o);
+                if (relu && !(ld(out + o) > 0.f)) dy = 0.f;
+                s1 += dy; s2 += dy * (ld(x + o) - mean) * istd;
+            } else {
+                float v = ld(x + o); s1 += v; s2 += v * v;
+            }
+        }
+    }
+    __shared__ float sh1[8][33], sh2[8][33];
+    sh1[threadIdx.y][threadIdx.x] = s1; sh2[threadIdx.y][threadIdx.x] = s2;
+    __syncthreads();
+    if (threadIdx.y == 0 && c < C) {
+        float a = 0.f, b = 0.f;
+        for (int i = 0; i < 8; ++i) { a += sh1[i][threadIdx.x]; b += sh2[i][threadIdx.x]; }
+        size_t o = (((size_t)blockIdx.y * nw + w) * C + c) * 2;
+        part[o] = a; part[o + 1] = b;
+    }
+}
+// forward: stats[w][c] = (mean, invstd).  One thread per (w, c).
+__global__ void bn_stats_final(const float* __restrict__ part, float* __restrict__ stats, int chunks, int nwC, long rpw) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= nwC) return;
+    double s1 = 0.0, s2 = 0.0;
+    for (int k = 0; k < chunks; ++k) { s1 += part[((size_t)k * nwC + i) * 2]; s2 += part[((size_t)k * nwC + i) * 2 + 1]; }
+    double mean = s1 / (double)rpw, var = s2 / (double)rpw - mean * mean;
+    if (var < 0.0) var = 0.0;
+    stats[(size_t)i * 2] = (float)mean;
+    stats[(size_t)i * 2 + 1] = (float)(1.0 / sqrt(var + 1e-5));
+}
+// backward: red[w][c] = (sum dy, sum dy xhat); dgamma[c] = sum_w red[w][c].y; dbeta[c] = sum_w red[w][c].x
+__global__ void bn_bwd_final(const float* __restrict__ part, float* __restrict__ red, float* __restrict__ dgamma,
+                             float* __restrict__ dbeta, int chunks, int nw, int C) {
+    int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    float g = 0.f, b = 0.f;
+    for (int w = 0; w < nw; ++w) {
+        float s1 = 0.f, s2 = 0.f;
+        for (int k = 0; k < chunks; ++k) { size_t o = (((size_t)k * nw + w) * C + c) * 2; s1 += part[o]; s2 += part[o + 1]; }
+        red[((size_t)w * C + c) * 2] = s1; red[((size_t)w * C + c) * 2 + 1] = s2;
+        b += s1; g += s2;
+    }
+    dgamma[c] = g; dbeta[c] = b;
+}
+template <typename T>
+__global__ void bn_apply_k(const T* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+                           const T* __restrict__ res, T* __restrict__ y, const float* __restrict__ stats,
+                           long rpw, int C, size_t total, bool relu) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    int c = i % C; size_t row = i / C; int w = (int)(row / rpw);
+    float mean = stats[((size_t)w * C + c) * 2], istd = stats[((size_t)w * C + c) * 2 + 1];
+    float v = gamma[c] * (ld(x + i) - mean) * istd + beta[c];
+    if (res) v += ld(res + i);
+    if (relu) v = fmaxf(v, 0.f);
+    st(y + i, v);
+}
+template <typename T>
+__global__ void bn_bwd_apply_k(const T* __restrict__ x, const T* __restrict__ out, const T* __restrict__ dout,
+                               const float* __restrict__ gamma, const float* __restrict__ stats, const float* __restrict__ red,
+                               T* __restrict__ dx, bool accum_dx, T* __restrict__ dres, bool accum_dres,
+                               long rpw, int C, size_t total, bool relu) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    int c = i % C; size_t row = i / C; int w = (int)(row / rpw);
+    size_t so = ((size_t)w * C + c) * 2;
+    float mean = stats[so], istd = stats[so + 1];
+    float dy = ld(dout + i);
+    if (relu && !(ld(out + i) > 0.f)) dy = 0.f;
+    float xh = (ld(x + i) - mean) * istd;
+    float inv_n = 1.f / (float)rpw;
+    float v = gamma[c] * istd * (dy - red[so] * inv_n - xh * red[so + 1] * inv_n);
+    if (accum_dx) v += ld(dx + i);
+    st(dx + i, v);
+    if (dres) { float r = dy; if (accum_dres) r += ld(dres + i); st(dres + i, r); }
+}
+
+void bn_forward(int dt, const void* x, const float* gamma, const float* beta, const void* res, void* y, float* stats,
+                float* scratch, int nw, long rpw, int C, bool relu, cudaStream_t s) {
+    int chunks = (int)(rpw < RED_CHUNKS ? rpw : RED_CHUNKS);
+    dim3 grid(cdiv(C, 32), chunks, nw), blk(32, 8);
+    if (dt) bn_reduce_partial<bf16, false><<<grid, blk, 0, s>>>((const bf16*)x, nullptr, nullptr, nullptr, scratch, rpw, C, false);
+    else bn_reduce_partial<float, false><<<grid, blk, 0, s>>>((const float*)x, nullptr, nullptr, nullptr, scratch, rpw, C, false);
+    COUNT_LAUNCH();
+    bn_stats_final<<<cdiv((size_t)nw * C, 128), 128, 0, s>>>(scratch, stats, chunks, nw * C, rpw);
+    COUNT_LAUNCH();
+    size_t total = (size_t)nw * rpw * C;
+    if (dt) bn_apply_k<bf16><<<cdiv(total, 256), 256, 0, s>>>((const bf16*)x, gamma, beta, (const bf16*)res, (bf16*)y, stats, rpw, C, total, relu);
+    else bn_apply_k<float><<<cdiv(total, 256), 256, 0, s>>>((const float*)x, gamma, beta, (const float*)res, (float*)y, stats, rpw, C, total, relu);
+    COUNT_LAUNCH();
+}
+
+void bn_backward(int dt, const void* x, const void* out, const void* dout, const float* gamma, const float* stats,
+                 void* dx, bool accum_dx, void* dres, bool accum_dres, float* dgamma, float* dbeta, float* red,
+                 float* scratch, int nw, long rpw, int C, bool relu, cudaStream_t s) {
+    int chunks = (int)(rpw < RED_CHUNKS ? rpw : RED_CHUNKS);
+    dim3 grid(cdiv(C, 32), chunks, nw), blk(32, 8);
+    if (dt) bn_reduce_partial<bf16, true><<<grid, blk, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, stats, scratch, rpw, C, relu);
+    else bn_reduce_partial<float, true><<<grid, blk, 0, s>>>((const float*)x, (const float*)out, (const float*)dout, stats, scratch, rpw, C, relu);
+    COUNT_LAUNCH();
+    bn_bwd_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C);
+    COUNT_LAUNCH();
+    size_t total = (size_t)nw * rpw * C;
+    if (dt) bn_bwd_apply_k<bf16><<<cdiv(total, 256), 256, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, gamma, stats, red,
+                                                                  (bf16*)dx, accum_dx, (bf16*)dres, accum_dres, rpw, C, total, relu);
+    else bn_bwd_apply_k<float><<<cdiv(total, 256), 256, 0, s>>>((const float*)x, (const float*)out, (const float*)dout, gamma, stats, red,
+                                                                (float*)dx, accum_dx, (float*)dres, accum_dres, rpw, C, total, relu);
+    COUNT_LAUNCH();
+}
+
+// ------------------------------------------------------------------------------------------
+// softmax cross-entropy: one block; thread i handles rows i, i+256, ...; fixed-order tree sum
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void softmax_ce_k(const float* __restrict__ z, const int32_t* __restrict__ labels, T* __restrict__ dz,
+                             float* __restrict__ loss_out, int M, int C) {
+    __shared__ float sh[256];
+    float local = 0.f;
+    float inv_m = 1.f / (float)M;
+    for (int r = threadIdx.x; r < M; r += blockDim.x) {
+        const float* zr = z + (size_t)r * C;
+        float m = zr[0];
+        for (int c = 1; c < C; ++c) m = fmaxf(m, zr[c]);
+        float se = 0.f;
+        for (int c = 0; c < C; ++c) se += expf(zr[c] - m);
+        float lse = m + logf(se);
+        int y = labels[r];
+        local += lse - zr[y];
+        for (int c = 0; c < C; ++c) st(dz + (size_t)r * C + c, (expf(zr[c] - lse) - (c == y ? 1.f : 0.f)) * inv_m);
+    }
+    sh[threadIdx.x] = local;
+    __syncthreads();
+    for (int s = 128; s > 0; s >>= 1) { if ((int)threadIdx.x < s) sh[threadIdx.x] += sh[threadIdx.x + s]; __syncthreads(); }
+    if (threadIdx.x == 0) *loss_out = sh[0] * inv_m;
+}
+void softmax_ce(int dt, const float* logits, const int32_t* labels, void* dlogits, float* loss_out, int M, int classes, cudaStream_t s) {
+    if (dt) softmax_ce_k<bf16><<<1, 256, 0, s>>>(logits, labels, (bf16*)dlogits, loss_out, M, classes);
+    else softmax_ce_k<float><<<1, 256, 0, s>>>(logits, labels, (float*)dlogits, loss_out, M, classes);
+    COUNT_LAUNCH();
+}
+
+// ------------------------------------------------------------------------------------------
+// SGD update fused with the emission of the next weight version (Eq. dl_update with P = 11^T/N)
+// 128-bit loads and stores; grid sized to a multiple of the SM count by the grid-stride loop.
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void sgd_k(float4* __restrict__ master, const float4* __restrict__ grad, T* __restrict__ copy, size_t n4, float lr) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        float4 w = master[i];
+        if (grad) {
+            float4 g = grad[i];
+            w.x = fmaf(-lr, g.x, w.x); w.y = fmaf(-lr, g.y, w.y); w.z = fmaf(-lr, g.z, w.z); w.w = fmaf(-lr, g.w, w.w);
+            master[i] = w;
+        }
+        if (sizeof(T) == 4) {
+            ((float4*)copy)[i] = w;
+        } else {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
+            uint2 pk; pk.x = *(unsigned*)&lo; pk.y = *(unsigned*)&hi;
+            ((uint2*)copy)[i] = pk;
+        }
+    }
+}
+void sgd_update(int dt, float* master, const float* grad, void* copy_next, size_t n, float lr, cudaStream_t s) {
+    size_t n4 = n / 4;
+    if (n4 == 0) return;
+    unsigned blocks = cdiv(n4, 256);
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (dt) sgd_k<bf16><<<blocks, 256, 0, s>>>((float4*)master, (const float4*)grad, (bf16*)copy_next, n4, lr);
+    else sgd_k<float><<<blocks, 256, 0, s>>>((float4*)master, (const float4*)grad, (float*)copy_next, n4, lr);
+    COUNT_LAUNCH();
+}
+
+// ------------------------------------------------------------------------------------------
+// schedule tags
+// ------------------------------------------------------------------------------------------
+__global__ void tags_k(TagOps o) {
+    if (threadIdx.x != 0) return;
+    // tags of what this step produces first: the last module reads the stash slot it fills itself
+    if (o.wr_in) { o.wr_in[0] = o.version_now; o.wr_in[1] = -1; }      // module 1: the batch sampled now
+    if (o.wr_out) { o.wr_out[0] = o.fwd_batch; o.wr_out[1] = -1; }
+    if (o.wr_stash) { o.wr_stash[0] = o.fwd_batch; o.wr_stash[1] = o.version_now; }
+    if (o.wr_grad) { o.wr_grad[0] = o.bwd_batch; o.wr_grad[1] = -1; }
+    if (o.wr_wnext) { o.wr_wnext[0] = -1; o.wr_wnext[1] = o.version_now + 1; }
+    int64_t fb = o.rd_act ? o.rd_act[0] : -1;
+    int64_t bb = -1, bv = -1;
+    if (o.rd_stash) {
+        bb = o.rd_stash[0];
+        if (o.rd_grad && o.rd_grad[0] != bb) bb = -2;
+        bv = o.rd_wbwd ? o.rd_wbwd[1] : -1;
+        if (o.rd_stash[1] != bv) bv = -2;                 // the stash records the version the forward used
+    }
+    o.trace[0] = fb; o.trace[1] = bb; o.trace[2] = bv; o.trace[3] = o.rd_wfwd ? o.rd_wfwd[1] : -1;
+}
+void tags_step(const TagOps& ops, cudaStream_t s) { tags_k<<<1, 32, 0, s>>>(ops); COUNT_LAUNCH(); }
+
+__global__ void fill_k(float* p, float v, size_t n) { size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; if (i < n) p[i] = v; }
+void fill_f32(float* p, float v, size_t n, cudaStream_t s) { if (!n) return; fill_k<<<cdiv(n, 256), 256, 0, s>>>(p, v, n); COUNT_LAUNCH(); }
+
+}  // namespace fdg

@@ -1,0 +1,74 @@
+// Internal launch interface between the step executor (fdg_api.cu) and the kernels.
+// All pointers are device pointers; `dt` is 0 for fp32 storage, 1 for bf16 storage.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace fdg {
+
+struct ConvGeom {            // x: [N,H,W,C]  ->  y: [N,Ho,Wo,Co], R x R window
+    int N, H, W, C, Ho, Wo, Co, R, stride, pad;
+};
+
+enum { EPI_RELU = 1, EPI_ACCUM = 2, EPI_OUT_F32 = 4 };
+
+// Number of k-splits the weight-gradient kernel will use for this geometry (>= 1) and the
+// fp32 workspace elements it needs (splits * Co * R*R*C when splits > 1, else 0).
+int    wgrad_splits(const ConvGeom& g);
+size_t wgrad_workspace_elems(const ConvGeom& g);
+
+// y = conv(x, W) (+ bias) (relu)            (Eq. forward_step for linear / conv layers)
+void conv_forward(int dt, const void* x, const void* w, const float* bias, void* y, const ConvGeom& g,
+                  int epi, cudaStream_t st);
+// dx (+)= conv_transpose(dy, W)             (Eq. backward_step, gradient w.r.t. the layer input)
+void conv_dgrad(int dt, const void* dy, const void* w, void* dx, const ConvGeom& g, int epi, cudaStream_t st);
+// dW = sum over all N*Ho*Wo rows of dy^T (x) patches(x), fp32 out; the reduction runs over the
+// worker x batch axis, which is the worker average of Eq. dl_update (b) for P = 11^T/N.
+void conv_wgrad(int dt, const void* x, const void* dy, float* dw, float* workspace, const ConvGeom& g, cudaStream_t st);
+// db[c] = sum over rows of dy[row][c]; scratch: fp32 [64 * C]
+void bias_grad(int dt, const void* dy, float* db, float* scratch, long rows, int C, cudaStream_t st);
+
+void relu_forward(int dt, const void* x, void* y, size_t n, cudaStream_t st);
+// dx (+)= dy * (y > 0)
+void relu_backward(int dt, const void* y, const void* dy, void* dx, size_t n, bool accum, cudaStream_t st);
+// y = a + b ; backward is two copies / accumulations
+void add_forward(int dt, const void* a, const void* b, void* y, size_t n, cudaStream_t st);
+void copy_or_accumulate(int dt, const void* src, void* dst, size_t n, bool accum, cudaStream_t st);
+void maxpool_forward(int dt, const void* x, void* y, int N, int H, int W, int C, cudaStream_t st);
+void maxpool_backward(int dt, const void* x, const void* dy, void* dx, int N, int H, int W, int C, bool accum, cudaStream_t st);
+void gap_forward(int dt, const void* x, void* y, int N, int HW, int C, cudaStream_t st);
+void gap_backward(int dt, const void* dy, void* dx, int N, int HW, int C, bool accum, cudaStream_t st);
+
+// Batch-norm with per-worker statistics.  x: [n_workers * rows_per_worker, C].
+// stats: fp32 [n_workers][C][2] = (mean, invstd).  scratch: fp32 [64 * n_workers * C * 2].
+void bn_forward(int dt, const void* x, const float* gamma, const float* beta, const void* residual_or_null,
+                void* y, float* stats, float* scratch, int n_workers, long rows_per_worker, int C, bool relu,
+                cudaStream_t st);
+// dy_eff = dout * (out > 0 if relu).  dx (+)= BN backward of dy_eff; dres (+)= dy_eff;
+// dgamma, dbeta (fp32) = sums over all workers.  red: fp32 [n_workers][C][2] scratch for (sum dy, sum dy xhat).
+void bn_backward(int dt, const void* x, const void* out, const void* dout, const float* gamma, const float* stats,
+                 void* dx, bool accum_dx, void* dres_or_null, bool accum_dres, float* dgamma, float* dbeta,
+                 float* red, float* scratch, int n_workers, long rows_per_worker, int C, bool relu, cudaStream_t st);
+
+// Softmax cross-entropy over fp32 logits [M, classes]: dlogits (storage dtype) = (softmax - onehot) / M,
+// *loss_out = mean loss.  Deterministic single-block reduction.
+void softmax_ce(int dt, const float* logits, const int32_t* labels, void* dlogits, float* loss_out, int M, int classes,
+                cudaStream_t st);
+
+// master -= lr * grad (skipped when grad == nullptr: w(t+1) = w(t)); copy_next = storage-dtype copy of
+// the new master (the next weight version).  n must be a multiple of 4; pointers 16-byte aligned.
+void sgd_update(int dt, float* master, const float* grad, void* copy_next, size_t n, float lr, cudaStream_t st);
+
+// Schedule tags (see fdg_trace).  tags are int64 pairs {batch id, weight version}.
+struct TagOps {
+    const int64_t* rd_act;  const int64_t* rd_stash; const int64_t* rd_grad; const int64_t* rd_wbwd; const int64_t* rd_wfwd;
+    int64_t* wr_in; int64_t* wr_out; int64_t* wr_stash; int64_t* wr_grad; int64_t* wr_wnext;
+    int64_t fwd_batch, bwd_batch, version_now;   // what this step produces (-1: nothing)
+    int64_t* trace;                              // [4]: fwd batch, bwd batch, bwd weight version, fwd weight version
+};
+void tags_step(const TagOps& ops, cudaStream_t st);
+
+void fill_f32(float* p, float v, size_t n, cudaStream_t st);
+uint64_t launches();     // kernels launched so far through this interface
+
+}  // namespace fdg

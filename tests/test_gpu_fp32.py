@@ -1,0 +1,97 @@
+"""fp32 path of the library against the oracle: bit-exact schedule, parameters within max
+relative error 1e-5 after every step (per tensor, |a-b| / max(|b|, 1e-3 rms(b)))."""
+import numpy as np
+import pytest
+
+from paper_2509_05679_b200 import synth as sy
+from harness import run_parity, make_ctx
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+def as_fp32(net):
+    net.dtype = "fp32"
+    return net
+
+
+def test_config1_mlp_20_iterations(orc):
+    net = sy.config(0)
+    rec = run_parity(orc, net, net.steps, param_tol=TOL, loss_tol=1e-5, perturb=False)
+    assert len(rec) == 20 and not np.isnan(rec[-1]["loss_g"])
+
+
+def test_mlp_four_modules_ragged_sizes(orc):
+    net = sy.Net("mlp-k4", sy.mlp_layers([70, 33, 65, 17, 5]), [2, 4, 6], 1, 1, 70, 5, 3, 7, 0.05, "fp32")
+    run_parity(orc, net, 4 * net.K + 2, param_tol=TOL, loss_tol=1e-5)
+
+
+def test_vgg_shaped_four_modules(orc):
+    layers, starts = sy.vgg_layers(widths=(6, 10, 12, 20), in_c=3, classes=10)
+    net = sy.Net("vgg-small", layers, starts[1:], 16, 16, 3, 10, 2, 3, 0.05, "fp32")
+    run_parity(orc, net, 4 * net.K, param_tol=TOL, loss_tol=1e-5)
+
+
+def test_resnet_shaped_four_modules_per_worker_batchnorm(orc):
+    net = as_fp32(sy.config(3, n_workers=2, batch=3, width_div=8))
+    rec = run_parity(orc, net, 4 * net.K, param_tol=TOL, loss_tol=1e-5, grad_tol=1e-4)
+    assert rec[-1]["grad_err"] > 0
+
+
+def test_resnet_shaped_eight_modules_max_delay(orc):
+    net = as_fp32(sy.config(4, n_workers=2, batch=2, width_div=16))
+    run_parity(orc, net, 2 * net.K + 3, param_tol=TOL, loss_tol=1e-5)
+
+
+def test_single_module_single_worker_is_plain_sgd(orc):
+    net = as_fp32(sy.config(3, n_workers=1, batch=4, width_div=8, K=1))
+    run_parity(orc, net, 3, param_tol=TOL, loss_tol=1e-5)
+
+
+def test_serial_and_concurrent_modes_are_bit_identical():
+    import torch
+    from paper_2509_05679_b200 import binding
+    net = as_fp32(sy.config(3, n_workers=2, batch=4, width_div=8))
+    p0 = sy.perturb_params(sy.init_params(net.layers, 0), net.layers, 7, 0.1)
+    outs = []
+    for serial in (False, True):
+        ctx = make_ctx(net, p0, serial=serial)
+        for t in range(3 * net.K):
+            ctx.step(binding.to_device("fp32", sy.batch_inputs(net, t)), torch.from_numpy(sy.batch_labels(net, t)).cuda())
+        outs.append(ctx.params())
+        ctx.close()
+    assert np.array_equal(outs[0], outs[1])
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    import torch
+    from paper_2509_05679_b200 import binding
+    net = sy.config(0)
+    p0 = sy.init_params(net.layers, 0)
+    a, b = make_ctx(net, p0), make_ctx(net, p0)
+    for t in range(5):
+        x, y = sy.batch_inputs(net, t), sy.batch_labels(net, t)
+        la = a.step(binding.to_device("fp32", x), torch.from_numpy(y).cuda(), want_loss=True)
+        lb = b.step_host(x, y, want_loss=True)
+        assert la == lb or (np.isnan(la) and np.isnan(lb))
+    assert np.array_equal(a.params(), b.params())
+    a.close(); b.close()
+
+
+def test_error_paths_do_not_touch_the_gpu_state():
+    from paper_2509_05679_b200 import binding
+    layers, bs = sy.resnet_layers(widths=(8, 16), blocks=1, in_c=3, classes=10)
+    with pytest.raises(binding.FdgError) as e:
+        binding.Context(layers, [bs[0] + 2], 1, 2, 0.1, dtype="fp32", in_shape=(8, 8, 3))      # cuts a residual block
+    assert e.value.status == 2
+    with pytest.raises(binding.FdgError) as e:
+        binding.Context(layers, [5, 5], 1, 2, 0.1, dtype="fp32", in_shape=(8, 8, 3))           # not increasing
+    assert e.value.status == 2
+    with pytest.raises(binding.FdgError) as e:
+        binding.Context(sy.mlp_layers([8, 4, 3]), [], 1, 2, 0.1, dtype="fp32", in_shape=(1, 1, 9), num_classes=3)
+    assert e.value.status == 3
+    ctx = binding.Context(sy.mlp_layers([8, 4, 3]), [], 1, 2, 0.1, dtype="fp32", in_shape=(1, 1, 8), num_classes=3)
+    with pytest.raises(binding.FdgError) as e:
+        ctx.step(1, 1)                                                                          # no parameters yet
+    assert e.value.status == 8
+    ctx.close()
