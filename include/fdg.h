@@ -116,8 +116,11 @@ FDG_API fdg_status fdg_set_params(fdg_ctx* ctx, const float* host_params, size_t
 
 /* One iteration t of Algorithm 1 for all modules and workers (steps listed at the top).
  *   dev_inputs : device, [M, in_h, in_w, in_c] in the context's dtype (fp32 or bf16), the
- *                batch sampled at iteration t; must be complete before the call (the library
- *                copies it into its own FIFO on module 1's stream and does not keep the pointer).
+ *                batch sampled at iteration t.  Its contents must be complete before the call
+ *                (the library's streams do not synchronise with the caller's), and the buffer
+ *                must stay valid and unchanged until the library has copied it into its own FIFO:
+ *                that copy is enqueued on module 1's stream; fdg_wait_ingest() blocks until it
+ *                is done.  The library does not keep the pointer.
  *   dev_labels : device, int32 [M].
  *   host_loss_or_null : if non-NULL the call waits for the last module and stores the mean
  *                loss of the batch it processed in this iteration (tau = t-K+1; NaN while
@@ -129,6 +132,10 @@ FDG_API fdg_status fdg_step(fdg_ctx* ctx, const void* dev_inputs, const int32_t*
  * host-to-device copies go straight into the FIFO slot, ordered on module 1's stream. */
 FDG_API fdg_status fdg_step_host(fdg_ctx* ctx, const void* host_inputs, const int32_t* host_labels,
                          float* host_loss_or_null);
+
+/* Block the host until the input/label copies of the most recent step have executed; after
+ * that the caller may overwrite or free the buffers it passed to that step. */
+FDG_API fdg_status fdg_wait_ingest(fdg_ctx* ctx);
 
 /* Wait for all modules, then copy the fp32 master weights w(t) (t = number of steps done) to a
  * host array in canonical order.  count receives the number of floats written. */

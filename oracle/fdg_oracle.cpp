@@ -49,6 +49,10 @@ struct Layer { int32_t kind, c_in, c_out, stride, flags; };
 constexpr double BN_EPS = 1e-5;
 
 int g_threads = 0;   // 0 = hardware_concurrency
+// Smallest distance of any value from a kink seen since the last reset: |x| at a ReLU, the gap
+// between the two largest values of a max-pool window.  Tests use it to tell whether a lower
+// precision could legitimately take the other branch somewhere.
+double g_kink_margin = 1e300;
 
 int num_threads() {
     int n = g_threads > 0 ? g_threads : (int)std::thread::hardware_concurrency();
@@ -161,7 +165,11 @@ void conv_bwd(const Tensor& x, const Tensor& gy, const double* W, int R, int st,
 // A linear layer is a 1x1 convolution over the flattened sample.
 Tensor flatten(const Tensor& x) { Tensor y = x; y.c = (int)x.per_sample(); y.h = y.w = 1; return y; }
 
-Tensor relu_fwd(const Tensor& x) { Tensor y = x; for (auto& e : y.v) e = e > 0.0 ? e : 0.0; return y; }
+Tensor relu_fwd(const Tensor& x) {
+    Tensor y = x;
+    for (auto& e : y.v) { g_kink_margin = std::min(g_kink_margin, std::fabs(e)); e = e > 0.0 ? e : 0.0; }
+    return y;
+}
 Tensor relu_bwd(const Tensor& x, const Tensor& gy) {
     Tensor g = gy; for (size_t i = 0; i < g.v.size(); ++i) if (!(x.v[i] > 0.0)) g.v[i] = 0.0; return g;
 }
@@ -170,8 +178,10 @@ Tensor maxpool_fwd(const Tensor& x) {
     Tensor y(x.n, x.h / 2, x.w / 2, x.c);
     for (int i = 0; i < x.n; ++i) for (int oy = 0; oy < y.h; ++oy) for (int ox = 0; ox < y.w; ++ox)
         for (int c = 0; c < x.c; ++c) {
-            double m = x.at(i, 2 * oy, 2 * ox)[c];
-            for (int r = 0; r < 2; ++r) for (int s = 0; s < 2; ++s) m = std::max(m, x.at(i, 2 * oy + r, 2 * ox + s)[c]);
+            double v[4] = {x.at(i, 2 * oy, 2 * ox)[c], x.at(i, 2 * oy, 2 * ox + 1)[c], x.at(i, 2 * oy + 1, 2 * ox)[c], x.at(i, 2 * oy + 1, 2 * ox + 1)[c]};
+            double m = std::max(std::max(v[0], v[1]), std::max(v[2], v[3]));
+            std::sort(v, v + 4);
+            g_kink_margin = std::min(g_kink_margin, v[3] - v[2]);
             y.at(i, oy, ox)[c] = m;
         }
     return y;
@@ -406,6 +416,7 @@ void* orc_create(const int32_t* layers, int n_layers, const int32_t* splits, int
 }
 void orc_destroy(void* h) { delete (Oracle*)h; }
 void orc_set_threads(int n) { g_threads = n; }
+double orc_kink_margin(int reset) { double m = g_kink_margin; if (reset) g_kink_margin = 1e300; return m; }
 int orc_threads() { return num_threads(); }
 size_t orc_param_count(void* h) { return ((Oracle*)h)->poff.back(); }
 void orc_set_flag_use_current_weights(void* h, int on) { ((Oracle*)h)->use_current_weights = on != 0; }

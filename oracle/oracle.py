@@ -35,6 +35,8 @@ def lib():
         L.orc_destroy.argtypes = [C.c_void_p]
         L.orc_set_threads.argtypes = [C.c_int]
         L.orc_threads.restype = C.c_int
+        L.orc_kink_margin.restype = C.c_double
+        L.orc_kink_margin.argtypes = [C.c_int]
         L.orc_param_count.restype = C.c_size_t
         L.orc_param_count.argtypes = [C.c_void_p]
         L.orc_set_flag_use_current_weights.argtypes = [C.c_void_p, C.c_int]
@@ -70,6 +72,11 @@ def threads() -> int:
     return int(lib().orc_threads())
 
 
+def kink_margin(reset: bool = True) -> float:
+    """Smallest |x| at a ReLU / top-2 gap in a max-pool window since the last reset."""
+    return float(lib().orc_kink_margin(int(reset)))
+
+
 def set_threads(n: int) -> None:
     lib().orc_set_threads(int(n))
 
@@ -98,7 +105,7 @@ class Oracle:
         self.n_params = int(lib().orc_param_count(self.h))
 
     def __del__(self):
-        if getattr(self, "h", None):
+        if getattr(self, "h", None) and lib is not None:
             lib().orc_destroy(self.h)
             self.h = None
 

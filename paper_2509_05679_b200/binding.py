@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libfdg.so")
 STATUS = {0: "FDG_OK", 1: "FDG_ERR_INVALID_ARG", 2: "FDG_ERR_BAD_SPLIT", 3: "FDG_ERR_UNSUPPORTED",
           4: "FDG_ERR_ARCH", 5: "FDG_ERR_OOM", 6: "FDG_ERR_CUDA", 7: "FDG_ERR_TIMEOUT", 8: "FDG_ERR_STATE"}
 
-EXPORTS = ["fdg_create", "fdg_param_count", "fdg_set_params", "fdg_step", "fdg_step_host", "fdg_params",
+EXPORTS = ["fdg_create", "fdg_param_count", "fdg_set_params", "fdg_step", "fdg_step_host", "fdg_wait_ingest", "fdg_params",
            "fdg_grads", "fdg_trace", "fdg_set_lr", "fdg_stats", "fdg_module_times", "fdg_last_error", "fdg_destroy"]
 
 
@@ -75,6 +75,8 @@ def lib():
         L.fdg_trace.argtypes = [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.c_int32]
         L.fdg_set_lr.restype = C.c_int
         L.fdg_set_lr.argtypes = [vp, C.c_float]
+        L.fdg_wait_ingest.restype = C.c_int
+        L.fdg_wait_ingest.argtypes = [vp]
         L.fdg_stats.restype = C.c_int
         L.fdg_stats.argtypes = [vp, C.POINTER(C.c_size_t), C.POINTER(C.c_uint64)]
         L.fdg_module_times.restype = C.c_int
@@ -180,6 +182,9 @@ class Context:
         self._ck(lib().fdg_step_host(self.h, _ptr(host_inputs), _ptr(host_labels), C.byref(loss) if want_loss else None))
         return loss.value if want_loss else None
 
+    def wait_ingest(self):
+        self._ck(lib().fdg_wait_ingest(self.h))
+
     def _vec(self, fn) -> np.ndarray:
         out = np.empty(self.n_params, dtype=np.float32)
         n = C.c_size_t()
@@ -216,4 +221,6 @@ def to_device(net_dtype: str, x: np.ndarray):
     """Copy a host fp32 batch to the device in the context's storage dtype (plumbing for callers)."""
     import torch
     t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).cuda()
-    return t.to(torch.bfloat16).contiguous() if net_dtype == "bf16" else t
+    t = t.to(torch.bfloat16).contiguous() if net_dtype == "bf16" else t
+    torch.cuda.current_stream().synchronize()      # the library's streams do not wait for torch's
+    return t

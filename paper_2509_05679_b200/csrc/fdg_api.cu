@@ -96,6 +96,7 @@ struct fdg_ctx {
     char* dlogits;
     float* loss_ring;
     int64_t* tags;
+    cudaEvent_t ingested;
     std::string err;
 };
 
@@ -402,6 +403,7 @@ fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, boo
         CK(cudaMemcpyAsync(m0.in_ring + (size_t)(t % m0.in_depth) * m0.in_slot_bytes, inputs,
                            (size_t)ctx->M * m0.in_elems * ctx->esz, kind, m0.stream));
         CK(cudaMemcpyAsync(ctx->labels + (size_t)(t % ctx->label_depth) * ctx->M, labels, (size_t)ctx->M * sizeof(int32_t), kind, m0.stream));
+        CK(cudaEventRecord(ctx->ingested, m0.stream));
     }
     // 3. every module: forward on tau_f, backward on tau_b, update
     for (int kk = 0; kk < K; ++kk) {
@@ -470,6 +472,7 @@ void fdg_destroy(fdg_ctx* ctx) {
         if (m.ev0) cudaEventDestroy(m.ev0);
         if (m.ev1) cudaEventDestroy(m.ev1);
     }
+    if (ctx->ingested) cudaEventDestroy(ctx->ingested);
     for (cudaStream_t s : ctx->owned) cudaStreamDestroy(s);
     for (void* p : ctx->blocks) ctx->alloc.free(p, ctx->alloc.user);
     delete ctx;
@@ -503,6 +506,7 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
     ctx->alloc = alloc ? *alloc : fdg_allocator{default_alloc, default_free, nullptr};
     ctx->own_streams = opt->streams == nullptr;
     ctx->device_bytes = 0;
+    ctx->ingested = nullptr;
     ctx->mod.resize(K);
     auto bail = [&](fdg_status s, const std::string& msg) { g_create_error = msg; fdg_destroy(ctx); return s; };
 
@@ -577,7 +581,14 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
         if (e == cudaSuccess) e = cudaMemset(m.master, 0, (m.n_big + m.n_small) * sizeof(float));
         if (e != cudaSuccess) return bail(FDG_ERR_CUDA, cudaGetErrorString(e));
     }
+    if (cudaEventCreateWithFlags(&ctx->ingested, cudaEventDisableTiming) != cudaSuccess) return bail(FDG_ERR_CUDA, "cudaEventCreate failed");
     *out = ctx;
+    return FDG_OK;
+}
+
+fdg_status fdg_wait_ingest(fdg_ctx* ctx) {
+    if (!ctx) return FDG_ERR_INVALID_ARG;
+    if (ctx->t > 0) CK(cudaEventSynchronize(ctx->ingested));
     return FDG_OK;
 }
 

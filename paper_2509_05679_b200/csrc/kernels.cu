@@ -59,11 +59,13 @@ __global__ void __launch_bounds__(256) igemm_simt(const T* __restrict__ P0, cons
     int b_r = 0, b_s = 0, b_c = 0;       // WGRAD: n -> (r, s, ci)
     if (MODE == M_WGRAD && bn < Ng) { b_r = bn / RC; int q = bn - b_r * RC; b_s = q / g.C; b_c = q - b_s * g.C; }
 
-    float acc[4][4];
+    // acc + comp: compensated (Kahan) running sum of the per-slice partial sums, so that the rounding
+    // error of a long contraction (3072 terms in the first MLP layer) stays at a few ulps
+    float acc[4][4], comp[4][4];
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+        for (int j = 0; j < 4; ++j) { acc[i][j] = 0.f; comp[i][j] = 0.f; }
     const int tx = tid & 15, ty = tid >> 4;
 
     for (int k0 = kbeg; k0 < kend; k0 += BK) {
@@ -108,6 +110,11 @@ __global__ void __launch_bounds__(256) igemm_simt(const T* __restrict__ P0, cons
             Bs[b_kq * 4 + j][b_col] = v;
         }
         __syncthreads();
+        float part[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) part[i][j] = 0.f;
 #pragma unroll
         for (int kk = 0; kk < BK; ++kk) {
             float a[4], b[4];
@@ -118,8 +125,17 @@ __global__ void __launch_bounds__(256) igemm_simt(const T* __restrict__ P0, cons
 #pragma unroll
             for (int i = 0; i < 4; ++i)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+                for (int j = 0; j < 4; ++j) part[i][j] = fmaf(a[i], b[j], part[i][j]);
         }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float y = part[i][j] - comp[i][j];
+                float t = acc[i][j] + y;
+                comp[i][j] = (t - acc[i][j]) - y;
+                acc[i][j] = t;
+            }
         __syncthreads();
     }
     (void)RCo;
@@ -561,7 +577,6 @@ __global__ void tags_k(TagOps o) {
     if (o.wr_out) { o.wr_out[0] = o.fwd_batch; o.wr_out[1] = -1; }
     if (o.wr_stash) { o.wr_stash[0] = o.fwd_batch; o.wr_stash[1] = o.version_now; }
     if (o.wr_grad) { o.wr_grad[0] = o.bwd_batch; o.wr_grad[1] = -1; }
-    if (o.wr_wnext) { o.wr_wnext[0] = -1; o.wr_wnext[1] = o.version_now + 1; }
     int64_t fb = o.rd_act ? o.rd_act[0] : -1;
     int64_t bb = -1, bv = -1;
     if (o.rd_stash) {
@@ -571,6 +586,8 @@ __global__ void tags_k(TagOps o) {
         if (o.rd_stash[1] != bv) bv = -2;                 // the stash records the version the forward used
     }
     o.trace[0] = fb; o.trace[1] = bb; o.trace[2] = bv; o.trace[3] = o.rd_wfwd ? o.rd_wfwd[1] : -1;
+    // the next weight version replaces a slot only at the end of the step, after the reads above
+    if (o.wr_wnext) { o.wr_wnext[0] = -1; o.wr_wnext[1] = o.version_now + 1; }
 }
 void tags_step(const TagOps& ops, cudaStream_t s) { tags_k<<<1, 32, 0, s>>>(ops); COUNT_LAUNCH(); }
 

@@ -126,16 +126,16 @@ def perturb_params(params: np.ndarray, layers: Sequence[Layer], seed: int, scale
     return p
 
 
-def batch_inputs(net: Net, t: int) -> np.ndarray:
+def batch_inputs(net: Net, t: int, stream: int = 0) -> np.ndarray:
     """Inputs of iteration t: [M, in_h, in_w, in_c] i.i.d. N(0,1), fp32 (bf16-representable
-    when the configuration computes in bf16)."""
-    x = _rng(1000 + t).standard_normal((net.M, net.in_h, net.in_w, net.in_c)).astype(np.float32)
+    when the configuration computes in bf16).  `stream` selects an independent data stream."""
+    x = _rng(1000 + t + 1000003 * stream).standard_normal((net.M, net.in_h, net.in_w, net.in_c)).astype(np.float32)
     return round_to_bf16(x) if net.dtype == "bf16" else x
 
 
-def batch_labels(net: Net, t: int) -> np.ndarray:
+def batch_labels(net: Net, t: int, stream: int = 0) -> np.ndarray:
     """Labels of iteration t: int32[M], uniform in 0..classes-1."""
-    return _rng(2000 + t).integers(0, net.classes, size=net.M, dtype=np.int32)
+    return _rng(2000 + t + 1000003 * stream).integers(0, net.classes, size=net.M, dtype=np.int32)
 
 
 # ----------------------------------------------------------------------------- networks
