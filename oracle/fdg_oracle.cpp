@@ -79,6 +79,27 @@ struct Tensor {                       // [n, h, w, c], c fastest
     const double* at(int i, int y, int x) const { return v.data() + (((size_t)i * h + y) * w + x) * c; }
 };
 
+// ---- optional storage model of the bf16 configurations -------------------------------------
+// "bf16 activations and weights with fp32 master weights and accumulation": arithmetic stays
+// fp64 here, but every tensor the configuration STORES in bf16 is rounded when it is stored:
+// value -> fp32 (round to nearest even) -> bf16 (round to nearest even).  Storage points:
+//   forward : output of a linear/conv layer (after bias), of batch-norm (after the residual add
+//             that directly follows it, if any), of the shortcut's projection conv and batch-norm,
+//             of the residual add, of the pooling layers; NOT the logits of the last layer;
+//             ReLU commutes with rounding, so it needs no point of its own;
+//   weights : the matrices W (biases, gamma, beta stay unrounded);
+//   backward: softmax-CE gradient, every input-gradient a layer hands on (a conv that opens a
+//             residual block hands its gradient to the add unrounded; the sum is rounded once).
+double round_bf16(double v) {
+    float f = (float)v;
+    uint32_t u; std::memcpy(&u, &f, 4);
+    if ((u & 0x7f800000u) == 0x7f800000u) return f;              // inf / nan unchanged
+    u += 0x7fffu + ((u >> 16) & 1u); u &= 0xffff0000u;
+    std::memcpy(&f, &u, 4);
+    return f;
+}
+template <class TensorT> void store(TensorT& t, bool q) { if (q) for (auto& e : t.v) e = round_bf16(e); }
+
 size_t layer_param_count(const Layer& L) {
     switch (L.kind) {
         case LINEAR:  return (size_t)L.c_in * L.c_out + ((L.flags & 1) ? L.c_out : 0);
@@ -270,7 +291,7 @@ struct Saved {                         // h~_k(tau): what the backward pass of t
 };
 
 // Forward layers [p,q) on ONE worker's batch x with parameters `prm` (the group's slice).
-Tensor group_forward(const std::vector<Layer>& L, int p, int q, const double* prm, const Tensor& x0, Saved* sv) {
+Tensor group_forward(const std::vector<Layer>& L, int p, int q, const double* prm, const Tensor& x0, Saved* sv, bool sq = false) {
     int n = q - p;
     sv->in.assign(n, Tensor()); sv->bn.assign(n, BnSaved()); sv->sc_in.assign(n, Tensor()); sv->sc_conv.assign(n, Tensor());
     std::vector<Tensor> shortcut;
@@ -280,26 +301,33 @@ Tensor group_forward(const std::vector<Layer>& L, int p, int q, const double* pr
         const double* w = prm;
         switch (Y.kind) {
             case LINEAR: { sv->in[j] = x; Tensor f = flatten(x);
-                x = conv_fwd(f, w, (Y.flags & 1) ? w + (size_t)Y.c_in * Y.c_out : nullptr, Y.c_out, 1, 1, 0); break; }
+                x = conv_fwd(f, w, (Y.flags & 1) ? w + (size_t)Y.c_in * Y.c_out : nullptr, Y.c_out, 1, 1, 0);
+                store(x, sq && l + 1 < (int)L.size()); break; }
             case CONV3X3: sv->in[j] = x;
-                x = conv_fwd(x, w, (Y.flags & 1) ? w + (size_t)9 * Y.c_in * Y.c_out : nullptr, Y.c_out, 3, Y.stride, 1); break;
+                x = conv_fwd(x, w, (Y.flags & 1) ? w + (size_t)9 * Y.c_in * Y.c_out : nullptr, Y.c_out, 3, Y.stride, 1);
+                store(x, sq); break;
             case CONV1X1: sv->in[j] = x;
-                x = conv_fwd(x, w, (Y.flags & 1) ? w + (size_t)Y.c_in * Y.c_out : nullptr, Y.c_out, 1, Y.stride, 0); break;
+                x = conv_fwd(x, w, (Y.flags & 1) ? w + (size_t)Y.c_in * Y.c_out : nullptr, Y.c_out, 1, Y.stride, 0);
+                store(x, sq); break;
             case RELU: sv->in[j] = x; x = relu_fwd(x); break;
             case MAXPOOL2: sv->in[j] = x; x = maxpool_fwd(x); break;
-            case GLOBAL_AVGPOOL: sv->in[j] = x; x = gap_fwd(x); break;
-            case BATCHNORM: sv->in[j] = x; x = bn_fwd(x, w, w + Y.c_in, &sv->bn[j]); break;
+            case GLOBAL_AVGPOOL: sv->in[j] = x; x = gap_fwd(x); store(x, sq); break;
+            case BATCHNORM: sv->in[j] = x; x = bn_fwd(x, w, w + Y.c_in, &sv->bn[j]);
+                store(x, sq && !(l + 1 < q && L[l + 1].kind == RES_ADD)); break;
             case RES_BEGIN: shortcut.push_back(x); break;
             case RES_ADD: {
                 Tensor s = shortcut.back(); shortcut.pop_back();
                 sv->sc_in[j] = s;
                 if (Y.flags & 1) {
                     Tensor cv = conv_fwd(s, w, nullptr, Y.c_out, 1, Y.stride, 0);
+                    store(cv, sq);
                     sv->sc_conv[j] = cv;
                     const double* gb = w + (size_t)Y.c_in * Y.c_out;
                     s = bn_fwd(cv, gb, gb + Y.c_out, &sv->bn[j]);
+                    store(s, sq);
                 }
                 for (size_t i = 0; i < x.v.size(); ++i) x.v[i] += s.v[i];
+                store(x, sq);
                 break; }
         }
         prm += layer_param_count(Y);
@@ -309,7 +337,7 @@ Tensor group_forward(const std::vector<Layer>& L, int p, int q, const double* pr
 
 // Backward layers q-1..p with the SAME parameters the forward used; accumulates into gprm.
 Tensor group_backward(const std::vector<Layer>& L, int p, int q, const double* prm, const Saved& sv,
-                      const Tensor& gout, double* gprm, bool need_gin) {
+                      const Tensor& gout, double* gprm, bool need_gin, bool sq = false) {
     std::vector<size_t> off(q - p + 1, 0);
     for (int l = p; l < q; ++l) off[l - p + 1] = off[l - p] + layer_param_count(L[l]);
     std::vector<Tensor> gshort;
@@ -326,19 +354,24 @@ Tensor group_backward(const std::vector<Layer>& L, int p, int q, const double* p
                 const Tensor& xs = sv.in[j];
                 Tensor xin = Y.kind == LINEAR ? flatten(xs) : xs;
                 conv_bwd(xin, g, w, R, st, pad, want ? &gx : nullptr, gw, (Y.flags & 1) ? gw + nw : nullptr);
-                if (want) { gx.h = xs.h; gx.w = xs.w; gx.c = xs.c; g = gx; }   // undo the flattening
+                if (want) {
+                    gx.h = xs.h; gx.w = xs.w; gx.c = xs.c; g = gx;               // undo the flattening
+                    store(g, sq && !(l > p && L[l - 1].kind == RES_BEGIN));       // the add rounds the sum once
+                }
                 break; }
             case RELU: g = relu_bwd(sv.in[j], g); break;
             case MAXPOOL2: g = maxpool_bwd(sv.in[j], g); break;
-            case GLOBAL_AVGPOOL: g = gap_bwd(sv.in[j], g); break;
-            case BATCHNORM: g = bn_bwd(sv.in[j], g, w, sv.bn[j], gw, gw + Y.c_in); break;
+            case GLOBAL_AVGPOOL: g = gap_bwd(sv.in[j], g); store(g, sq); break;
+            case BATCHNORM: g = bn_bwd(sv.in[j], g, w, sv.bn[j], gw, gw + Y.c_in); store(g, sq); break;
             case RES_ADD: {
                 Tensor gs = g;                     // d(a + s)/ds = 1
                 if (Y.flags & 1) {
                     size_t nw = (size_t)Y.c_in * Y.c_out;
                     Tensor gc = bn_bwd(sv.sc_conv[j], gs, w + nw, sv.bn[j], gw + nw, gw + nw + Y.c_out);
+                    store(gc, sq);
                     Tensor gx;
                     conv_bwd(sv.sc_in[j], gc, w, 1, Y.stride, 0, &gx, gw, nullptr);
+                    store(gx, sq);
                     gs = gx;
                 }
                 gshort.push_back(gs);
@@ -346,6 +379,7 @@ Tensor group_backward(const std::vector<Layer>& L, int p, int q, const double* p
             case RES_BEGIN: {
                 Tensor gs = gshort.back(); gshort.pop_back();
                 for (size_t i = 0; i < g.v.size(); ++i) g.v[i] += gs.v[i];
+                store(g, sq);
                 break; }
         }
     }
@@ -373,6 +407,7 @@ struct Oracle {
     double scale = 1.0;                            // c: per-sample gradient scale
     std::vector<double> P;                         // S x S mixing matrix
     bool use_current_weights = false;              // planted-mistake switch for tests
+    bool storage_bf16 = false;                     // round at the storage points listed above
     long t = 0;
     std::vector<std::vector<Agent>> ag;            // [s][k]
     std::vector<size_t> poff;                      // parameter offset of module k in the full vector
@@ -383,6 +418,24 @@ struct Oracle {
 };
 
 size_t module_params(const Oracle& o, int k) { return o.poff[k + 1] - o.poff[k]; }
+
+// The copy of a module's weights that the passes read: matrices rounded to bf16 when the storage
+// model is on, everything else as it is.
+std::vector<double> pass_weights(const Oracle& o, int p, int q, const std::vector<double>& w) {
+    std::vector<double> c = w;
+    if (!o.storage_bf16) return c;
+    size_t off = 0;
+    for (int l = p; l < q; ++l) {
+        const Layer& Y = o.layers[l];
+        size_t nmat = 0;
+        if (Y.kind == LINEAR || Y.kind == CONV1X1) nmat = (size_t)Y.c_in * Y.c_out;
+        else if (Y.kind == CONV3X3) nmat = (size_t)9 * Y.c_in * Y.c_out;
+        else if (Y.kind == RES_ADD && (Y.flags & 1)) nmat = (size_t)Y.c_in * Y.c_out;
+        for (size_t i = 0; i < nmat; ++i) c[off + i] = round_bf16(c[off + i]);
+        off += layer_param_count(Y);
+    }
+    return c;
+}
 
 }  // namespace
 
@@ -420,6 +473,8 @@ double orc_kink_margin(int reset) { double m = g_kink_margin; if (reset) g_kink_
 int orc_threads() { return num_threads(); }
 size_t orc_param_count(void* h) { return ((Oracle*)h)->poff.back(); }
 void orc_set_flag_use_current_weights(void* h, int on) { ((Oracle*)h)->use_current_weights = on != 0; }
+void orc_set_storage_bf16(void* h, int on) { ((Oracle*)h)->storage_bf16 = on != 0; }
+void orc_round_bf16(const double* in, double* out, size_t n) { for (size_t i = 0; i < n; ++i) out[i] = round_bf16(in[i]); }
 
 // worker < 0: set every replica to the same vector.
 void orc_set_params(void* h, int worker, const double* p) {
@@ -465,14 +520,15 @@ int orc_step(void* h, const double* inputs, const int32_t* labels, double eta, d
             // ---- forward pass on whatever arrived (Algorithm 1: "compute h_l(t-k+1)")
             Tensor gout; long bwd_batch = -1;
             if (a.act_in.batch >= 0) {
-                StashEntry e; e.version = o.t; e.w = a.w; e.labels = a.act_in.labels;
-                Tensor out = group_forward(o.layers, p, q, a.w.data(), a.act_in.t, &e.sv);
+                StashEntry e; e.version = o.t; e.w = pass_weights(o, p, q, a.w); e.labels = a.act_in.labels;
+                Tensor out = group_forward(o.layers, p, q, e.w.data(), a.act_in.t, &e.sv, o.storage_bf16);
                 if (s == 0) o.tr_fwd[k] = a.act_in.batch;
                 if (k + 1 < K) {                       // send h_{q_k} to (s,k+1): it is read at t+1
                     Message nx; nx.batch = a.act_in.batch; nx.t = out; nx.labels = a.act_in.labels;
                     o.ag[s][k + 1].act_next = std::move(nx);
                 } else {                               // last module: evaluate phi and its gradient
                     loss_sum += softmax_ce(out, e.labels.data(), o.scale, &gout);
+                    store(gout, o.storage_bf16);
                     loss_batch = a.act_in.batch; bwd_batch = a.act_in.batch;
                 }
                 a.stash[a.act_in.batch] = std::move(e);
@@ -484,8 +540,8 @@ int orc_step(void* h, const double* inputs, const int32_t* labels, double eta, d
             std::fill(a.g.begin(), a.g.end(), 0.0);    // gradient is 0 while tau < 0
             if (bwd_batch >= 0) {
                 StashEntry& e = a.stash.at(bwd_batch);
-                const std::vector<double>& wb = o.use_current_weights ? a.w : e.w;
-                Tensor gin = group_backward(o.layers, p, q, wb.data(), e.sv, gout, a.g.data(), k > 0);
+                const std::vector<double> wb = o.use_current_weights ? pass_weights(o, p, q, a.w) : e.w;
+                Tensor gin = group_backward(o.layers, p, q, wb.data(), e.sv, gout, a.g.data(), k > 0, o.storage_bf16);
                 if (s == 0) { o.tr_bwd[k] = bwd_batch; o.tr_ver[k] = e.version; }
                 if (k > 0) {                           // send dphi/d(module input) to (s,k-1): read at t+1
                     Message nx; nx.batch = bwd_batch;

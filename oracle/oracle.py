@@ -40,6 +40,8 @@ def lib():
         L.orc_param_count.restype = C.c_size_t
         L.orc_param_count.argtypes = [C.c_void_p]
         L.orc_set_flag_use_current_weights.argtypes = [C.c_void_p, C.c_int]
+        L.orc_set_storage_bf16.argtypes = [C.c_void_p, C.c_int]
+        L.orc_round_bf16.argtypes = [dp, dp, C.c_size_t]
         L.orc_set_params.argtypes = [C.c_void_p, C.c_int, dp]
         L.orc_get_params.argtypes = [C.c_void_p, C.c_int, dp]
         L.orc_get_grads.argtypes = [C.c_void_p, C.c_int, dp]
@@ -127,6 +129,10 @@ class Oracle:
     def use_current_weights(self, on: bool):
         lib().orc_set_flag_use_current_weights(self.h, int(on))
 
+    def storage_bf16(self, on: bool):
+        """Round every tensor the bf16 configurations store in bf16 (see the C++ header comment)."""
+        lib().orc_set_storage_bf16(self.h, int(on))
+
     def step(self, inputs, labels, lr):
         x = np.ascontiguousarray(inputs, dtype=np.float64)
         y = np.ascontiguousarray(labels, dtype=np.int32)
@@ -162,6 +168,13 @@ def plain_logits(layers, n_workers, batch, in_shape, params, inputs, classes):
     x = np.ascontiguousarray(inputs, dtype=np.float64)
     out = np.empty((n_workers * batch, classes), dtype=np.float64)
     lib().orc_plain_logits(_i(L), len(L), n_workers, batch, *in_shape, _d(p), _d(x), _d(out))
+    return out
+
+
+def round_bf16(x) -> np.ndarray:
+    a = np.ascontiguousarray(x, dtype=np.float64)
+    out = np.empty_like(a)
+    lib().orc_round_bf16(_d(a), _d(out), a.size)
     return out
 
 

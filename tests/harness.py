@@ -47,8 +47,10 @@ def grad_rel_l2(a, b, layers, min_norm=1e-12):
     return worst, where, per
 
 
-def make_oracle(orc, net: sy.Net, params):
+def make_oracle(orc, net: sy.Net, params, storage_model=True):
+    """The oracle for a configuration; bf16 configurations get the bf16 storage model."""
     o = orc.Oracle(net.layers, net.splits, net.n_workers, net.batch, (net.in_h, net.in_w, net.in_c), net.classes)
+    o.storage_bf16(storage_model and net.dtype == "bf16")
     o.set_params(params)
     return o
 
@@ -84,14 +86,19 @@ def closed_form_trace(K, t):
 
 
 def run_parity(orc, net: sy.Net, steps: int, *, param_tol=None, grad_tol=None, grad_best_tol=None, loss_tol=None,
-               perturb=True, kink_guard=None, **ctx_kw):
+               perturb=True, kink_guard=None, grad_steps=None, grad_tail=None, **ctx_kw):
     """Step both implementations `steps` times; check the schedule bit-exactly after every step and
     parameters / gradients / loss within the given tolerances.  Returns the per-step records.
 
     Gradients: every tensor must be within `grad_tol` at every step.  `grad_best_tol` is a much
     tighter bound on each tensor's BEST step: a pre-activation that lands on the other side of a
     ReLU / max-pool kink in one precision but not the other legitimately changes a few terms of a
-    gradient sum in that step, whereas a wrong formula is wrong at every step."""
+    gradient sum in that step, whereas a wrong formula is wrong at every step.
+    `grad_steps`: check gradients only while t < grad_steps (afterwards the two trajectories have
+    moved apart and a gradient comparison compares different weights).  `grad_tail`: hold only the
+    last `grad_tail` tensors to `grad_tol` and ask the whole gradient for a cosine similarity of 0.7
+    (deep batch-norm networks amplify a single rounding difference by orders of magnitude on the
+    way back to the first layers)."""
     from paper_2509_05679_b200 import binding
     bf16 = net.dtype == "bf16"
     p0 = sy.init_params(net.layers, 0, bf16=False)
@@ -119,12 +126,21 @@ def run_parity(orc, net: sy.Net, steps: int, *, param_tol=None, grad_tol=None, g
                 assert np.isnan(lg)
             elif loss_tol is not None:
                 assert abs(lg - lo) <= loss_tol * max(abs(lo), 1e-6), (t, lg, lo)
-            if grad_tol is not None:
+            if grad_tol is not None and (grad_steps is None or t < grad_steps):
                 g_avg = np.mean([o.grads(s) for s in range(net.n_workers)], axis=0)     # P = 11^T/N averages the workers
-                r["grad_err"], r["grad_where"], per = grad_rel_l2(ctx.grads(), g_avg, net.layers)
+                g_gpu = ctx.grads()
+                r["grad_err"], r["grad_where"], per = grad_rel_l2(g_gpu, g_avg, net.layers)
                 for k_, e_ in per.items():
                     best[k_] = min(best.get(k_, np.inf), e_)
-                assert r["grad_err"] <= grad_tol, (t, r)
+                if grad_tail is None:
+                    assert r["grad_err"] <= grad_tol, (t, r)
+                elif per:
+                    tail = list(per.items())[-grad_tail:]
+                    assert all(e_ <= grad_tol for _, e_ in tail), (t, tail)
+                    nz = np.abs(g_avg) > 0
+                    cos = float(np.dot(g_gpu[nz], g_avg[nz]) / (np.linalg.norm(g_gpu[nz]) * np.linalg.norm(g_avg[nz]) + 1e-300))
+                    r["grad_cos"] = cos
+                    assert cos >= 0.7, (t, cos)
             if param_tol is not None:
                 r["param_err"], r["param_where"] = max_rel_err(ctx.params(), o.params(0), net.layers)
                 assert r["param_err"] <= param_tol, (t, r)

@@ -154,3 +154,36 @@ def test_softmax_cross_entropy_closed_forms(orc):
     z2 = np.array([[0.3, -1.1]])
     l, _ = orc.softmax_ce(z2, np.array([0], np.int32), 1.0)
     assert abs(l - np.log1p(np.exp(-1.4))) < 1e-14
+
+
+def test_bf16_storage_rounding_matches_torch_and_its_properties(orc):
+    g = np.random.default_rng(3)
+    x = np.concatenate([g.standard_normal(4000) * 10.0 ** g.integers(-6, 6, 4000),
+                        [0.0, -0.0, 1.0, 1.00390625, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 3.3895313892515355e38]])
+    got = orc.round_bf16(x)
+    want = torch.tensor(x, dtype=torch.float64).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    np.testing.assert_array_equal(got, want)
+    np.testing.assert_array_equal(orc.round_bf16(got), got)                 # idempotent
+    assert np.all(np.abs(got - x) <= np.abs(x) * 2.0 ** -8)                 # half an ulp of 8 significand bits
+    assert orc.round_bf16([1.0 + 2.0 ** -8])[0] == 1.0                      # tie -> even
+    assert orc.round_bf16([1.0 + 3 * 2.0 ** -8])[0] == 1.0 + 2.0 ** -6      # tie -> even (up)
+
+
+def test_bf16_storage_model_stays_close_to_the_fp64_run_and_is_off_by_default(orc):
+    layers, bs = sy.resnet_layers(widths=(4, 8), blocks=1, in_c=2, classes=3)
+    S, B, in_shape = 2, 3, (4, 4, 2)
+    p = sy.round_to_bf16(sy.perturb_params(sy.init_params(layers, 1), layers, 2, 0.2))
+    runs = {}
+    for mode in (False, True):
+        o = orc.Oracle(layers, [bs[0], bs[1]], S, B, in_shape, 3)
+        o.storage_bf16(mode)
+        o.set_params(p)
+        g = np.random.default_rng(0)
+        for t in range(7):
+            x = sy.round_to_bf16(g.standard_normal((S * B,) + in_shape).astype(np.float32))
+            loss, _ = o.step(x, g.integers(0, 3, S * B), 0.05)
+        runs[mode] = (loss, o.grads(0))
+    assert runs[True][0] != runs[False][0]
+    assert abs(runs[True][0] - runs[False][0]) < 2e-2 * runs[False][0]
+    d = np.linalg.norm(runs[True][1] - runs[False][1]) / np.linalg.norm(runs[False][1])
+    assert 0 < d < 0.1
