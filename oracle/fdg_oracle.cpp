@@ -38,6 +38,7 @@
 #include <functional>
 #include <map>
 #include <memory>
+#include <mutex>
 #include <string>
 #include <thread>
 #include <vector>
@@ -53,19 +54,23 @@ int g_threads = 0;   // 0 = hardware_concurrency
 // between the two largest values of a max-pool window.  Tests use it to tell whether a lower
 // precision could legitimately take the other branch somewhere.
 double g_kink_margin = 1e300;
+std::mutex g_kink_mu;
+void note_kink(double m) { std::lock_guard<std::mutex> lk(g_kink_mu); g_kink_margin = std::min(g_kink_margin, m); }
 
 int num_threads() {
     int n = g_threads > 0 ? g_threads : (int)std::thread::hardware_concurrency();
     return n < 1 ? 1 : n;
 }
 
-// Run fn(i) for i in [0,n) on up to num_threads() threads (static interleaving).
+// Run fn(i) for i in [0,n) on up to num_threads() threads (static interleaving).  A parallel_for
+// reached from inside another one runs serially: the outer level (the workers) owns the threads.
+thread_local bool t_inside_parallel = false;
 void parallel_for(int n, const std::function<void(int)>& fn) {
     int nt = std::min(num_threads(), n);
-    if (nt <= 1) { for (int i = 0; i < n; ++i) fn(i); return; }
+    if (nt <= 1 || t_inside_parallel) { for (int i = 0; i < n; ++i) fn(i); return; }
     std::vector<std::thread> th;
     for (int w = 0; w < nt; ++w)
-        th.emplace_back([=, &fn] { for (int i = w; i < n; i += nt) fn(i); });
+        th.emplace_back([=, &fn] { t_inside_parallel = true; for (int i = w; i < n; i += nt) fn(i); });
     for (auto& t : th) t.join();
 }
 
@@ -188,7 +193,9 @@ Tensor flatten(const Tensor& x) { Tensor y = x; y.c = (int)x.per_sample(); y.h =
 
 Tensor relu_fwd(const Tensor& x) {
     Tensor y = x;
-    for (auto& e : y.v) { g_kink_margin = std::min(g_kink_margin, std::fabs(e)); e = e > 0.0 ? e : 0.0; }
+    double margin = 1e300;
+    for (auto& e : y.v) { margin = std::min(margin, std::fabs(e)); e = e > 0.0 ? e : 0.0; }
+    note_kink(margin);
     return y;
 }
 Tensor relu_bwd(const Tensor& x, const Tensor& gy) {
@@ -197,14 +204,16 @@ Tensor relu_bwd(const Tensor& x, const Tensor& gy) {
 
 Tensor maxpool_fwd(const Tensor& x) {
     Tensor y(x.n, x.h / 2, x.w / 2, x.c);
+    double margin = 1e300;
     for (int i = 0; i < x.n; ++i) for (int oy = 0; oy < y.h; ++oy) for (int ox = 0; ox < y.w; ++ox)
         for (int c = 0; c < x.c; ++c) {
             double v[4] = {x.at(i, 2 * oy, 2 * ox)[c], x.at(i, 2 * oy, 2 * ox + 1)[c], x.at(i, 2 * oy + 1, 2 * ox)[c], x.at(i, 2 * oy + 1, 2 * ox + 1)[c]};
             double m = std::max(std::max(v[0], v[1]), std::max(v[2], v[3]));
             std::sort(v, v + 4);
-            g_kink_margin = std::min(g_kink_margin, v[3] - v[2]);
+            margin = std::min(margin, v[3] - v[2]);
             y.at(i, oy, ox)[c] = m;
         }
+    note_kink(margin);
     return y;
 }
 Tensor maxpool_bwd(const Tensor& x, const Tensor& gy) {
@@ -504,10 +513,12 @@ int orc_step(void* h, const double* inputs, const int32_t* labels, double eta, d
     Oracle& o = *(Oracle*)h;
     const int K = o.K, S = o.S, B = o.B;
     const size_t in_per = (size_t)o.in_h * o.in_w * o.in_c;
-    double loss_sum = 0.0; long loss_batch = -1;
+    std::vector<double> loss_of(S, 0.0); std::vector<long> batch_of(S, -1);
     std::fill(o.tr_fwd.begin(), o.tr_fwd.end(), -1); std::fill(o.tr_bwd.begin(), o.tr_bwd.end(), -1); std::fill(o.tr_ver.begin(), o.tr_ver.end(), -1);
 
-    for (int s = 0; s < S; ++s) {
+    // the data-groups are independent within an iteration (Algorithm 1: all agents in parallel)
+    parallel_for(S, [&](int s) {
+        double& loss_sum = loss_of[s]; long& loss_batch = batch_of[s];
         // agent (s,1) samples B_s(t): here, takes its rows of the caller's batch
         Message m; m.batch = o.t; m.t = Tensor(B, o.in_h, o.in_w, o.in_c);
         std::copy(inputs + (size_t)s * B * in_per, inputs + (size_t)(s + 1) * B * in_per, m.t.v.begin());
@@ -551,7 +562,9 @@ int orc_step(void* h, const double* inputs, const int32_t* labels, double eta, d
                 a.stash.erase(bwd_batch);
             }
         }
-    }
+    });
+    double loss_sum = 0.0; long loss_batch = -1;
+    for (int s = 0; s < S; ++s) { loss_sum += loss_of[s]; loss_batch = std::max(loss_batch, batch_of[s]); }
     // ---- u_{s,k} = w_{s,k} - eta g_{s,k};  w_{s,k}(t+1) = sum_r P_sr u_{r,k}   (Eq. dl_update a, b)
     for (int k = 0; k < K; ++k) {
         size_t n = module_params(o, k);

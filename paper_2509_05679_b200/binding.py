@@ -20,7 +20,8 @@ STATUS = {0: "FDG_OK", 1: "FDG_ERR_INVALID_ARG", 2: "FDG_ERR_BAD_SPLIT", 3: "FDG
           4: "FDG_ERR_ARCH", 5: "FDG_ERR_OOM", 6: "FDG_ERR_CUDA", 7: "FDG_ERR_TIMEOUT", 8: "FDG_ERR_STATE"}
 
 EXPORTS = ["fdg_create", "fdg_param_count", "fdg_set_params", "fdg_step", "fdg_step_host", "fdg_wait_ingest", "fdg_params",
-           "fdg_grads", "fdg_trace", "fdg_set_lr", "fdg_stats", "fdg_module_times", "fdg_last_error", "fdg_destroy"]
+           "fdg_grads", "fdg_trace", "fdg_set_lr", "fdg_stats", "fdg_module_times", "fdg_profile", "fdg_profile_read",
+           "fdg_last_error", "fdg_destroy"]
 
 
 class FdgError(RuntimeError):
@@ -39,6 +40,10 @@ FREE_FN = C.CFUNCTYPE(None, C.c_void_p, C.c_void_p)
 
 class fdg_allocator(C.Structure):
     _fields_ = [("alloc", ALLOC_FN), ("free", FREE_FN), ("user", C.c_void_p)]
+
+
+class fdg_kernel_stat(C.Structure):
+    _fields_ = [("name", C.c_char * 48), ("launches", C.c_uint64), ("ms", C.c_double), ("flops", C.c_double), ("bytes", C.c_double)]
 
 
 class fdg_options(C.Structure):
@@ -81,6 +86,10 @@ def lib():
         L.fdg_stats.argtypes = [vp, C.POINTER(C.c_size_t), C.POINTER(C.c_uint64)]
         L.fdg_module_times.restype = C.c_int
         L.fdg_module_times.argtypes = [vp, fp, C.c_int32]
+        L.fdg_profile.restype = C.c_int
+        L.fdg_profile.argtypes = [vp, C.c_int32]
+        L.fdg_profile_read.restype = C.c_int
+        L.fdg_profile_read.argtypes = [vp, C.POINTER(fdg_kernel_stat), C.c_int32, C.POINTER(C.c_int32)]
         L.fdg_last_error.restype = C.c_char_p
         L.fdg_last_error.argtypes = [vp]
         L.fdg_destroy.restype = None
@@ -128,7 +137,8 @@ class Context:
 
     def __init__(self, layers: Sequence[Sequence[int]], split_points: Sequence[int], n_workers: int,
                  per_worker_batch: int, lr: float, *, dtype: str = "bf16", in_shape=(32, 32, 3), num_classes: int = 10,
-                 serial: bool = False, kernel_path: int = 0, device: int = 0, use_torch_allocator: bool = True):
+                 serial: bool = False, kernel_path: int = 0, device: int = 0, use_torch_allocator: bool = True,
+                 streams: Optional[Sequence[int]] = None):
         import torch
         L = lib()
         if not torch.cuda.is_available():
@@ -140,8 +150,13 @@ class Context:
         self.in_shape = tuple(in_shape)
         arr = (fdg_layer * len(layers))(*[fdg_layer(*[int(v) for v in l]) for l in layers])
         sp = (C.c_int32 * max(1, len(split_points)))(*[int(s) for s in split_points])
+        self._streams = None
+        if streams is not None:          # K cudaStream_t handles owned by the caller
+            assert len(streams) == self.K
+            self._streams = (C.c_void_p * self.K)(*[C.c_void_p(int(h_)) for h_ in streams])
         opt = fdg_options({"fp32": 0, "bf16": 1}[dtype], int(in_shape[0]), int(in_shape[1]), int(in_shape[2]),
-                          int(num_classes), int(serial), int(kernel_path), None)
+                          int(num_classes), int(serial), int(kernel_path),
+                          C.cast(self._streams, C.POINTER(C.c_void_p)) if self._streams is not None else None)
         self._alloc = _TorchAllocator(torch.device("cuda", device)) if use_torch_allocator else None
         h = C.c_void_p()
         st = L.fdg_create(arr, len(layers), sp, self.K, n_workers, per_worker_batch, float(lr), C.byref(opt),
@@ -210,6 +225,17 @@ class Context:
         nb, nl = C.c_size_t(), C.c_uint64()
         self._ck(lib().fdg_stats(self.h, C.byref(nb), C.byref(nl)))
         return nb.value, nl.value
+
+    def profile(self, enable: bool):
+        self._ck(lib().fdg_profile(self.h, int(enable)))
+
+    def profile_read(self):
+        """{kernel class: dict(launches, ms, flops, bytes)} since profile(True)."""
+        arr = (fdg_kernel_stat * 64)()
+        n = C.c_int32()
+        self._ck(lib().fdg_profile_read(self.h, arr, 64, C.byref(n)))
+        return {arr[i].name.decode(): dict(launches=int(arr[i].launches), ms=arr[i].ms, flops=arr[i].flops, bytes=arr[i].bytes)
+                for i in range(n.value)}
 
     def module_times(self) -> np.ndarray:
         ms = np.empty(self.K, dtype=np.float32)

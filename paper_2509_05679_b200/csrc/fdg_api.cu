@@ -667,6 +667,28 @@ fdg_status fdg_stats(const fdg_ctx* ctx, size_t* device_bytes, uint64_t* kernel_
     return FDG_OK;
 }
 
+fdg_status fdg_profile(fdg_ctx* ctx, int32_t enable) {
+    if (!ctx) return FDG_ERR_INVALID_ARG;
+    CK(cudaDeviceSynchronize());
+    profile_enable(enable != 0);
+    return FDG_OK;
+}
+
+fdg_status fdg_profile_read(fdg_ctx* ctx, fdg_kernel_stat* out, int32_t capacity, int32_t* count) {
+    if (!ctx || !out || !count) return FDG_ERR_INVALID_ARG;
+    KernelStat st[KC_COUNT]; const char* names[KC_COUNT];
+    int n = profile_read(st, names), w = 0;
+    for (int i = 0; i < n && w < capacity; ++i) {
+        if (!st[i].launches) continue;
+        std::memset(&out[w], 0, sizeof out[w]);
+        std::strncpy(out[w].name, names[i], sizeof(out[w].name) - 1);
+        out[w].launches = st[i].launches; out[w].ms = st[i].ms; out[w].flops = st[i].flops; out[w].bytes = st[i].bytes;
+        ++w;
+    }
+    *count = w;
+    return FDG_OK;
+}
+
 fdg_status fdg_module_times(fdg_ctx* ctx, float* ms, int32_t K) {
     if (!ctx || !ms || K != ctx->K) return FDG_ERR_INVALID_ARG;
     if (ctx->t == 0) return fail(ctx, FDG_ERR_STATE, "no step has run yet");

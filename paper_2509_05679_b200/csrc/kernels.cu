@@ -6,12 +6,64 @@
 
 #include <cuda_bf16.h>
 #include <atomic>
+#include <mutex>
+#include <vector>
 
 namespace fdg {
 
 static std::atomic<uint64_t> g_launches{0};
 uint64_t launches() { return g_launches.load(); }
-#define COUNT_LAUNCH() g_launches.fetch_add(1, std::memory_order_relaxed)
+
+// ---- per-kernel-class device timing (off by default): every launcher opens a Scope, which counts the
+// launch and, while profiling is on, brackets it with two events on the launching stream.
+static const char* kClassNames[KC_COUNT] = {
+    "igemm_fma_fwd", "igemm_fma_dgrad", "igemm_fma_wgrad", "splitk_reduce", "bias_grad", "relu_fwd", "relu_bwd", "add_fwd",
+    "copy_accumulate", "maxpool_fwd", "maxpool_bwd", "gap_fwd", "gap_bwd", "bn_fwd_stats", "bn_fwd_apply", "bn_bwd_reduce",
+    "bn_bwd_apply", "softmax_ce", "sgd_update", "tags", "fill", "tc_gemm_fwd", "tc_gemm_dgrad", "tc_gemm_wgrad", "tc_aux"};
+namespace prof {
+struct Rec { int cls; cudaEvent_t a, b; };
+static bool g_on = false;
+static std::mutex g_mu;
+static std::vector<Rec> g_recs;
+static std::vector<cudaEvent_t> g_pool;
+static KernelStat g_stat[KC_COUNT];
+static cudaEvent_t get_event() {
+    if (!g_pool.empty()) { cudaEvent_t e = g_pool.back(); g_pool.pop_back(); return e; }
+    cudaEvent_t e = nullptr; cudaEventCreate(&e); return e;
+}
+}  // namespace prof
+Scope::Scope(int cls_, double flops, double bytes, cudaStream_t s) : cls(cls_), st(s), a(nullptr) {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (!prof::g_on) return;
+    std::lock_guard<std::mutex> lk(prof::g_mu);
+    prof::g_stat[cls].launches += 1; prof::g_stat[cls].flops += flops; prof::g_stat[cls].bytes += bytes;
+    a = prof::get_event();
+    cudaEventRecord(a, st);
+}
+Scope::~Scope() {
+    if (!a) return;
+    std::lock_guard<std::mutex> lk(prof::g_mu);
+    cudaEvent_t b = prof::get_event();
+    cudaEventRecord(b, st);
+    prof::g_recs.push_back({cls, a, b});
+}
+void profile_enable(bool on) {
+    std::lock_guard<std::mutex> lk(prof::g_mu);
+    if (on) for (auto& k : prof::g_stat) k = KernelStat{};
+    prof::g_on = on;
+}
+int profile_read(KernelStat* out, const char** names) {
+    cudaDeviceSynchronize();
+    std::lock_guard<std::mutex> lk(prof::g_mu);
+    for (auto& r : prof::g_recs) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess) prof::g_stat[r.cls].ms += ms;
+        prof::g_pool.push_back(r.a); prof::g_pool.push_back(r.b);
+    }
+    prof::g_recs.clear();
+    for (int i = 0; i < KC_COUNT; ++i) { out[i] = prof::g_stat[i]; names[i] = kClassNames[i]; }
+    return KC_COUNT;
+}
 
 typedef __nv_bfloat16 bf16;
 
@@ -173,6 +225,11 @@ __global__ void splitk_reduce(const float* __restrict__ partial, float* __restri
     out[i] = s;
 }
 
+void splitk_reduce_launch(const float* partial, float* out, size_t n, int splits, cudaStream_t s) {
+    Scope sc(KC_SPLITK, 0.0, 4.0 * n * (splits + 1), s);
+    splitk_reduce<<<cdiv(n, 256), 256, 0, s>>>(partial, out, n, splits);
+}
+
 int wgrad_splits(const ConvGeom& g) {
     long Kg = (long)g.N * g.Ho * g.Wo;
     int tiles = (int)(cdiv(g.Co, BM) * cdiv((size_t)g.R * g.R * g.C, BN));
@@ -192,8 +249,8 @@ template <typename T>
 static void conv_forward_t(const void* x, const void* w, const float* bias, void* y, const ConvGeom& g, int epi, cudaStream_t s) {
     int Mg = g.N * g.Ho * g.Wo, Ng = g.Co, Kg = g.R * g.R * g.C;
     dim3 grid(cdiv(Ng, BN), cdiv(Mg, BM), 1);
+    Scope sc(KC_FMA_FWD, 2.0 * Mg * Ng * Kg, sizeof(T) * ((double)g.N * g.H * g.W * g.C + (double)Ng * Kg + (double)Mg * Ng), s);
     igemm_simt<T, M_FWD><<<grid, 256, 0, s>>>((const T*)x, (const T*)w, y, bias, nullptr, g, Mg, Ng, Kg, Kg, epi);
-    COUNT_LAUNCH();
 }
 void conv_forward(int dt, const void* x, const void* w, const float* bias, void* y, const ConvGeom& g, int epi, cudaStream_t s) {
     if (dt) conv_forward_t<bf16>(x, w, bias, y, g, epi, s); else conv_forward_t<float>(x, w, bias, y, g, epi, s);
@@ -203,8 +260,8 @@ template <typename T>
 static void conv_dgrad_t(const void* dy, const void* w, void* dx, const ConvGeom& g, int epi, cudaStream_t s) {
     int Mg = g.N * g.H * g.W, Ng = g.C, Kg = g.R * g.R * g.Co;
     dim3 grid(cdiv(Ng, BN), cdiv(Mg, BM), 1);
+    Scope sc(KC_FMA_DGRAD, 2.0 * Mg * Ng * Kg, sizeof(T) * ((double)g.N * g.Ho * g.Wo * g.Co + (double)Ng * Kg + (double)Mg * Ng), s);
     igemm_simt<T, M_DGRAD><<<grid, 256, 0, s>>>((const T*)dy, (const T*)w, dx, nullptr, nullptr, g, Mg, Ng, Kg, Kg, epi);
-    COUNT_LAUNCH();
 }
 void conv_dgrad(int dt, const void* dy, const void* w, void* dx, const ConvGeom& g, int epi, cudaStream_t s) {
     if (dt) conv_dgrad_t<bf16>(dy, w, dx, g, epi, s); else conv_dgrad_t<float>(dy, w, dx, g, epi, s);
@@ -217,15 +274,14 @@ static void conv_wgrad_t(const void* x, const void* dy, float* dw, float* ws, co
     int kps = ((Kg + splits - 1) / splits + BK - 1) / BK * BK;
     splits = (Kg + kps - 1) / kps;
     dim3 grid(cdiv(Ng, BN), cdiv(Mg, BM), splits);
+    double flops = 2.0 * Mg * Ng * Kg, bytes = sizeof(T) * ((double)g.N * g.H * g.W * g.C + (double)Kg * Mg) + 4.0 * Mg * Ng;
     if (splits == 1) {
+        Scope sc(KC_FMA_WGRAD, flops, bytes, s);
         igemm_simt<T, M_WGRAD><<<grid, 256, 0, s>>>((const T*)dy, (const T*)x, dw, nullptr, nullptr, g, Mg, Ng, Kg, kps, EPI_OUT_F32);
-        COUNT_LAUNCH();
     } else {
-        igemm_simt<T, M_WGRAD><<<grid, 256, 0, s>>>((const T*)dy, (const T*)x, dw, nullptr, ws, g, Mg, Ng, Kg, kps, EPI_OUT_F32);
-        COUNT_LAUNCH();
-        size_t n = (size_t)Mg * Ng;
-        splitk_reduce<<<cdiv(n, 256), 256, 0, s>>>(ws, dw, n, splits);
-        COUNT_LAUNCH();
+        { Scope sc(KC_FMA_WGRAD, flops, bytes, s);
+          igemm_simt<T, M_WGRAD><<<grid, 256, 0, s>>>((const T*)dy, (const T*)x, dw, nullptr, ws, g, Mg, Ng, Kg, kps, EPI_OUT_F32); }
+        splitk_reduce_launch(ws, dw, (size_t)Mg * Ng, splits, s);
     }
 }
 void conv_wgrad(int dt, const void* x, const void* dy, float* dw, float* ws, const ConvGeom& g, cudaStream_t s) {
@@ -263,11 +319,11 @@ __global__ void colsum_final(const float* __restrict__ part, float* __restrict__
 void bias_grad(int dt, const void* dy, float* db, float* scratch, long rows, int C, cudaStream_t s) {
     int chunks = (int)(rows < RED_CHUNKS ? rows : RED_CHUNKS);
     dim3 grid(cdiv(C, 32), chunks), blk(32, 8);
-    if (dt) colsum_partial<bf16><<<grid, blk, 0, s>>>((const bf16*)dy, scratch, rows, C);
-    else colsum_partial<float><<<grid, blk, 0, s>>>((const float*)dy, scratch, rows, C);
-    COUNT_LAUNCH();
+    { Scope sc(KC_BIAS_GRAD, 0.0, (dt ? 2.0 : 4.0) * rows * C, s);
+      if (dt) colsum_partial<bf16><<<grid, blk, 0, s>>>((const bf16*)dy, scratch, rows, C);
+      else colsum_partial<float><<<grid, blk, 0, s>>>((const float*)dy, scratch, rows, C); }
+    Scope sc(KC_BIAS_GRAD, 0.0, 4.0 * chunks * C, s);
     colsum_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, db, chunks, C);
-    COUNT_LAUNCH();
 }
 
 // ------------------------------------------------------------------------------------------
@@ -285,24 +341,32 @@ template <typename T> __global__ void copy_acc_k(const T* src, T* dst, size_t n,
     if (i < n) { float v = ld(src + i); if (accum) v += ld(dst + i); st(dst + i, v); } }
 
 void relu_forward(int dt, const void* x, void* y, size_t n, cudaStream_t s) {
+    const double esz_ = dt ? 2.0 : 4.0; (void)esz_;
+    Scope sc(KC_RELU_FWD, 0.0, 2 * esz_ * n, s);
     if (dt) relu_fwd_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)x, (bf16*)y, n);
     else relu_fwd_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)x, (float*)y, n);
-    COUNT_LAUNCH();
+    
 }
 void relu_backward(int dt, const void* y, const void* dy, void* dx, size_t n, bool accum, cudaStream_t s) {
+    const double esz_ = dt ? 2.0 : 4.0; (void)esz_;
+    Scope sc(KC_RELU_BWD, 0.0, 3 * esz_ * n, s);
     if (dt) relu_bwd_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)y, (const bf16*)dy, (bf16*)dx, n, accum);
     else relu_bwd_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)y, (const float*)dy, (float*)dx, n, accum);
-    COUNT_LAUNCH();
+    
 }
 void add_forward(int dt, const void* a, const void* b, void* y, size_t n, cudaStream_t s) {
+    const double esz_ = dt ? 2.0 : 4.0; (void)esz_;
+    Scope sc(KC_ADD_FWD, 0.0, 3 * esz_ * n, s);
     if (dt) add_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)a, (const bf16*)b, (bf16*)y, n);
     else add_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)a, (const float*)b, (float*)y, n);
-    COUNT_LAUNCH();
+    
 }
 void copy_or_accumulate(int dt, const void* src, void* dst, size_t n, bool accum, cudaStream_t s) {
+    const double esz_ = dt ? 2.0 : 4.0; (void)esz_;
+    Scope sc(KC_COPY_ACC, 0.0, (accum ? 3 : 2) * esz_ * n, s);
     if (dt) copy_acc_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)src, (bf16*)dst, n, accum);
     else copy_acc_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)src, (float*)dst, n, accum);
-    COUNT_LAUNCH();
+    
 }
 
 template <typename T>
@@ -334,16 +398,20 @@ __global__ void maxpool_bwd_k(const T* x, const T* dy, T* dx, int N, int H, int 
     for (int j = 0; j < 4; ++j) { float v = (j == best) ? g : 0.f; if (accum) v += ld(dx + o[j]); st(dx + o[j], v); }
 }
 void maxpool_forward(int dt, const void* x, void* y, int N, int H, int W, int C, cudaStream_t s) {
+    const double esz_ = dt ? 2.0 : 4.0; (void)esz_;
+    Scope sc(KC_POOL_FWD, 0.0, 1.25 * esz_ * (double)N * H * W * C, s);
     size_t n = (size_t)N * (H / 2) * (W / 2) * C;
     if (dt) maxpool_fwd_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)x, (bf16*)y, N, H, W, C);
     else maxpool_fwd_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)x, (float*)y, N, H, W, C);
-    COUNT_LAUNCH();
+    
 }
 void maxpool_backward(int dt, const void* x, const void* dy, void* dx, int N, int H, int W, int C, bool accum, cudaStream_t s) {
+    const double esz_ = dt ? 2.0 : 4.0; (void)esz_;
+    Scope sc(KC_POOL_BWD, 0.0, 2.25 * esz_ * (double)N * H * W * C, s);
     size_t n = (size_t)N * (H / 2) * (W / 2) * C;
     if (dt) maxpool_bwd_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)x, (const bf16*)dy, (bf16*)dx, N, H, W, C, accum);
     else maxpool_bwd_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)x, (const float*)dy, (float*)dx, N, H, W, C, accum);
-    COUNT_LAUNCH();
+    
 }
 
 template <typename T>
@@ -365,16 +433,20 @@ __global__ void gap_bwd_k(const T* dy, T* dx, int N, int HW, int C, bool accum) 
     st(dx + i, v);
 }
 void gap_forward(int dt, const void* x, void* y, int N, int HW, int C, cudaStream_t s) {
+    const double esz_ = dt ? 2.0 : 4.0; (void)esz_;
+    Scope sc(KC_GAP_FWD, 0.0, esz_ * (double)N * (HW + 1) * C, s);
     size_t n = (size_t)N * C;
     if (dt) gap_fwd_k<bf16><<<cdiv(n, 128), 128, 0, s>>>((const bf16*)x, (bf16*)y, N, HW, C);
     else gap_fwd_k<float><<<cdiv(n, 128), 128, 0, s>>>((const float*)x, (float*)y, N, HW, C);
-    COUNT_LAUNCH();
+    
 }
 void gap_backward(int dt, const void* dy, void* dx, int N, int HW, int C, bool accum, cudaStream_t s) {
+    const double esz_ = dt ? 2.0 : 4.0; (void)esz_;
+    Scope sc(KC_GAP_BWD, 0.0, esz_ * (double)N * (HW + 1) * C, s);
     size_t n = (size_t)N * HW * C;
     if (dt) gap_bwd_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)dy, (bf16*)dx, N, HW, C, accum);
     else gap_bwd_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)dy, (float*)dx, N, HW, C, accum);
-    COUNT_LAUNCH();
+    
 }
 
 // ------------------------------------------------------------------------------------------
@@ -475,15 +547,16 @@ void bn_forward(int dt, const void* x, const float* gamma, const float* beta, co
                 float* scratch, int nw, long rpw, int C, bool relu, cudaStream_t s) {
     int chunks = (int)(rpw < RED_CHUNKS ? rpw : RED_CHUNKS);
     dim3 grid(cdiv(C, 32), chunks, nw), blk(32, 8);
-    if (dt) bn_reduce_partial<bf16, false><<<grid, blk, 0, s>>>((const bf16*)x, nullptr, nullptr, nullptr, scratch, rpw, C, false);
-    else bn_reduce_partial<float, false><<<grid, blk, 0, s>>>((const float*)x, nullptr, nullptr, nullptr, scratch, rpw, C, false);
-    COUNT_LAUNCH();
-    bn_stats_final<<<cdiv((size_t)nw * C, 128), 128, 0, s>>>(scratch, stats, chunks, nw * C, rpw);
-    COUNT_LAUNCH();
+    const double esz_ = dt ? 2.0 : 4.0;
     size_t total = (size_t)nw * rpw * C;
+    { Scope sc(KC_BN_FWD_STATS, 0.0, esz_ * total, s);
+      if (dt) bn_reduce_partial<bf16, false><<<grid, blk, 0, s>>>((const bf16*)x, nullptr, nullptr, nullptr, scratch, rpw, C, false);
+      else bn_reduce_partial<float, false><<<grid, blk, 0, s>>>((const float*)x, nullptr, nullptr, nullptr, scratch, rpw, C, false); }
+    { Scope sc(KC_BN_FWD_STATS, 0.0, 8.0 * chunks * nw * C, s);
+      bn_stats_final<<<cdiv((size_t)nw * C, 128), 128, 0, s>>>(scratch, stats, chunks, nw * C, rpw); }
+    Scope sc(KC_BN_FWD_APPLY, 0.0, esz_ * total * (res ? 3 : 2), s);
     if (dt) bn_apply_k<bf16><<<cdiv(total, 256), 256, 0, s>>>((const bf16*)x, gamma, beta, (const bf16*)res, (bf16*)y, stats, rpw, C, total, relu);
     else bn_apply_k<float><<<cdiv(total, 256), 256, 0, s>>>((const float*)x, gamma, beta, (const float*)res, (float*)y, stats, rpw, C, total, relu);
-    COUNT_LAUNCH();
 }
 
 void bn_backward(int dt, const void* x, const void* out, const void* dout, const float* gamma, const float* stats,
@@ -491,17 +564,18 @@ void bn_backward(int dt, const void* x, const void* out, const void* dout, const
                  float* scratch, int nw, long rpw, int C, bool relu, cudaStream_t s) {
     int chunks = (int)(rpw < RED_CHUNKS ? rpw : RED_CHUNKS);
     dim3 grid(cdiv(C, 32), chunks, nw), blk(32, 8);
-    if (dt) bn_reduce_partial<bf16, true><<<grid, blk, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, stats, scratch, rpw, C, relu);
-    else bn_reduce_partial<float, true><<<grid, blk, 0, s>>>((const float*)x, (const float*)out, (const float*)dout, stats, scratch, rpw, C, relu);
-    COUNT_LAUNCH();
-    bn_bwd_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C);
-    COUNT_LAUNCH();
+    const double esz_ = dt ? 2.0 : 4.0;
     size_t total = (size_t)nw * rpw * C;
+    { Scope sc(KC_BN_BWD_REDUCE, 0.0, esz_ * total * (relu ? 3 : 2), s);
+      if (dt) bn_reduce_partial<bf16, true><<<grid, blk, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, stats, scratch, rpw, C, relu);
+      else bn_reduce_partial<float, true><<<grid, blk, 0, s>>>((const float*)x, (const float*)out, (const float*)dout, stats, scratch, rpw, C, relu); }
+    { Scope sc(KC_BN_BWD_REDUCE, 0.0, 8.0 * chunks * nw * C, s);
+      bn_bwd_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C); }
+    Scope sc(KC_BN_BWD_APPLY, 0.0, esz_ * total * ((relu ? 3 : 2) + 1 + (dres ? (accum_dres ? 2 : 1) : 0) + (accum_dx ? 1 : 0)), s);
     if (dt) bn_bwd_apply_k<bf16><<<cdiv(total, 256), 256, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, gamma, stats, red,
                                                                   (bf16*)dx, accum_dx, (bf16*)dres, accum_dres, rpw, C, total, relu);
     else bn_bwd_apply_k<float><<<cdiv(total, 256), 256, 0, s>>>((const float*)x, (const float*)out, (const float*)dout, gamma, stats, red,
                                                                 (float*)dx, accum_dx, (float*)dres, accum_dres, rpw, C, total, relu);
-    COUNT_LAUNCH();
 }
 
 // ------------------------------------------------------------------------------------------
@@ -530,9 +604,9 @@ __global__ void softmax_ce_k(const float* __restrict__ z, const int32_t* __restr
     if (threadIdx.x == 0) *loss_out = sh[0] * inv_m;
 }
 void softmax_ce(int dt, const float* logits, const int32_t* labels, void* dlogits, float* loss_out, int M, int classes, cudaStream_t s) {
+    Scope sc(KC_SOFTMAX_CE, 0.0, (double)M * classes * (dt ? 6.0 : 8.0) + 4.0 * M, s);
     if (dt) softmax_ce_k<bf16><<<1, 256, 0, s>>>(logits, labels, (bf16*)dlogits, loss_out, M, classes);
     else softmax_ce_k<float><<<1, 256, 0, s>>>(logits, labels, (float*)dlogits, loss_out, M, classes);
-    COUNT_LAUNCH();
 }
 
 // ------------------------------------------------------------------------------------------
@@ -562,9 +636,10 @@ void sgd_update(int dt, float* master, const float* grad, void* copy_next, size_
     if (n4 == 0) return;
     unsigned blocks = cdiv(n4, 256);
     if (blocks > 148 * 8) blocks = 148 * 8;
+    // per parameter: read master (4) [+ read grad (4) + write master (4)] + write the copy (2 or 4)
+    Scope sc(KC_SGD, 0.0, (double)n * ((grad ? 12.0 : 4.0) + (dt ? 2.0 : 4.0)), s);
     if (dt) sgd_k<bf16><<<blocks, 256, 0, s>>>((float4*)master, (const float4*)grad, (bf16*)copy_next, n4, lr);
     else sgd_k<float><<<blocks, 256, 0, s>>>((float4*)master, (const float4*)grad, (float*)copy_next, n4, lr);
-    COUNT_LAUNCH();
 }
 
 // ------------------------------------------------------------------------------------------
@@ -589,9 +664,9 @@ __global__ void tags_k(TagOps o) {
     // the next weight version replaces a slot only at the end of the step, after the reads above
     if (o.wr_wnext) { o.wr_wnext[0] = -1; o.wr_wnext[1] = o.version_now + 1; }
 }
-void tags_step(const TagOps& ops, cudaStream_t s) { tags_k<<<1, 32, 0, s>>>(ops); COUNT_LAUNCH(); }
+void tags_step(const TagOps& ops, cudaStream_t s) { Scope sc(KC_TAGS, 0.0, 128.0, s); tags_k<<<1, 32, 0, s>>>(ops); }
 
 __global__ void fill_k(float* p, float v, size_t n) { size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; if (i < n) p[i] = v; }
-void fill_f32(float* p, float v, size_t n, cudaStream_t s) { if (!n) return; fill_k<<<cdiv(n, 256), 256, 0, s>>>(p, v, n); COUNT_LAUNCH(); }
+void fill_f32(float* p, float v, size_t n, cudaStream_t s) { if (!n) return; Scope sc(KC_FILL, 0.0, 4.0 * n, s); fill_k<<<cdiv(n, 256), 256, 0, s>>>(p, v, n); }
 
 }  // namespace fdg

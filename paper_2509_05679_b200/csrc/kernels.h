@@ -69,6 +69,24 @@ struct TagOps {
 void tags_step(const TagOps& ops, cudaStream_t st);
 
 void fill_f32(float* p, float v, size_t n, cudaStream_t st);
+void splitk_reduce_launch(const float* partial, float* out, size_t n, int splits, cudaStream_t st);
 uint64_t launches();     // kernels launched so far through this interface
+
+// Kernel classes for launch counting and optional device timing.
+enum KernelClass {
+    KC_FMA_FWD, KC_FMA_DGRAD, KC_FMA_WGRAD, KC_SPLITK, KC_BIAS_GRAD, KC_RELU_FWD, KC_RELU_BWD, KC_ADD_FWD, KC_COPY_ACC,
+    KC_POOL_FWD, KC_POOL_BWD, KC_GAP_FWD, KC_GAP_BWD, KC_BN_FWD_STATS, KC_BN_FWD_APPLY, KC_BN_BWD_REDUCE, KC_BN_BWD_APPLY,
+    KC_SOFTMAX_CE, KC_SGD, KC_TAGS, KC_FILL, KC_TC_FWD, KC_TC_DGRAD, KC_TC_WGRAD, KC_TC_AUX, KC_COUNT
+};
+struct KernelStat { uint64_t launches; double ms, flops, bytes; };
+// Opened around every launch: counts it and, while profiling is enabled, records an event before and
+// after it on the launching stream.  flops / bytes are the launch's ALGORITHMIC work.
+struct Scope {
+    int cls; cudaStream_t st; cudaEvent_t a;
+    Scope(int cls, double flops, double bytes, cudaStream_t s);
+    ~Scope();
+};
+void profile_enable(bool on);                               // on: clears the statistics
+int  profile_read(KernelStat* out, const char** names);     // synchronises the device; returns KC_COUNT
 
 }  // namespace fdg
