@@ -18,6 +18,7 @@
 // at the end of iteration t.
 #include "../../include/fdg.h"
 #include "kernels.h"
+#include "tc_gemm.h"
 
 #include <cmath>
 #include <cstdarg>
@@ -54,6 +55,15 @@ struct Op {
     size_t stats_off;              // byte offset of saved (mean, invstd) inside the stash slot (OP_BN)
     bool acc_in, acc_in2;          // backward accumulates into an already written gradient
     bool need_dgrad;
+    // tensor-core plan (bf16 storage, channel counts that are multiples of 64, power-of-two images)
+    bool tc;
+    int n_tile_f, n_tile_d, n_tile_w, wg_splits;
+    tc::KmParams kf;
+    std::vector<tc::KmParams> kd;                            // one per output-parity class (1 for stride 1, up to 4 for stride 2)
+    bool dgrad_needs_zero;                                   // some parity classes receive no gradient (1x1 stride 2)
+    tc::WgParams kw;
+    std::vector<char*> a_ptrs, dy_ptrs;                      // the buffers the A / dY maps below were built for
+    std::vector<tc::TensorMap> fa, fb, da, db, wx, wdy;      // fwd A, fwd B (per weight slot), dgrad A, dgrad B, wgrad X, wgrad dY
 };
 
 struct Segment { size_t canon, internal, count; bool big; };
@@ -67,7 +77,7 @@ struct Module {
     size_t in_elems;               // per-sample elements of the input / output tensor
     size_t stash_slot_bytes, wslot_bytes, grad_pool_bytes, in_slot_bytes;
     size_t ws_elems, scratch_elems, red_elems;
-    char *in_ring, *stash, *gradpool, *d2, *wring;
+    char *in_ring, *stash, *gradpool, *d2, *wring, *wtring;
     float *master, *grad, *ws, *scratch, *red;
     int64_t *tag_in, *tag_stash, *tag_d2, *tag_w, *trace;
     cudaStream_t stream;
@@ -96,6 +106,8 @@ struct fdg_ctx {
     char* dlogits;
     float* loss_ring;
     int64_t* tags;
+    int* tc_err;                   // device word: set by a tensor-core kernel whose bounded wait gave up
+    bool any_tc;
     cudaEvent_t ingested;
     std::string err;
 };
@@ -149,6 +161,24 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
         o.w_off = seg((size_t)g.R * g.R * g.C * g.Co, true);
         if (bias) o.b_off = seg(cout, false);
         o.out = add_tensor(g.Ho, g.Wo, cout);
+        // tensor-core eligibility
+        int wt, ht, nt;
+        o.tc = ctx->dt == 1 && ctx->kernel_path == 0 && g.C % 64 == 0 && g.Co % 64 == 0 &&
+               tc::pixel_tile(g.Ho, g.Wo, 128, &wt, &ht, &nt) && g.Ho % ht == 0 && 2 * wt <= 256 && tc::init();
+        if (o.tc) {
+            o.n_tile_f = g.Co % 128 == 0 ? 128 : 64;
+            o.n_tile_d = g.C % 128 == 0 ? 128 : 64;
+            o.n_tile_w = g.Co % 256 == 0 ? 256 : (g.Co % 128 == 0 ? 128 : 64);
+            tc::pixel_tile(g.Ho, g.Wo, 64, &wt, &ht, &nt);
+            int row_blocks = g.R * g.R * g.C / 64;
+            long ptiles = (long)(g.Wo / wt) * (g.Ho / ht) * ((g.N + nt - 1) / nt);
+            int tiles = ((row_blocks + 1) / 2) * (g.Co / o.n_tile_w);
+            long want = (2 * 148 + tiles - 1) / tiles;
+            long splits = want < 1 ? 1 : want;
+            if (splits > ptiles) splits = ptiles;
+            long pps = (ptiles + splits - 1) / splits;
+            o.wg_splits = (int)((ptiles + pps - 1) / pps);
+        }
         m.ops.push_back(o);
         return "";
     };
@@ -252,6 +282,7 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
             m.red_elems = std::max(m.red_elems, (size_t)ctx->n_workers * o.g.C * 2);
         }
         if (o.type == OP_CONV) {
+            if (o.tc) m.ws_elems = std::max(m.ws_elems, (size_t)o.wg_splits * o.g.R * o.g.R * o.g.C * o.g.Co);
             m.ws_elems = std::max(m.ws_elems, wgrad_workspace_elems(o.g));
             m.scratch_elems = std::max(m.scratch_elems, (size_t)64 * o.g.Co);
         }
@@ -290,6 +321,56 @@ char* wslot(fdg_ctx* c, Module& m, int64_t version) { return m.wring + (size_t)(
 char* wbig(fdg_ctx* c, Module& m, int64_t version, size_t off) { return wslot(c, m, version) + off * c->esz; }
 float* wsmall(fdg_ctx* c, Module& m, int64_t version, size_t off) { return (float*)(wslot(c, m, version) + m.n_big * c->esz) + off; }
 
+char* wtslot(Module& m, int64_t version, size_t off) { return m.wtring + ((size_t)(version % m.D) * m.n_big + off) * 2; }
+
+int find_buf(const std::vector<char*>& v, const char* p) {
+    for (size_t i = 0; i < v.size(); ++i) if (v[i] == p) return (int)i;
+    return -1;
+}
+
+// forward conv / linear on the tensor cores; false if the buffers are not the ones planned for
+bool tc_forward(fdg_ctx* c, Module& m, const Op& o, char* x, char* y, int64_t version, cudaStream_t s) {
+    int ia = find_buf(o.a_ptrs, x);
+    if (ia < 0) return false;
+    tc::KmParams p = o.kf;
+    p.bias = o.bias ? wsmall(c, m, version, o.b_off) : nullptr;
+    p.out = y; p.epi = o.relu ? EPI_RELU : 0; p.err = c->tc_err;
+    const ConvGeom& g = o.g;
+    double rows = (double)g.N * g.Ho * g.Wo;
+    Scope sc(KC_TC_FWD, 2.0 * rows * g.Co * g.R * g.R * g.C, 2.0 * ((double)g.N * g.H * g.W * g.C + (double)g.Co * g.R * g.R * g.C + rows * g.Co), s);
+    return tc::run_km(o.fa[ia], o.fb[version % m.D], p, o.n_tile_f, s) == cudaSuccess;
+}
+bool tc_dgrad(fdg_ctx* c, Module& m, const Op& o, char* dy, char* dx, int64_t version, bool accum, cudaStream_t s) {
+    int ia = find_buf(o.dy_ptrs, dy);
+    if (ia < 0) return false;
+    const ConvGeom& g = o.g;
+    double rows = (double)g.N * g.H * g.W;
+    if (o.dgrad_needs_zero && !accum) {
+        Scope sc(KC_TC_AUX, 0.0, 2.0 * rows * g.C, s);
+        cudaMemsetAsync(dx, 0, (size_t)rows * g.C * 2, s);
+    }
+    bool ok = true;
+    for (const tc::KmParams& cls : o.kd) {
+        tc::KmParams p = cls;
+        p.bias = nullptr; p.out = dx; p.epi = accum ? EPI_ACCUM : 0; p.err = c->tc_err;
+        double crows = (double)g.N * p.Hd * p.Wd;
+        Scope sc(KC_TC_DGRAD, 2.0 * crows * g.C * p.ntaps * g.Co,
+                 2.0 * ((double)g.N * g.Ho * g.Wo * g.Co + (double)g.Co * p.ntaps * g.C + crows * g.C * (accum ? 2 : 1)), s);
+        ok = ok && tc::run_km(o.da[ia], o.db[version % m.D], p, o.n_tile_d, s) == cudaSuccess;
+    }
+    return ok;
+}
+bool tc_wgrad(fdg_ctx* c, Module& m, const Op& o, char* x, char* dy, float* dw, cudaStream_t s) {
+    int ix = find_buf(o.a_ptrs, x), id = find_buf(o.dy_ptrs, dy);
+    if (ix < 0 || id < 0) return false;
+    tc::WgParams p = o.kw;
+    p.partial = m.ws; p.err = c->tc_err;
+    const ConvGeom& g = o.g;
+    double rows = (double)g.N * g.Ho * g.Wo, R = (double)g.R * g.R * g.C;
+    Scope sc(KC_TC_WGRAD, 2.0 * rows * g.Co * R, 2.0 * ((double)g.N * g.H * g.W * g.C + rows * g.Co) + 4.0 * R * g.Co, s);
+    return tc::run_wg(o.wx[ix], o.wdy[id], p, o.n_tile_w, o.wg_splits, dw, s) == cudaSuccess;
+}
+
 void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version) {
     Module& m = c->mod[kk];
     StepPtrs P{c, &m, kk, batch};
@@ -302,6 +383,7 @@ void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version) {
         switch (o.type) {
             case OP_CONV: {
                 int epi = (o.relu ? EPI_RELU : 0) | (to.loc == LOC_LOGITS ? EPI_OUT_F32 : 0);
+                if (o.tc && tc_forward(c, m, o, P.tensor(o.in), P.tensor(o.out), version, s)) break;
                 conv_forward(dt, P.tensor(o.in), wbig(c, m, version, o.w_off), o.bias ? wsmall(c, m, version, o.b_off) : nullptr,
                              P.tensor(o.out), o.g, epi, s);
                 break; }
@@ -344,9 +426,11 @@ void backward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int64_t
         switch (o.type) {
             case OP_CONV: {
                 if (o.relu) relu_backward(dt, P.tensor(o.out), gout, gout, n_out, false, s);       // in place: dZ = dA * (A > 0)
-                conv_wgrad(dt, P.tensor(o.in), gout, m.grad + o.w_off, m.ws, o.g, s);
+                if (!(o.tc && tc_wgrad(c, m, o, P.tensor(o.in), gout, m.grad + o.w_off, s)))
+                    conv_wgrad(dt, P.tensor(o.in), gout, m.grad + o.w_off, m.ws, o.g, s);
                 if (o.bias) bias_grad(dt, gout, m.grad + m.n_big + o.b_off, m.scratch, (long)o.g.N * o.g.Ho * o.g.Wo, o.g.Co, s);
-                if (gin) conv_dgrad(dt, gout, wbig(c, m, version, o.w_off), gin, o.g, o.acc_in ? EPI_ACCUM : 0, s);
+                if (gin && !(o.tc && tc_dgrad(c, m, o, gout, gin, version, o.acc_in, s)))
+                    conv_dgrad(dt, gout, wbig(c, m, version, o.w_off), gin, o.g, o.acc_in ? EPI_ACCUM : 0, s);
                 break; }
             case OP_BN: {
                 char* gres = o.has_res ? grad_ptr(c, kk, o.in2, t) : nullptr;
@@ -366,6 +450,88 @@ void backward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int64_t
     }
 }
 
+// Emit the transposed (and tap-flipped) copies of weight version `version` that the input-gradient kernel reads.
+void emit_transposed_weights(fdg_ctx* c, Module& m, int64_t version) {
+    for (const Op& o : m.ops)
+        if (o.type == OP_CONV && o.tc) {
+            Scope sc(KC_TC_AUX, 0.0, 4.0 * o.g.R * o.g.R * o.g.C * o.g.Co, m.stream);
+            tc::run_flip_transpose(wbig(c, m, version, o.w_off), wtslot(m, version, o.w_off), o.g.Co, o.g.R * o.g.R, o.g.C, m.stream);
+        }
+}
+
+// Build the TMA tensor maps of every tensor-core op (needs the final device addresses).
+bool build_tc_plans(fdg_ctx* c) {
+    for (int kk = 0; kk < c->K; ++kk) {
+        Module& m = c->mod[kk];
+        for (Op& o : m.ops) {
+            if (o.type != OP_CONV || !o.tc) continue;
+            const ConvGeom& g = o.g;
+            const TensorDesc& ti = m.t[o.in];
+            const TensorDesc& to = m.t[o.out];
+            // where the input activation can live
+            if (ti.loc == LOC_IN) for (int i = 0; i < m.in_depth; ++i) o.a_ptrs.push_back(m.in_ring + (size_t)i * m.in_slot_bytes);
+            else for (int i = 0; i < m.D; ++i) o.a_ptrs.push_back(m.stash + (size_t)i * m.stash_slot_bytes + ti.off);
+            // where the output gradient can live
+            if (to.own_grad) o.dy_ptrs.push_back(m.gradpool + to.goff);
+            else if (to.loc == LOC_NEXT) { Module& n = c->mod[kk + 1]; for (int i = 0; i < 2; ++i) o.dy_ptrs.push_back(n.d2 + (size_t)i * n.in_slot_bytes); }
+            else { o.tc = false; continue; }
+            int wt, ht, nt;
+            const int taps = g.R * g.R, Ktot = taps * g.C;
+            bool ok = true;
+            // ---- forward: A = x (128-pixel boxes), B = W [Co][taps*C]
+            tc::pixel_tile(g.Ho, g.Wo, 128, &wt, &ht, &nt);
+            tc::KmParams& f = o.kf; f = tc::KmParams{};
+            f.Wt = wt; f.Ht = ht; f.Nt = nt; f.tiles_w = g.Wo / wt; f.tiles_h = g.Ho / ht; f.tiles_n = (g.N + nt - 1) / nt;
+            f.ntaps = taps; f.kchunks = g.C / 64; f.xs = g.stride;
+            for (int t = 0; t < taps; ++t) { f.dh[t] = t / g.R - g.pad; f.dw[t] = t % g.R - g.pad; f.koff[t] = t * g.C; }
+            f.N = g.N; f.Hd = g.Ho; f.Wd = g.Wo; f.Ho = g.Ho; f.Wo = g.Wo; f.Co = g.Co; f.os = 1; f.oph = 0; f.opw = 0; f.Cn = g.Co;
+            o.fa.resize(o.a_ptrs.size());
+            for (size_t i = 0; i < o.a_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.fa[i], o.a_ptrs[i], g.C, g.W, g.H, g.N, 64, wt, ht, nt, g.stride);
+            o.fb.resize(m.D);
+            for (int v = 0; v < m.D; ++v) ok = ok && tc::make_map_2d(&o.fb[v], wbig(c, m, v, o.w_off), Ktot, g.Co, 64, o.n_tile_f);
+            // ---- input gradient: dx[n, h, w, :] = sum over taps (r, s) with (h + pad - r), (w + pad - s) divisible by
+            // the stride of dy[n, (h + pad - r) / stride, (w + pad - s) / stride, :] . W[:, r, s, :].
+            // One launch per parity class (h mod stride, w mod stride); the class's pixels form a dense grid of the
+            // size of dy.  A = dy (dense boxes), B = Wt [C][taps * Co] with flipped taps, output strided into dx.
+            o.kd.clear(); o.dgrad_needs_zero = false;
+            for (int ph = 0; ph < g.stride; ++ph) for (int pw = 0; pw < g.stride; ++pw) {
+                tc::KmParams d = f;
+                d.kchunks = g.Co / 64; d.xs = 1; d.ntaps = 0;
+                for (int r = 0; r < g.R; ++r) for (int q = 0; q < g.R; ++q) {
+                    int a = ph + g.pad - r, b = pw + g.pad - q;
+                    if (a % g.stride != 0 || b % g.stride != 0) continue;
+                    d.dh[d.ntaps] = a / g.stride; d.dw[d.ntaps] = b / g.stride;
+                    d.koff[d.ntaps] = (taps - 1 - (r * g.R + q)) * g.Co;
+                    ++d.ntaps;
+                }
+                if (d.ntaps == 0) { o.dgrad_needs_zero = true; continue; }
+                d.Hd = g.H / g.stride; d.Wd = g.W / g.stride; d.Ho = g.H; d.Wo = g.W; d.Co = g.C; d.Cn = g.C;
+                d.os = g.stride; d.oph = ph; d.opw = pw;
+                o.kd.push_back(d);
+            }
+            o.da.resize(o.dy_ptrs.size());
+            for (size_t i = 0; i < o.dy_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.da[i], o.dy_ptrs[i], g.Co, g.Wo, g.Ho, g.N, 64, wt, ht, nt, 1);
+            o.db.resize(m.D);
+            for (int v = 0; v < m.D; ++v) ok = ok && tc::make_map_2d(&o.db[v], wtslot(m, v, o.w_off), (long)taps * g.Co, g.C, 64, o.n_tile_d);
+            // ---- weight gradient: 64-pixel boxes of x (shifted per tap) and of dy
+            tc::pixel_tile(g.Ho, g.Wo, 64, &wt, &ht, &nt);
+            tc::WgParams& w = o.kw; w = tc::WgParams{};
+            w.Wt = wt; w.Ht = ht; w.Nt = nt; w.tiles_w = g.Wo / wt; w.tiles_h = g.Ho / ht; w.tiles_n = (g.N + nt - 1) / nt;
+            w.ptiles = w.tiles_w * w.tiles_h * w.tiles_n;
+            w.ptiles_per_split = (w.ptiles + o.wg_splits - 1) / o.wg_splits;
+            w.kchunks = g.C / 64; w.row_blocks = taps * w.kchunks; w.xs = g.stride; w.Co = g.Co;
+            for (int t = 0; t < taps; ++t) { w.dh[t] = t / g.R - g.pad; w.dw[t] = t % g.R - g.pad; }
+            o.wx.resize(o.a_ptrs.size());
+            for (size_t i = 0; i < o.a_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.wx[i], o.a_ptrs[i], g.C, g.W, g.H, g.N, 64, wt, ht, nt, g.stride);
+            o.wdy.resize(o.dy_ptrs.size());
+            for (size_t i = 0; i < o.dy_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.wdy[i], o.dy_ptrs[i], g.Co, g.Wo, g.Ho, g.N, 64, wt, ht, nt, 1);
+            if (!ok) return false;
+            c->any_tc = true;
+        }
+    }
+    return true;
+}
+
 fdg_status reset_state(fdg_ctx* ctx) {
     // tags: everything -1 (empty); weight slot 0 carries version 0
     size_t n_tags = 0;
@@ -378,8 +544,18 @@ fdg_status reset_state(fdg_ctx* ctx) {
         pos += 2 * (size_t)m.D + 4;
     }
     CK(cudaMemcpy(ctx->tags, h.data(), n_tags * sizeof(int64_t), cudaMemcpyHostToDevice));
+    CK(cudaDeviceSynchronize());
     ctx->t = 0;
     for (Module& m : ctx->mod) m.had_bwd = false;
+    return FDG_OK;
+}
+
+// Reads the device error word (the caller has synchronised the stream it cares about).
+fdg_status check_device_error(fdg_ctx* ctx) {
+    if (!ctx->any_tc) return FDG_OK;
+    int e = 0;
+    CK(cudaMemcpy(&e, ctx->tc_err, sizeof(int), cudaMemcpyDeviceToHost));
+    if (e) return fail(ctx, FDG_ERR_TIMEOUT, "a tensor-core kernel gave up waiting on an mbarrier (code %d)", e);
     return FDG_OK;
 }
 
@@ -445,6 +621,7 @@ fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, boo
         if (m.n_small)
             sgd_update(0, m.master + m.n_big, tau_b >= 0 ? m.grad + m.n_big : nullptr,
                        wsmall(ctx, m, t + 1, 0), m.n_small, ctx->lr, m.stream);
+        emit_transposed_weights(ctx, m, t + 1);
         m.had_bwd = tau_b >= 0;
         CK(cudaEventRecord(m.ev1, m.stream));
         CK(cudaEventRecord(m.done, m.stream));
@@ -453,7 +630,11 @@ fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, boo
     ctx->t = t + 1;
     if (host_loss) {
         CK(cudaStreamSynchronize(ctx->mod[K - 1].stream));
-        CK(cudaMemcpy(host_loss, ctx->loss_ring + (t % 64), sizeof(float), cudaMemcpyDeviceToHost));
+        float l = 0.f;
+        CK(cudaMemcpy(&l, ctx->loss_ring + (t % 64), sizeof(float), cudaMemcpyDeviceToHost));
+        fdg_status es = check_device_error(ctx);
+        if (es != FDG_OK) return es;
+        *host_loss = l;
     }
     return FDG_OK;
 }
@@ -547,6 +728,7 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
     ctx->logits = (float*)get((size_t)ctx->M * ctx->classes * sizeof(float));
     ctx->dlogits = get((size_t)ctx->M * ctx->classes * ctx->esz);
     ctx->loss_ring = (float*)get(64 * sizeof(float));
+    ctx->tc_err = (int*)get(256);
     size_t tpos = 0;
     for (int kk = 0; kk < K && !oom; ++kk) {
         Module& m = ctx->mod[kk];
@@ -555,6 +737,7 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
         m.gradpool = get(m.grad_pool_bytes);
         m.d2 = kk > 0 ? get(2 * m.in_slot_bytes) : nullptr;
         m.wring = get((size_t)m.D * m.wslot_bytes);
+        m.wtring = ctx->dt == 1 ? get((size_t)m.D * m.n_big * 2) : nullptr;
         m.master = (float*)get((m.n_big + m.n_small) * sizeof(float));
         m.grad = (float*)get((m.n_big + m.n_small) * sizeof(float));
         m.ws = (float*)get(m.ws_elems * sizeof(float));
@@ -582,6 +765,9 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
         if (e != cudaSuccess) return bail(FDG_ERR_CUDA, cudaGetErrorString(e));
     }
     if (cudaEventCreateWithFlags(&ctx->ingested, cudaEventDisableTiming) != cudaSuccess) return bail(FDG_ERR_CUDA, "cudaEventCreate failed");
+    if (cudaMemset(ctx->tc_err, 0, 256) != cudaSuccess) return bail(FDG_ERR_CUDA, "cudaMemset failed");
+    ctx->any_tc = false;
+    if (!build_tc_plans(ctx)) return bail(FDG_ERR_CUDA, "cuTensorMapEncodeTiled rejected a tensor map");
     *out = ctx;
     return FDG_OK;
 }
@@ -606,10 +792,14 @@ fdg_status fdg_set_params(fdg_ctx* ctx, const float* host_params, size_t count) 
         std::vector<float> h(m.n_big + m.n_small, 0.f);
         for (const Segment& s : m.segs)
             std::memcpy(h.data() + (s.big ? 0 : m.n_big) + s.internal, host_params + s.canon, s.count * sizeof(float));
-        CK(cudaMemcpy(m.master, h.data(), h.size() * sizeof(float), cudaMemcpyHostToDevice));
+        // in-stream copy, then wait: a plain cudaMemcpy from pageable memory may return before the DMA has
+        // landed, and the module streams are non-blocking streams that do not order behind the default stream
+        CK(cudaMemcpyAsync(m.master, h.data(), h.size() * sizeof(float), cudaMemcpyHostToDevice, m.stream));
+        CK(cudaStreamSynchronize(m.stream));
         // version 0 into weight slot 0
         sgd_update(ctx->dt, m.master, nullptr, wslot(ctx, m, 0), m.n_big, 0.f, m.stream);
         if (m.n_small) sgd_update(0, m.master + m.n_big, nullptr, wsmall(ctx, m, 0, 0), m.n_small, 0.f, m.stream);
+        emit_transposed_weights(ctx, m, 0);
         CK(cudaMemsetAsync(m.grad, 0, (m.n_big + m.n_small) * sizeof(float), m.stream));
     }
     fdg_status s = reset_state(ctx);
@@ -630,6 +820,7 @@ static fdg_status gather(fdg_ctx* ctx, bool grads, float* host_out, size_t capac
     if (!ctx || !host_out) return FDG_ERR_INVALID_ARG;
     if (capacity < ctx->n_params) return fail(ctx, FDG_ERR_INVALID_ARG, "capacity %zu < %zu parameters", capacity, ctx->n_params);
     CK(cudaDeviceSynchronize());
+    { fdg_status es = check_device_error(ctx); if (es != FDG_OK) return es; }
     for (Module& m : ctx->mod) {
         std::vector<float> h(m.n_big + m.n_small, 0.f);
         if (!grads || m.had_bwd) CK(cudaMemcpy(h.data(), grads ? m.grad : m.master, h.size() * sizeof(float), cudaMemcpyDeviceToHost));

@@ -1,0 +1,473 @@
+// Tensor-core kernels for sm_100a: implicit-GEMM convolution / linear layers on tcgen05.mma with
+// accumulators in tensor memory, operands staged in shared memory by TMA (cp.async.bulk.tensor,
+// 128-byte swizzle), a 3-4 stage mbarrier pipeline, and warp-specialised roles:
+//   warp 0 : TMA producer (one elected thread)
+//   warp 1 : tensor-memory allocation, MMA issue (one elected thread), deallocation
+//   warps 2-5 : epilogue (tcgen05.ld -> registers -> global)
+//
+// Two kernels:
+//   km_kernel  (forward and input-gradient): D[pixel][c_out] = sum_{tap, c} A[pixel + tap][c] * B[c_out][tap, c]
+//              A is an NHWC activation read through a 4-D tensor map (one box per filter tap, shifted by
+//              the tap; out-of-bounds elements are zero-filled, which is the padding), B a K-major weight
+//              matrix.  Both operands are K-major in shared memory.
+//   wg_kernel  (weight gradient): D[(tap, c_in)][c_out] = sum_{pixel} X[pixel + tap][c_in] * dY[pixel][c_out]
+//              The contraction runs over pixels = worker x batch x H x W, so the average over workers is
+//              part of the contraction.  Both operands are MN-major in shared memory (channel contiguous).
+//              Split over pixels across CTAs; partial sums are reduced in a fixed order by a second kernel.
+// Every wait on an mbarrier is bounded; a wait that gives up sets an error word and the CTA leaves
+// through the common exit (tensor memory is always released).
+#include "tc_gemm.h"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cstdio>
+#include <cstring>
+
+namespace fdg {
+namespace tc {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int BLOCK_M = 128;      // rows of an accumulator tile (= tensor-memory lanes)
+constexpr int BLOCK_K = 64;       // bf16 elements per 128-byte swizzle row
+constexpr int UMMA_K = 16;
+constexpr int NUM_THREADS = 192;
+constexpr long long WAIT_CYCLES = 4000000000LL;   // ~2 s at 2 GHz
+
+// ------------------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok;
+}
+// Bounded wait: false (and *err set) if the phase did not complete within WAIT_CYCLES.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* err, int code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > WAIT_CYCLES) { atomicCAS(err, 0, code); return false; }
+    }
+    return true;
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* tm, uint64_t* bar, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(tm), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, uint64_t* bar, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(tm), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tm) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t* slot, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulate
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// the mbarrier receives one arrival when all previously issued MMAs of this thread have completed
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns -> 32 registers per thread (thread = lane)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                   "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                   "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
+//   K-major operand  [rows][64 bf16]: 8-row groups are `sbo` bytes apart (1024); lbo unused.
+//   MN-major operand [k rows][64 bf16 of the M/N axis]: groups of 8 k-rows are `sbo` bytes apart (1024),
+//                    consecutive 64-element chunks of the M/N axis are `lbo` bytes apart.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((sbo >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// Instruction descriptor for kind::f16: fp32 accumulator, bf16 A and B, dense.
+__device__ __forceinline__ uint32_t make_idesc(int M, int N, int a_mn_major, int b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+           ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+__device__ __forceinline__ uint8_t* align1024(uint8_t* p) {
+    return (uint8_t*)(((uintptr_t)p + 1023) & ~(uintptr_t)1023);
+}
+
+// ------------------------------------------------------------------------------------------ forward / dgrad
+template <int N_TILE, int STAGES>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, KmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align1024(smem_raw);
+    constexpr int A_BYTES = BLOCK_M * BLOCK_K * 2, B_BYTES = N_TILE * BLOCK_K * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+    uint64_t* full = (uint64_t*)(smem + STAGES * STAGE_BYTES);
+    uint64_t* empty = full + STAGES;
+    uint64_t* accum_bar = empty + STAGES;
+    uint32_t* tmem_slot = (uint32_t*)(accum_bar + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // tile coordinates: blockIdx.x enumerates pixel tiles (w fastest), blockIdx.y output-channel tiles
+    int tm = blockIdx.x;
+    const int tw = tm % p.tiles_w; tm /= p.tiles_w;
+    const int th = tm % p.tiles_h; const int tn = tm / p.tiles_h;
+    const int w0 = tw * p.Wt, h0 = th * p.Ht, n0 = tn * p.Nt;
+    const int co0 = blockIdx.y * N_TILE;
+    const int num_kb = p.ntaps * p.kchunks;
+
+    if (threadIdx.x == 0) {
+        tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB);
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        mbar_init(accum_bar, 1);
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, N_TILE < 32 ? 32 : N_TILE);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % STAGES, it = kb / STAGES;
+                if (it > 0 && !mbar_wait(&empty[s], (it - 1) & 1, p.err, 1)) break;
+                const int tap = kb / p.kchunks, kc = kb - tap * p.kchunks;
+                uint8_t* a = smem + s * STAGE_BYTES;
+                mbar_expect_tx(&full[s], STAGE_BYTES);
+                tma_load_4d(a, &tmA, &full[s], kc * BLOCK_K, w0 * p.xs + p.dw[tap], h0 * p.xs + p.dh[tap], n0);
+                tma_load_2d(a + A_BYTES, &tmB, &full[s], p.koff[tap] + kc * BLOCK_K, co0);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(BLOCK_M, N_TILE, 0, 0);
+            bool ok = true;
+            for (int kb = 0; kb < num_kb && ok; ++kb) {
+                const int s = kb % STAGES, it = kb / STAGES;
+                ok = mbar_wait(&full[s], it & 1, p.err, 2);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a = smem_u32(smem + s * STAGE_BYTES), b = a + A_BYTES;
+#pragma unroll
+                for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                    umma_bf16(tmem_base, make_desc(a + k * UMMA_K * 2, 16, 1024), make_desc(b + k * UMMA_K * 2, 16, 1024), idesc,
+                              (kb | k) != 0);
+                umma_commit(&empty[s]);
+            }
+            umma_commit(accum_bar);           // arrives once every MMA issued above has finished
+        }
+    } else {
+        // ---- epilogue: warp q = warp % 4 owns tensor-memory lanes 32q .. 32q+31 (= tile rows)
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const bool ok = mbar_wait(accum_bar, 0, p.err, 3);
+        tc_fence_after();
+        // row -> pixel of the tile -> output address
+        const int pw = row % p.Wt, ph = (row / p.Wt) % p.Ht, pn = row / (p.Wt * p.Ht);
+        const int n = n0 + pn, h = h0 + ph, w = w0 + pw;
+        const bool valid = ok && n < p.N && h < p.Hd && w < p.Wd;
+        bf16* out = (bf16*)p.out + (((size_t)n * p.Ho + (h * p.os + p.oph)) * p.Wo + (w * p.os + p.opw)) * p.Co + co0;
+#pragma unroll 1
+        for (int c = 0; c < N_TILE; c += 32) {
+            uint32_t v[32];
+            tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + c, v);
+            if (!valid) continue;
+            float f[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v[j]);
+            if (p.bias) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) f[j] += p.bias[co0 + c + j];
+            }
+            if (p.epi & EPI_RELU) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) f[j] = fmaxf(f[j], 0.f);
+            }
+            uint4* o4 = (uint4*)(out + c);
+            if (p.epi & EPI_ACCUM) {
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    uint4 old = o4[g];
+                    const __nv_bfloat162* ob = (const __nv_bfloat162*)&old;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) { float2 t = __bfloat1622float2(ob[j]); f[g * 8 + 2 * j] += t.x; f[g * 8 + 2 * j + 1] += t.y; }
+                }
+            }
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                uint4 pk;
+                __nv_bfloat162 t0 = __floats2bfloat162_rn(f[g * 8 + 0], f[g * 8 + 1]), t1 = __floats2bfloat162_rn(f[g * 8 + 2], f[g * 8 + 3]);
+                __nv_bfloat162 t2 = __floats2bfloat162_rn(f[g * 8 + 4], f[g * 8 + 5]), t3 = __floats2bfloat162_rn(f[g * 8 + 6], f[g * 8 + 7]);
+                pk.x = *(uint32_t*)&t0; pk.y = *(uint32_t*)&t1; pk.z = *(uint32_t*)&t2; pk.w = *(uint32_t*)&t3;
+                o4[g] = pk;
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, N_TILE < 32 ? 32 : N_TILE); }
+}
+
+// ------------------------------------------------------------------------------------------ weight gradient
+// Tile: rows = two 64-row blocks of the (tap, c_in chunk) axis, columns = N_TILE output channels.
+// blockIdx.x = row-block pair, blockIdx.y = column tile, blockIdx.z = pixel split.
+template <int N_TILE, int STAGES>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+wg_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmDY, WgParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align1024(smem_raw);
+    constexpr int BOX_BYTES = 64 * 64 * 2;                 // 64 pixels x 64 channels
+    constexpr int A_BYTES = 2 * BOX_BYTES, B_BYTES = (N_TILE / 64) * BOX_BYTES, STAGE_BYTES = A_BYTES + B_BYTES;
+    uint64_t* full = (uint64_t*)(smem + STAGES * STAGE_BYTES);
+    uint64_t* empty = full + STAGES;
+    uint64_t* accum_bar = empty + STAGES;
+    uint32_t* tmem_slot = (uint32_t*)(accum_bar + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rb0 = blockIdx.x * 2;
+    const int rb1 = min(rb0 + 1, p.row_blocks - 1);       // an odd count: the last tile's upper half repeats a block and is not stored
+    const int co0 = blockIdx.y * N_TILE;
+    const int pt_begin = blockIdx.z * p.ptiles_per_split;
+    const int pt_end = min(p.ptiles, pt_begin + p.ptiles_per_split);
+    const int num_kb = pt_end - pt_begin;
+
+    if (threadIdx.x == 0) {
+        tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmDY);
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        mbar_init(accum_bar, 1);
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, N_TILE < 32 ? 32 : N_TILE);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const int tap0 = rb0 / p.kchunks, cc0 = rb0 - tap0 * p.kchunks;
+            const int tap1 = rb1 / p.kchunks, cc1 = rb1 - tap1 * p.kchunks;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % STAGES, it = kb / STAGES;
+                if (it > 0 && !mbar_wait(&empty[s], (it - 1) & 1, p.err, 4)) break;
+                int pt = pt_begin + kb;
+                const int tw = pt % p.tiles_w; pt /= p.tiles_w;
+                const int th = pt % p.tiles_h; const int tn = pt / p.tiles_h;
+                const int w0 = tw * p.Wt, h0 = th * p.Ht, n0 = tn * p.Nt;
+                uint8_t* a = smem + s * STAGE_BYTES;
+                mbar_expect_tx(&full[s], STAGE_BYTES);
+                tma_load_4d(a, &tmX, &full[s], cc0 * 64, w0 * p.xs + p.dw[tap0], h0 * p.xs + p.dh[tap0], n0);
+                tma_load_4d(a + BOX_BYTES, &tmX, &full[s], cc1 * 64, w0 * p.xs + p.dw[tap1], h0 * p.xs + p.dh[tap1], n0);
+#pragma unroll
+                for (int j = 0; j < N_TILE / 64; ++j)
+                    tma_load_4d(a + A_BYTES + j * BOX_BYTES, &tmDY, &full[s], co0 + j * 64, w0, h0, n0);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(BLOCK_M, N_TILE, 1, 1);
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % STAGES, it = kb / STAGES;
+                if (!mbar_wait(&full[s], it & 1, p.err, 5)) break;
+                tc_fence_after();
+                const uint32_t a = smem_u32(smem + s * STAGE_BYTES), b = a + A_BYTES;
+#pragma unroll
+                for (int k = 0; k < 64 / UMMA_K; ++k)      // 16 pixels = 16 rows of 128 bytes per MMA
+                    umma_bf16(tmem_base, make_desc(a + k * UMMA_K * 128, BOX_BYTES, 1024), make_desc(b + k * UMMA_K * 128, BOX_BYTES, 1024),
+                              idesc, (kb | k) != 0);
+                umma_commit(&empty[s]);
+            }
+            umma_commit(accum_bar);
+        }
+    } else {
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const bool ok = num_kb > 0 ? mbar_wait(accum_bar, 0, p.err, 6) : true;
+        tc_fence_after();
+        const int rb = rb0 + (row >> 6);
+        const bool valid = ok && rb < p.row_blocks;
+        // partial[z][row-block][64][c_out]
+        float* out = p.partial + (((size_t)blockIdx.z * p.row_blocks + rb) * 64 + (row & 63)) * p.Co + co0;
+#pragma unroll 1
+        for (int c = 0; c < N_TILE; c += 32) {
+            uint32_t v[32];
+            if (num_kb > 0) tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + c, v);
+            else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = 0u;
+            }
+            if (!valid) continue;
+            uint4* o4 = (uint4*)(out + c);
+#pragma unroll
+            for (int g = 0; g < 8; ++g) o4[g] = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, N_TILE < 32 ? 32 : N_TILE); }
+}
+
+// dW[co][tap][ci] = sum_z partial[z][(tap, cc)][ci % 64][co], z ascending.  32x32 transposing tiles.
+__global__ void wg_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dw, int splits, int row_blocks, int Co) {
+    __shared__ float t[32][33];
+    const int R = row_blocks * 64;                       // = taps * Cin
+    const int r0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+    const int tx = threadIdx.x, ty = threadIdx.y;        // 32 x 8
+    for (int i = ty; i < 32; i += 8) {
+        float s = 0.f;
+        const size_t o = (size_t)(r0 + i) * Co + c0 + tx;
+        for (int z = 0; z < splits; ++z) s += partial[(size_t)z * R * Co + o];
+        t[i][tx] = s;
+    }
+    __syncthreads();
+    for (int i = ty; i < 32; i += 8) dw[(size_t)(c0 + i) * R + r0 + tx] = t[tx][i];
+}
+
+// Wt[ci][R*R-1-tap][co] = W[co][tap][ci]: the weights of the transposed convolution, K-major for km_kernel.
+__global__ void flip_transpose_kernel(const bf16* __restrict__ w, bf16* __restrict__ wt, int Co, int taps, int Ci) {
+    __shared__ bf16 t[32][34];
+    const int tap = blockIdx.z;
+    const int ci0 = blockIdx.x * 32, co0 = blockIdx.y * 32;
+    const int tx = threadIdx.x, ty = threadIdx.y;
+    for (int i = ty; i < 32; i += 8) t[i][tx] = w[((size_t)(co0 + i) * taps + tap) * Ci + ci0 + tx];
+    __syncthreads();
+    for (int i = ty; i < 32; i += 8) wt[((size_t)(ci0 + i) * taps + (taps - 1 - tap)) * Co + co0 + tx] = t[tx][i];
+}
+
+// ------------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn g_encode = nullptr;
+
+bool init() {
+    if (g_encode) return true;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn) return false;
+    g_encode = (EncodeTiledFn)fn;
+    return true;
+}
+
+bool make_map_4d(TensorMap* out, const void* base, int C, int W, int H, int N, int boxC, int boxW, int boxH, int boxN, int stride) {
+    static_assert(sizeof(TensorMap) == sizeof(CUtensorMap), "tensor map size");
+    if (!init()) return false;
+    cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
+    cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+    cuuint32_t box[4] = {(cuuint32_t)boxC, (cuuint32_t)(boxW * stride), (cuuint32_t)(boxH * stride), (cuuint32_t)boxN};
+    cuuint32_t estr[4] = {1, (cuuint32_t)stride, (cuuint32_t)stride, 1};
+    CUresult r = g_encode((CUtensorMap*)out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+bool make_map_2d(TensorMap* out, const void* base, long inner, long outer, int box_inner, int box_outer) {
+    if (!init()) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+    cuuint64_t strides[1] = {(cuuint64_t)inner * 2};
+    cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode((CUtensorMap*)out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+bool pixel_tile(int H, int W, int pixels, int* Wt, int* Ht, int* Nt) {
+    auto pow2 = [](int v) { return v > 0 && (v & (v - 1)) == 0; };
+    if (!pow2(W) || !pow2(H)) return false;
+    int wt = W < pixels ? W : pixels;
+    int ht = H < pixels / wt ? H : pixels / wt;
+    *Wt = wt; *Ht = ht; *Nt = pixels / (wt * ht);
+    return true;
+}
+
+template <int N_TILE, int STAGES>
+static cudaError_t launch_km(const TensorMap& a, const TensorMap& b, const KmParams& p, dim3 grid, cudaStream_t s) {
+    constexpr int smem = STAGES * (BLOCK_M * BLOCK_K * 2 + N_TILE * BLOCK_K * 2) + 1024 + 256;
+    static bool attr = false;
+    if (!attr) {
+        cudaError_t e = cudaFuncSetAttribute(km_kernel<N_TILE, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        attr = true;
+    }
+    km_kernel<N_TILE, STAGES><<<grid, NUM_THREADS, smem, s>>>(*(const CUtensorMap*)&a, *(const CUtensorMap*)&b, p);
+    return cudaGetLastError();
+}
+
+cudaError_t run_km(const TensorMap& a, const TensorMap& b, const KmParams& p, int n_tile, cudaStream_t s) {
+    dim3 grid(p.tiles_w * p.tiles_h * p.tiles_n, p.Cn / n_tile, 1);
+    if (n_tile == 64) return launch_km<64, 4>(a, b, p, grid, s);
+    if (n_tile == 128) return launch_km<128, 4>(a, b, p, grid, s);
+    return cudaErrorInvalidValue;
+}
+
+template <int N_TILE, int STAGES>
+static cudaError_t launch_wg(const TensorMap& x, const TensorMap& dy, const WgParams& p, dim3 grid, cudaStream_t s) {
+    constexpr int smem = STAGES * (2 + N_TILE / 64) * 8192 + 1024 + 256;
+    static bool attr = false;
+    if (!attr) {
+        cudaError_t e = cudaFuncSetAttribute(wg_kernel<N_TILE, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        attr = true;
+    }
+    wg_kernel<N_TILE, STAGES><<<grid, NUM_THREADS, smem, s>>>(*(const CUtensorMap*)&x, *(const CUtensorMap*)&dy, p);
+    return cudaGetLastError();
+}
+
+cudaError_t run_wg(const TensorMap& x, const TensorMap& dy, const WgParams& p, int n_tile, int splits, float* dw, cudaStream_t s) {
+    dim3 grid((p.row_blocks + 1) / 2, p.Co / n_tile, splits);
+    cudaError_t e;
+    if (n_tile == 64) e = launch_wg<64, 6>(x, dy, p, grid, s);
+    else if (n_tile == 128) e = launch_wg<128, 5>(x, dy, p, grid, s);
+    else if (n_tile == 256) e = launch_wg<256, 4>(x, dy, p, grid, s);
+    else return cudaErrorInvalidValue;
+    if (e != cudaSuccess) return e;
+    dim3 rgrid(p.row_blocks * 2, p.Co / 32), rblk(32, 8);
+    wg_reduce_kernel<<<rgrid, rblk, 0, s>>>(p.partial, dw, splits, p.row_blocks, p.Co);
+    return cudaGetLastError();
+}
+
+cudaError_t run_flip_transpose(const void* w, void* wt, int Co, int taps, int Ci, cudaStream_t s) {
+    dim3 grid(Ci / 32, Co / 32, taps), blk(32, 8);
+    flip_transpose_kernel<<<grid, blk, 0, s>>>((const bf16*)w, (bf16*)wt, Co, taps, Ci);
+    return cudaGetLastError();
+}
+
+}  // namespace tc
+}  // namespace fdg

@@ -1,0 +1,50 @@
+// Launch interface of the tcgen05 / TMA kernels (tc_gemm.cu).  bf16 storage only.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kernels.h"
+
+namespace fdg {
+namespace tc {
+
+struct alignas(64) TensorMap { unsigned char bytes[128]; };     // a CUtensorMap, opaque here
+
+// Forward / input-gradient kernel.  The "tile domain" is the pixel grid the M tiles enumerate
+// (output pixels for forward; for a stride-2 input gradient one parity class of the input pixels).
+struct KmParams {
+    int Wt, Ht, Nt, tiles_w, tiles_h, tiles_n;   // 128-pixel tile = Wt x Ht x Nt, and how many tiles per axis
+    int ntaps, kchunks, xs;                      // filter taps, 64-channel chunks per tap, coordinate scale of the A map
+    int dh[9], dw[9], koff[9];                   // per tap: spatial shift of the A box, column offset into B
+    int N, Hd, Wd;                               // extents of the tile domain (rows outside are not stored)
+    int Ho, Wo, Co, os, oph, opw;                // output tensor [N,Ho,Wo,Co]; domain pixel (h,w) -> (h*os+oph, w*os+opw)
+    int Cn;                                      // output channels computed (multiple of the column tile)
+    int epi;                                     // EPI_RELU | EPI_ACCUM
+    const float* bias;                           // or nullptr
+    void* out;
+    int* err;                                    // device word, set non-zero if a bounded wait gave up
+};
+
+struct WgParams {
+    int Wt, Ht, Nt, tiles_w, tiles_h, tiles_n;   // 64-pixel tile of the dY pixel grid
+    int ptiles, ptiles_per_split;
+    int kchunks, row_blocks, xs;                 // 64-channel chunks of c_in; row blocks = taps * kchunks
+    int dh[9], dw[9];
+    int Co;
+    float* partial;                              // [splits][row_blocks * 64][Co]
+    int* err;
+};
+
+bool init();     // resolves the driver's tensor-map encoder; false if unavailable
+// NHWC bf16 tensor [N,H,W,C]; box = boxC channels x (boxW x boxH x boxN) pixels; stride 2 samples every other pixel
+bool make_map_4d(TensorMap* out, const void* base, int C, int W, int H, int N, int boxC, int boxW, int boxH, int boxN, int stride);
+bool make_map_2d(TensorMap* out, const void* base, long inner, long outer, int box_inner, int box_outer);
+// Wt x Ht x Nt = pixels, Wt = min(W, pixels) ...; false unless H and W are powers of two
+bool pixel_tile(int H, int W, int pixels, int* Wt, int* Ht, int* Nt);
+
+cudaError_t run_km(const TensorMap& a, const TensorMap& b, const KmParams& p, int n_tile, cudaStream_t s);
+cudaError_t run_wg(const TensorMap& x, const TensorMap& dy, const WgParams& p, int n_tile, int splits, float* dw, cudaStream_t s);
+cudaError_t run_flip_transpose(const void* w, void* wt, int Co, int taps, int Ci, cudaStream_t s);
+
+}  // namespace tc
+}  // namespace fdg

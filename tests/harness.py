@@ -78,6 +78,10 @@ def pick_data_stream(orc, net: sy.Net, p0, steps: int, guard: float, tries: int 
     raise AssertionError("no data stream keeps every pre-activation away from the kinks")
 
 
+def module_bounds(net):
+    return [0] + list(net.splits) + [len(net.layers)]
+
+
 def closed_form_trace(K, t):
     f = np.array([t - k + 1 if t - k + 1 >= 0 else -1 for k in range(1, K + 1)])
     b = np.array([t - 2 * K + k + 1 if t - 2 * K + k + 1 >= 0 else -1 for k in range(1, K + 1)])
@@ -86,7 +90,7 @@ def closed_form_trace(K, t):
 
 
 def run_parity(orc, net: sy.Net, steps: int, *, param_tol=None, grad_tol=None, grad_best_tol=None, loss_tol=None,
-               perturb=True, kink_guard=None, grad_steps=None, grad_tail=None, **ctx_kw):
+               perturb=True, kink_guard=None, grad_steps=None, grad_tail=None, grad_tol_later=None, **ctx_kw):
     """Step both implementations `steps` times; check the schedule bit-exactly after every step and
     parameters / gradients / loss within the given tolerances.  Returns the per-step records.
 
@@ -98,7 +102,9 @@ def run_parity(orc, net: sy.Net, steps: int, *, param_tol=None, grad_tol=None, g
     moved apart and a gradient comparison compares different weights).  `grad_tail`: hold only the
     last `grad_tail` tensors to `grad_tol` and ask the whole gradient for a cosine similarity of 0.7
     (deep batch-norm networks amplify a single rounding difference by orders of magnitude on the
-    way back to the first layers)."""
+    way back to the first layers).  `grad_tol_later`: tolerance after the run's first backward pass
+    (t = K-1, held to `grad_tol`): from then on the weights of the two runs differ by their
+    earlier gradient differences."""
     from paper_2509_05679_b200 import binding
     bf16 = net.dtype == "bf16"
     p0 = sy.init_params(net.layers, 0, bf16=False)
@@ -132,8 +138,11 @@ def run_parity(orc, net: sy.Net, steps: int, *, param_tol=None, grad_tol=None, g
                 r["grad_err"], r["grad_where"], per = grad_rel_l2(g_gpu, g_avg, net.layers)
                 for k_, e_ in per.items():
                     best[k_] = min(best.get(k_, np.inf), e_)
-                if grad_tail is None:
+                if grad_tail is None and grad_tol_later is None:
                     assert r["grad_err"] <= grad_tol, (t, r)
+                elif grad_tail is None:
+                    first = t == net.K - 1          # the first backward pass of the run: no weight has changed yet
+                    assert r["grad_err"] <= (grad_tol if first else grad_tol_later), (t, r)
                 elif per:
                     tail = list(per.items())[-grad_tail:]
                     assert all(e_ <= grad_tol for _, e_ in tail), (t, tail)
