@@ -174,6 +174,35 @@ typedef struct { char name[48]; uint64_t launches; double ms, flops, bytes; } fd
 FDG_API fdg_status fdg_profile(fdg_ctx* ctx, int32_t enable);
 FDG_API fdg_status fdg_profile_read(fdg_ctx* ctx, fdg_kernel_stat* out, int32_t capacity, int32_t* count);
 
+/* Bias gradient without any allocation.  (The paper has no counterpart: this is a service entry
+ * point, not a step of its method.)
+ *
+ * For whom: code that must not allocate device memory while it runs -- a plug-in living inside
+ * another framework's memory pool, a latency-critical loop that forbids cudaMalloc/cudaFree because
+ * they synchronise the whole device, a process whose memory budget was handed out up front.  Such a
+ * caller cannot create an fdg_ctx (which allocates its FIFOs), yet may still need the reduction the
+ * step uses for bias gradients:  dev_db[c] = sum over rows of dev_dy[row][c].
+ *
+ *   dev_dy  : device, [rows][channels] row-major, fp32 (dtype 0) or bf16 (dtype 1)
+ *   dev_db  : device, fp32 [channels], overwritten
+ *   stream  : a cudaStream_t (NULL = default stream); the call only enqueues two kernels
+ * Limits and behaviour
+ *   - channels <= FDG_STATIC_MAX_CHANNELS, rows >= 1; anything else returns FDG_ERR_INVALID_ARG and
+ *     fdg_static_last_error() says why.  Nothing is launched in that case.
+ *   - The partial sums go to a fixed 1 MiB array inside the library image (present on every GPU
+ *     that loads the library, for the life of the process).  The entry point calls no cudaMalloc,
+ *     cudaFree or any allocating routine.
+ *   - All calls on a device share that array.  It keeps the previous call's contents; nothing in it
+ *     has to start at zero, because the first kernel writes every slot the second one reads.  Two
+ *     calls that may overlap on the GPU (different streams, no ordering) race on it: order them.
+ *   - The first call on each device looks the array's device address up (cudaGetSymbolAddress, with
+ *     that device current).  Make that first call before starting any stream capture.
+ *   - Same summation order on every call, so equal inputs give equal bits. */
+#define FDG_STATIC_MAX_CHANNELS 4096
+FDG_API fdg_status fdg_bias_grad_static(const void* dev_dy, int32_t dtype, int64_t rows, int32_t channels,
+                                        float* dev_db, void* stream);
+FDG_API const char* fdg_static_last_error(void);
+
 FDG_API const char* fdg_last_error(const fdg_ctx* ctx);   /* ctx may be NULL: last create error */
 FDG_API void        fdg_destroy(fdg_ctx* ctx);
 

@@ -21,6 +21,7 @@ STATUS = {0: "FDG_OK", 1: "FDG_ERR_INVALID_ARG", 2: "FDG_ERR_BAD_SPLIT", 3: "FDG
 
 EXPORTS = ["fdg_create", "fdg_param_count", "fdg_set_params", "fdg_step", "fdg_step_host", "fdg_wait_ingest", "fdg_params",
            "fdg_grads", "fdg_trace", "fdg_set_lr", "fdg_stats", "fdg_module_times", "fdg_profile", "fdg_profile_read",
+           "fdg_bias_grad_static", "fdg_static_last_error",
            "fdg_last_error", "fdg_destroy"]
 
 
@@ -90,6 +91,10 @@ def lib():
         L.fdg_profile.argtypes = [vp, C.c_int32]
         L.fdg_profile_read.restype = C.c_int
         L.fdg_profile_read.argtypes = [vp, C.POINTER(fdg_kernel_stat), C.c_int32, C.POINTER(C.c_int32)]
+        L.fdg_bias_grad_static.restype = C.c_int
+        L.fdg_bias_grad_static.argtypes = [vp, C.c_int32, C.c_int64, C.c_int32, vp, vp]
+        L.fdg_static_last_error.restype = C.c_char_p
+        L.fdg_static_last_error.argtypes = []
         L.fdg_last_error.restype = C.c_char_p
         L.fdg_last_error.argtypes = [vp]
         L.fdg_destroy.restype = None
@@ -241,6 +246,15 @@ class Context:
         ms = np.empty(self.K, dtype=np.float32)
         self._ck(lib().fdg_module_times(self.h, ms.ctypes.data_as(C.POINTER(C.c_float)), self.K))
         return ms
+
+
+def bias_grad_static(dev_dy, dtype: str, rows: int, channels: int, dev_db, stream: int = 0) -> None:
+    """dev_db[c] = sum_rows dev_dy[row][c] through fdg_bias_grad_static: no device memory is allocated
+    by the call (its scratch is a fixed array inside the library).  Arguments are device tensors /
+    addresses owned by the caller; raises FdgError with the library's message on a rejected call."""
+    st = lib().fdg_bias_grad_static(_ptr(dev_dy), {"fp32": 0, "bf16": 1}[dtype], int(rows), int(channels), _ptr(dev_db), stream or None)
+    if st != 0:
+        raise FdgError(st, (lib().fdg_static_last_error() or b"").decode())
 
 
 def to_device(net_dtype: str, x: np.ndarray):
