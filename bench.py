@@ -123,6 +123,7 @@ def main():
     ap.add_argument("--kernel-path", type=int, default=0, help="0: tensor-core kernels where shapes allow, 1: plain FMA kernels only")
     ap.add_argument("--batch", type=int, default=None, help="per-worker batch override (testing only; changes the workload name)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--serial", action="store_true", help="diagnosis: all modules on one stream (uncontended per-kernel times)")
     args = ap.parse_args()
 
     net = sy.config(args.config, batch=args.batch)
@@ -148,7 +149,7 @@ def main():
     streams = [torch.cuda.Stream() for _ in range(net.K)]
     ctx = binding.Context(net.layers, net.splits, net.n_workers, net.batch, net.lr, dtype=net.dtype,
                           in_shape=(net.in_h, net.in_w, net.in_c), num_classes=net.classes, device=local,
-                          kernel_path=args.kernel_path, streams=[s.cuda_stream for s in streams])
+                          kernel_path=args.kernel_path, streams=[s.cuda_stream for s in streams], serial=args.serial)
     ctx.set_params(sy.init_params(net.layers, 0, bf16=net.dtype == "bf16"))
 
     # a pool of distinct batches, resident in HBM (device arm) and in pinned host memory (e2e arm)
@@ -198,7 +199,9 @@ def main():
     barrier()
     ms = start.elapsed_time(end)
     ctx.profile(False)
-    kstats = ctx.profile_read()
+    kall = ctx.profile_read()
+    kstats = {k: v for k, v in kall.items() if "[" not in k}
+    kshapes = {k: v for k, v in kall.items() if "[" in k}
     clocks = sampler.stop()
     _, launches1 = ctx.stats()
     mod_ms = [float(v) for v in ctx.module_times()]
@@ -250,14 +253,20 @@ def main():
             "config": {"workload": net.name + ("" if args.batch is None else f"-B{args.batch}"), "K": net.K, "n_workers": net.n_workers,
                        "per_worker_batch": net.batch, "M": net.M, "lr": net.lr, "pipeline_fill_steps": fill,
                        "l2": "inputs rotate over 4 batches; each step streams the multi-GB activation stash, far larger than L2",
-                       "multi_gpu": "independent replicas (no exchange between GPUs)", "kernel_path": args.kernel_path},
+                       "multi_gpu": "independent replicas (no exchange between GPUs)", "kernel_path": args.kernel_path, "serial": bool(args.serial)},
             "clocks": clocks,
             "step_tensor_roofline": {"flop_per_step": flops_step, "tflops_achieved": flops_step / (ms / args.steps * 1e-3) / 1e12 * 1.0,
                                      "frac_of_burst_peak": flops_step / (ms / args.steps * 1e-3) / 1e12 / pk["tensor_burst"],
                                      "frac_of_sustained_peak": flops_step / (ms / args.steps * 1e-3) / 1e12 / pk["tensor"],
                                      "peak_source": pk["source"]},
             "roofline": roof,
-            "kernels": {k: {"launches": v["launches"], "ms": round(v["ms"], 4)} for k, v in sorted(kstats.items(), key=lambda kv: -kv[1]["ms"])},
+            "kernels": {k: {"launches": v["launches"], "ms": round(v["ms"], 4),
+                            "tflops": round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 2) if v["ms"] > 0 else None,
+                            "gbs": round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1) if v["ms"] > 0 else None}
+                        for k, v in sorted(kstats.items(), key=lambda kv: -kv[1]["ms"])},
+            "kernel_shapes": {k: {"launches": v["launches"], "ms": round(v["ms"], 4),
+                                  "tflops": round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 1) if v["ms"] > 0 else None}
+                              for k, v in sorted(kshapes.items(), key=lambda kv: -kv[1]["ms"])},
             "module_ms_last_step": mod_ms,
             "gpu_launches": int(launches1 - launches0),
             "e2e": {"value": total_samples / e2e_s, "unit": UNIT,

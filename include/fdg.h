@@ -169,7 +169,8 @@ FDG_API fdg_status fdg_module_times(fdg_ctx* ctx, float* ms, int32_t K);
  * makes every later launch record a CUDA event before and after itself on its own stream;
  * fdg_profile(ctx, 0) stops that.  fdg_profile_read waits for the device and returns one record
  * per kernel class that was launched: its launches, the summed event time (ms) and the summed
- * ALGORITHMIC flops and bytes of those launches.  The statistics are process-wide. */
+ * ALGORITHMIC flops and bytes of those launches, followed by records named "class[layer shape]"
+ * that break the GEMM / convolution classes down by layer shape.  The statistics are process-wide. */
 typedef struct { char name[48]; uint64_t launches; double ms, flops, bytes; } fdg_kernel_stat;
 FDG_API fdg_status fdg_profile(fdg_ctx* ctx, int32_t enable);
 FDG_API fdg_status fdg_profile_read(fdg_ctx* ctx, fdg_kernel_stat* out, int32_t capacity, int32_t* count);

@@ -236,9 +236,9 @@ class Context:
 
     def profile_read(self):
         """{kernel class: dict(launches, ms, flops, bytes)} since profile(True)."""
-        arr = (fdg_kernel_stat * 64)()
+        arr = (fdg_kernel_stat * 256)()
         n = C.c_int32()
-        self._ck(lib().fdg_profile_read(self.h, arr, 64, C.byref(n)))
+        self._ck(lib().fdg_profile_read(self.h, arr, 256, C.byref(n)))
         return {arr[i].name.decode(): dict(launches=int(arr[i].launches), ms=arr[i].ms, flops=arr[i].flops, bytes=arr[i].bytes)
                 for i in range(n.value)}
 

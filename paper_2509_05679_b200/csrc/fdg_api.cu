@@ -57,6 +57,7 @@ struct Op {
     bool need_dgrad;
     // tensor-core plan (bf16 storage, channel counts that are multiples of 64, power-of-two images)
     bool tc;
+    char shape[40];                                          // "HxW Cin->Cout kR sS", the profiler's detail tag
     int n_tile_f, n_tile_d, n_tile_w, wg_splits;
     tc::KmParams kf;
     std::vector<tc::KmParams> kd;                            // one per output-parity class (1 for stride 1, up to 4 for stride 2)
@@ -161,6 +162,7 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
         o.w_off = seg((size_t)g.R * g.R * g.C * g.Co, true);
         if (bias) o.b_off = seg(cout, false);
         o.out = add_tensor(g.Ho, g.Wo, cout);
+        std::snprintf(o.shape, sizeof o.shape, "%dx%d %d->%d k%d s%d", g.H, g.W, g.C, g.Co, g.R, g.stride);
         // tensor-core eligibility
         int wt, ht, nt;
         o.tc = ctx->dt == 1 && ctx->kernel_path == 0 && g.C % 64 == 0 && g.Co % 64 == 0 &&
@@ -278,7 +280,7 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
     for (Op& o : m.ops) {
         if (o.type == OP_BN) {
             o.stats_off = soff; soff += align_up((size_t)ctx->n_workers * o.g.C * 2 * sizeof(float), 256);
-            m.scratch_elems = std::max(m.scratch_elems, (size_t)64 * ctx->n_workers * o.g.C * 2);
+            m.scratch_elems = std::max(m.scratch_elems, (size_t)128 * ctx->n_workers * o.g.C * 2);
             m.red_elems = std::max(m.red_elems, (size_t)ctx->n_workers * o.g.C * 2);
         }
         if (o.type == OP_CONV) {
@@ -383,9 +385,11 @@ void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version) {
         switch (o.type) {
             case OP_CONV: {
                 int epi = (o.relu ? EPI_RELU : 0) | (to.loc == LOC_LOGITS ? EPI_OUT_F32 : 0);
-                if (o.tc && tc_forward(c, m, o, P.tensor(o.in), P.tensor(o.out), version, s)) break;
+                profile_detail(o.shape);
+                if (o.tc && tc_forward(c, m, o, P.tensor(o.in), P.tensor(o.out), version, s)) { profile_detail(nullptr); break; }
                 conv_forward(dt, P.tensor(o.in), wbig(c, m, version, o.w_off), o.bias ? wsmall(c, m, version, o.b_off) : nullptr,
                              P.tensor(o.out), o.g, epi, s);
+                profile_detail(nullptr);
                 break; }
             case OP_BN:
                 bn_forward(dt, P.tensor(o.in), wsmall(c, m, version, o.gamma_off), wsmall(c, m, version, o.beta_off),
@@ -426,17 +430,19 @@ void backward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int64_t
         switch (o.type) {
             case OP_CONV: {
                 if (o.relu) relu_backward(dt, P.tensor(o.out), gout, gout, n_out, false, s);       // in place: dZ = dA * (A > 0)
+                profile_detail(o.shape);
                 if (!(o.tc && tc_wgrad(c, m, o, P.tensor(o.in), gout, m.grad + o.w_off, s)))
                     conv_wgrad(dt, P.tensor(o.in), gout, m.grad + o.w_off, m.ws, o.g, s);
                 if (o.bias) bias_grad(dt, gout, m.grad + m.n_big + o.b_off, m.scratch, (long)o.g.N * o.g.Ho * o.g.Wo, o.g.Co, s);
                 if (gin && !(o.tc && tc_dgrad(c, m, o, gout, gin, version, o.acc_in, s)))
                     conv_dgrad(dt, gout, wbig(c, m, version, o.w_off), gin, o.g, o.acc_in ? EPI_ACCUM : 0, s);
+                profile_detail(nullptr);
                 break; }
             case OP_BN: {
                 char* gres = o.has_res ? grad_ptr(c, kk, o.in2, t) : nullptr;
-                bn_backward(dt, P.tensor(o.in), P.tensor(o.out), gout, wsmall(c, m, version, o.gamma_off), P.stats(o),
-                            gin, o.acc_in, gres, o.acc_in2, m.grad + m.n_big + o.gamma_off, m.grad + m.n_big + o.beta_off,
-                            m.red, m.scratch, c->n_workers, (long)c->B * ti.h * ti.w, ti.c, o.relu, s);
+                bn_backward(dt, P.tensor(o.in), P.tensor(o.out), gout, wsmall(c, m, version, o.gamma_off), wsmall(c, m, version, o.beta_off),
+                            P.stats(o), gin, o.acc_in, gres, o.acc_in2, m.grad + m.n_big + o.gamma_off, m.grad + m.n_big + o.beta_off,
+                            m.red, m.scratch, c->n_workers, (long)c->B * ti.h * ti.w, ti.c, o.relu, o.has_res, s);
                 break; }
             case OP_RELU: if (gin) relu_backward(dt, P.tensor(o.out), gout, gin, n_out, o.acc_in, s); break;
             case OP_POOL: if (gin) maxpool_backward(dt, P.tensor(o.in), gout, gin, c->M, ti.h, ti.w, ti.c, o.acc_in, s); break;
@@ -874,6 +880,15 @@ fdg_status fdg_profile_read(fdg_ctx* ctx, fdg_kernel_stat* out, int32_t capacity
         std::memset(&out[w], 0, sizeof out[w]);
         std::strncpy(out[w].name, names[i], sizeof(out[w].name) - 1);
         out[w].launches = st[i].launches; out[w].ms = st[i].ms; out[w].flops = st[i].flops; out[w].bytes = st[i].bytes;
+        ++w;
+    }
+    // then the per-shape breakdown of the classes that carry a detail tag
+    static KernelStat ds[192]; static char dn[192][48];
+    int nd = profile_read_detail(ds, dn, 192);
+    for (int i = 0; i < nd && w < capacity; ++i) {
+        std::memset(&out[w], 0, sizeof out[w]);
+        std::strncpy(out[w].name, dn[i], sizeof(out[w].name) - 1);
+        out[w].launches = ds[i].launches; out[w].ms = ds[i].ms; out[w].flops = ds[i].flops; out[w].bytes = ds[i].bytes;
         ++w;
     }
     *count = w;

@@ -6,7 +6,10 @@
 
 #include <cuda_bf16.h>
 #include <atomic>
+#include <cstdio>
+#include <map>
 #include <mutex>
+#include <string>
 #include <vector>
 
 namespace fdg {
@@ -27,16 +30,25 @@ static std::mutex g_mu;
 static std::vector<Rec> g_recs;
 static std::vector<cudaEvent_t> g_pool;
 static KernelStat g_stat[KC_COUNT];
+static std::map<std::string, KernelStat> g_detail;          // "class[detail]" -> statistics
+static thread_local const char* t_detail = nullptr;
+struct DRec { std::string key; cudaEvent_t a, b; };
+static std::vector<DRec> g_drecs;
 static cudaEvent_t get_event() {
     if (!g_pool.empty()) { cudaEvent_t e = g_pool.back(); g_pool.pop_back(); return e; }
     cudaEvent_t e = nullptr; cudaEventCreate(&e); return e;
 }
 }  // namespace prof
-Scope::Scope(int cls_, double flops, double bytes, cudaStream_t s) : cls(cls_), st(s), a(nullptr) {
+void profile_detail(const char* d) { prof::t_detail = d; }
+Scope::Scope(int cls_, double flops, double bytes, cudaStream_t s) : cls(cls_), st(s), a(nullptr), detail(prof::t_detail) {
     g_launches.fetch_add(1, std::memory_order_relaxed);
     if (!prof::g_on) return;
     std::lock_guard<std::mutex> lk(prof::g_mu);
     prof::g_stat[cls].launches += 1; prof::g_stat[cls].flops += flops; prof::g_stat[cls].bytes += bytes;
+    if (detail) {
+        KernelStat& d = prof::g_detail[std::string(kClassNames[cls]) + "[" + detail + "]"];
+        d.launches += 1; d.flops += flops; d.bytes += bytes;
+    }
     a = prof::get_event();
     cudaEventRecord(a, st);
 }
@@ -46,15 +58,21 @@ Scope::~Scope() {
     cudaEvent_t b = prof::get_event();
     cudaEventRecord(b, st);
     prof::g_recs.push_back({cls, a, b});
+    if (detail) prof::g_drecs.push_back({std::string(kClassNames[cls]) + "[" + detail + "]", a, b});
 }
 void profile_enable(bool on) {
     std::lock_guard<std::mutex> lk(prof::g_mu);
-    if (on) for (auto& k : prof::g_stat) k = KernelStat{};
+    if (on) { for (auto& k : prof::g_stat) k = KernelStat{}; prof::g_detail.clear(); }
     prof::g_on = on;
 }
 int profile_read(KernelStat* out, const char** names) {
     cudaDeviceSynchronize();
     std::lock_guard<std::mutex> lk(prof::g_mu);
+    for (auto& r : prof::g_drecs) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess) prof::g_detail[r.key].ms += ms;
+    }
+    prof::g_drecs.clear();
     for (auto& r : prof::g_recs) {
         float ms = 0.f;
         if (cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess) prof::g_stat[r.cls].ms += ms;
@@ -63,6 +81,17 @@ int profile_read(KernelStat* out, const char** names) {
     prof::g_recs.clear();
     for (int i = 0; i < KC_COUNT; ++i) { out[i] = prof::g_stat[i]; names[i] = kClassNames[i]; }
     return KC_COUNT;
+}
+int profile_read_detail(KernelStat* out, char (*names)[48], int capacity) {
+    std::lock_guard<std::mutex> lk(prof::g_mu);
+    int n = 0;
+    for (auto& kv : prof::g_detail) {
+        if (n >= capacity) break;
+        out[n] = kv.second;
+        std::snprintf(names[n], 48, "%s", kv.first.c_str());
+        ++n;
+    }
+    return n;
 }
 
 typedef __nv_bfloat16 bf16;
@@ -543,8 +572,236 @@ __global__ void bn_bwd_apply_k(const T* __restrict__ x, const T* __restrict__ ou
     if (dres) { float r = dy; if (accum_dres) r += ld(dres + i); st(dres + i, r); }
 }
 
+// ------------------------------------------------------------------------------------------
+// batch-norm, bf16 storage, 128-bit accesses: a thread owns 8 consecutive channels and walks down
+// the rows of one worker, four rows in flight; grid = (row chunks, workers).  Used when C/8 is a
+// power of two <= 256.
+// ------------------------------------------------------------------------------------------
+constexpr int BNV_THREADS = 256;
+constexpr int BNV_MAX_CHUNKS = 128;
+constexpr int BNV_UNROLL = 4;
+
+__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
+    const __nv_bfloat162* h = (const __nv_bfloat162*)&v;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { float2 t = __bfloat1622float2(h[j]); f[2 * j] = t.x; f[2 * j + 1] = t.y; }
+}
+__device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
+    uint4 v; __nv_bfloat162* h = (__nv_bfloat162*)&v;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) h[j] = __floats2bfloat162_rn(f[2 * j], f[2 * j + 1]);
+    return v;
+}
+__device__ __forceinline__ uint4 ldg16(const bf16* p) { return __ldg((const uint4*)p); }
+// the one expression both passes use for the normalised value, so that the backward pass can
+// recompute the sign of the forward output from x alone
+__device__ __forceinline__ float bn_value(float x, float mean, float istd, float g, float b) {
+    return __fmaf_rn(g, (x - mean) * istd, b);
+}
+
+// MODE 0: (sum x, sum x^2).  MODE 1: (sum dy, sum dy * xhat) with dy = dout * [forward output > 0] if relu.
+// mask_from_x: the forward output had no residual, so its sign is the sign of bn_value(x).
+template <int MODE>
+__global__ void __launch_bounds__(BNV_THREADS) bnv_reduce(const bf16* __restrict__ x, const bf16* __restrict__ out,
+                                                          const bf16* __restrict__ dout, const float* __restrict__ gamma,
+                                                          const float* __restrict__ beta, const float* __restrict__ stats,
+                                                          float* __restrict__ part, long rpw, int C, int relu, int mask_from_x) {
+    __shared__ float sh[BNV_THREADS][17];
+    const int cgs = C >> 3, rows_it = BNV_THREADS / cgs;
+    const int cg = threadIdx.x % cgs, r = threadIdx.x / cgs;
+    const int w = blockIdx.y, nw = gridDim.y;
+    const long per = (rpw + gridDim.x - 1) / gridDim.x;
+    const long r0 = (long)blockIdx.x * per, r1 = min(rpw, r0 + per);
+    float s1[8], s2[8], mean[8], istd[8], g[8], b[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        s1[j] = 0.f; s2[j] = 0.f;
+        if (MODE == 1) {
+            const int c = cg * 8 + j;
+            mean[j] = stats[((size_t)w * C + c) * 2]; istd[j] = stats[((size_t)w * C + c) * 2 + 1];
+            g[j] = gamma[c]; b[j] = beta[c];
+        }
+    }
+    const size_t base = (size_t)w * rpw * C + (size_t)cg * 8;
+    const bool need_out = MODE == 1 && relu && !mask_from_x;
+    for (long row = r0 + r; row < r1; row += (long)rows_it * BNV_UNROLL) {
+        uint4 xr[BNV_UNROLL], dr[BNV_UNROLL], orr[BNV_UNROLL];
+#pragma unroll
+        for (int u = 0; u < BNV_UNROLL; ++u) {
+            const long rr = row + (long)u * rows_it;
+            if (rr < r1) {
+                const size_t o = base + (size_t)rr * C;
+                xr[u] = ldg16(x + o);
+                if (MODE == 1) dr[u] = ldg16(dout + o);
+                if (need_out) orr[u] = ldg16(out + o);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < BNV_UNROLL; ++u) {
+            if (row + (long)u * rows_it >= r1) break;
+            float xv[8];
+            unpack8(xr[u], xv);
+            if (MODE == 0) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { s1[j] += xv[j]; s2[j] = fmaf(xv[j], xv[j], s2[j]); }
+            } else {
+                float dv[8], ov[8];
+                unpack8(dr[u], dv);
+                if (need_out) unpack8(orr[u], ov);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    float dy = dv[j];
+                    if (relu) { float f = mask_from_x ? bn_value(xv[j], mean[j], istd[j], g[j], b[j]) : ov[j]; if (!(f > 0.f)) dy = 0.f; }
+                    s1[j] += dy; s2[j] = fmaf(dy, (xv[j] - mean[j]) * istd[j], s2[j]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { sh[threadIdx.x][j] = s1[j]; sh[threadIdx.x][8 + j] = s2[j]; }
+    __syncthreads();
+    // thread t < 16 * cgs sums one (channel group, value) column over the rows_it row lanes, in a fixed order
+    for (int t = threadIdx.x; t < cgs * 16; t += BNV_THREADS) {
+        const int q = t >> 4, k = t & 15;
+        float acc = 0.f;
+        for (int rr = 0; rr < rows_it; ++rr) acc += sh[rr * cgs + q][k];
+        const int c = q * 8 + (k & 7);
+        part[(((size_t)blockIdx.x * nw + w) * C + c) * 2 + (k >> 3)] = acc;
+    }
+}
+
+__global__ void __launch_bounds__(BNV_THREADS) bnv_apply(const bf16* __restrict__ x, const float* __restrict__ gamma,
+                                                         const float* __restrict__ beta, const bf16* __restrict__ res,
+                                                         bf16* __restrict__ y, const float* __restrict__ stats, long rpw, int C, int relu) {
+    const int cgs = C >> 3, rows_it = BNV_THREADS / cgs;
+    const int cg = threadIdx.x % cgs, r = threadIdx.x / cgs;
+    const int w = blockIdx.y;
+    const long per = (rpw + gridDim.x - 1) / gridDim.x;
+    const long r0 = (long)blockIdx.x * per, r1 = min(rpw, r0 + per);
+    float mean[8], istd[8], g[8], b[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int c = cg * 8 + j;
+        mean[j] = stats[((size_t)w * C + c) * 2]; istd[j] = stats[((size_t)w * C + c) * 2 + 1];
+        g[j] = gamma[c]; b[j] = beta[c];
+    }
+    const size_t base = (size_t)w * rpw * C + (size_t)cg * 8;
+    for (long row = r0 + r; row < r1; row += (long)rows_it * BNV_UNROLL) {
+        uint4 xr[BNV_UNROLL], rr_[BNV_UNROLL];
+#pragma unroll
+        for (int u = 0; u < BNV_UNROLL; ++u) {
+            const long rr = row + (long)u * rows_it;
+            if (rr < r1) { const size_t o = base + (size_t)rr * C; xr[u] = ldg16(x + o); if (res) rr_[u] = ldg16(res + o); }
+        }
+#pragma unroll
+        for (int u = 0; u < BNV_UNROLL; ++u) {
+            const long rr = row + (long)u * rows_it;
+            if (rr >= r1) break;
+            float xv[8], rv[8];
+            unpack8(xr[u], xv);
+            if (res) unpack8(rr_[u], rv);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                float v = bn_value(xv[j], mean[j], istd[j], g[j], b[j]);
+                if (res) v += rv[j];
+                if (relu) v = fmaxf(v, 0.f);
+                xv[j] = v;
+            }
+            *(uint4*)(y + base + (size_t)rr * C) = pack8(xv);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(BNV_THREADS) bnv_bwd_apply(const bf16* __restrict__ x, const bf16* __restrict__ out,
+                                                             const bf16* __restrict__ dout, const float* __restrict__ gamma,
+                                                             const float* __restrict__ beta, const float* __restrict__ stats,
+                                                             const float* __restrict__ red, bf16* __restrict__ dx, int accum_dx,
+                                                             bf16* __restrict__ dres, int accum_dres, long rpw, int C, int relu,
+                                                             int mask_from_x) {
+    const int cgs = C >> 3, rows_it = BNV_THREADS / cgs;
+    const int cg = threadIdx.x % cgs, r = threadIdx.x / cgs;
+    const int w = blockIdx.y;
+    const long per = (rpw + gridDim.x - 1) / gridDim.x;
+    const long r0 = (long)blockIdx.x * per, r1 = min(rpw, r0 + per);
+    const float inv_n = 1.f / (float)rpw;
+    float mean[8], istd[8], g[8], b[8], c1[8], c2[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int c = cg * 8 + j;
+        const size_t so = ((size_t)w * C + c) * 2;
+        mean[j] = stats[so]; istd[j] = stats[so + 1];
+        g[j] = gamma[c]; b[j] = beta[c];
+        c1[j] = red[so] * inv_n; c2[j] = red[so + 1] * inv_n;
+    }
+    const size_t base = (size_t)w * rpw * C + (size_t)cg * 8;
+    const bool need_out = relu && !mask_from_x;
+    constexpr int U = 2;
+    for (long row = r0 + r; row < r1; row += (long)rows_it * U) {
+        uint4 xr[U], dr[U], orr[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long rr = row + (long)u * rows_it;
+            if (rr < r1) {
+                const size_t o = base + (size_t)rr * C;
+                xr[u] = ldg16(x + o); dr[u] = ldg16(dout + o);
+                if (need_out) orr[u] = ldg16(out + o);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long rr = row + (long)u * rows_it;
+            if (rr >= r1) break;
+            const size_t o = base + (size_t)rr * C;
+            float xv[8], dv[8], ov[8], t[8];
+            unpack8(xr[u], xv); unpack8(dr[u], dv);
+            if (need_out) unpack8(orr[u], ov);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (relu) { float f = mask_from_x ? bn_value(xv[j], mean[j], istd[j], g[j], b[j]) : ov[j]; if (!(f > 0.f)) dv[j] = 0.f; }
+                const float xh = (xv[j] - mean[j]) * istd[j];
+                t[j] = g[j] * istd[j] * (dv[j] - c1[j] - xh * c2[j]);
+            }
+            if (accum_dx) {
+                float old[8]; unpack8(*(const uint4*)(dx + o), old);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) t[j] += old[j];
+            }
+            *(uint4*)(dx + o) = pack8(t);
+            if (dres) {
+                if (accum_dres) {
+                    float old[8]; unpack8(*(const uint4*)(dres + o), old);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) dv[j] += old[j];
+                }
+                *(uint4*)(dres + o) = pack8(dv);
+            }
+        }
+    }
+}
+
+static bool bnv_ok(int dt, int C) { int cgs = C >> 3; return dt == 1 && C % 8 == 0 && cgs <= BNV_THREADS && (cgs & (cgs - 1)) == 0; }
+static int bnv_chunks(int nw, long rpw, int C) {
+    long rows_it = BNV_THREADS / (C >> 3);
+    long want = (148 * 6 + nw - 1) / nw, maxc = (rpw + rows_it * 4 - 1) / (rows_it * 4);
+    long c = want < maxc ? want : maxc;
+    if (c > BNV_MAX_CHUNKS) c = BNV_MAX_CHUNKS;
+    return (int)(c < 1 ? 1 : c);
+}
+
 void bn_forward(int dt, const void* x, const float* gamma, const float* beta, const void* res, void* y, float* stats,
                 float* scratch, int nw, long rpw, int C, bool relu, cudaStream_t s) {
+    if (bnv_ok(dt, C)) {
+        const int chunks = bnv_chunks(nw, rpw, C);
+        const double total = (double)nw * rpw * C;
+        dim3 grid(chunks, nw);
+        { Scope sc(KC_BN_FWD_STATS, 0.0, 2.0 * total, s);
+          bnv_reduce<0><<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, nullptr, nullptr, nullptr, nullptr, nullptr, scratch, rpw, C, 0, 0); }
+        { Scope sc(KC_BN_FWD_STATS, 0.0, 8.0 * chunks * nw * C, s);
+          bn_stats_final<<<cdiv((size_t)nw * C, 128), 128, 0, s>>>(scratch, stats, chunks, nw * C, rpw); }
+        Scope sc(KC_BN_FWD_APPLY, 0.0, 2.0 * total * (res ? 3 : 2), s);
+        bnv_apply<<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, gamma, beta, (const bf16*)res, (bf16*)y, stats, rpw, C, relu);
+        return;
+    }
     int chunks = (int)(rpw < RED_CHUNKS ? rpw : RED_CHUNKS);
     dim3 grid(cdiv(C, 32), chunks, nw), blk(32, 8);
     const double esz_ = dt ? 2.0 : 4.0;
@@ -559,9 +816,25 @@ void bn_forward(int dt, const void* x, const float* gamma, const float* beta, co
     else bn_apply_k<float><<<cdiv(total, 256), 256, 0, s>>>((const float*)x, gamma, beta, (const float*)res, (float*)y, stats, rpw, C, total, relu);
 }
 
-void bn_backward(int dt, const void* x, const void* out, const void* dout, const float* gamma, const float* stats,
-                 void* dx, bool accum_dx, void* dres, bool accum_dres, float* dgamma, float* dbeta, float* red,
-                 float* scratch, int nw, long rpw, int C, bool relu, cudaStream_t s) {
+void bn_backward(int dt, const void* x, const void* out, const void* dout, const float* gamma, const float* beta,
+                 const float* stats, void* dx, bool accum_dx, void* dres, bool accum_dres, float* dgamma, float* dbeta, float* red,
+                 float* scratch, int nw, long rpw, int C, bool relu, bool has_res, cudaStream_t s) {
+    if (bnv_ok(dt, C)) {
+        const int chunks = bnv_chunks(nw, rpw, C);
+        const double total = (double)nw * rpw * C;
+        const int mask_from_x = relu && !has_res;
+        const int reads = 2 + ((relu && !mask_from_x) ? 1 : 0);
+        dim3 grid(chunks, nw);
+        { Scope sc(KC_BN_BWD_REDUCE, 0.0, 2.0 * total * reads, s);
+          bnv_reduce<1><<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, gamma, beta, stats, scratch, rpw, C,
+                                                      relu, mask_from_x); }
+        { Scope sc(KC_BN_BWD_REDUCE, 0.0, 8.0 * chunks * nw * C, s);
+          bn_bwd_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C); }
+        Scope sc(KC_BN_BWD_APPLY, 0.0, 2.0 * total * (reads + 1 + (accum_dx ? 1 : 0) + (dres ? (accum_dres ? 2 : 1) : 0)), s);
+        bnv_bwd_apply<<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, gamma, beta, stats, red, (bf16*)dx,
+                                                   accum_dx, (bf16*)dres, accum_dres, rpw, C, relu, mask_from_x);
+        return;
+    }
     int chunks = (int)(rpw < RED_CHUNKS ? rpw : RED_CHUNKS);
     dim3 grid(cdiv(C, 32), chunks, nw), blk(32, 8);
     const double esz_ = dt ? 2.0 : 4.0;

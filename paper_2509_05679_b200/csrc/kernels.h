@@ -40,15 +40,15 @@ void gap_forward(int dt, const void* x, void* y, int N, int HW, int C, cudaStrea
 void gap_backward(int dt, const void* dy, void* dx, int N, int HW, int C, bool accum, cudaStream_t st);
 
 // Batch-norm with per-worker statistics.  x: [n_workers * rows_per_worker, C].
-// stats: fp32 [n_workers][C][2] = (mean, invstd).  scratch: fp32 [64 * n_workers * C * 2].
+// stats: fp32 [n_workers][C][2] = (mean, invstd).  scratch: fp32 [128 * n_workers * C * 2].
 void bn_forward(int dt, const void* x, const float* gamma, const float* beta, const void* residual_or_null,
                 void* y, float* stats, float* scratch, int n_workers, long rows_per_worker, int C, bool relu,
                 cudaStream_t st);
 // dy_eff = dout * (out > 0 if relu).  dx (+)= BN backward of dy_eff; dres (+)= dy_eff;
 // dgamma, dbeta (fp32) = sums over all workers.  red: fp32 [n_workers][C][2] scratch for (sum dy, sum dy xhat).
-void bn_backward(int dt, const void* x, const void* out, const void* dout, const float* gamma, const float* stats,
-                 void* dx, bool accum_dx, void* dres_or_null, bool accum_dres, float* dgamma, float* dbeta,
-                 float* red, float* scratch, int n_workers, long rows_per_worker, int C, bool relu, cudaStream_t st);
+void bn_backward(int dt, const void* x, const void* out, const void* dout, const float* gamma, const float* beta,
+                 const float* stats, void* dx, bool accum_dx, void* dres_or_null, bool accum_dres, float* dgamma, float* dbeta,
+                 float* red, float* scratch, int n_workers, long rows_per_worker, int C, bool relu, bool has_res, cudaStream_t st);
 
 // Softmax cross-entropy over fp32 logits [M, classes]: dlogits (storage dtype) = (softmax - onehot) / M,
 // *loss_out = mean loss.  Deterministic single-block reduction.
@@ -82,10 +82,12 @@ struct KernelStat { uint64_t launches; double ms, flops, bytes; };
 // Opened around every launch: counts it and, while profiling is enabled, records an event before and
 // after it on the launching stream.  flops / bytes are the launch's ALGORITHMIC work.
 struct Scope {
-    int cls; cudaStream_t st; cudaEvent_t a;
+    int cls; cudaStream_t st; cudaEvent_t a; const char* detail;
     Scope(int cls, double flops, double bytes, cudaStream_t s);
     ~Scope();
 };
+void profile_detail(const char* detail);                    // tag (e.g. a layer shape) for the Scopes this thread opens next; nullptr clears
+int  profile_read_detail(KernelStat* out, char (*names)[48], int capacity);   // call after profile_read
 void profile_enable(bool on);                               // on: clears the statistics
 int  profile_read(KernelStat* out, const char** names);     // synchronises the device; returns KC_COUNT
 
