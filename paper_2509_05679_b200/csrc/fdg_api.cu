@@ -168,8 +168,8 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
         o.tc = ctx->dt == 1 && ctx->kernel_path == 0 && g.C % 64 == 0 && g.Co % 64 == 0 &&
                tc::pixel_tile(g.Ho, g.Wo, 128, &wt, &ht, &nt) && g.Ho % ht == 0 && 2 * wt <= 256 && tc::init();
         if (o.tc) {
-            o.n_tile_f = g.Co % 128 == 0 ? 128 : 64;
-            o.n_tile_d = g.C % 128 == 0 ? 128 : 64;
+            o.n_tile_f = g.Co % 256 == 0 ? 256 : (g.Co % 128 == 0 ? 128 : 64);
+            o.n_tile_d = g.C % 256 == 0 ? 256 : (g.C % 128 == 0 ? 128 : 64);
             o.n_tile_w = g.Co % 256 == 0 ? 256 : (g.Co % 128 == 0 ? 128 : 64);
             tc::pixel_tile(g.Ho, g.Wo, 64, &wt, &ht, &nt);
             int row_blocks = g.R * g.R * g.C / 64;

@@ -779,10 +779,49 @@ __global__ void __launch_bounds__(BNV_THREADS) bnv_bwd_apply(const bf16* __restr
     }
 }
 
+// stats[w][c] = (mean, invstd) from the chunk partials; one thread per (w, c), independent loads
+__global__ void bnv_stats_final(const float* __restrict__ part, float* __restrict__ stats, int chunks, int nwC, long rpw) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= nwC) return;
+    double s1 = 0.0, s2 = 0.0;
+#pragma unroll 8
+    for (int k = 0; k < chunks; ++k) {
+        const float2 v = *(const float2*)(part + ((size_t)k * nwC + i) * 2);
+        s1 += v.x; s2 += v.y;
+    }
+    const double mean = s1 / (double)rpw;
+    double var = s2 / (double)rpw - mean * mean;
+    if (var < 0.0) var = 0.0;
+    *(float2*)(stats + (size_t)i * 2) = make_float2((float)mean, (float)(1.0 / sqrt(var + 1e-5)));
+}
+// block = 32 channels x nw workers: thread (c, w) sums its chunk partials into red[w][c]; then the w == 0
+// threads add the workers in ascending order into dgamma / dbeta
+__global__ void bnv_bwd_final(const float* __restrict__ part, float* __restrict__ red, float* __restrict__ dgamma,
+                              float* __restrict__ dbeta, int chunks, int nw, int C) {
+    __shared__ float sh[32][33][2];
+    const int c = blockIdx.x * 32 + threadIdx.x, w = threadIdx.y;
+    float s1 = 0.f, s2 = 0.f;
+    if (c < C) {
+#pragma unroll 8
+        for (int k = 0; k < chunks; ++k) {
+            const float2 v = *(const float2*)(part + (((size_t)k * nw + w) * C + c) * 2);
+            s1 += v.x; s2 += v.y;
+        }
+        *(float2*)(red + ((size_t)w * C + c) * 2) = make_float2(s1, s2);
+    }
+    sh[w][threadIdx.x][0] = s1; sh[w][threadIdx.x][1] = s2;
+    __syncthreads();
+    if (w == 0 && c < C) {
+        float g = 0.f, b = 0.f;
+        for (int i = 0; i < nw; ++i) { b += sh[i][threadIdx.x][0]; g += sh[i][threadIdx.x][1]; }
+        dgamma[c] = g; dbeta[c] = b;
+    }
+}
+
 static bool bnv_ok(int dt, int C) { int cgs = C >> 3; return dt == 1 && C % 8 == 0 && cgs <= BNV_THREADS && (cgs & (cgs - 1)) == 0; }
 static int bnv_chunks(int nw, long rpw, int C) {
     long rows_it = BNV_THREADS / (C >> 3);
-    long want = (148 * 6 + nw - 1) / nw, maxc = (rpw + rows_it * 4 - 1) / (rows_it * 4);
+    long want = (148 * 4 + nw - 1) / nw, maxc = (rpw + rows_it * 4 - 1) / (rows_it * 4);
     long c = want < maxc ? want : maxc;
     if (c > BNV_MAX_CHUNKS) c = BNV_MAX_CHUNKS;
     return (int)(c < 1 ? 1 : c);
@@ -797,7 +836,7 @@ void bn_forward(int dt, const void* x, const float* gamma, const float* beta, co
         { Scope sc(KC_BN_FWD_STATS, 0.0, 2.0 * total, s);
           bnv_reduce<0><<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, nullptr, nullptr, nullptr, nullptr, nullptr, scratch, rpw, C, 0, 0); }
         { Scope sc(KC_BN_FWD_STATS, 0.0, 8.0 * chunks * nw * C, s);
-          bn_stats_final<<<cdiv((size_t)nw * C, 128), 128, 0, s>>>(scratch, stats, chunks, nw * C, rpw); }
+          bnv_stats_final<<<cdiv((size_t)nw * C, 64), 64, 0, s>>>(scratch, stats, chunks, nw * C, rpw); }
         Scope sc(KC_BN_FWD_APPLY, 0.0, 2.0 * total * (res ? 3 : 2), s);
         bnv_apply<<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, gamma, beta, (const bf16*)res, (bf16*)y, stats, rpw, C, relu);
         return;
@@ -829,7 +868,8 @@ void bn_backward(int dt, const void* x, const void* out, const void* dout, const
           bnv_reduce<1><<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, gamma, beta, stats, scratch, rpw, C,
                                                       relu, mask_from_x); }
         { Scope sc(KC_BN_BWD_REDUCE, 0.0, 8.0 * chunks * nw * C, s);
-          bn_bwd_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C); }
+          if (nw <= 32) bnv_bwd_final<<<cdiv(C, 32), dim3(32, nw), 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C);
+          else bn_bwd_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C); }
         Scope sc(KC_BN_BWD_APPLY, 0.0, 2.0 * total * (reads + 1 + (accum_dx ? 1 : 0) + (dres ? (accum_dres ? 2 : 1) : 0)), s);
         bnv_bwd_apply<<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, gamma, beta, stats, red, (bf16*)dx,
                                                    accum_dx, (bf16*)dres, accum_dres, rpw, C, relu, mask_from_x);

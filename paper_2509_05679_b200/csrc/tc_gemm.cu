@@ -128,33 +128,43 @@ __device__ __forceinline__ uint8_t* align1024(uint8_t* p) {
 }
 
 // ------------------------------------------------------------------------------------------ forward / dgrad
+// Persistent: one CTA per SM walks over output tiles (column tile fastest, so CTAs running side by side
+// read the same activation tile through L2).  Two accumulator buffers in tensor memory let the MMA warp
+// start the next tile while the epilogue warps drain the previous one.  The epilogue stages each
+// 32-column slice through shared memory so that a warp's global stores cover whole rows.
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+constexpr int EPI_ROW_WORDS = 36;                 // 32 fp32 + 4 padding: conflict-free 128-bit rows
+
 template <int N_TILE, int STAGES>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, KmParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
     constexpr int A_BYTES = BLOCK_M * BLOCK_K * 2, B_BYTES = N_TILE * BLOCK_K * 2, STAGE_BYTES = A_BYTES + B_BYTES;
-    uint64_t* full = (uint64_t*)(smem + STAGES * STAGE_BYTES);
+    constexpr int EPI_BYTES = 4 * 32 * EPI_ROW_WORDS * 4;
+    constexpr uint32_t TMEM_COLS = 2 * N_TILE;
+    float* epi_smem = (float*)(smem + STAGES * STAGE_BYTES);
+    uint64_t* full = (uint64_t*)(smem + STAGES * STAGE_BYTES + EPI_BYTES);
     uint64_t* empty = full + STAGES;
-    uint64_t* accum_bar = empty + STAGES;
-    uint32_t* tmem_slot = (uint32_t*)(accum_bar + 1);
+    uint64_t* tmem_full = empty + STAGES;        // [2]
+    uint64_t* tmem_empty = tmem_full + 2;        // [2]
+    uint32_t* tmem_slot = (uint32_t*)(tmem_empty + 2);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // tile coordinates: blockIdx.x enumerates pixel tiles (w fastest), blockIdx.y output-channel tiles
-    int tm = blockIdx.x;
-    const int tw = tm % p.tiles_w; tm /= p.tiles_w;
-    const int th = tm % p.tiles_h; const int tn = tm / p.tiles_h;
-    const int w0 = tw * p.Wt, h0 = th * p.Ht, n0 = tn * p.Nt;
-    const int co0 = blockIdx.y * N_TILE;
+    const int tiles_m = p.tiles_w * p.tiles_h * p.tiles_n;
+    const int tiles_c = p.Cn / N_TILE;
+    const int total = tiles_m * tiles_c;
     const int num_kb = p.ntaps * p.kchunks;
 
     if (threadIdx.x == 0) {
         tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB);
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        mbar_init(accum_bar, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 4); }
         fence_barrier_init();
     }
-    if (warp == 1) tmem_alloc(tmem_slot, N_TILE < 32 ? 32 : N_TILE);
+    if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -162,84 +172,115 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % STAGES, it = kb / STAGES;
-                if (it > 0 && !mbar_wait(&empty[s], (it - 1) & 1, p.err, 1)) break;
-                const int tap = kb / p.kchunks, kc = kb - tap * p.kchunks;
-                uint8_t* a = smem + s * STAGE_BYTES;
-                mbar_expect_tx(&full[s], STAGE_BYTES);
-                tma_load_4d(a, &tmA, &full[s], kc * BLOCK_K, w0 * p.xs + p.dw[tap], h0 * p.xs + p.dh[tap], n0);
-                tma_load_2d(a + A_BYTES, &tmB, &full[s], p.koff[tap] + kc * BLOCK_K, co0);
+            int kbg = 0;                                              // k-blocks issued so far, over all tiles
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+                int tm = tile / tiles_c; const int co0 = (tile - tm * tiles_c) * N_TILE;
+                const int tw = tm % p.tiles_w; tm /= p.tiles_w;
+                const int th = tm % p.tiles_h; const int tn = tm / p.tiles_h;
+                const int w0 = tw * p.Wt, h0 = th * p.Ht, n0 = tn * p.Nt;
+                for (int kb = 0; kb < num_kb; ++kb, ++kbg) {
+                    const int s = kbg % STAGES, it = kbg / STAGES;
+                    if (it > 0 && !mbar_wait(&empty[s], (it - 1) & 1, p.err, 1)) { ok = false; break; }
+                    const int tap = kb / p.kchunks, kc = kb - tap * p.kchunks;
+                    uint8_t* a = smem + s * STAGE_BYTES;
+                    mbar_expect_tx(&full[s], STAGE_BYTES);
+                    tma_load_4d(a, &tmA, &full[s], kc * BLOCK_K, w0 * p.xs + p.dw[tap], h0 * p.xs + p.dh[tap], n0);
+                    tma_load_2d(a + A_BYTES, &tmB, &full[s], p.koff[tap] + kc * BLOCK_K, co0);
+                }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = make_idesc(BLOCK_M, N_TILE, 0, 0);
+            int kbg = 0, ti = 0;
             bool ok = true;
-            for (int kb = 0; kb < num_kb && ok; ++kb) {
-                const int s = kb % STAGES, it = kb / STAGES;
-                ok = mbar_wait(&full[s], it & 1, p.err, 2);
-                if (!ok) break;
+            for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++ti) {
+                const int buf = ti & 1, use = ti >> 1;
+                if (use > 0 && !mbar_wait(&tmem_empty[buf], (use - 1) & 1, p.err, 7)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t a = smem_u32(smem + s * STAGE_BYTES), b = a + A_BYTES;
+                const uint32_t d = tmem_base + buf * N_TILE;
+                for (int kb = 0; kb < num_kb; ++kb, ++kbg) {
+                    const int s = kbg % STAGES, it = kbg / STAGES;
+                    if (!mbar_wait(&full[s], it & 1, p.err, 2)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a = smem_u32(smem + s * STAGE_BYTES), b = a + A_BYTES;
 #pragma unroll
-                for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                    umma_bf16(tmem_base, make_desc(a + k * UMMA_K * 2, 16, 1024), make_desc(b + k * UMMA_K * 2, 16, 1024), idesc,
-                              (kb | k) != 0);
-                umma_commit(&empty[s]);
+                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                        umma_bf16(d, make_desc(a + k * UMMA_K * 2, 16, 1024), make_desc(b + k * UMMA_K * 2, 16, 1024), idesc, (kb | k) != 0);
+                    umma_commit(&empty[s]);
+                }
+                umma_commit(&tmem_full[buf]);      // arrives once every MMA of this tile has finished
             }
-            umma_commit(accum_bar);           // arrives once every MMA issued above has finished
         }
     } else {
         // ---- epilogue: warp q = warp % 4 owns tensor-memory lanes 32q .. 32q+31 (= tile rows)
         const int q = warp & 3;
-        const int row = q * 32 + lane;
-        const bool ok = mbar_wait(accum_bar, 0, p.err, 3);
-        tc_fence_after();
-        // row -> pixel of the tile -> output address
-        const int pw = row % p.Wt, ph = (row / p.Wt) % p.Ht, pn = row / (p.Wt * p.Ht);
-        const int n = n0 + pn, h = h0 + ph, w = w0 + pw;
-        const bool valid = ok && n < p.N && h < p.Hd && w < p.Wd;
-        bf16* out = (bf16*)p.out + (((size_t)n * p.Ho + (h * p.os + p.oph)) * p.Wo + (w * p.os + p.opw)) * p.Co + co0;
+        float* stage = epi_smem + q * 32 * EPI_ROW_WORDS;
+        int ti = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++ti) {
+            const int buf = ti & 1, use = ti >> 1;
+            int tm = tile / tiles_c; const int co0 = (tile - tm * tiles_c) * N_TILE;
+            const int tw = tm % p.tiles_w; tm /= p.tiles_w;
+            const int th = tm % p.tiles_h; const int tn = tm / p.tiles_h;
+            // this lane's row of the tile -> output address (0 = row outside the tensor)
+            const int row = q * 32 + lane;
+            const int pw = row % p.Wt, ph = (row / p.Wt) % p.Ht, pn = row / (p.Wt * p.Ht);
+            const int n = tn * p.Nt + pn, h = th * p.Ht + ph, w = tw * p.Wt + pw;
+            const bool valid = n < p.N && h < p.Hd && w < p.Wd;
+            const unsigned long long rowptr = valid ? (unsigned long long)((bf16*)p.out + (((size_t)n * p.Ho + (h * p.os + p.oph)) * p.Wo +
+                                                                                                (w * p.os + p.opw)) * p.Co + co0) : 0ull;
+            ok = mbar_wait(&tmem_full[buf], use & 1, p.err, 3);
+            tc_fence_after();
 #pragma unroll 1
-        for (int c = 0; c < N_TILE; c += 32) {
-            uint32_t v[32];
-            tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + c, v);
-            if (!valid) continue;
-            float f[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v[j]);
-            if (p.bias) {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) f[j] += p.bias[co0 + c + j];
-            }
-            if (p.epi & EPI_RELU) {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) f[j] = fmaxf(f[j], 0.f);
-            }
-            uint4* o4 = (uint4*)(out + c);
-            if (p.epi & EPI_ACCUM) {
-#pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    uint4 old = o4[g];
-                    const __nv_bfloat162* ob = (const __nv_bfloat162*)&old;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) { float2 t = __bfloat1622float2(ob[j]); f[g * 8 + 2 * j] += t.x; f[g * 8 + 2 * j + 1] += t.y; }
+            for (int c = 0; c < N_TILE; c += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * N_TILE + c, v);
+                if (c + 32 >= N_TILE) {            // last read of this accumulator: hand the buffer back to the MMA warp
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&tmem_empty[buf]);
                 }
-            }
+                // bias / ReLU on this lane's row, then into the staging rows
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-                uint4 pk;
-                __nv_bfloat162 t0 = __floats2bfloat162_rn(f[g * 8 + 0], f[g * 8 + 1]), t1 = __floats2bfloat162_rn(f[g * 8 + 2], f[g * 8 + 3]);
-                __nv_bfloat162 t2 = __floats2bfloat162_rn(f[g * 8 + 4], f[g * 8 + 5]), t3 = __floats2bfloat162_rn(f[g * 8 + 6], f[g * 8 + 7]);
-                pk.x = *(uint32_t*)&t0; pk.y = *(uint32_t*)&t1; pk.z = *(uint32_t*)&t2; pk.w = *(uint32_t*)&t3;
-                o4[g] = pk;
+                for (int j = 0; j < 32; j += 4) {
+                    float4 f = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                    if (p.bias) { const float4 bb = __ldg((const float4*)(p.bias + co0 + c + j)); f.x += bb.x; f.y += bb.y; f.z += bb.z; f.w += bb.w; }
+                    if (p.epi & EPI_RELU) { f.x = fmaxf(f.x, 0.f); f.y = fmaxf(f.y, 0.f); f.z = fmaxf(f.z, 0.f); f.w = fmaxf(f.w, 0.f); }
+                    *(float4*)(stage + lane * EPI_ROW_WORDS + j) = f;
+                }
+                __syncwarp();
+                // transposed read-out: 4 lanes cover one row's 32 columns (64 bytes of bf16), 8 rows per pass
+#pragma unroll
+                for (int pass = 0; pass < 4; ++pass) {
+                    const int r = pass * 8 + (lane >> 2), piece = lane & 3;
+                    const unsigned long long rp = __shfl_sync(0xffffffffu, rowptr, r);
+                    const float4 f0 = *(const float4*)(stage + r * EPI_ROW_WORDS + piece * 8);
+                    const float4 f1 = *(const float4*)(stage + r * EPI_ROW_WORDS + piece * 8 + 4);
+                    if (rp && ok) {
+                        float f[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
+                        uint4* o = (uint4*)((bf16*)rp + c + piece * 8);
+                        if (p.epi & EPI_ACCUM) {
+                            const uint4 old = *o;
+                            const __nv_bfloat162* ob = (const __nv_bfloat162*)&old;
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) { const float2 t = __bfloat1622float2(ob[j]); f[2 * j] += t.x; f[2 * j + 1] += t.y; }
+                        }
+                        uint4 pk;
+                        __nv_bfloat162 t0 = __floats2bfloat162_rn(f[0], f[1]), t1 = __floats2bfloat162_rn(f[2], f[3]);
+                        __nv_bfloat162 t2 = __floats2bfloat162_rn(f[4], f[5]), t3 = __floats2bfloat162_rn(f[6], f[7]);
+                        pk.x = *(uint32_t*)&t0; pk.y = *(uint32_t*)&t1; pk.z = *(uint32_t*)&t2; pk.w = *(uint32_t*)&t3;
+                        *o = pk;
+                    }
+                }
+                __syncwarp();
             }
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, N_TILE < 32 ? 32 : N_TILE); }
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, TMEM_COLS); }
 }
 
 // ------------------------------------------------------------------------------------------ weight gradient
@@ -417,23 +458,31 @@ bool pixel_tile(int H, int W, int pixels, int* Wt, int* Ht, int* Nt) {
     return true;
 }
 
+static int sm_count() {
+    static int n = 0;
+    if (!n) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev); if (n <= 0) n = 148; }
+    return n;
+}
+
 template <int N_TILE, int STAGES>
-static cudaError_t launch_km(const TensorMap& a, const TensorMap& b, const KmParams& p, dim3 grid, cudaStream_t s) {
-    constexpr int smem = STAGES * (BLOCK_M * BLOCK_K * 2 + N_TILE * BLOCK_K * 2) + 1024 + 256;
+static cudaError_t launch_km(const TensorMap& a, const TensorMap& b, const KmParams& p, cudaStream_t s) {
+    constexpr int smem = STAGES * (BLOCK_M * BLOCK_K * 2 + N_TILE * BLOCK_K * 2) + 4 * 32 * EPI_ROW_WORDS * 4 + 1024 + 256;
     static bool attr = false;
     if (!attr) {
         cudaError_t e = cudaFuncSetAttribute(km_kernel<N_TILE, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         attr = true;
     }
+    const int total = p.tiles_w * p.tiles_h * p.tiles_n * (p.Cn / N_TILE);
+    const int grid = total < sm_count() ? total : sm_count();
     km_kernel<N_TILE, STAGES><<<grid, NUM_THREADS, smem, s>>>(*(const CUtensorMap*)&a, *(const CUtensorMap*)&b, p);
     return cudaGetLastError();
 }
 
 cudaError_t run_km(const TensorMap& a, const TensorMap& b, const KmParams& p, int n_tile, cudaStream_t s) {
-    dim3 grid(p.tiles_w * p.tiles_h * p.tiles_n, p.Cn / n_tile, 1);
-    if (n_tile == 64) return launch_km<64, 4>(a, b, p, grid, s);
-    if (n_tile == 128) return launch_km<128, 4>(a, b, p, grid, s);
+    if (n_tile == 64) return launch_km<64, 6>(a, b, p, s);
+    if (n_tile == 128) return launch_km<128, 6>(a, b, p, s);
+    if (n_tile == 256) return launch_km<256, 4>(a, b, p, s);
     return cudaErrorInvalidValue;
 }
 
