@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfdg.so")
-SOURCES = ["fdg_api.cu", "kernels.cu", "tc_gemm.cu", "noalloc.cu"]
+SOURCES = ["fdg_api.cu", "kernels.cu", "tc_gemm.cu", "stem.cu", "noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--use_fast_math=false"]
 

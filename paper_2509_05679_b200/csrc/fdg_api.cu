@@ -57,6 +57,7 @@ struct Op {
     bool need_dgrad;
     // tensor-core plan (bf16 storage, channel counts that are multiples of 64, power-of-two images)
     bool tc;
+    bool stem;                                               // thin first-layer conv: dedicated FMA kernels
     char shape[40];                                          // "HxW Cin->Cout kR sS", the profiler's detail tag
     int n_tile_f, n_tile_d, n_tile_w, wg_splits;
     tc::KmParams kf;
@@ -163,6 +164,7 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
         if (bias) o.b_off = seg(cout, false);
         o.out = add_tensor(g.Ho, g.Wo, cout);
         std::snprintf(o.shape, sizeof o.shape, "%dx%d %d->%d k%d s%d", g.H, g.W, g.C, g.Co, g.R, g.stride);
+        o.stem = ctx->kernel_path == 0 && kind == FDG_CONV3X3 && stem_supported(ctx->dt, g);
         // tensor-core eligibility
         int wt, ht, nt;
         o.tc = ctx->dt == 1 && ctx->kernel_path == 0 && g.C % 64 == 0 && g.Co % 64 == 0 &&
@@ -175,7 +177,7 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
             int row_blocks = g.R * g.R * g.C / 64;
             long ptiles = (long)(g.Wo / wt) * (g.Ho / ht) * ((g.N + nt - 1) / nt);
             int tiles = ((row_blocks + 1) / 2) * (g.Co / o.n_tile_w);
-            long want = (2 * 148 + tiles - 1) / tiles;
+            long want = (2 * 148) / tiles;              // CTAs = tiles * splits fill at most two full waves of the 148 SMs
             long splits = want < 1 ? 1 : want;
             if (splits > ptiles) splits = ptiles;
             long pps = (ptiles + splits - 1) / splits;
@@ -285,6 +287,7 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
         }
         if (o.type == OP_CONV) {
             if (o.tc) m.ws_elems = std::max(m.ws_elems, (size_t)o.wg_splits * o.g.R * o.g.R * o.g.C * o.g.Co);
+            if (o.stem) m.ws_elems = std::max(m.ws_elems, stem_wgrad_workspace_elems(o.g));
             m.ws_elems = std::max(m.ws_elems, wgrad_workspace_elems(o.g));
             m.scratch_elems = std::max(m.scratch_elems, (size_t)64 * o.g.Co);
         }
@@ -387,6 +390,12 @@ void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version) {
                 int epi = (o.relu ? EPI_RELU : 0) | (to.loc == LOC_LOGITS ? EPI_OUT_F32 : 0);
                 profile_detail(o.shape);
                 if (o.tc && tc_forward(c, m, o, P.tensor(o.in), P.tensor(o.out), version, s)) { profile_detail(nullptr); break; }
+                if (o.stem) {
+                    stem_forward(P.tensor(o.in), wbig(c, m, version, o.w_off), o.bias ? wsmall(c, m, version, o.b_off) : nullptr,
+                                 P.tensor(o.out), o.g, o.relu, s);
+                    profile_detail(nullptr);
+                    break;
+                }
                 conv_forward(dt, P.tensor(o.in), wbig(c, m, version, o.w_off), o.bias ? wsmall(c, m, version, o.b_off) : nullptr,
                              P.tensor(o.out), o.g, epi, s);
                 profile_detail(nullptr);
@@ -431,7 +440,8 @@ void backward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int64_t
             case OP_CONV: {
                 if (o.relu) relu_backward(dt, P.tensor(o.out), gout, gout, n_out, false, s);       // in place: dZ = dA * (A > 0)
                 profile_detail(o.shape);
-                if (!(o.tc && tc_wgrad(c, m, o, P.tensor(o.in), gout, m.grad + o.w_off, s)))
+                if (o.stem) stem_wgrad(P.tensor(o.in), gout, m.grad + o.w_off, m.ws, o.g, s);
+                else if (!(o.tc && tc_wgrad(c, m, o, P.tensor(o.in), gout, m.grad + o.w_off, s)))
                     conv_wgrad(dt, P.tensor(o.in), gout, m.grad + o.w_off, m.ws, o.g, s);
                 if (o.bias) bias_grad(dt, gout, m.grad + m.n_big + o.b_off, m.scratch, (long)o.g.N * o.g.Ho * o.g.Wo, o.g.Co, s);
                 if (gin && !(o.tc && tc_dgrad(c, m, o, gout, gin, version, o.acc_in, s)))

@@ -28,6 +28,12 @@ void conv_wgrad(int dt, const void* x, const void* dy, float* dw, float* workspa
 // db[c] = sum over rows of dy[row][c]; scratch: fp32 [64 * C]
 void bias_grad(int dt, const void* dy, float* db, float* scratch, long rows, int C, cudaStream_t st);
 
+// First-layer convolution (3x3, stride 1, <= 4 input channels, bf16): dedicated kernels (stem.cu).
+bool   stem_supported(int dt, const ConvGeom& g);
+size_t stem_wgrad_workspace_elems(const ConvGeom& g);
+void   stem_forward(const void* x, const void* w, const float* bias, void* y, const ConvGeom& g, bool relu, cudaStream_t st);
+void   stem_wgrad(const void* x, const void* dy, float* dw, float* workspace, const ConvGeom& g, cudaStream_t st);
+
 void relu_forward(int dt, const void* x, void* y, size_t n, cudaStream_t st);
 // dx (+)= dy * (y > 0)
 void relu_backward(int dt, const void* y, const void* dy, void* dx, size_t n, bool accum, cudaStream_t st);

@@ -474,13 +474,14 @@ static cudaError_t launch_km(const TensorMap& a, const TensorMap& b, const KmPar
         attr = true;
     }
     const int total = p.tiles_w * p.tiles_h * p.tiles_n * (p.Cn / N_TILE);
-    const int grid = total < sm_count() ? total : sm_count();
+    const int slots = sm_count() * (smem <= 100 * 1024 ? 2 : 1);       // the 64-column variant fits twice on an SM
+    const int grid = total < slots ? total : slots;
     km_kernel<N_TILE, STAGES><<<grid, NUM_THREADS, smem, s>>>(*(const CUtensorMap*)&a, *(const CUtensorMap*)&b, p);
     return cudaGetLastError();
 }
 
 cudaError_t run_km(const TensorMap& a, const TensorMap& b, const KmParams& p, int n_tile, cudaStream_t s) {
-    if (n_tile == 64) return launch_km<64, 6>(a, b, p, s);
+    if (n_tile == 64) return launch_km<64, 3>(a, b, p, s);
     if (n_tile == 128) return launch_km<128, 6>(a, b, p, s);
     if (n_tile == 256) return launch_km<256, 4>(a, b, p, s);
     return cudaErrorInvalidValue;
