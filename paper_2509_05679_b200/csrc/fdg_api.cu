@@ -177,7 +177,7 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
             int row_blocks = g.R * g.R * g.C / 64;
             long ptiles = (long)(g.Wo / wt) * (g.Ho / ht) * ((g.N + nt - 1) / nt);
             int tiles = ((row_blocks + 1) / 2) * (g.Co / o.n_tile_w);
-            long want = (2 * 148) / tiles;              // CTAs = tiles * splits fill at most two full waves of the 148 SMs
+            long want = ((o.n_tile_w == 64 ? 4 : 2) * 148) / tiles;   // CTAs = tiles * splits fill whole waves of the SMs (two CTAs per SM fit for the 64-column tile)
             long splits = want < 1 ? 1 : want;
             if (splits > ptiles) splits = ptiles;
             long pps = (ptiles + splits - 1) / splits;

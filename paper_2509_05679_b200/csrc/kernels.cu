@@ -602,7 +602,7 @@ __device__ __forceinline__ float bn_value(float x, float mean, float istd, float
 // MODE 0: (sum x, sum x^2).  MODE 1: (sum dy, sum dy * xhat) with dy = dout * [forward output > 0] if relu.
 // mask_from_x: the forward output had no residual, so its sign is the sign of bn_value(x).
 template <int MODE>
-__global__ void __launch_bounds__(BNV_THREADS) bnv_reduce(const bf16* __restrict__ x, const bf16* __restrict__ out,
+__global__ void __launch_bounds__(BNV_THREADS, MODE == 1 ? 2 : 3) bnv_reduce(const bf16* __restrict__ x, const bf16* __restrict__ out,
                                                           const bf16* __restrict__ dout, const float* __restrict__ gamma,
                                                           const float* __restrict__ beta, const float* __restrict__ stats,
                                                           float* __restrict__ part, long rpw, int C, int relu, int mask_from_x) {
@@ -624,6 +624,7 @@ __global__ void __launch_bounds__(BNV_THREADS) bnv_reduce(const bf16* __restrict
     }
     const size_t base = (size_t)w * rpw * C + (size_t)cg * 8;
     const bool need_out = MODE == 1 && relu && !mask_from_x;
+    constexpr int BNV_UNROLL = MODE == 1 ? 2 : 4;
     for (long row = r0 + r; row < r1; row += (long)rows_it * BNV_UNROLL) {
         uint4 xr[BNV_UNROLL], dr[BNV_UNROLL], orr[BNV_UNROLL];
 #pragma unroll
@@ -712,7 +713,7 @@ __global__ void __launch_bounds__(BNV_THREADS) bnv_apply(const bf16* __restrict_
     }
 }
 
-__global__ void __launch_bounds__(BNV_THREADS) bnv_bwd_apply(const bf16* __restrict__ x, const bf16* __restrict__ out,
+__global__ void __launch_bounds__(BNV_THREADS, 2) bnv_bwd_apply(const bf16* __restrict__ x, const bf16* __restrict__ out,
                                                              const bf16* __restrict__ dout, const float* __restrict__ gamma,
                                                              const float* __restrict__ beta, const float* __restrict__ stats,
                                                              const float* __restrict__ red, bf16* __restrict__ dx, int accum_dx,
@@ -779,41 +780,40 @@ __global__ void __launch_bounds__(BNV_THREADS) bnv_bwd_apply(const bf16* __restr
     }
 }
 
-// stats[w][c] = (mean, invstd) from the chunk partials; one thread per (w, c), independent loads
-__global__ void bnv_stats_final(const float* __restrict__ part, float* __restrict__ stats, int chunks, int nwC, long rpw) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= nwC) return;
-    double s1 = 0.0, s2 = 0.0;
-#pragma unroll 8
-    for (int k = 0; k < chunks; ++k) {
-        const float2 v = *(const float2*)(part + ((size_t)k * nwC + i) * 2);
-        s1 += v.x; s2 += v.y;
-    }
-    const double mean = s1 / (double)rpw;
-    double var = s2 / (double)rpw - mean * mean;
-    if (var < 0.0) var = 0.0;
-    *(float2*)(stats + (size_t)i * 2) = make_float2((float)mean, (float)(1.0 / sqrt(var + 1e-5)));
+// One warp per (worker, channel): lanes take the chunk partials round-robin, then a fixed shuffle tree adds the
+// lanes, so the summation order never changes.  stats[w][c] = (mean, invstd).
+__device__ __forceinline__ float2 warp_sum2(float2 v) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) { v.x += __shfl_xor_sync(0xffffffffu, v.x, d); v.y += __shfl_xor_sync(0xffffffffu, v.y, d); }
+    return v;
 }
-// block = 32 channels x nw workers: thread (c, w) sums its chunk partials into red[w][c]; then the w == 0
-// threads add the workers in ascending order into dgamma / dbeta
+__global__ void bnv_stats_final(const float* __restrict__ part, float* __restrict__ stats, int chunks, int nwC, long rpw) {
+    const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (i >= nwC) return;
+    float2 a = make_float2(0.f, 0.f);
+    for (int k = lane; k < chunks; k += 32) { const float2 v = *(const float2*)(part + ((size_t)k * nwC + i) * 2); a.x += v.x; a.y += v.y; }
+    a = warp_sum2(a);
+    if (lane == 0) {
+        const double mean = (double)a.x / (double)rpw;
+        double var = (double)a.y / (double)rpw - mean * mean;
+        if (var < 0.0) var = 0.0;
+        *(float2*)(stats + (size_t)i * 2) = make_float2((float)mean, (float)(1.0 / sqrt(var + 1e-5)));
+    }
+}
+// block = one channel, one warp per worker (nw <= 32): red[w][c] = (sum dy, sum dy xhat); warp 0 then adds the
+// workers in ascending order into dgamma / dbeta
 __global__ void bnv_bwd_final(const float* __restrict__ part, float* __restrict__ red, float* __restrict__ dgamma,
                               float* __restrict__ dbeta, int chunks, int nw, int C) {
-    __shared__ float sh[32][33][2];
-    const int c = blockIdx.x * 32 + threadIdx.x, w = threadIdx.y;
-    float s1 = 0.f, s2 = 0.f;
-    if (c < C) {
-#pragma unroll 8
-        for (int k = 0; k < chunks; ++k) {
-            const float2 v = *(const float2*)(part + (((size_t)k * nw + w) * C + c) * 2);
-            s1 += v.x; s2 += v.y;
-        }
-        *(float2*)(red + ((size_t)w * C + c) * 2) = make_float2(s1, s2);
-    }
-    sh[w][threadIdx.x][0] = s1; sh[w][threadIdx.x][1] = s2;
+    __shared__ float2 sh[32];
+    const int c = blockIdx.x, w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float2 a = make_float2(0.f, 0.f);
+    for (int k = lane; k < chunks; k += 32) { const float2 v = *(const float2*)(part + (((size_t)k * nw + w) * C + c) * 2); a.x += v.x; a.y += v.y; }
+    a = warp_sum2(a);
+    if (lane == 0) { *(float2*)(red + ((size_t)w * C + c) * 2) = a; sh[w] = a; }
     __syncthreads();
-    if (w == 0 && c < C) {
+    if (threadIdx.x == 0) {
         float g = 0.f, b = 0.f;
-        for (int i = 0; i < nw; ++i) { b += sh[i][threadIdx.x][0]; g += sh[i][threadIdx.x][1]; }
+        for (int i = 0; i < nw; ++i) { b += sh[i].x; g += sh[i].y; }
         dgamma[c] = g; dbeta[c] = b;
     }
 }
@@ -836,7 +836,7 @@ void bn_forward(int dt, const void* x, const float* gamma, const float* beta, co
         { Scope sc(KC_BN_FWD_STATS, 0.0, 2.0 * total, s);
           bnv_reduce<0><<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, nullptr, nullptr, nullptr, nullptr, nullptr, scratch, rpw, C, 0, 0); }
         { Scope sc(KC_BN_FWD_STATS, 0.0, 8.0 * chunks * nw * C, s);
-          bnv_stats_final<<<cdiv((size_t)nw * C, 64), 64, 0, s>>>(scratch, stats, chunks, nw * C, rpw); }
+          bnv_stats_final<<<cdiv((size_t)nw * C * 32, 256), 256, 0, s>>>(scratch, stats, chunks, nw * C, rpw); }
         Scope sc(KC_BN_FWD_APPLY, 0.0, 2.0 * total * (res ? 3 : 2), s);
         bnv_apply<<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, gamma, beta, (const bf16*)res, (bf16*)y, stats, rpw, C, relu);
         return;
@@ -868,7 +868,7 @@ void bn_backward(int dt, const void* x, const void* out, const void* dout, const
           bnv_reduce<1><<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, gamma, beta, stats, scratch, rpw, C,
                                                       relu, mask_from_x); }
         { Scope sc(KC_BN_BWD_REDUCE, 0.0, 8.0 * chunks * nw * C, s);
-          if (nw <= 32) bnv_bwd_final<<<cdiv(C, 32), dim3(32, nw), 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C);
+          if (nw <= 32) bnv_bwd_final<<<C, 32 * nw, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C);
           else bn_bwd_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C); }
         Scope sc(KC_BN_BWD_APPLY, 0.0, 2.0 * total * (reads + 1 + (accum_dx ? 1 : 0) + (dres ? (accum_dres ? 2 : 1) : 0)), s);
         bnv_bwd_apply<<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, gamma, beta, stats, red, (bf16*)dx,

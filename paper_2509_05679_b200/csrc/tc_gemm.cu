@@ -382,20 +382,27 @@ wg_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUten
     if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, N_TILE < 32 ? 32 : N_TILE); }
 }
 
-// dW[co][tap][ci] = sum_z partial[z][(tap, cc)][ci % 64][co], z ascending.  32x32 transposing tiles.
-__global__ void wg_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dw, int splits, int row_blocks, int Co) {
+// dW[co][tap][ci] = sum_z partial[z][(tap, cc)][ci % 64][co], z ascending.  32x32 transposing tiles; a thread owns
+// one (row, column) per pass and keeps eight independent loads in flight along z.
+__global__ void __launch_bounds__(1024) wg_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dw, int splits, int row_blocks, int Co) {
     __shared__ float t[32][33];
     const int R = row_blocks * 64;                       // = taps * Cin
     const int r0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
-    const int tx = threadIdx.x, ty = threadIdx.y;        // 32 x 8
-    for (int i = ty; i < 32; i += 8) {
-        float s = 0.f;
-        const size_t o = (size_t)(r0 + i) * Co + c0 + tx;
-        for (int z = 0; z < splits; ++z) s += partial[(size_t)z * R * Co + o];
-        t[i][tx] = s;
+    const int tx = threadIdx.x, ty = threadIdx.y;        // 32 x 32
+    const size_t o = (size_t)(r0 + ty) * Co + c0 + tx, zs = (size_t)R * Co;
+    float s = 0.f;
+    int z = 0;
+    for (; z + 8 <= splits; z += 8) {
+        float v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = __ldg(partial + (size_t)(z + j) * zs + o);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) s += v[j];
     }
+    for (; z < splits; ++z) s += __ldg(partial + (size_t)z * zs + o);
+    t[ty][tx] = s;
     __syncthreads();
-    for (int i = ty; i < 32; i += 8) dw[(size_t)(c0 + i) * R + r0 + tx] = t[tx][i];
+    dw[(size_t)(c0 + ty) * R + r0 + tx] = t[tx][ty];
 }
 
 // Wt[ci][R*R-1-tap][co] = W[co][tap][ci]: the weights of the transposed convolution, K-major for km_kernel.
@@ -503,12 +510,12 @@ static cudaError_t launch_wg(const TensorMap& x, const TensorMap& dy, const WgPa
 cudaError_t run_wg(const TensorMap& x, const TensorMap& dy, const WgParams& p, int n_tile, int splits, float* dw, cudaStream_t s) {
     dim3 grid((p.row_blocks + 1) / 2, p.Co / n_tile, splits);
     cudaError_t e;
-    if (n_tile == 64) e = launch_wg<64, 6>(x, dy, p, grid, s);
+    if (n_tile == 64) e = launch_wg<64, 4>(x, dy, p, grid, s);      // 96 KB of stages: two CTAs per SM
     else if (n_tile == 128) e = launch_wg<128, 5>(x, dy, p, grid, s);
     else if (n_tile == 256) e = launch_wg<256, 4>(x, dy, p, grid, s);
     else return cudaErrorInvalidValue;
     if (e != cudaSuccess) return e;
-    dim3 rgrid(p.row_blocks * 2, p.Co / 32), rblk(32, 8);
+    dim3 rgrid(p.row_blocks * 2, p.Co / 32), rblk(32, 32);
     wg_reduce_kernel<<<rgrid, rblk, 0, s>>>(p.partial, dw, splits, p.row_blocks, p.Co);
     return cudaGetLastError();
 }
