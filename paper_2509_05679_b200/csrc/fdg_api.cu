@@ -63,6 +63,8 @@ struct Op {
     tc::KmParams kf;
     std::vector<tc::KmParams> kd;                            // one per output-parity class (1 for stride 1, up to 4 for stride 2)
     bool dgrad_needs_zero;                                   // some parity classes receive no gradient (1x1 stride 2)
+    int stat_chunks;                                         // > 0: the forward epilogue also leaves batch-norm partial sums
+                                                             //      (this many per worker) for the batch-norm that follows
     tc::WgParams kw;
     std::vector<char*> a_ptrs, dy_ptrs;                      // the buffers the A / dY maps below were built for
     std::vector<tc::TensorMap> fa, fb, da, db, wx, wdy;      // fwd A, fwd B (per weight slot), dgrad A, dgrad B, wgrad X, wgrad dY
@@ -80,7 +82,9 @@ struct Module {
     size_t stash_slot_bytes, wslot_bytes, grad_pool_bytes, in_slot_bytes;
     size_t ws_elems, scratch_elems, red_elems;
     char *in_ring, *stash, *gradpool, *d2, *wring, *wtring;
-    float *master, *grad, *ws, *scratch, *red;
+    float *master, *grad, *ws, *scratch, *red, *cstat;
+    size_t cstat_elems;
+    int fused_stats_tensor, fused_stats_chunks;   // set by a conv that produced statistics partials for this tensor
     int64_t *tag_in, *tag_stash, *tag_d2, *tag_w, *trace;
     cudaStream_t stream;
     cudaEvent_t done, ev0, ev1;
@@ -292,6 +296,20 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
             m.scratch_elems = std::max(m.scratch_elems, (size_t)64 * o.g.Co);
         }
     }
+    // a tensor-core conv whose output goes straight into a batch-norm computes that batch-norm's statistics
+    // in its epilogue, if its 128-row tiles never straddle two workers
+    m.cstat_elems = 0;
+    for (size_t i = 0; i + 1 < m.ops.size(); ++i) {
+        Op& o = m.ops[i];
+        const Op& nx = m.ops[i + 1];
+        o.stat_chunks = 0;
+        if (o.type != OP_CONV || !o.tc || nx.type != OP_BN || nx.in != o.out || !bn_accepts_conv_partials(ctx->dt, o.g.Co)) continue;
+        int wt, ht, nt;
+        tc::pixel_tile(o.g.Ho, o.g.Wo, 128, &wt, &ht, &nt);
+        if (ctx->B % nt != 0) continue;
+        o.stat_chunks = (ctx->B / nt) * (o.g.Ho / ht) * (o.g.Wo / wt) * 4;
+        m.cstat_elems = std::max(m.cstat_elems, (size_t)ctx->n_workers * o.stat_chunks * o.g.Co * 2);
+    }
     m.stash_slot_bytes = align_up(soff, 256);
     m.grad_pool_bytes = align_up(goff, 256);
     // backward write/accumulate analysis: walking the ops in reverse, the first op that touches a
@@ -340,10 +358,14 @@ bool tc_forward(fdg_ctx* c, Module& m, const Op& o, char* x, char* y, int64_t ve
     tc::KmParams p = o.kf;
     p.bias = o.bias ? wsmall(c, m, version, o.b_off) : nullptr;
     p.out = y; p.epi = o.relu ? EPI_RELU : 0; p.err = c->tc_err;
+    p.stat_part = o.stat_chunks ? m.cstat : nullptr;
+
     const ConvGeom& g = o.g;
     double rows = (double)g.N * g.Ho * g.Wo;
     Scope sc(KC_TC_FWD, 2.0 * rows * g.Co * g.R * g.R * g.C, 2.0 * ((double)g.N * g.H * g.W * g.C + (double)g.Co * g.R * g.R * g.C + rows * g.Co), s);
-    return tc::run_km(o.fa[ia], o.fb[version % m.D], p, o.n_tile_f, s) == cudaSuccess;
+    const bool ok = tc::run_km(o.fa[ia], o.fb[version % m.D], p, o.n_tile_f, s) == cudaSuccess;
+    if (ok && o.stat_chunks) { m.fused_stats_tensor = o.out; m.fused_stats_chunks = o.stat_chunks; }
+    return ok;
 }
 bool tc_dgrad(fdg_ctx* c, Module& m, const Op& o, char* dy, char* dx, int64_t version, bool accum, cudaStream_t s) {
     int ia = find_buf(o.dy_ptrs, dy);
@@ -357,7 +379,7 @@ bool tc_dgrad(fdg_ctx* c, Module& m, const Op& o, char* dy, char* dx, int64_t ve
     bool ok = true;
     for (const tc::KmParams& cls : o.kd) {
         tc::KmParams p = cls;
-        p.bias = nullptr; p.out = dx; p.epi = accum ? EPI_ACCUM : 0; p.err = c->tc_err;
+        p.bias = nullptr; p.out = dx; p.epi = accum ? EPI_ACCUM : 0; p.err = c->tc_err; p.stat_part = nullptr;
         double crows = (double)g.N * p.Hd * p.Wd;
         Scope sc(KC_TC_DGRAD, 2.0 * crows * g.C * p.ntaps * g.Co,
                  2.0 * ((double)g.N * g.Ho * g.Wo * g.Co + (double)g.Co * p.ntaps * g.C + crows * g.C * (accum ? 2 : 1)), s);
@@ -381,6 +403,7 @@ void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version) {
     StepPtrs P{c, &m, kk, batch};
     cudaStream_t s = m.stream;
     const int dt = c->dt;
+    m.fused_stats_tensor = -1;
     for (const Op& o : m.ops) {
         const TensorDesc& ti = m.t[o.in];
         const TensorDesc& to = m.t[o.out];
@@ -400,11 +423,13 @@ void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version) {
                              P.tensor(o.out), o.g, epi, s);
                 profile_detail(nullptr);
                 break; }
-            case OP_BN:
+            case OP_BN: {
+                const bool fused = m.fused_stats_tensor == o.in;
                 bn_forward(dt, P.tensor(o.in), wsmall(c, m, version, o.gamma_off), wsmall(c, m, version, o.beta_off),
                            o.has_res ? P.tensor(o.in2) : nullptr, P.tensor(o.out), P.stats(o), m.scratch, c->n_workers,
-                           (long)c->B * ti.h * ti.w, ti.c, o.relu, s);
-                break;
+                           (long)c->B * ti.h * ti.w, ti.c, o.relu, fused ? m.cstat : nullptr, fused ? m.fused_stats_chunks : 0, s);
+                m.fused_stats_tensor = -1;
+                break; }
             case OP_RELU: relu_forward(dt, P.tensor(o.in), P.tensor(o.out), n_out, s); break;
             case OP_POOL: maxpool_forward(dt, P.tensor(o.in), P.tensor(o.out), c->M, ti.h, ti.w, ti.c, s); break;
             case OP_GAP: gap_forward(dt, P.tensor(o.in), P.tensor(o.out), c->M, ti.h * ti.w, ti.c, s); break;
@@ -759,6 +784,7 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
         m.ws = (float*)get(m.ws_elems * sizeof(float));
         m.scratch = (float*)get(m.scratch_elems * sizeof(float));
         m.red = (float*)get(m.red_elems * sizeof(float));
+        m.cstat = m.cstat_elems ? (float*)get(m.cstat_elems * sizeof(float)) : nullptr;
         if (oom) break;
         m.tag_in = ctx->tags + tpos; tpos += 2 * (size_t)m.in_depth;
         m.tag_stash = ctx->tags + tpos; tpos += 2 * (size_t)m.D;

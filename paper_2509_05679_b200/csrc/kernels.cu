@@ -800,6 +800,33 @@ __global__ void bnv_stats_final(const float* __restrict__ part, float* __restric
         *(float2*)(stats + (size_t)i * 2) = make_float2((float)mean, (float)(1.0 / sqrt(var + 1e-5)));
     }
 }
+// same, from the partials a convolution epilogue left: [w * cpw + k][C][2], k < cpw.  One block of 128 threads per
+// (worker, channel): strided partial sums, then a fixed-order tree in shared memory.
+__global__ void __launch_bounds__(128) bnv_stats_final_tiles(const float* __restrict__ part, float* __restrict__ stats, int cpw, int nw, int C, long rpw) {
+    __shared__ float2 sh[128];
+    const int i = blockIdx.x, w = i / C, c = i - w * C, tid = threadIdx.x;
+    const float* p = part + ((size_t)w * cpw * C + c) * 2;
+    float2 a = make_float2(0.f, 0.f);
+    int k = tid;
+    for (; k + 384 < cpw; k += 512) {                      // four independent loads in flight
+        const float2 v0 = *(const float2*)(p + (size_t)k * C * 2), v1 = *(const float2*)(p + (size_t)(k + 128) * C * 2);
+        const float2 v2 = *(const float2*)(p + (size_t)(k + 256) * C * 2), v3 = *(const float2*)(p + (size_t)(k + 384) * C * 2);
+        a.x += (v0.x + v1.x) + (v2.x + v3.x); a.y += (v0.y + v1.y) + (v2.y + v3.y);
+    }
+    for (; k < cpw; k += 128) { const float2 v = *(const float2*)(p + (size_t)k * C * 2); a.x += v.x; a.y += v.y; }
+    sh[tid] = a;
+    __syncthreads();
+    for (int d = 64; d > 0; d >>= 1) {
+        if (tid < d) { sh[tid].x += sh[tid + d].x; sh[tid].y += sh[tid + d].y; }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        const double mean = (double)sh[0].x / (double)rpw;
+        double var = (double)sh[0].y / (double)rpw - mean * mean;
+        if (var < 0.0) var = 0.0;
+        *(float2*)(stats + (size_t)i * 2) = make_float2((float)mean, (float)(1.0 / sqrt(var + 1e-5)));
+    }
+}
 // block = one channel, one warp per worker (nw <= 32): red[w][c] = (sum dy, sum dy xhat); warp 0 then adds the
 // workers in ascending order into dgamma / dbeta
 __global__ void bnv_bwd_final(const float* __restrict__ part, float* __restrict__ red, float* __restrict__ dgamma,
@@ -827,16 +854,23 @@ static int bnv_chunks(int nw, long rpw, int C) {
     return (int)(c < 1 ? 1 : c);
 }
 
+bool bn_accepts_conv_partials(int dt, int C) { return bnv_ok(dt, C); }
+
 void bn_forward(int dt, const void* x, const float* gamma, const float* beta, const void* res, void* y, float* stats,
-                float* scratch, int nw, long rpw, int C, bool relu, cudaStream_t s) {
+                float* scratch, int nw, long rpw, int C, bool relu, const float* conv_part, int conv_chunks, cudaStream_t s) {
     if (bnv_ok(dt, C)) {
         const int chunks = bnv_chunks(nw, rpw, C);
         const double total = (double)nw * rpw * C;
         dim3 grid(chunks, nw);
-        { Scope sc(KC_BN_FWD_STATS, 0.0, 2.0 * total, s);
-          bnv_reduce<0><<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, nullptr, nullptr, nullptr, nullptr, nullptr, scratch, rpw, C, 0, 0); }
-        { Scope sc(KC_BN_FWD_STATS, 0.0, 8.0 * chunks * nw * C, s);
-          bnv_stats_final<<<cdiv((size_t)nw * C * 32, 256), 256, 0, s>>>(scratch, stats, chunks, nw * C, rpw); }
+        if (conv_part) {
+            Scope sc(KC_BN_FWD_STATS, 0.0, 8.0 * conv_chunks * nw * C, s);
+            bnv_stats_final_tiles<<<nw * C, 128, 0, s>>>(conv_part, stats, conv_chunks, nw, C, rpw);
+        } else {
+            { Scope sc(KC_BN_FWD_STATS, 0.0, 2.0 * total, s);
+              bnv_reduce<0><<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, nullptr, nullptr, nullptr, nullptr, nullptr, scratch, rpw, C, 0, 0); }
+            { Scope sc(KC_BN_FWD_STATS, 0.0, 8.0 * chunks * nw * C, s);
+              bnv_stats_final<<<cdiv((size_t)nw * C * 32, 256), 256, 0, s>>>(scratch, stats, chunks, nw * C, rpw); }
+        }
         Scope sc(KC_BN_FWD_APPLY, 0.0, 2.0 * total * (res ? 3 : 2), s);
         bnv_apply<<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, gamma, beta, (const bf16*)res, (bf16*)y, stats, rpw, C, relu);
         return;

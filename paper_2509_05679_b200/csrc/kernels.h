@@ -47,9 +47,12 @@ void gap_backward(int dt, const void* dy, void* dx, int N, int HW, int C, bool a
 
 // Batch-norm with per-worker statistics.  x: [n_workers * rows_per_worker, C].
 // stats: fp32 [n_workers][C][2] = (mean, invstd).  scratch: fp32 [128 * n_workers * C * 2].
+// conv_part / conv_chunks: if non-null, the producing convolution already left per-tile (sum, sum of squares)
+// partials [n_workers * conv_chunks][C][2] (worker-major); the statistics pass over x is skipped.
 void bn_forward(int dt, const void* x, const float* gamma, const float* beta, const void* residual_or_null,
                 void* y, float* stats, float* scratch, int n_workers, long rows_per_worker, int C, bool relu,
-                cudaStream_t st);
+                const float* conv_part, int conv_chunks, cudaStream_t st);
+bool bn_accepts_conv_partials(int dt, int C);
 // dy_eff = dout * (out > 0 if relu).  dx (+)= BN backward of dy_eff; dres (+)= dy_eff;
 // dgamma, dbeta (fp32) = sums over all workers.  red: fp32 [n_workers][C][2] scratch for (sum dy, sum dy xhat).
 void bn_backward(int dt, const void* x, const void* out, const void* dout, const float* gamma, const float* beta,

@@ -222,6 +222,7 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++ti) {
             const int buf = ti & 1, use = ti >> 1;
             int tm = tile / tiles_c; const int co0 = (tile - tm * tiles_c) * N_TILE;
+            const int tmi = tm;
             const int tw = tm % p.tiles_w; tm /= p.tiles_w;
             const int th = tm % p.tiles_h; const int tn = tm / p.tiles_h;
             // this lane's row of the tile -> output address (0 = row outside the tensor)
@@ -231,6 +232,7 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             const bool valid = n < p.N && h < p.Hd && w < p.Wd;
             const unsigned long long rowptr = valid ? (unsigned long long)((bf16*)p.out + (((size_t)n * p.Ho + (h * p.os + p.oph)) * p.Wo +
                                                                                                 (w * p.os + p.opw)) * p.Co + co0) : 0ull;
+            const unsigned vmask = __ballot_sync(0xffffffffu, rowptr != 0ull);
             ok = mbar_wait(&tmem_full[buf], use & 1, p.err, 3);
             tc_fence_after();
 #pragma unroll 1
@@ -251,6 +253,16 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     *(float4*)(stage + lane * EPI_ROW_WORDS + j) = f;
                 }
                 __syncwarp();
+                if (p.stat_part) {
+                    // batch-norm statistics of the layer's output, fused: lane j adds column j over this warp's rows
+                    float s1 = 0.f, s2 = 0.f;
+#pragma unroll 8
+                    for (int r = 0; r < 32; ++r) {
+                        const float vr = __bfloat162float(__float2bfloat16_rn(stage[r * EPI_ROW_WORDS + lane]));
+                        if ((vmask >> r) & 1u) { s1 += vr; s2 = fmaf(vr, vr, s2); }
+                    }
+                    *(float2*)(p.stat_part + (((size_t)tmi * 4 + q) * p.Cn + co0 + c + lane) * 2) = make_float2(s1, s2);
+                }
                 // transposed read-out: 4 lanes cover one row's 32 columns (64 bytes of bf16), 8 rows per pass
 #pragma unroll
                 for (int pass = 0; pass < 4; ++pass) {

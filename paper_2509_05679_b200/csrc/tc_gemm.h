@@ -22,6 +22,8 @@ struct KmParams {
     int epi;                                     // EPI_RELU | EPI_ACCUM
     const float* bias;                           // or nullptr
     void* out;
+    float* stat_part;                            // or nullptr: [tile_m * 4 + warp][Cn][2] = (sum, sum of squares) over the
+                                                 // warp's 32 output rows, of the values as stored (rounded to bf16)
     int* err;                                    // device word, set non-zero if a bounded wait gave up
 };
 
