@@ -32,6 +32,27 @@ UNIT = "samples/s"
 FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 148 SMs x 128 fp32 FMA lanes x 2 flop x 1.965 GHz
 
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel classes, from the ncu
+# capture summarised under profiles/ (taken at per-worker batch 64 and scaled x2 to the bench's 128: every operand of
+# these kernels grows in proportion to the batch).  Valid only for the kernel source it was taken from.
+NCU_TRAFFIC = {}        # kernel class -> {"bytes_per_launch": float, "sha1": sha1 of csrc/tc_gemm.cu + csrc/kernels.cu at capture}
+
+
+def _kernel_source_sha1():
+    import hashlib
+    h = hashlib.sha1()
+    for f in ("tc_gemm.cu", "kernels.cu"):
+        h.update(open(os.path.join(ROOT, "paper_2509_05679_b200", "csrc", f), "rb").read())
+    return h.hexdigest()
+
+
+def traffic_per_launch(kernel_class):
+    rec = NCU_TRAFFIC.get(kernel_class)
+    if not rec or rec.get("sha1") != _kernel_source_sha1():
+        return None            # never captured, or the kernel has changed since the counters were taken
+    return rec["bytes_per_launch"]
+
+
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -123,6 +144,7 @@ def main():
     ap.add_argument("--kernel-path", type=int, default=0, help="0: tensor-core kernels where shapes allow, 1: plain FMA kernels only")
     ap.add_argument("--batch", type=int, default=None, help="per-worker batch override (testing only; changes the workload name)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-uncontended", action="store_true", help="skip the extra one-stream pass that times kernels alone")
     ap.add_argument("--serial", action="store_true", help="diagnosis: all modules on one stream (uncontended per-kernel times)")
     args = ap.parse_args()
 
@@ -217,6 +239,23 @@ def main():
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
+    # ---- uncontended kernel times: the same workload with every module on one stream (rank 0, N=1 only)
+    kstats_alone, alone_steps = None, 3
+    if world == 1 and not args.serial and not args.no_uncontended:
+        ctx.close()
+        ctx = binding.Context(net.layers, net.splits, net.n_workers, net.batch, net.lr, dtype=net.dtype,
+                              in_shape=(net.in_h, net.in_w, net.in_c), num_classes=net.classes, device=local,
+                              kernel_path=args.kernel_path, serial=True)
+        ctx.set_params(sy.init_params(net.layers, 0, bf16=net.dtype == "bf16"))
+        for i in range(fill + 3):
+            ctx.step(dev_x[i % pool], dev_y[i % pool])
+        torch.cuda.synchronize()
+        ctx.profile(True)
+        for i in range(alone_steps):
+            ctx.step(dev_x[i % pool], dev_y[i % pool])
+        ctx.profile(False)
+        kstats_alone = {k: v for k, v in ctx.profile_read().items() if "[" not in k}
+
     if dist:
         tt = torch.tensor([ms, e2e_s], device="cuda", dtype=torch.float64)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
@@ -227,25 +266,32 @@ def main():
         total_samples = net.M * args.steps * world
         value = total_samples / (ms * 1e-3)
         flops_step = sy.flops_per_sample(net) * net.M
-        # dominant kernel class by device time
-        top = max(kstats.items(), key=lambda kv: kv[1]["ms"]) if kstats else (None, None)
-        roof = None
-        if top[0]:
-            name, st = top
-            per_launch_ms = st["ms"] / st["launches"]
-            tensor_bound = name.startswith("tc_gemm")
-            if tensor_bound or name.startswith("igemm_fma"):
+        def roofline_of(stats, which=None):
+            """Roofline entry of the kernel class with the largest summed event time (or of class `which`)."""
+            if not stats:
+                return None
+            name, st = (which, stats[which]) if which in stats else max(stats.items(), key=lambda kv: kv[1]["ms"])
+            total_ms = sum(v["ms"] for v in stats.values())
+            base = {"kernel": name, "launches": st["launches"], "avg_launch_ms": st["ms"] / st["launches"],
+                    "share_of_kernel_time": st["ms"] / total_ms, "traffic": traffic_per_launch(name)}
+            if name.startswith("tc_gemm") or name.startswith("igemm_fma"):
+                tensor = name.startswith("tc_gemm")
                 ach = st["flops"] / (st["ms"] * 1e-3) / 1e12
-                peak = pk["tensor"] if tensor_bound else FMA_PEAK_TFLOPS
-                roof = {"kernel": name, "bound": "tensor" if tensor_bound else "alu", "achieved": ach, "peak": peak, "unit": "TFLOP/s",
-                        "frac": ach / peak, "traffic": None, "launches": st["launches"], "avg_launch_ms": per_launch_ms,
-                        "peak_source": (pk["source"] + " (sustained bf16 GEMM)") if tensor_bound else "derived: 148 SMs x 128 FMA x 2 x 1.965 GHz",
-                        "share_of_kernel_time": st["ms"] / sum(v["ms"] for v in kstats.values())}
+                peak = pk["tensor"] if tensor else FMA_PEAK_TFLOPS
+                base.update({"bound": "tensor" if tensor else "alu", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
+                             "peak_source": (pk["source"] + ", sustained bf16 GEMM (kernel timed inside a long step)") if tensor
+                             else "derived: 148 SMs x 128 FMA x 2 x 1.965 GHz"})
             else:
                 ach = st["bytes"] / (st["ms"] * 1e-3) / 1e9
-                roof = {"kernel": name, "bound": "hbm", "achieved": ach, "peak": pk["hbm"], "unit": "GB/s", "frac": ach / pk["hbm"],
-                        "traffic": None, "launches": st["launches"], "avg_launch_ms": per_launch_ms, "peak_source": pk["source"],
-                        "share_of_kernel_time": st["ms"] / sum(v["ms"] for v in kstats.values())}
+                base.update({"bound": "hbm", "achieved": ach, "peak": pk["hbm"], "unit": "GB/s", "frac": ach / pk["hbm"], "peak_source": pk["source"]})
+            return base
+
+        roof = roofline_of(kstats)
+        if roof:
+            roof["timing"] = "CUDA events around every launch of the class inside the timed region; K module streams run concurrently, so a launch shares the GPU with other modules' kernels"
+        roof_alone = roofline_of(kstats_alone, roof["kernel"]) if (roof and kstats_alone) else None
+        if roof_alone:
+            roof_alone["timing"] = f"same class, separate pass of {alone_steps} steps with all modules on one stream (kernels do not share the GPU)"
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -260,6 +306,7 @@ def main():
                                      "frac_of_sustained_peak": flops_step / (ms / args.steps * 1e-3) / 1e12 / pk["tensor"],
                                      "peak_source": pk["source"]},
             "roofline": roof,
+            "roofline_uncontended": roof_alone,
             "kernels": {k: {"launches": v["launches"], "ms": round(v["ms"], 4),
                             "tflops": round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 2) if v["ms"] > 0 else None,
                             "gbs": round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1) if v["ms"] > 0 else None}
