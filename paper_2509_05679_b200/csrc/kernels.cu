@@ -573,26 +573,25 @@ __global__ void bn_bwd_apply_k(const T* __restrict__ x, const T* __restrict__ ou
 }
 
 // ------------------------------------------------------------------------------------------
-// batch-norm, bf16 storage, 128-bit accesses: a thread owns 8 consecutive channels and walks down
-// the rows of one worker, four rows in flight; grid = (row chunks, workers).  Used when C/8 is a
+// batch-norm, bf16 storage, 64-bit accesses: a thread owns 4 consecutive channels and walks down
+// the rows of one worker, four rows in flight; grid = (row chunks, workers).  Used when C/4 is a
 // power of two <= 256.
 // ------------------------------------------------------------------------------------------
 constexpr int BNV_THREADS = 256;
 constexpr int BNV_MAX_CHUNKS = 128;
-constexpr int BNV_UNROLL = 4;
+constexpr int BV = 4;                               // channels per thread (one 64-bit access)
 
-__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
-    const __nv_bfloat162* h = (const __nv_bfloat162*)&v;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) { float2 t = __bfloat1622float2(h[j]); f[2 * j] = t.x; f[2 * j + 1] = t.y; }
+__device__ __forceinline__ void unpack4(const uint2& v, float (&f)[BV]) {
+    const float2 a = __bfloat1622float2(*(const __nv_bfloat162*)&v.x), b = __bfloat1622float2(*(const __nv_bfloat162*)&v.y);
+    f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y;
 }
-__device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
-    uint4 v; __nv_bfloat162* h = (__nv_bfloat162*)&v;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) h[j] = __floats2bfloat162_rn(f[2 * j], f[2 * j + 1]);
+__device__ __forceinline__ uint2 pack4(const float (&f)[BV]) {
+    uint2 v;
+    __nv_bfloat162 a = __floats2bfloat162_rn(f[0], f[1]), b = __floats2bfloat162_rn(f[2], f[3]);
+    v.x = *(uint32_t*)&a; v.y = *(uint32_t*)&b;
     return v;
 }
-__device__ __forceinline__ uint4 ldg16(const bf16* p) { return __ldg((const uint4*)p); }
+__device__ __forceinline__ uint2 ldg8(const bf16* p) { return __ldg((const uint2*)p); }
 // the one expression both passes use for the normalised value, so that the backward pass can
 // recompute the sign of the forward output from x alone
 __device__ __forceinline__ float bn_value(float x, float mean, float istd, float g, float b) {
@@ -602,55 +601,55 @@ __device__ __forceinline__ float bn_value(float x, float mean, float istd, float
 // MODE 0: (sum x, sum x^2).  MODE 1: (sum dy, sum dy * xhat) with dy = dout * [forward output > 0] if relu.
 // mask_from_x: the forward output had no residual, so its sign is the sign of bn_value(x).
 template <int MODE>
-__global__ void __launch_bounds__(BNV_THREADS, MODE == 1 ? 2 : 3) bnv_reduce(const bf16* __restrict__ x, const bf16* __restrict__ out,
-                                                          const bf16* __restrict__ dout, const float* __restrict__ gamma,
-                                                          const float* __restrict__ beta, const float* __restrict__ stats,
-                                                          float* __restrict__ part, long rpw, int C, int relu, int mask_from_x) {
-    __shared__ float sh[BNV_THREADS][17];
-    const int cgs = C >> 3, rows_it = BNV_THREADS / cgs;
+__global__ void __launch_bounds__(BNV_THREADS, 3) bnv_reduce(const bf16* __restrict__ x, const bf16* __restrict__ out,
+                                                             const bf16* __restrict__ dout, const float* __restrict__ gamma,
+                                                             const float* __restrict__ beta, const float* __restrict__ stats,
+                                                             float* __restrict__ part, long rpw, int C, int relu, int mask_from_x) {
+    __shared__ float sh[BNV_THREADS][2 * BV + 1];
+    const int cgs = C / BV, rows_it = BNV_THREADS / cgs;
     const int cg = threadIdx.x % cgs, r = threadIdx.x / cgs;
     const int w = blockIdx.y, nw = gridDim.y;
     const long per = (rpw + gridDim.x - 1) / gridDim.x;
     const long r0 = (long)blockIdx.x * per, r1 = min(rpw, r0 + per);
-    float s1[8], s2[8], mean[8], istd[8], g[8], b[8];
+    float s1[BV], s2[BV], mean[BV], istd[BV], g[BV], b[BV];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
+    for (int j = 0; j < BV; ++j) {
         s1[j] = 0.f; s2[j] = 0.f;
         if (MODE == 1) {
-            const int c = cg * 8 + j;
+            const int c = cg * BV + j;
             mean[j] = stats[((size_t)w * C + c) * 2]; istd[j] = stats[((size_t)w * C + c) * 2 + 1];
             g[j] = gamma[c]; b[j] = beta[c];
         }
     }
-    const size_t base = (size_t)w * rpw * C + (size_t)cg * 8;
+    const size_t base = (size_t)w * rpw * C + (size_t)cg * BV;
     const bool need_out = MODE == 1 && relu && !mask_from_x;
-    constexpr int BNV_UNROLL = MODE == 1 ? 2 : 4;
-    for (long row = r0 + r; row < r1; row += (long)rows_it * BNV_UNROLL) {
-        uint4 xr[BNV_UNROLL], dr[BNV_UNROLL], orr[BNV_UNROLL];
+    constexpr int U = 4;
+    for (long row = r0 + r; row < r1; row += (long)rows_it * U) {
+        uint2 xr[U], dr[U], orr[U];
 #pragma unroll
-        for (int u = 0; u < BNV_UNROLL; ++u) {
+        for (int u = 0; u < U; ++u) {
             const long rr = row + (long)u * rows_it;
             if (rr < r1) {
                 const size_t o = base + (size_t)rr * C;
-                xr[u] = ldg16(x + o);
-                if (MODE == 1) dr[u] = ldg16(dout + o);
-                if (need_out) orr[u] = ldg16(out + o);
+                xr[u] = ldg8(x + o);
+                if (MODE == 1) dr[u] = ldg8(dout + o);
+                if (need_out) orr[u] = ldg8(out + o);
             }
         }
 #pragma unroll
-        for (int u = 0; u < BNV_UNROLL; ++u) {
+        for (int u = 0; u < U; ++u) {
             if (row + (long)u * rows_it >= r1) break;
-            float xv[8];
-            unpack8(xr[u], xv);
+            float xv[BV];
+            unpack4(xr[u], xv);
             if (MODE == 0) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) { s1[j] += xv[j]; s2[j] = fmaf(xv[j], xv[j], s2[j]); }
+                for (int j = 0; j < BV; ++j) { s1[j] += xv[j]; s2[j] = fmaf(xv[j], xv[j], s2[j]); }
             } else {
-                float dv[8], ov[8];
-                unpack8(dr[u], dv);
-                if (need_out) unpack8(orr[u], ov);
+                float dv[BV], ov[BV];
+                unpack4(dr[u], dv);
+                if (need_out) unpack4(orr[u], ov);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
+                for (int j = 0; j < BV; ++j) {
                     float dy = dv[j];
                     if (relu) { float f = mask_from_x ? bn_value(xv[j], mean[j], istd[j], g[j], b[j]) : ov[j]; if (!(f > 0.f)) dy = 0.f; }
                     s1[j] += dy; s2[j] = fmaf(dy, (xv[j] - mean[j]) * istd[j], s2[j]);
@@ -659,93 +658,94 @@ __global__ void __launch_bounds__(BNV_THREADS, MODE == 1 ? 2 : 3) bnv_reduce(con
         }
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) { sh[threadIdx.x][j] = s1[j]; sh[threadIdx.x][8 + j] = s2[j]; }
+    for (int j = 0; j < BV; ++j) { sh[threadIdx.x][j] = s1[j]; sh[threadIdx.x][BV + j] = s2[j]; }
     __syncthreads();
-    // thread t < 16 * cgs sums one (channel group, value) column over the rows_it row lanes, in a fixed order
-    for (int t = threadIdx.x; t < cgs * 16; t += BNV_THREADS) {
-        const int q = t >> 4, k = t & 15;
+    // thread t < 2*BV*cgs sums one (channel group, value) column over the rows_it row lanes, in a fixed order
+    for (int t = threadIdx.x; t < cgs * 2 * BV; t += BNV_THREADS) {
+        const int q = t / (2 * BV), k = t % (2 * BV);
         float acc = 0.f;
         for (int rr = 0; rr < rows_it; ++rr) acc += sh[rr * cgs + q][k];
-        const int c = q * 8 + (k & 7);
-        part[(((size_t)blockIdx.x * nw + w) * C + c) * 2 + (k >> 3)] = acc;
+        const int c = q * BV + (k % BV);
+        part[(((size_t)blockIdx.x * nw + w) * C + c) * 2 + (k / BV)] = acc;
     }
 }
 
-__global__ void __launch_bounds__(BNV_THREADS) bnv_apply(const bf16* __restrict__ x, const float* __restrict__ gamma,
-                                                         const float* __restrict__ beta, const bf16* __restrict__ res,
-                                                         bf16* __restrict__ y, const float* __restrict__ stats, long rpw, int C, int relu) {
-    const int cgs = C >> 3, rows_it = BNV_THREADS / cgs;
+__global__ void __launch_bounds__(BNV_THREADS, 4) bnv_apply(const bf16* __restrict__ x, const float* __restrict__ gamma,
+                                                            const float* __restrict__ beta, const bf16* __restrict__ res,
+                                                            bf16* __restrict__ y, const float* __restrict__ stats, long rpw, int C, int relu) {
+    const int cgs = C / BV, rows_it = BNV_THREADS / cgs;
     const int cg = threadIdx.x % cgs, r = threadIdx.x / cgs;
     const int w = blockIdx.y;
     const long per = (rpw + gridDim.x - 1) / gridDim.x;
     const long r0 = (long)blockIdx.x * per, r1 = min(rpw, r0 + per);
-    float mean[8], istd[8], g[8], b[8];
+    float mean[BV], istd[BV], g[BV], b[BV];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const int c = cg * 8 + j;
+    for (int j = 0; j < BV; ++j) {
+        const int c = cg * BV + j;
         mean[j] = stats[((size_t)w * C + c) * 2]; istd[j] = stats[((size_t)w * C + c) * 2 + 1];
         g[j] = gamma[c]; b[j] = beta[c];
     }
-    const size_t base = (size_t)w * rpw * C + (size_t)cg * 8;
-    for (long row = r0 + r; row < r1; row += (long)rows_it * BNV_UNROLL) {
-        uint4 xr[BNV_UNROLL], rr_[BNV_UNROLL];
+    const size_t base = (size_t)w * rpw * C + (size_t)cg * BV;
+    constexpr int U = 4;
+    for (long row = r0 + r; row < r1; row += (long)rows_it * U) {
+        uint2 xr[U], rr_[U];
 #pragma unroll
-        for (int u = 0; u < BNV_UNROLL; ++u) {
+        for (int u = 0; u < U; ++u) {
             const long rr = row + (long)u * rows_it;
-            if (rr < r1) { const size_t o = base + (size_t)rr * C; xr[u] = ldg16(x + o); if (res) rr_[u] = ldg16(res + o); }
+            if (rr < r1) { const size_t o = base + (size_t)rr * C; xr[u] = ldg8(x + o); if (res) rr_[u] = ldg8(res + o); }
         }
 #pragma unroll
-        for (int u = 0; u < BNV_UNROLL; ++u) {
+        for (int u = 0; u < U; ++u) {
             const long rr = row + (long)u * rows_it;
             if (rr >= r1) break;
-            float xv[8], rv[8];
-            unpack8(xr[u], xv);
-            if (res) unpack8(rr_[u], rv);
+            float xv[BV], rv[BV];
+            unpack4(xr[u], xv);
+            if (res) unpack4(rr_[u], rv);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
+            for (int j = 0; j < BV; ++j) {
                 float v = bn_value(xv[j], mean[j], istd[j], g[j], b[j]);
                 if (res) v += rv[j];
                 if (relu) v = fmaxf(v, 0.f);
                 xv[j] = v;
             }
-            *(uint4*)(y + base + (size_t)rr * C) = pack8(xv);
+            *(uint2*)(y + base + (size_t)rr * C) = pack4(xv);
         }
     }
 }
 
-__global__ void __launch_bounds__(BNV_THREADS, 2) bnv_bwd_apply(const bf16* __restrict__ x, const bf16* __restrict__ out,
-                                                             const bf16* __restrict__ dout, const float* __restrict__ gamma,
-                                                             const float* __restrict__ beta, const float* __restrict__ stats,
-                                                             const float* __restrict__ red, bf16* __restrict__ dx, int accum_dx,
-                                                             bf16* __restrict__ dres, int accum_dres, long rpw, int C, int relu,
-                                                             int mask_from_x) {
-    const int cgs = C >> 3, rows_it = BNV_THREADS / cgs;
+__global__ void __launch_bounds__(BNV_THREADS, 3) bnv_bwd_apply(const bf16* __restrict__ x, const bf16* __restrict__ out,
+                                                                const bf16* __restrict__ dout, const float* __restrict__ gamma,
+                                                                const float* __restrict__ beta, const float* __restrict__ stats,
+                                                                const float* __restrict__ red, bf16* __restrict__ dx, int accum_dx,
+                                                                bf16* __restrict__ dres, int accum_dres, long rpw, int C, int relu,
+                                                                int mask_from_x) {
+    const int cgs = C / BV, rows_it = BNV_THREADS / cgs;
     const int cg = threadIdx.x % cgs, r = threadIdx.x / cgs;
     const int w = blockIdx.y;
     const long per = (rpw + gridDim.x - 1) / gridDim.x;
     const long r0 = (long)blockIdx.x * per, r1 = min(rpw, r0 + per);
     const float inv_n = 1.f / (float)rpw;
-    float mean[8], istd[8], g[8], b[8], c1[8], c2[8];
+    float mean[BV], istd[BV], g[BV], b[BV], c1[BV], c2[BV];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const int c = cg * 8 + j;
+    for (int j = 0; j < BV; ++j) {
+        const int c = cg * BV + j;
         const size_t so = ((size_t)w * C + c) * 2;
         mean[j] = stats[so]; istd[j] = stats[so + 1];
         g[j] = gamma[c]; b[j] = beta[c];
         c1[j] = red[so] * inv_n; c2[j] = red[so + 1] * inv_n;
     }
-    const size_t base = (size_t)w * rpw * C + (size_t)cg * 8;
+    const size_t base = (size_t)w * rpw * C + (size_t)cg * BV;
     const bool need_out = relu && !mask_from_x;
     constexpr int U = 2;
     for (long row = r0 + r; row < r1; row += (long)rows_it * U) {
-        uint4 xr[U], dr[U], orr[U];
+        uint2 xr[U], dr[U], orr[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const long rr = row + (long)u * rows_it;
             if (rr < r1) {
                 const size_t o = base + (size_t)rr * C;
-                xr[u] = ldg16(x + o); dr[u] = ldg16(dout + o);
-                if (need_out) orr[u] = ldg16(out + o);
+                xr[u] = ldg8(x + o); dr[u] = ldg8(dout + o);
+                if (need_out) orr[u] = ldg8(out + o);
             }
         }
 #pragma unroll
@@ -753,28 +753,28 @@ __global__ void __launch_bounds__(BNV_THREADS, 2) bnv_bwd_apply(const bf16* __re
             const long rr = row + (long)u * rows_it;
             if (rr >= r1) break;
             const size_t o = base + (size_t)rr * C;
-            float xv[8], dv[8], ov[8], t[8];
-            unpack8(xr[u], xv); unpack8(dr[u], dv);
-            if (need_out) unpack8(orr[u], ov);
+            float xv[BV], dv[BV], ov[BV], t[BV];
+            unpack4(xr[u], xv); unpack4(dr[u], dv);
+            if (need_out) unpack4(orr[u], ov);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
+            for (int j = 0; j < BV; ++j) {
                 if (relu) { float f = mask_from_x ? bn_value(xv[j], mean[j], istd[j], g[j], b[j]) : ov[j]; if (!(f > 0.f)) dv[j] = 0.f; }
                 const float xh = (xv[j] - mean[j]) * istd[j];
                 t[j] = g[j] * istd[j] * (dv[j] - c1[j] - xh * c2[j]);
             }
             if (accum_dx) {
-                float old[8]; unpack8(*(const uint4*)(dx + o), old);
+                float old[BV]; unpack4(*(const uint2*)(dx + o), old);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) t[j] += old[j];
+                for (int j = 0; j < BV; ++j) t[j] += old[j];
             }
-            *(uint4*)(dx + o) = pack8(t);
+            *(uint2*)(dx + o) = pack4(t);
             if (dres) {
                 if (accum_dres) {
-                    float old[8]; unpack8(*(const uint4*)(dres + o), old);
+                    float old[BV]; unpack4(*(const uint2*)(dres + o), old);
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) dv[j] += old[j];
+                    for (int j = 0; j < BV; ++j) dv[j] += old[j];
                 }
-                *(uint4*)(dres + o) = pack8(dv);
+                *(uint2*)(dres + o) = pack4(dv);
             }
         }
     }
@@ -845,10 +845,17 @@ __global__ void bnv_bwd_final(const float* __restrict__ part, float* __restrict_
     }
 }
 
-static bool bnv_ok(int dt, int C) { int cgs = C >> 3; return dt == 1 && C % 8 == 0 && cgs <= BNV_THREADS && (cgs & (cgs - 1)) == 0; }
-static int bnv_chunks(int nw, long rpw, int C) {
-    long rows_it = BNV_THREADS / (C >> 3);
-    long want = (148 * 4 + nw - 1) / nw, maxc = (rpw + rows_it * 4 - 1) / (rows_it * 4);
+static bool bnv_ok(int dt, int C) { int cgs = C / BV; return dt == 1 && C % BV == 0 && cgs <= BNV_THREADS && (cgs & (cgs - 1)) == 0; }
+// Row chunks per worker such that chunks * nw CTAs fill the GPU exactly once (no partial second wave).
+template <typename K>
+static int bnv_chunks(K kernel, int which, int nw, long rpw, int C) {
+    static int occ_cache[4] = {0, 0, 0, 0}, sms = 0;
+    if (!sms) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); if (sms <= 0) sms = 148; }
+    if (!occ_cache[which] && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_cache[which], kernel, BNV_THREADS, 0) != cudaSuccess || occ_cache[which] < 1))
+        occ_cache[which] = 2;
+    const int occ = occ_cache[which];
+    long rows_it = BNV_THREADS / (C / BV);
+    long want = ((long)sms * occ) / nw, maxc = (rpw + rows_it * 4 - 1) / (rows_it * 4);
     long c = want < maxc ? want : maxc;
     if (c > BNV_MAX_CHUNKS) c = BNV_MAX_CHUNKS;
     return (int)(c < 1 ? 1 : c);
@@ -859,9 +866,10 @@ bool bn_accepts_conv_partials(int dt, int C) { return bnv_ok(dt, C); }
 void bn_forward(int dt, const void* x, const float* gamma, const float* beta, const void* res, void* y, float* stats,
                 float* scratch, int nw, long rpw, int C, bool relu, const float* conv_part, int conv_chunks, cudaStream_t s) {
     if (bnv_ok(dt, C)) {
-        const int chunks = bnv_chunks(nw, rpw, C);
+        const int chunks = bnv_chunks(bnv_reduce<0>, 0, nw, rpw, C);
+        const int chunks_a = bnv_chunks(bnv_apply, 1, nw, rpw, C);
         const double total = (double)nw * rpw * C;
-        dim3 grid(chunks, nw);
+        dim3 grid(chunks, nw), grid_a(chunks_a, nw);
         if (conv_part) {
             Scope sc(KC_BN_FWD_STATS, 0.0, 8.0 * conv_chunks * nw * C, s);
             bnv_stats_final_tiles<<<nw * C, 128, 0, s>>>(conv_part, stats, conv_chunks, nw, C, rpw);
@@ -872,7 +880,7 @@ void bn_forward(int dt, const void* x, const float* gamma, const float* beta, co
               bnv_stats_final<<<cdiv((size_t)nw * C * 32, 256), 256, 0, s>>>(scratch, stats, chunks, nw * C, rpw); }
         }
         Scope sc(KC_BN_FWD_APPLY, 0.0, 2.0 * total * (res ? 3 : 2), s);
-        bnv_apply<<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, gamma, beta, (const bf16*)res, (bf16*)y, stats, rpw, C, relu);
+        bnv_apply<<<grid_a, BNV_THREADS, 0, s>>>((const bf16*)x, gamma, beta, (const bf16*)res, (bf16*)y, stats, rpw, C, relu);
         return;
     }
     int chunks = (int)(rpw < RED_CHUNKS ? rpw : RED_CHUNKS);
@@ -893,7 +901,8 @@ void bn_backward(int dt, const void* x, const void* out, const void* dout, const
                  const float* stats, void* dx, bool accum_dx, void* dres, bool accum_dres, float* dgamma, float* dbeta, float* red,
                  float* scratch, int nw, long rpw, int C, bool relu, bool has_res, cudaStream_t s) {
     if (bnv_ok(dt, C)) {
-        const int chunks = bnv_chunks(nw, rpw, C);
+        const int chunks = bnv_chunks(bnv_reduce<1>, 2, nw, rpw, C);
+        const int chunks_a = bnv_chunks(bnv_bwd_apply, 3, nw, rpw, C);
         const double total = (double)nw * rpw * C;
         const int mask_from_x = relu && !has_res;
         const int reads = 2 + ((relu && !mask_from_x) ? 1 : 0);
@@ -905,7 +914,7 @@ void bn_backward(int dt, const void* x, const void* out, const void* dout, const
           if (nw <= 32) bnv_bwd_final<<<C, 32 * nw, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C);
           else bn_bwd_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C); }
         Scope sc(KC_BN_BWD_APPLY, 0.0, 2.0 * total * (reads + 1 + (accum_dx ? 1 : 0) + (dres ? (accum_dres ? 2 : 1) : 0)), s);
-        bnv_bwd_apply<<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, gamma, beta, stats, red, (bf16*)dx,
+        bnv_bwd_apply<<<dim3(chunks_a, nw), BNV_THREADS, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, gamma, beta, stats, red, (bf16*)dx,
                                                    accum_dx, (bf16*)dres, accum_dres, rpw, C, relu, mask_from_x);
         return;
     }
