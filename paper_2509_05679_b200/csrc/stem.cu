@@ -18,7 +18,7 @@ bool stem_supported(int dt, const ConvGeom& g) {
     if (!pow2(g.W) || g.W < 8 || g.W > 64) return false;
     return g.H % (ST_THREADS / g.W) == 0;
 }
-int stem_wgrad_blocks() { return 2 * 148; }
+int stem_wgrad_blocks() { return 4 * 148; }
 size_t stem_wgrad_workspace_elems(const ConvGeom& g) { return (size_t)stem_wgrad_blocks() * 64 * 9 * g.C * (g.Co / 64); }
 
 // x tile with a one-pixel zero border, as fp32: xs[(TH+2)][(W+2)][C]
@@ -121,17 +121,20 @@ __global__ void __launch_bounds__(ST_THREADS) stem_wgrad_kernel(const bf16* __re
             *(uint4*)(dys + pix * 64 + part * 8) = *(const uint4*)(src + (size_t)pix * Co + part * 8);
         }
         __syncthreads();
+#pragma unroll 4
         for (int pi = 0; pi < 64; ++pi) {
             const int pix = ps * 64 + pi;
             const int row = pix / W, col = pix - row * W;
             const uint2 raw = *(const uint2*)(dys + pix * 64 + cg * 4);
             const float2 d01 = __bfloat1622float2(*(const __nv_bfloat162*)&raw.x), d23 = __bfloat1622float2(*(const __nv_bfloat162*)&raw.y);
             const float* xb = xs + (row * tw + col) * C;
+            float xv[7];
+#pragma unroll
+            for (int j = 0; j < 7; ++j) xv[j] = xb[off[j]];          // off[j] of a padded column points at a valid (unused) slot
 #pragma unroll
             for (int j = 0; j < 7; ++j) {
-                const float xv = kv[j] ? xb[off[j]] : 0.f;
-                acc[j][0] = fmaf(d01.x, xv, acc[j][0]); acc[j][1] = fmaf(d01.y, xv, acc[j][1]);
-                acc[j][2] = fmaf(d23.x, xv, acc[j][2]); acc[j][3] = fmaf(d23.y, xv, acc[j][3]);
+                acc[j][0] = fmaf(d01.x, xv[j], acc[j][0]); acc[j][1] = fmaf(d01.y, xv[j], acc[j][1]);
+                acc[j][2] = fmaf(d23.x, xv[j], acc[j][2]); acc[j][3] = fmaf(d23.y, xv[j], acc[j][3]);
             }
         }
     }

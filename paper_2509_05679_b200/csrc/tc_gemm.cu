@@ -137,13 +137,15 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 }
 constexpr int EPI_ROW_WORDS = 36;                 // 32 fp32 + 4 padding: conflict-free 128-bit rows
 
-template <int N_TILE, int STAGES>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+// EPI_WARPS = 4 or 8: with 8, two warps share each quarter of the tensor-memory lanes and take alternate 32-column slices.
+template <int N_TILE, int STAGES, int EPI_WARPS>
+__global__ void __launch_bounds__(64 + 32 * EPI_WARPS, 1)
 km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, KmParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
     constexpr int A_BYTES = BLOCK_M * BLOCK_K * 2, B_BYTES = N_TILE * BLOCK_K * 2, STAGE_BYTES = A_BYTES + B_BYTES;
-    constexpr int EPI_BYTES = 4 * 32 * EPI_ROW_WORDS * 4;
+    constexpr int EPI_BYTES = EPI_WARPS * 32 * EPI_ROW_WORDS * 4;
+    constexpr int COL_STEP = 32 * (EPI_WARPS / 4);
     constexpr uint32_t TMEM_COLS = 2 * N_TILE;
     float* epi_smem = (float*)(smem + STAGES * STAGE_BYTES);
     uint64_t* full = (uint64_t*)(smem + STAGES * STAGE_BYTES + EPI_BYTES);
@@ -161,7 +163,7 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     if (threadIdx.x == 0) {
         tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB);
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], EPI_WARPS); }
         fence_barrier_init();
     }
     if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);
@@ -215,8 +217,8 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         }
     } else {
         // ---- epilogue: warp q = warp % 4 owns tensor-memory lanes 32q .. 32q+31 (= tile rows)
-        const int q = warp & 3;
-        float* stage = epi_smem + q * 32 * EPI_ROW_WORDS;
+        const int q = warp & 3, half = (warp - 2) >> 2;
+        float* stage = epi_smem + (warp - 2) * 32 * EPI_ROW_WORDS;
         int ti = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++ti) {
@@ -236,10 +238,10 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             ok = mbar_wait(&tmem_full[buf], use & 1, p.err, 3);
             tc_fence_after();
 #pragma unroll 1
-            for (int c = 0; c < N_TILE; c += 32) {
+            for (int c = half * 32; c < N_TILE; c += COL_STEP) {
                 uint32_t v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * N_TILE + c, v);
-                if (c + 32 >= N_TILE) {            // last read of this accumulator: hand the buffer back to the MMA warp
+                if (c + COL_STEP >= N_TILE) {      // this warp's last read of the accumulator: hand the buffer back to the MMA warp
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&tmem_empty[buf]);
@@ -483,26 +485,26 @@ static int sm_count() {
     return n;
 }
 
-template <int N_TILE, int STAGES>
+template <int N_TILE, int STAGES, int EPI_WARPS>
 static cudaError_t launch_km(const TensorMap& a, const TensorMap& b, const KmParams& p, cudaStream_t s) {
-    constexpr int smem = STAGES * (BLOCK_M * BLOCK_K * 2 + N_TILE * BLOCK_K * 2) + 4 * 32 * EPI_ROW_WORDS * 4 + 1024 + 256;
+    constexpr int smem = STAGES * (BLOCK_M * BLOCK_K * 2 + N_TILE * BLOCK_K * 2) + EPI_WARPS * 32 * EPI_ROW_WORDS * 4 + 1024 + 256;
     static bool attr = false;
     if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(km_kernel<N_TILE, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaError_t e = cudaFuncSetAttribute(km_kernel<N_TILE, STAGES, EPI_WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         attr = true;
     }
     const int total = p.tiles_w * p.tiles_h * p.tiles_n * (p.Cn / N_TILE);
-    const int slots = sm_count() * (smem <= 100 * 1024 ? 2 : 1);       // the 64-column variant fits twice on an SM
+    const int slots = sm_count() * (smem <= 113 * 1024 ? 2 : 1);       // the 64-column variant fits twice on an SM
     const int grid = total < slots ? total : slots;
-    km_kernel<N_TILE, STAGES><<<grid, NUM_THREADS, smem, s>>>(*(const CUtensorMap*)&a, *(const CUtensorMap*)&b, p);
+    km_kernel<N_TILE, STAGES, EPI_WARPS><<<grid, 64 + 32 * EPI_WARPS, smem, s>>>(*(const CUtensorMap*)&a, *(const CUtensorMap*)&b, p);
     return cudaGetLastError();
 }
 
 cudaError_t run_km(const TensorMap& a, const TensorMap& b, const KmParams& p, int n_tile, cudaStream_t s) {
-    if (n_tile == 64) return launch_km<64, 3>(a, b, p, s);
-    if (n_tile == 128) return launch_km<128, 6>(a, b, p, s);
-    if (n_tile == 256) return launch_km<256, 4>(a, b, p, s);
+    if (n_tile == 64) return launch_km<64, 3, 4>(a, b, p, s);
+    if (n_tile == 128) return launch_km<128, 5, 8>(a, b, p, s);
+    if (n_tile == 256) return launch_km<256, 4, 4>(a, b, p, s);
     return cudaErrorInvalidValue;
 }
 
