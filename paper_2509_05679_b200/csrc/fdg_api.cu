@@ -61,7 +61,7 @@ struct Op {
     char shape[40];                                          // "HxW Cin->Cout kR sS", the profiler's detail tag
     int n_tile_f, n_tile_d, n_tile_w, wg_splits;
     tc::KmParams kf;
-    std::vector<tc::KmParams> kd;                            // one per output-parity class (1 for stride 1, up to 4 for stride 2)
+    tc::KmParams kd;                                         // all output-parity classes of the input gradient in one launch
     bool dgrad_needs_zero;                                   // some parity classes receive no gradient (1x1 stride 2)
     int stat_chunks;                                         // > 0: the forward epilogue also leaves batch-norm partial sums
                                                              //      (this many per worker) for the batch-norm that follows
@@ -376,16 +376,12 @@ bool tc_dgrad(fdg_ctx* c, Module& m, const Op& o, char* dy, char* dx, int64_t ve
         Scope sc(KC_TC_AUX, 0.0, 2.0 * rows * g.C, s);
         cudaMemsetAsync(dx, 0, (size_t)rows * g.C * 2, s);
     }
-    bool ok = true;
-    for (const tc::KmParams& cls : o.kd) {
-        tc::KmParams p = cls;
-        p.bias = nullptr; p.out = dx; p.epi = accum ? EPI_ACCUM : 0; p.err = c->tc_err; p.stat_part = nullptr;
-        double crows = (double)g.N * p.Hd * p.Wd;
-        Scope sc(KC_TC_DGRAD, 2.0 * crows * g.C * p.ntaps * g.Co,
-                 2.0 * ((double)g.N * g.Ho * g.Wo * g.Co + (double)g.Co * p.ntaps * g.C + crows * g.C * (accum ? 2 : 1)), s);
-        ok = ok && tc::run_km(o.da[ia], o.db[version % m.D], p, o.n_tile_d, s) == cudaSuccess;
-    }
-    return ok;
+    tc::KmParams p = o.kd;
+    p.bias = nullptr; p.out = dx; p.epi = accum ? EPI_ACCUM : 0; p.err = c->tc_err; p.stat_part = nullptr;
+    const double crows = (double)g.N * p.Hd * p.Wd;          // pixels of one class; every tap belongs to exactly one class
+    Scope sc(KC_TC_DGRAD, 2.0 * crows * g.C * p.ntaps * g.Co,
+             2.0 * ((double)g.N * g.Ho * g.Wo * g.Co + (double)g.Co * p.ntaps * g.C + crows * p.ncls * g.C * (accum ? 2 : 1)), s);
+    return tc::run_km(o.da[ia], o.db[version % m.D], p, o.n_tile_d, s) == cudaSuccess;
 }
 bool tc_wgrad(fdg_ctx* c, Module& m, const Op& o, char* x, char* dy, float* dw, cudaStream_t s) {
     int ix = find_buf(o.a_ptrs, x), id = find_buf(o.dy_ptrs, dy);
@@ -525,7 +521,8 @@ bool build_tc_plans(fdg_ctx* c) {
             f.Wt = wt; f.Ht = ht; f.Nt = nt; f.tiles_w = g.Wo / wt; f.tiles_h = g.Ho / ht; f.tiles_n = (g.N + nt - 1) / nt;
             f.ntaps = taps; f.kchunks = g.C / 64; f.xs = g.stride;
             for (int t = 0; t < taps; ++t) { f.dh[t] = t / g.R - g.pad; f.dw[t] = t % g.R - g.pad; f.koff[t] = t * g.C; }
-            f.N = g.N; f.Hd = g.Ho; f.Wd = g.Wo; f.Ho = g.Ho; f.Wo = g.Wo; f.Co = g.Co; f.os = 1; f.oph = 0; f.opw = 0; f.Cn = g.Co;
+            f.N = g.N; f.Hd = g.Ho; f.Wd = g.Wo; f.Ho = g.Ho; f.Wo = g.Wo; f.Co = g.Co; f.os = 1; f.Cn = g.Co;
+            f.ncls = 1; f.cls_tap0[0] = 0; f.cls_tap0[1] = taps; f.cls_oph[0] = 0; f.cls_opw[0] = 0;
             o.fa.resize(o.a_ptrs.size());
             for (size_t i = 0; i < o.a_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.fa[i], o.a_ptrs[i], g.C, g.W, g.H, g.N, 64, wt, ht, nt, g.stride);
             o.fb.resize(m.D);
@@ -534,10 +531,12 @@ bool build_tc_plans(fdg_ctx* c) {
             // the stride of dy[n, (h + pad - r) / stride, (w + pad - s) / stride, :] . W[:, r, s, :].
             // One launch per parity class (h mod stride, w mod stride); the class's pixels form a dense grid of the
             // size of dy.  A = dy (dense boxes), B = Wt [C][taps * Co] with flipped taps, output strided into dx.
-            o.kd.clear(); o.dgrad_needs_zero = false;
+            o.dgrad_needs_zero = false;
+            tc::KmParams& d = o.kd; d = f;
+            d.kchunks = g.Co / 64; d.xs = 1; d.ntaps = 0; d.ncls = 0;
+            d.Hd = g.H / g.stride; d.Wd = g.W / g.stride; d.Ho = g.H; d.Wo = g.W; d.Co = g.C; d.Cn = g.C; d.os = g.stride;
             for (int ph = 0; ph < g.stride; ++ph) for (int pw = 0; pw < g.stride; ++pw) {
-                tc::KmParams d = f;
-                d.kchunks = g.Co / 64; d.xs = 1; d.ntaps = 0;
+                const int first = d.ntaps;
                 for (int r = 0; r < g.R; ++r) for (int q = 0; q < g.R; ++q) {
                     int a = ph + g.pad - r, b = pw + g.pad - q;
                     if (a % g.stride != 0 || b % g.stride != 0) continue;
@@ -545,10 +544,9 @@ bool build_tc_plans(fdg_ctx* c) {
                     d.koff[d.ntaps] = (taps - 1 - (r * g.R + q)) * g.Co;
                     ++d.ntaps;
                 }
-                if (d.ntaps == 0) { o.dgrad_needs_zero = true; continue; }
-                d.Hd = g.H / g.stride; d.Wd = g.W / g.stride; d.Ho = g.H; d.Wo = g.W; d.Co = g.C; d.Cn = g.C;
-                d.os = g.stride; d.oph = ph; d.opw = pw;
-                o.kd.push_back(d);
+                if (d.ntaps == first) { o.dgrad_needs_zero = true; continue; }
+                d.cls_tap0[d.ncls] = first; d.cls_oph[d.ncls] = ph; d.cls_opw[d.ncls] = pw; ++d.ncls;
+                d.cls_tap0[d.ncls] = d.ntaps;
             }
             o.da.resize(o.dy_ptrs.size());
             for (size_t i = 0; i < o.dy_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.da[i], o.dy_ptrs[i], g.Co, g.Wo, g.Ho, g.N, 64, wt, ht, nt, 1);

@@ -157,8 +157,8 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tiles_m = p.tiles_w * p.tiles_h * p.tiles_n;
     const int tiles_c = p.Cn / N_TILE;
-    const int total = tiles_m * tiles_c;
-    const int num_kb = p.ntaps * p.kchunks;
+    const int per_cls = tiles_m * tiles_c;
+    const int total = per_cls * p.ncls;                 // tile index = (class, pixel tile, column tile), column tile fastest
 
     if (threadIdx.x == 0) {
         tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB);
@@ -177,14 +177,16 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             int kbg = 0;                                              // k-blocks issued so far, over all tiles
             bool ok = true;
             for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
-                int tm = tile / tiles_c; const int co0 = (tile - tm * tiles_c) * N_TILE;
+                const int cls = tile / per_cls, tl = tile - cls * per_cls;
+                int tm = tl / tiles_c; const int co0 = (tl - tm * tiles_c) * N_TILE;
                 const int tw = tm % p.tiles_w; tm /= p.tiles_w;
                 const int th = tm % p.tiles_h; const int tn = tm / p.tiles_h;
                 const int w0 = tw * p.Wt, h0 = th * p.Ht, n0 = tn * p.Nt;
+                const int tap0 = p.cls_tap0[cls], num_kb = (p.cls_tap0[cls + 1] - tap0) * p.kchunks;
                 for (int kb = 0; kb < num_kb; ++kb, ++kbg) {
                     const int s = kbg % STAGES, it = kbg / STAGES;
                     if (it > 0 && !mbar_wait(&empty[s], (it - 1) & 1, p.err, 1)) { ok = false; break; }
-                    const int tap = kb / p.kchunks, kc = kb - tap * p.kchunks;
+                    const int tq = kb / p.kchunks, kc = kb - tq * p.kchunks, tap = tap0 + tq;
                     uint8_t* a = smem + s * STAGE_BYTES;
                     mbar_expect_tx(&full[s], STAGE_BYTES);
                     tma_load_4d(a, &tmA, &full[s], kc * BLOCK_K, w0 * p.xs + p.dw[tap], h0 * p.xs + p.dh[tap], n0);
@@ -199,6 +201,8 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             bool ok = true;
             for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++ti) {
                 const int buf = ti & 1, use = ti >> 1;
+                const int cls = tile / per_cls;
+                const int num_kb = (p.cls_tap0[cls + 1] - p.cls_tap0[cls]) * p.kchunks;
                 if (use > 0 && !mbar_wait(&tmem_empty[buf], (use - 1) & 1, p.err, 7)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d = tmem_base + buf * N_TILE;
@@ -223,7 +227,8 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         bool ok = true;
         for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++ti) {
             const int buf = ti & 1, use = ti >> 1;
-            int tm = tile / tiles_c; const int co0 = (tile - tm * tiles_c) * N_TILE;
+            const int cls = tile / per_cls, tl = tile - cls * per_cls;
+            int tm = tl / tiles_c; const int co0 = (tl - tm * tiles_c) * N_TILE;
             const int tmi = tm;
             const int tw = tm % p.tiles_w; tm /= p.tiles_w;
             const int th = tm % p.tiles_h; const int tn = tm / p.tiles_h;
@@ -232,8 +237,8 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             const int pw = row % p.Wt, ph = (row / p.Wt) % p.Ht, pn = row / (p.Wt * p.Ht);
             const int n = tn * p.Nt + pn, h = th * p.Ht + ph, w = tw * p.Wt + pw;
             const bool valid = n < p.N && h < p.Hd && w < p.Wd;
-            const unsigned long long rowptr = valid ? (unsigned long long)((bf16*)p.out + (((size_t)n * p.Ho + (h * p.os + p.oph)) * p.Wo +
-                                                                                                (w * p.os + p.opw)) * p.Co + co0) : 0ull;
+            const unsigned long long rowptr = valid ? (unsigned long long)((bf16*)p.out + (((size_t)n * p.Ho + (h * p.os + p.cls_oph[cls])) * p.Wo +
+                                                                                                (w * p.os + p.cls_opw[cls])) * p.Co + co0) : 0ull;
             const unsigned vmask = __ballot_sync(0xffffffffu, rowptr != 0ull);
             ok = mbar_wait(&tmem_full[buf], use & 1, p.err, 3);
             tc_fence_after();
@@ -494,7 +499,7 @@ static cudaError_t launch_km(const TensorMap& a, const TensorMap& b, const KmPar
         if (e != cudaSuccess) return e;
         attr = true;
     }
-    const int total = p.tiles_w * p.tiles_h * p.tiles_n * (p.Cn / N_TILE);
+    const int total = p.tiles_w * p.tiles_h * p.tiles_n * (p.Cn / N_TILE) * p.ncls;
     const int slots = sm_count() * (smem <= 113 * 1024 ? 2 : 1);       // the 64-column variant fits twice on an SM
     const int grid = total < slots ? total : slots;
     km_kernel<N_TILE, STAGES, EPI_WARPS><<<grid, 64 + 32 * EPI_WARPS, smem, s>>>(*(const CUtensorMap*)&a, *(const CUtensorMap*)&b, p);

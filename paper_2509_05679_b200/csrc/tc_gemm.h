@@ -14,10 +14,13 @@ struct alignas(64) TensorMap { unsigned char bytes[128]; };     // a CUtensorMap
 // (output pixels for forward; for a stride-2 input gradient one parity class of the input pixels).
 struct KmParams {
     int Wt, Ht, Nt, tiles_w, tiles_h, tiles_n;   // 128-pixel tile = Wt x Ht x Nt, and how many tiles per axis
-    int ntaps, kchunks, xs;                      // filter taps, 64-channel chunks per tap, coordinate scale of the A map
+    int ntaps, kchunks, xs;                      // filter taps (all classes), 64-channel chunks per tap, coordinate scale of the A map
     int dh[9], dw[9], koff[9];                   // per tap: spatial shift of the A box, column offset into B
+    int ncls;                                    // output-parity classes handled by one launch (1, or up to 4 for a stride-2 input gradient)
+    int cls_tap0[5];                             // class c uses taps [cls_tap0[c], cls_tap0[c+1])
+    int cls_oph[4], cls_opw[4];                  // class c writes domain pixel (h, w) to (h*os + cls_oph[c], w*os + cls_opw[c])
     int N, Hd, Wd;                               // extents of the tile domain (rows outside are not stored)
-    int Ho, Wo, Co, os, oph, opw;                // output tensor [N,Ho,Wo,Co]; domain pixel (h,w) -> (h*os+oph, w*os+opw)
+    int Ho, Wo, Co, os;                          // output tensor [N,Ho,Wo,Co] and the output stride of a domain pixel
     int Cn;                                      // output channels computed (multiple of the column tile)
     int epi;                                     // EPI_RELU | EPI_ACCUM
     const float* bias;                           // or nullptr
