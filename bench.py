@@ -100,6 +100,21 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (the job is as slow as its slowest replica)."""
+    if dist is None:
+        return [float(v) for v in values]
+    import torch
+    t = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_throughput(samples_per_rank_step: int, steps: int, world: int, seconds: float) -> float:
+    """samples/s of the whole job: every rank is an independent replica processing its own batches."""
+    return samples_per_rank_step * steps * world / seconds
+
+
 def oracle_sample(net: sy.Net, timed_steps: int, warm_steps: int):
     """The CPU oracle, as it stands, on a bounded sample of the workload: same network, same K, same
     number of workers, ONE sample per worker; the pipeline is filled first, then `timed_steps`
@@ -256,15 +271,12 @@ def main():
         ctx.profile(False)
         kstats_alone = {k: v for k, v in ctx.profile_read().items() if "[" not in k}
 
-    if dist:
-        tt = torch.tensor([ms, e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms, e2e_s = float(tt[0]), float(tt[1])
+    ms, e2e_s = max_over_ranks([ms, e2e_s], dist, "cuda")
 
     if rank == 0:
         pk = peaks()
         total_samples = net.M * args.steps * world
-        value = total_samples / (ms * 1e-3)
+        value = whole_job_throughput(net.M, args.steps, world, ms * 1e-3)
         flops_step = sy.flops_per_sample(net) * net.M
         def roofline_of(stats, which=None):
             """Roofline entry of the kernel class with the largest summed event time (or of class `which`)."""
