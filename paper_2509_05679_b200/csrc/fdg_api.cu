@@ -14,8 +14,10 @@
 //              vectors); version v lives in slot v mod D.
 //   d2       : 2 slots of the error gradient w.r.t. the module's input; written in iteration t to
 //              slot t&1, read by module k-1 in iteration t+1.
-// Streams: module k's work of iteration t+1 waits only for the events modules k-1 and k+1 recorded
-// at the end of iteration t.
+// Streams: every module has a forward stream and a backward/update stream.  Iteration t+1 of module k waits only
+// for events of iteration t: its forward pass for its own update (weights, stash and ring slots it overwrites) and
+// for module k-1's forward pass (its input); its backward pass for the updates of modules k+1 (error gradient) and
+// k-1 (reader of the hand-off slot it overwrites); its update for its own forward pass.
 #include "../../include/fdg.h"
 #include "kernels.h"
 #include "tc_gemm.h"
@@ -86,8 +88,10 @@ struct Module {
     size_t cstat_elems;
     int fused_stats_tensor, fused_stats_chunks;   // set by a conv that produced statistics partials for this tensor
     int64_t *tag_in, *tag_stash, *tag_d2, *tag_w, *trace;
-    cudaStream_t stream;
-    cudaEvent_t done, ev0, ev1;
+    cudaStream_t stream;           // backward pass, loss, update (and everything in serial mode)
+    cudaStream_t fstream;          // forward pass: independent of the backward pass of the same iteration (other batch)
+    cudaEvent_t done, fdone, ev0, ev1;
+    float* scratch_f;              // reduction scratch of the forward stream
     bool had_bwd;
 };
 
@@ -397,7 +401,7 @@ bool tc_wgrad(fdg_ctx* c, Module& m, const Op& o, char* x, char* dy, float* dw, 
 void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version) {
     Module& m = c->mod[kk];
     StepPtrs P{c, &m, kk, batch};
-    cudaStream_t s = m.stream;
+    cudaStream_t s = m.fstream;
     const int dt = c->dt;
     m.fused_stats_tensor = -1;
     for (const Op& o : m.ops) {
@@ -422,7 +426,7 @@ void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version) {
             case OP_BN: {
                 const bool fused = m.fused_stats_tensor == o.in;
                 bn_forward(dt, P.tensor(o.in), wsmall(c, m, version, o.gamma_off), wsmall(c, m, version, o.beta_off),
-                           o.has_res ? P.tensor(o.in2) : nullptr, P.tensor(o.out), P.stats(o), m.scratch, c->n_workers,
+                           o.has_res ? P.tensor(o.in2) : nullptr, P.tensor(o.out), P.stats(o), m.scratch_f, c->n_workers,
                            (long)c->B * ti.h * ti.w, ti.c, o.relu, fused ? m.cstat : nullptr, fused ? m.fused_stats_chunks : 0, s);
                 m.fused_stats_tensor = -1;
                 break; }
@@ -608,17 +612,20 @@ fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, boo
     //    event recorded for THIS iteration)
     if (!ctx->serial && t > 0)
         for (int kk = 0; kk < K; ++kk) {
-            if (kk > 0) CK(cudaStreamWaitEvent(ctx->mod[kk].stream, ctx->mod[kk - 1].done, 0));
-            if (kk + 1 < K) CK(cudaStreamWaitEvent(ctx->mod[kk].stream, ctx->mod[kk + 1].done, 0));
+            Module& m = ctx->mod[kk];
+            CK(cudaStreamWaitEvent(m.fstream, m.done, 0));                                   // weights t; slots its forward overwrites
+            if (kk > 0) CK(cudaStreamWaitEvent(m.fstream, ctx->mod[kk - 1].fdone, 0));       // its input
+            if (kk > 0) CK(cudaStreamWaitEvent(m.stream, ctx->mod[kk - 1].done, 0));         // reader of the hand-off slot it overwrites
+            if (kk + 1 < K) CK(cudaStreamWaitEvent(m.stream, ctx->mod[kk + 1].done, 0));     // the error gradient it consumes
         }
     // 2. module 1 "samples" the batch of iteration t: copy into its FIFO slot; labels into the label FIFO
     {
         Module& m0 = ctx->mod[0];
         cudaMemcpyKind kind = host_src ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
         CK(cudaMemcpyAsync(m0.in_ring + (size_t)(t % m0.in_depth) * m0.in_slot_bytes, inputs,
-                           (size_t)ctx->M * m0.in_elems * ctx->esz, kind, m0.stream));
-        CK(cudaMemcpyAsync(ctx->labels + (size_t)(t % ctx->label_depth) * ctx->M, labels, (size_t)ctx->M * sizeof(int32_t), kind, m0.stream));
-        CK(cudaEventRecord(ctx->ingested, m0.stream));
+                           (size_t)ctx->M * m0.in_elems * ctx->esz, kind, m0.fstream));
+        CK(cudaMemcpyAsync(ctx->labels + (size_t)(t % ctx->label_depth) * ctx->M, labels, (size_t)ctx->M * sizeof(int32_t), kind, m0.fstream));
+        CK(cudaEventRecord(ctx->ingested, m0.fstream));
     }
     // 3. every module: forward on tau_f, backward on tau_b, update
     for (int kk = 0; kk < K; ++kk) {
@@ -648,6 +655,8 @@ fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, boo
         tags_step(tg, m.stream);
 
         if (tau_f >= 0) forward_module(ctx, kk, tau_f, t);
+        CK(cudaEventRecord(m.fdone, m.fstream));
+        if (lastm && m.fstream != m.stream) CK(cudaStreamWaitEvent(m.stream, m.fdone, 0));   // the last module back-propagates the batch it just forwarded
         if (lastm) {
             float* loss_slot = ctx->loss_ring + (t % 64);
             if (tau_f >= 0) softmax_ce(ctx->dt, ctx->logits, ctx->labels + (size_t)(tau_f % ctx->label_depth) * ctx->M, ctx->dlogits,
@@ -656,6 +665,8 @@ fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, boo
         }
         if (tau_b >= 0) backward_module(ctx, kk, tau_b, v_b, t);
         // Eq. dl_update with P = 11^T/N: w(t+1) = w(t) - lr * averaged gradient; also emits version t+1
+        // (after the forward pass has read version t: with a one-slot ring the update overwrites it)
+        if (!lastm && m.fstream != m.stream) CK(cudaStreamWaitEvent(m.stream, m.fdone, 0));
         sgd_update(ctx->dt, m.master, tau_b >= 0 ? m.grad : nullptr, wslot(ctx, m, t + 1), m.n_big, ctx->lr, m.stream);
         if (m.n_small)
             sgd_update(0, m.master + m.n_big, tau_b >= 0 ? m.grad + m.n_big : nullptr,
@@ -689,6 +700,7 @@ void fdg_destroy(fdg_ctx* ctx) {
     cudaDeviceSynchronize();
     for (Module& m : ctx->mod) {
         if (m.done) cudaEventDestroy(m.done);
+        if (m.fdone) cudaEventDestroy(m.fdone);
         if (m.ev0) cudaEventDestroy(m.ev0);
         if (m.ev1) cudaEventDestroy(m.ev1);
     }
@@ -782,6 +794,7 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
         m.ws = (float*)get(m.ws_elems * sizeof(float));
         m.scratch = (float*)get(m.scratch_elems * sizeof(float));
         m.red = (float*)get(m.red_elems * sizeof(float));
+        m.scratch_f = (float*)get(m.scratch_elems * sizeof(float));
         m.cstat = m.cstat_elems ? (float*)get(m.cstat_elems * sizeof(float)) : nullptr;
         if (oom) break;
         m.tag_in = ctx->tags + tpos; tpos += 2 * (size_t)m.in_depth;
@@ -797,7 +810,10 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
         if (opt->streams) m.stream = (cudaStream_t)opt->streams[ctx->serial ? 0 : kk];
         else if (ctx->serial && kk > 0) m.stream = ctx->mod[0].stream;
         else { e = cudaStreamCreateWithFlags(&m.stream, cudaStreamNonBlocking); if (e == cudaSuccess) ctx->owned.push_back(m.stream); }
+        m.fstream = m.stream;
+        if (e == cudaSuccess && !ctx->serial) { e = cudaStreamCreateWithFlags(&m.fstream, cudaStreamNonBlocking); if (e == cudaSuccess) ctx->owned.push_back(m.fstream); }
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.done, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.fdone, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreate(&m.ev0);
         if (e == cudaSuccess) e = cudaEventCreate(&m.ev1);
         if (e == cudaSuccess) e = cudaMemset(m.grad, 0, (m.n_big + m.n_small) * sizeof(float));
