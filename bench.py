@@ -33,9 +33,13 @@ FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 148 SMs x 128 fp32 FMA l
 
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel classes, from the ncu
-# capture summarised under profiles/ (taken at per-worker batch 64 and scaled x2 to the bench's 128: every operand of
-# these kernels grows in proportion to the batch).  Valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {}        # kernel class -> {"bytes_per_launch": float, "sha1": sha1 of csrc/tc_gemm.cu + csrc/kernels.cu at capture}
+# capture summarised under profiles/.  Valid only for the kernel source it was taken from: a changed source gives null.
+NCU_SHA1 = "353a7900d72b4567d3c7b26f512c0ca0a2cff654"
+NCU_TRAFFIC = {          # profiles/ncu_dram_bytes_C4_full_size.md: single-pass capture at the bench's own size (M = 1024)
+    "tc_gemm_fwd": {"bytes_per_launch": 111.0e6, "sha1": NCU_SHA1},      # km_kernel, average over the 76 forward + input-gradient launches
+    "tc_gemm_dgrad": {"bytes_per_launch": 111.0e6, "sha1": NCU_SHA1},
+    "tc_gemm_wgrad": {"bytes_per_launch": 125.6e6, "sha1": NCU_SHA1},    # wg_kernel, average over its 38 launches (wg_reduce_kernel not included)
+}
 
 
 def _kernel_source_sha1():

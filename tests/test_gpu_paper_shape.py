@@ -1,0 +1,42 @@
+"""The paper's experiment shape on synthetic data: a ResNet-20-style network (3 stages of 16/32/64 channels,
+3 basic blocks each) for 32x32x3 inputs, trained by the four methods it compares (Sec. 5):
+centralized (S=1, K=1), decoupled model (S=1, K=2), data parallel (S=4, K=1), proposed (S=4, K=2).
+fp32 path, every step compared with the oracle.  Also a step-size sequence (Strategy II style)."""
+import numpy as np
+import pytest
+
+from paper_2509_05679_b200 import synth as sy
+from harness import make_ctx, make_oracle, max_rel_err, run_parity
+
+pytestmark = pytest.mark.gpu
+
+
+def resnet20(S, K, batch):
+    layers, bs = sy.resnet_layers(widths=(16, 32, 64), blocks=3, in_c=3, classes=10)
+    splits = [] if K == 1 else [bs[4]]             # two model-groups: cut between blocks 4 and 5
+    return sy.Net(f"resnet20-S{S}-K{K}", layers, splits, 32, 32, 3, 10, S, batch, 0.1, "fp32")
+
+
+@pytest.mark.parametrize("S,K", [(1, 1), (1, 2), (4, 1), (4, 2)])
+def test_the_four_compared_methods_match_the_oracle(orc, S, K):
+    net = resnet20(S, K, 2)
+    rec = run_parity(orc, net, 2 * K + 3, param_tol=1e-5, loss_tol=1e-5)
+    assert not np.isnan(rec[-1]["loss_g"])
+
+
+def test_step_size_sequence(orc):
+    """eta_t changes between steps (the paper's Strategy II switches 0.1 -> 0.01 -> 0.001 -> 0.0001)."""
+    import torch
+    from paper_2509_05679_b200 import binding
+    net = sy.Net("mlp-lr-seq", sy.mlp_layers([24, 32, 16, 10]), [2], 1, 1, 24, 10, 2, 8, 0.1, "fp32")
+    p0 = sy.init_params(net.layers, 0)
+    o, ctx = make_oracle(orc, net, p0), make_ctx(net, p0)
+    etas = [0.1, 0.1, 0.01, 0.01, 0.001, 0.0001, 0.0001]
+    for t, eta in enumerate(etas):
+        x, y = sy.batch_inputs(net, t), sy.batch_labels(net, t)
+        ctx.set_lr(eta)
+        o.step(x, y, eta)
+        ctx.step(binding.to_device("fp32", x), torch.from_numpy(y).cuda(), want_loss=True)
+        err, where = max_rel_err(ctx.params(), o.params(0), net.layers)
+        assert err <= 1e-5, (t, err, where)
+    ctx.close()

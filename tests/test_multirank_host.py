@@ -1,6 +1,6 @@
 """Host-side logic of the multi-GPU bench path, exercised with two gloo ranks on the CPU.
 
-The method has no exchange between GPUs in this build: N ranks are N independent replicas, each with its
+This library has no exchange between GPUs: N ranks are N independent replicas, each with its
 own data stream; the only collective is the maximum of the timings over the ranks."""
 import os
 import subprocess
