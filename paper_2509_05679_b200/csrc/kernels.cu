@@ -493,6 +493,7 @@ __global__ void bn_reduce_partial(const T* __restrict__ x, const T* __restrict__
     if (c < C) {
         float mean = 0.f, istd = 0.f;
         if (BWD) { mean = stats[((size_t)w * C + c) * 2]; istd = stats[((size_t)w * C + c) * 2 + 1]; }
+        const float pivot = BWD ? 0.f : ld(x + (size_t)w * rpw * C + c);
         for (long r = r0 + threadIdx.y; r < r1; r += blockDim.y) {
             size_t o = ((size_t)w * rpw + r) * C + c;
             if (BWD) {
@@ -500,7 +501,9 @@ __global__ void bn_reduce_partial(const T* __restrict__ x, const T* __restrict__
                 if (relu && !(ld(out + o) > 0.f)) dy = 0.f;
                 s1 += dy; s2 += dy * (ld(x + o) - mean) * istd;
             } else {
-                float v = ld(x + o); s1 += v; s2 += v * v;
+                // sums of (x - pivot): the pivot (the worker's first value of the channel) keeps the variance
+                // formula E[d^2] - E[d]^2 from cancelling when |mean| >> std
+                float v = ld(x + o) - pivot; s1 += v; s2 += v * v;
             }
         }
     }
@@ -515,14 +518,18 @@ __global__ void bn_reduce_partial(const T* __restrict__ x, const T* __restrict__
     }
 }
 // forward: stats[w][c] = (mean, invstd).  One thread per (w, c).
-__global__ void bn_stats_final(const float* __restrict__ part, float* __restrict__ stats, int chunks, int nwC, long rpw) {
+template <typename T>
+__global__ void bn_stats_final(const float* __restrict__ part, const T* __restrict__ x, float* __restrict__ stats, int chunks, int nwC,
+                               int C, long rpw) {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= nwC) return;
     double s1 = 0.0, s2 = 0.0;
     for (int k = 0; k < chunks; ++k) { s1 += part[((size_t)k * nwC + i) * 2]; s2 += part[((size_t)k * nwC + i) * 2 + 1]; }
-    double mean = s1 / (double)rpw, var = s2 / (double)rpw - mean * mean;
+    const int w = i / C, c = i - w * C;
+    const double pivot = (double)ld(x + (size_t)w * rpw * C + c);       // the partial sums are sums of (x - pivot)
+    double dm = s1 / (double)rpw, var = s2 / (double)rpw - dm * dm;
     if (var < 0.0) var = 0.0;
-    stats[(size_t)i * 2] = (float)mean;
+    stats[(size_t)i * 2] = (float)(pivot + dm);
     stats[(size_t)i * 2 + 1] = (float)(1.0 / sqrt(var + 1e-5));
 }
 // backward: red[w][c] = (sum dy, sum dy xhat); dgamma[c] = sum_w red[w][c].y; dbeta[c] = sum_w red[w][c].x
@@ -891,7 +898,8 @@ void bn_forward(int dt, const void* x, const float* gamma, const float* beta, co
       if (dt) bn_reduce_partial<bf16, false><<<grid, blk, 0, s>>>((const bf16*)x, nullptr, nullptr, nullptr, scratch, rpw, C, false);
       else bn_reduce_partial<float, false><<<grid, blk, 0, s>>>((const float*)x, nullptr, nullptr, nullptr, scratch, rpw, C, false); }
     { Scope sc(KC_BN_FWD_STATS, 0.0, 8.0 * chunks * nw * C, s);
-      bn_stats_final<<<cdiv((size_t)nw * C, 128), 128, 0, s>>>(scratch, stats, chunks, nw * C, rpw); }
+      if (dt) bn_stats_final<bf16><<<cdiv((size_t)nw * C, 128), 128, 0, s>>>(scratch, (const bf16*)x, stats, chunks, nw * C, C, rpw);
+      else bn_stats_final<float><<<cdiv((size_t)nw * C, 128), 128, 0, s>>>(scratch, (const float*)x, stats, chunks, nw * C, C, rpw); }
     Scope sc(KC_BN_FWD_APPLY, 0.0, esz_ * total * (res ? 3 : 2), s);
     if (dt) bn_apply_k<bf16><<<cdiv(total, 256), 256, 0, s>>>((const bf16*)x, gamma, beta, (const bf16*)res, (bf16*)y, stats, rpw, C, total, relu);
     else bn_apply_k<float><<<cdiv(total, 256), 256, 0, s>>>((const float*)x, gamma, beta, (const float*)res, (float*)y, stats, rpw, C, total, relu);
@@ -943,16 +951,18 @@ __global__ void softmax_ce_k(const float* __restrict__ z, const int32_t* __restr
     __shared__ float sh[256];
     float local = 0.f;
     float inv_m = 1.f / (float)M;
+    // exp / log in double: a few thousand values per step, and it keeps the error of (softmax - onehot) at the rounding
+    // of the stored result instead of |z| * ulp(expf)
     for (int r = threadIdx.x; r < M; r += blockDim.x) {
         const float* zr = z + (size_t)r * C;
         float m = zr[0];
         for (int c = 1; c < C; ++c) m = fmaxf(m, zr[c]);
-        float se = 0.f;
-        for (int c = 0; c < C; ++c) se += expf(zr[c] - m);
-        float lse = m + logf(se);
+        double se = 0.0;
+        for (int c = 0; c < C; ++c) se += exp((double)zr[c] - (double)m);
+        const double lse = (double)m + log(se);
         int y = labels[r];
-        local += lse - zr[y];
-        for (int c = 0; c < C; ++c) st(dz + (size_t)r * C + c, (expf(zr[c] - lse) - (c == y ? 1.f : 0.f)) * inv_m);
+        local += (float)(lse - (double)zr[y]);
+        for (int c = 0; c < C; ++c) st(dz + (size_t)r * C + c, (float)((exp((double)zr[c] - lse) - (c == y ? 1.0 : 0.0)) * (double)inv_m));
     }
     sh[threadIdx.x] = local;
     __syncthreads();
