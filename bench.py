@@ -34,7 +34,7 @@ FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 148 SMs x 128 fp32 FMA l
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel classes, from the ncu
 # capture summarised under profiles/.  Valid only for the kernel source it was taken from: a changed source gives null.
-NCU_SHA1 = "353a7900d72b4567d3c7b26f512c0ca0a2cff654"
+NCU_SHA1 = "68072dbb385993dd7289f8470a575a07c2bfc997"   # sha1 of csrc/tc_gemm.cu when the counters were taken
 NCU_TRAFFIC = {          # profiles/ncu_dram_bytes_C4_full_size.md: single-pass capture at the bench's own size (M = 1024)
     "tc_gemm_fwd": {"bytes_per_launch": 111.0e6, "sha1": NCU_SHA1},      # km_kernel, average over the 76 forward + input-gradient launches
     "tc_gemm_dgrad": {"bytes_per_launch": 111.0e6, "sha1": NCU_SHA1},
@@ -45,8 +45,7 @@ NCU_TRAFFIC = {          # profiles/ncu_dram_bytes_C4_full_size.md: single-pass 
 def _kernel_source_sha1():
     import hashlib
     h = hashlib.sha1()
-    for f in ("tc_gemm.cu", "kernels.cu"):
-        h.update(open(os.path.join(ROOT, "paper_2509_05679_b200", "csrc", f), "rb").read())
+    h.update(open(os.path.join(ROOT, "paper_2509_05679_b200", "csrc", "tc_gemm.cu"), "rb").read())
     return h.hexdigest()
 
 
