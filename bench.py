@@ -159,6 +159,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=3, help="0..4 = the five configurations; 3 = ResNet-18-shaped K=4, 8 workers x 128")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--worker-groups", type=int, default=0, help="0: chosen by the library; n: every module but the last runs its layers once per n-th of the workers")
     ap.add_argument("--kernel-path", type=int, default=0, help="0: tensor-core kernels where shapes allow, 1: plain FMA kernels only")
     ap.add_argument("--batch", type=int, default=None, help="per-worker batch override (testing only; changes the workload name)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -189,7 +190,8 @@ def main():
     streams = [torch.cuda.Stream() for _ in range(net.K)]
     ctx = binding.Context(net.layers, net.splits, net.n_workers, net.batch, net.lr, dtype=net.dtype,
                           in_shape=(net.in_h, net.in_w, net.in_c), num_classes=net.classes, device=local,
-                          kernel_path=args.kernel_path, streams=[s.cuda_stream for s in streams], serial=args.serial)
+                          kernel_path=args.kernel_path, streams=[s.cuda_stream for s in streams], serial=args.serial,
+                          worker_groups=args.worker_groups)
     ctx.set_params(sy.init_params(net.layers, 0, bf16=net.dtype == "bf16"))
 
     # a pool of distinct batches, resident in HBM (device arm) and in pinned host memory (e2e arm)
@@ -263,7 +265,7 @@ def main():
         ctx.close()
         ctx = binding.Context(net.layers, net.splits, net.n_workers, net.batch, net.lr, dtype=net.dtype,
                               in_shape=(net.in_h, net.in_w, net.in_c), num_classes=net.classes, device=local,
-                              kernel_path=args.kernel_path, serial=True)
+                              kernel_path=args.kernel_path, serial=True, worker_groups=args.worker_groups)
         ctx.set_params(sy.init_params(net.layers, 0, bf16=net.dtype == "bf16"))
         for i in range(fill + 3):
             ctx.step(dev_x[i % pool], dev_y[i % pool])
@@ -314,7 +316,7 @@ def main():
             "config": {"workload": net.name + ("" if args.batch is None else f"-B{args.batch}"), "K": net.K, "n_workers": net.n_workers,
                        "per_worker_batch": net.batch, "M": net.M, "lr": net.lr, "pipeline_fill_steps": fill,
                        "l2": "inputs rotate over 4 batches; each step streams the multi-GB activation stash, far larger than L2",
-                       "multi_gpu": "independent replicas (no exchange between GPUs)", "kernel_path": args.kernel_path, "serial": bool(args.serial)},
+                       "multi_gpu": "independent replicas (no exchange between GPUs)", "kernel_path": args.kernel_path, "serial": bool(args.serial), "worker_groups": args.worker_groups},
             "clocks": clocks,
             "step_tensor_roofline": {"flop_per_step": flops_step, "tflops_achieved": flops_step / (ms / args.steps * 1e-3) / 1e12 * 1.0,
                                      "frac_of_burst_peak": flops_step / (ms / args.steps * 1e-3) / 1e12 / pk["tensor_burst"],

@@ -91,6 +91,13 @@ typedef struct {
                                   to the concurrent mode; used to test the event wiring)        */
     int32_t kernel_path;       /* 0: tensor-core kernels where shapes allow (bf16 only);
                                   1: plain FMA kernels only                                      */
+    int32_t worker_groups;     /* 0 or 1: every kernel covers all workers.  n > 1: every module but the last runs
+                                  its layers once per group of n_workers / n workers (n rounded down to a power
+                                  of two that divides n_workers; ignored where a group would cut a tensor-core
+                                  tile) and adds the groups' parameter gradients; results differ from n = 1 only
+                                  in fp32 summation order.  Smaller launches, more of them: on a B200 this was
+                                  slower at every n for the ResNet-18-shaped benchmark (7.2 ms per step at 1,
+                                  7.6 at 2, 8.6 at 4), so it is off by default                                  */
     void* const* streams;      /* K cudaStream_t of the caller, or NULL: the library creates K  */
 } fdg_options;
 

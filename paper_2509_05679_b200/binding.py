@@ -50,7 +50,7 @@ class fdg_kernel_stat(C.Structure):
 class fdg_options(C.Structure):
     _fields_ = [("dtype", C.c_int32), ("in_h", C.c_int32), ("in_w", C.c_int32), ("in_c", C.c_int32),
                 ("num_classes", C.c_int32), ("serial", C.c_int32), ("kernel_path", C.c_int32),
-                ("streams", C.POINTER(C.c_void_p))]
+                ("worker_groups", C.c_int32), ("streams", C.POINTER(C.c_void_p))]
 
 
 _lib = None
@@ -143,7 +143,7 @@ class Context:
     def __init__(self, layers: Sequence[Sequence[int]], split_points: Sequence[int], n_workers: int,
                  per_worker_batch: int, lr: float, *, dtype: str = "bf16", in_shape=(32, 32, 3), num_classes: int = 10,
                  serial: bool = False, kernel_path: int = 0, device: int = 0, use_torch_allocator: bool = True,
-                 streams: Optional[Sequence[int]] = None):
+                 streams: Optional[Sequence[int]] = None, worker_groups: int = 0):
         import torch
         L = lib()
         if not torch.cuda.is_available():
@@ -160,7 +160,7 @@ class Context:
             assert len(streams) == self.K
             self._streams = (C.c_void_p * self.K)(*[C.c_void_p(int(h_)) for h_ in streams])
         opt = fdg_options({"fp32": 0, "bf16": 1}[dtype], int(in_shape[0]), int(in_shape[1]), int(in_shape[2]),
-                          int(num_classes), int(serial), int(kernel_path),
+                          int(num_classes), int(serial), int(kernel_path), int(worker_groups),
                           C.cast(self._streams, C.POINTER(C.c_void_p)) if self._streams is not None else None)
         self._alloc = _TorchAllocator(torch.device("cuda", device)) if use_torch_allocator else None
         h = C.c_void_p()

@@ -76,6 +76,7 @@ struct Segment { size_t canon, internal, count; bool big; };
 
 struct Module {
     int p, q, D, in_depth;
+    int groups;                    // worker groups the op list is run for, one after the other (1 = all workers at once)
     std::vector<TensorDesc> t;
     std::vector<Op> ops;
     std::vector<Segment> segs;
@@ -356,84 +357,107 @@ int find_buf(const std::vector<char*>& v, const char* p) {
 }
 
 // forward conv / linear on the tensor cores; false if the buffers are not the ones planned for
-bool tc_forward(fdg_ctx* c, Module& m, const Op& o, char* x, char* y, int64_t version, cudaStream_t s) {
-    int ia = find_buf(o.a_ptrs, x);
+// A group of consecutive workers (rows n0 .. n0+n-1 of every [M, ...] tensor).  A module whose tensors are far
+// larger than L2 runs its op list once per group, so that what one kernel writes is still in L2 when the next
+// kernel reads it; weight / bias / gamma / beta gradients of the second and later groups add to the first's.
+struct Win { int n0, n, w0, nw; bool first; };
+
+Win group_window(const fdg_ctx* c, const Module& m, int g) {
+    const int nw = c->n_workers / m.groups;
+    return Win{g * nw * c->B, nw * c->B, g * nw, nw, g == 0};
+}
+
+bool tc_forward(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* y_base, int64_t version, const Win& wn, cudaStream_t s) {
+    int ia = find_buf(o.a_ptrs, x_base);
     if (ia < 0) return false;
     tc::KmParams p = o.kf;
     p.bias = o.bias ? wsmall(c, m, version, o.b_off) : nullptr;
-    p.out = y; p.epi = o.relu ? EPI_RELU : 0; p.err = c->tc_err;
+    p.out = y_base; p.epi = o.relu ? EPI_RELU : 0; p.err = c->tc_err;
     p.stat_part = o.stat_chunks ? m.cstat : nullptr;
-
+    p.n_base = wn.n0; p.N = wn.n0 + wn.n; p.tiles_n = (wn.n + p.Nt - 1) / p.Nt;
     const ConvGeom& g = o.g;
-    double rows = (double)g.N * g.Ho * g.Wo;
-    Scope sc(KC_TC_FWD, 2.0 * rows * g.Co * g.R * g.R * g.C, 2.0 * ((double)g.N * g.H * g.W * g.C + (double)g.Co * g.R * g.R * g.C + rows * g.Co), s);
+    double rows = (double)wn.n * g.Ho * g.Wo;
+    Scope sc(KC_TC_FWD, 2.0 * rows * g.Co * g.R * g.R * g.C, 2.0 * ((double)wn.n * g.H * g.W * g.C + (double)g.Co * g.R * g.R * g.C + rows * g.Co), s);
     const bool ok = tc::run_km(o.fa[ia], o.fb[version % m.D], p, o.n_tile_f, s) == cudaSuccess;
     if (ok && o.stat_chunks) { m.fused_stats_tensor = o.out; m.fused_stats_chunks = o.stat_chunks; }
     return ok;
 }
-bool tc_dgrad(fdg_ctx* c, Module& m, const Op& o, char* dy, char* dx, int64_t version, bool accum, cudaStream_t s) {
-    int ia = find_buf(o.dy_ptrs, dy);
+bool tc_dgrad(fdg_ctx* c, Module& m, const Op& o, char* dy_base, char* dx_base, int64_t version, bool accum, const Win& wn, cudaStream_t s) {
+    int ia = find_buf(o.dy_ptrs, dy_base);
     if (ia < 0) return false;
     const ConvGeom& g = o.g;
-    double rows = (double)g.N * g.H * g.W;
+    double rows = (double)wn.n * g.H * g.W;
     if (o.dgrad_needs_zero && !accum) {
         Scope sc(KC_TC_AUX, 0.0, 2.0 * rows * g.C, s);
-        cudaMemsetAsync(dx, 0, (size_t)rows * g.C * 2, s);
+        cudaMemsetAsync(dx_base + (size_t)wn.n0 * g.H * g.W * g.C * 2, 0, (size_t)rows * g.C * 2, s);
     }
     tc::KmParams p = o.kd;
-    p.bias = nullptr; p.out = dx; p.epi = accum ? EPI_ACCUM : 0; p.err = c->tc_err; p.stat_part = nullptr;
-    const double crows = (double)g.N * p.Hd * p.Wd;          // pixels of one class; every tap belongs to exactly one class
+    p.bias = nullptr; p.out = dx_base; p.epi = accum ? EPI_ACCUM : 0; p.err = c->tc_err; p.stat_part = nullptr;
+    p.n_base = wn.n0; p.N = wn.n0 + wn.n; p.tiles_n = (wn.n + p.Nt - 1) / p.Nt;
+    const double crows = (double)wn.n * p.Hd * p.Wd;         // pixels of one class; every tap belongs to exactly one class
     Scope sc(KC_TC_DGRAD, 2.0 * crows * g.C * p.ntaps * g.Co,
-             2.0 * ((double)g.N * g.Ho * g.Wo * g.Co + (double)g.Co * p.ntaps * g.C + crows * p.ncls * g.C * (accum ? 2 : 1)), s);
+             2.0 * ((double)wn.n * g.Ho * g.Wo * g.Co + (double)g.Co * p.ntaps * g.C + crows * p.ncls * g.C * (accum ? 2 : 1)), s);
     return tc::run_km(o.da[ia], o.db[version % m.D], p, o.n_tile_d, s) == cudaSuccess;
 }
-bool tc_wgrad(fdg_ctx* c, Module& m, const Op& o, char* x, char* dy, float* dw, cudaStream_t s) {
-    int ix = find_buf(o.a_ptrs, x), id = find_buf(o.dy_ptrs, dy);
+bool tc_wgrad(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* dy_base, float* dw, const Win& wn, cudaStream_t s) {
+    int ix = find_buf(o.a_ptrs, x_base), id = find_buf(o.dy_ptrs, dy_base);
     if (ix < 0 || id < 0) return false;
     tc::WgParams p = o.kw;
     p.partial = m.ws; p.err = c->tc_err;
+    p.n_base = wn.n0; p.tiles_n = (wn.n + p.Nt - 1) / p.Nt;
+    p.ptiles = p.tiles_w * p.tiles_h * p.tiles_n;
+    int splits = o.wg_splits < p.ptiles ? o.wg_splits : p.ptiles;
+    p.ptiles_per_split = (p.ptiles + splits - 1) / splits;
+    splits = (p.ptiles + p.ptiles_per_split - 1) / p.ptiles_per_split;
     const ConvGeom& g = o.g;
-    double rows = (double)g.N * g.Ho * g.Wo, R = (double)g.R * g.R * g.C;
-    Scope sc(KC_TC_WGRAD, 2.0 * rows * g.Co * R, 2.0 * ((double)g.N * g.H * g.W * g.C + rows * g.Co) + 4.0 * R * g.Co, s);
-    return tc::run_wg(o.wx[ix], o.wdy[id], p, o.n_tile_w, o.wg_splits, dw, s) == cudaSuccess;
+    double rows = (double)wn.n * g.Ho * g.Wo, R = (double)g.R * g.R * g.C;
+    Scope sc(KC_TC_WGRAD, 2.0 * rows * g.Co * R, 2.0 * ((double)wn.n * g.H * g.W * g.C + rows * g.Co) + 4.0 * R * g.Co, s);
+    return tc::run_wg(o.wx[ix], o.wdy[id], p, o.n_tile_w, splits, dw, !wn.first, s) == cudaSuccess;
 }
 
-void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version) {
+// byte offset of the group's first sample inside a tensor of the module
+size_t row_off(const fdg_ctx* c, const TensorDesc& d, const Win& wn) {
+    return (size_t)wn.n0 * d.elems() * (d.loc == LOC_LOGITS ? sizeof(float) : (size_t)c->esz);
+}
+
+void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int group) {
     Module& m = c->mod[kk];
     StepPtrs P{c, &m, kk, batch};
+    const Win wn = group_window(c, m, group);
     cudaStream_t s = m.fstream;
     const int dt = c->dt;
     m.fused_stats_tensor = -1;
+    auto T = [&](int id) { return P.tensor(id) + row_off(c, m.t[id], wn); };
     for (const Op& o : m.ops) {
         const TensorDesc& ti = m.t[o.in];
         const TensorDesc& to = m.t[o.out];
-        size_t n_out = to.elems() * c->M;
+        size_t n_out = to.elems() * wn.n;
         switch (o.type) {
             case OP_CONV: {
                 int epi = (o.relu ? EPI_RELU : 0) | (to.loc == LOC_LOGITS ? EPI_OUT_F32 : 0);
+                ConvGeom g = o.g; g.N = wn.n;
                 profile_detail(o.shape);
-                if (o.tc && tc_forward(c, m, o, P.tensor(o.in), P.tensor(o.out), version, s)) { profile_detail(nullptr); break; }
+                if (o.tc && tc_forward(c, m, o, P.tensor(o.in), P.tensor(o.out), version, wn, s)) { profile_detail(nullptr); break; }
                 if (o.stem) {
-                    stem_forward(P.tensor(o.in), wbig(c, m, version, o.w_off), o.bias ? wsmall(c, m, version, o.b_off) : nullptr,
-                                 P.tensor(o.out), o.g, o.relu, s);
+                    stem_forward(T(o.in), wbig(c, m, version, o.w_off), o.bias ? wsmall(c, m, version, o.b_off) : nullptr, T(o.out), g, o.relu, s);
                     profile_detail(nullptr);
                     break;
                 }
-                conv_forward(dt, P.tensor(o.in), wbig(c, m, version, o.w_off), o.bias ? wsmall(c, m, version, o.b_off) : nullptr,
-                             P.tensor(o.out), o.g, epi, s);
+                conv_forward(dt, T(o.in), wbig(c, m, version, o.w_off), o.bias ? wsmall(c, m, version, o.b_off) : nullptr, T(o.out), g, epi, s);
                 profile_detail(nullptr);
                 break; }
             case OP_BN: {
                 const bool fused = m.fused_stats_tensor == o.in;
-                bn_forward(dt, P.tensor(o.in), wsmall(c, m, version, o.gamma_off), wsmall(c, m, version, o.beta_off),
-                           o.has_res ? P.tensor(o.in2) : nullptr, P.tensor(o.out), P.stats(o), m.scratch_f, c->n_workers,
-                           (long)c->B * ti.h * ti.w, ti.c, o.relu, fused ? m.cstat : nullptr, fused ? m.fused_stats_chunks : 0, s);
+                const float* part = fused ? m.cstat + (size_t)wn.w0 * m.fused_stats_chunks * ti.c * 2 : nullptr;
+                bn_forward(dt, T(o.in), wsmall(c, m, version, o.gamma_off), wsmall(c, m, version, o.beta_off),
+                           o.has_res ? T(o.in2) : nullptr, T(o.out), P.stats(o) + (size_t)wn.w0 * ti.c * 2, m.scratch_f, wn.nw,
+                           (long)c->B * ti.h * ti.w, ti.c, o.relu, part, fused ? m.fused_stats_chunks : 0, s);
                 m.fused_stats_tensor = -1;
                 break; }
-            case OP_RELU: relu_forward(dt, P.tensor(o.in), P.tensor(o.out), n_out, s); break;
-            case OP_POOL: maxpool_forward(dt, P.tensor(o.in), P.tensor(o.out), c->M, ti.h, ti.w, ti.c, s); break;
-            case OP_GAP: gap_forward(dt, P.tensor(o.in), P.tensor(o.out), c->M, ti.h * ti.w, ti.c, s); break;
-            case OP_ADD: add_forward(dt, P.tensor(o.in), P.tensor(o.in2), P.tensor(o.out), n_out, s); break;
+            case OP_RELU: relu_forward(dt, T(o.in), T(o.out), n_out, s); break;
+            case OP_POOL: maxpool_forward(dt, T(o.in), T(o.out), wn.n, ti.h, ti.w, ti.c, s); break;
+            case OP_GAP: gap_forward(dt, T(o.in), T(o.out), wn.n, ti.h * ti.w, ti.c, s); break;
+            case OP_ADD: add_forward(dt, T(o.in), T(o.in2), T(o.out), n_out, s); break;
         }
     }
 }
@@ -449,42 +473,48 @@ char* grad_ptr(fdg_ctx* c, int kk, int id, int64_t t) {
     return n.d2 + (size_t)((t - 1) & 1) * n.in_slot_bytes;
 }
 
-void backward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int64_t t) {
+void backward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int64_t t, int group) {
     Module& m = c->mod[kk];
     StepPtrs P{c, &m, kk, batch};
+    const Win wn = group_window(c, m, group);
     cudaStream_t s = m.stream;
     const int dt = c->dt;
+    const bool acc_p = !wn.first;                       // parameter gradients of later groups add to the first group's
+    auto T = [&](int id) { return P.tensor(id) + row_off(c, m.t[id], wn); };
+    // gradients are stored in the storage dtype (also the one of the logits)
+    auto G = [&](int id) -> char* { char* b = grad_ptr(c, kk, id, t); return b ? b + (size_t)wn.n0 * m.t[id].elems() * c->esz : nullptr; };
     for (int i = (int)m.ops.size() - 1; i >= 0; --i) {
         const Op& o = m.ops[i];
         const TensorDesc& ti = m.t[o.in];
         const TensorDesc& to = m.t[o.out];
-        size_t n_out = to.elems() * c->M, n_in = ti.elems() * c->M;
-        char* gout = grad_ptr(c, kk, o.out, t);
-        char* gin = grad_ptr(c, kk, o.in, t);
+        size_t n_out = to.elems() * wn.n, n_in = ti.elems() * wn.n;
+        char* gout = G(o.out);
+        char* gin = G(o.in);
         switch (o.type) {
             case OP_CONV: {
-                if (o.relu) relu_backward(dt, P.tensor(o.out), gout, gout, n_out, false, s);       // in place: dZ = dA * (A > 0)
+                ConvGeom g = o.g; g.N = wn.n;
+                if (o.relu) relu_backward(dt, T(o.out), gout, gout, n_out, false, s);       // in place: dZ = dA * (A > 0)
                 profile_detail(o.shape);
-                if (o.stem) stem_wgrad(P.tensor(o.in), gout, m.grad + o.w_off, m.ws, o.g, s);
-                else if (!(o.tc && tc_wgrad(c, m, o, P.tensor(o.in), gout, m.grad + o.w_off, s)))
-                    conv_wgrad(dt, P.tensor(o.in), gout, m.grad + o.w_off, m.ws, o.g, s);
-                if (o.bias) bias_grad(dt, gout, m.grad + m.n_big + o.b_off, m.scratch, (long)o.g.N * o.g.Ho * o.g.Wo, o.g.Co, s);
-                if (gin && !(o.tc && tc_dgrad(c, m, o, gout, gin, version, o.acc_in, s)))
-                    conv_dgrad(dt, gout, wbig(c, m, version, o.w_off), gin, o.g, o.acc_in ? EPI_ACCUM : 0, s);
+                if (o.stem) stem_wgrad(T(o.in), gout, m.grad + o.w_off, m.ws, g, acc_p, s);
+                else if (!(o.tc && tc_wgrad(c, m, o, P.tensor(o.in), grad_ptr(c, kk, o.out, t), m.grad + o.w_off, wn, s)))
+                    conv_wgrad(dt, T(o.in), gout, m.grad + o.w_off, m.ws, g, acc_p, s);
+                if (o.bias) bias_grad(dt, gout, m.grad + m.n_big + o.b_off, m.scratch, (long)g.N * g.Ho * g.Wo, g.Co, acc_p, s);
+                if (gin && !(o.tc && tc_dgrad(c, m, o, grad_ptr(c, kk, o.out, t), grad_ptr(c, kk, o.in, t), version, o.acc_in, wn, s)))
+                    conv_dgrad(dt, gout, wbig(c, m, version, o.w_off), gin, g, o.acc_in ? EPI_ACCUM : 0, s);
                 profile_detail(nullptr);
                 break; }
             case OP_BN: {
-                char* gres = o.has_res ? grad_ptr(c, kk, o.in2, t) : nullptr;
-                bn_backward(dt, P.tensor(o.in), P.tensor(o.out), gout, wsmall(c, m, version, o.gamma_off), wsmall(c, m, version, o.beta_off),
-                            P.stats(o), gin, o.acc_in, gres, o.acc_in2, m.grad + m.n_big + o.gamma_off, m.grad + m.n_big + o.beta_off,
-                            m.red, m.scratch, c->n_workers, (long)c->B * ti.h * ti.w, ti.c, o.relu, o.has_res, s);
+                char* gres = o.has_res ? G(o.in2) : nullptr;
+                bn_backward(dt, T(o.in), T(o.out), gout, wsmall(c, m, version, o.gamma_off), wsmall(c, m, version, o.beta_off),
+                            P.stats(o) + (size_t)wn.w0 * ti.c * 2, gin, o.acc_in, gres, o.acc_in2, m.grad + m.n_big + o.gamma_off,
+                            m.grad + m.n_big + o.beta_off, m.red, m.scratch, wn.nw, (long)c->B * ti.h * ti.w, ti.c, o.relu, o.has_res, acc_p, s);
                 break; }
-            case OP_RELU: if (gin) relu_backward(dt, P.tensor(o.out), gout, gin, n_out, o.acc_in, s); break;
-            case OP_POOL: if (gin) maxpool_backward(dt, P.tensor(o.in), gout, gin, c->M, ti.h, ti.w, ti.c, o.acc_in, s); break;
-            case OP_GAP: if (gin) gap_backward(dt, gout, gin, c->M, ti.h * ti.w, ti.c, o.acc_in, s); break;
+            case OP_RELU: if (gin) relu_backward(dt, T(o.out), gout, gin, n_out, o.acc_in, s); break;
+            case OP_POOL: if (gin) maxpool_backward(dt, T(o.in), gout, gin, wn.n, ti.h, ti.w, ti.c, o.acc_in, s); break;
+            case OP_GAP: if (gin) gap_backward(dt, gout, gin, wn.n, ti.h * ti.w, ti.c, o.acc_in, s); break;
             case OP_ADD: {
                 if (gin) copy_or_accumulate(dt, gout, gin, n_in, o.acc_in, s);
-                char* g2 = grad_ptr(c, kk, o.in2, t);
+                char* g2 = G(o.in2);
                 if (g2) copy_or_accumulate(dt, gout, g2, n_in, o.acc_in2, s);
                 break; }
         }
@@ -654,7 +684,7 @@ fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, boo
         tg.trace = m.trace;
         tags_step(tg, m.stream);
 
-        if (tau_f >= 0) forward_module(ctx, kk, tau_f, t);
+        if (tau_f >= 0) for (int g = 0; g < m.groups; ++g) forward_module(ctx, kk, tau_f, t, g);
         CK(cudaEventRecord(m.fdone, m.fstream));
         if (lastm && m.fstream != m.stream) CK(cudaStreamWaitEvent(m.stream, m.fdone, 0));   // the last module back-propagates the batch it just forwarded
         if (lastm) {
@@ -663,7 +693,7 @@ fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, boo
                                        loss_slot, ctx->M, ctx->classes, m.stream);
             else fill_f32(loss_slot, NAN, 1, m.stream);
         }
-        if (tau_b >= 0) backward_module(ctx, kk, tau_b, v_b, t);
+        if (tau_b >= 0) for (int g = 0; g < m.groups; ++g) backward_module(ctx, kk, tau_b, v_b, t, g);
         // Eq. dl_update with P = 11^T/N: w(t+1) = w(t) - lr * averaged gradient; also emits version t+1
         // (after the forward pass has read version t: with a one-slot ring the update overwrites it)
         if (!lastm && m.fstream != m.stream) CK(cudaStreamWaitEvent(m.stream, m.fdone, 0));
@@ -755,6 +785,14 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
             char buf[256]; snprintf(buf, sizeof buf, "module %d: %s", kk + 1, e.c_str());
             return bail(s, buf);
         }
+        // worker groups (off unless asked for: measured slower on every configuration, see fdg_options.worker_groups):
+        // a group is a whole number of workers; the last module of a split network stays whole
+        m.groups = 1;
+        if (opt->worker_groups > 1 && (kk + 1 < K || K == 1)) {
+            int g = 1;
+            while (g * 2 <= opt->worker_groups && n_workers % (g * 2) == 0) g *= 2;
+            m.groups = g;
+        }
         m.in_slot_bytes = align_up((size_t)ctx->M * m.in_elems * ctx->esz, 256);
         m.wslot_bytes = align_up(m.n_big * ctx->esz + m.n_small * sizeof(float), 256);
     }
@@ -824,6 +862,12 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
     if (cudaMemset(ctx->tc_err, 0, 256) != cudaSuccess) return bail(FDG_ERR_CUDA, "cudaMemset failed");
     ctx->any_tc = false;
     if (!build_tc_plans(ctx)) return bail(FDG_ERR_CUDA, "cuTensorMapEncodeTiled rejected a tensor map");
+    // a group must hold whole image tiles of every tensor-core tiling: a ragged tile would reach into the next group's rows
+    for (Module& m : ctx->mod) {
+        const int n = ctx->M / m.groups;
+        for (const Op& o : m.ops)
+            if (o.tc && (n % o.kf.Nt || (o.kd.Nt && n % o.kd.Nt) || n % o.kw.Nt)) m.groups = 1;
+    }
     *out = ctx;
     return FDG_OK;
 }

@@ -246,17 +246,17 @@ __global__ void __launch_bounds__(256) igemm_simt(const T* __restrict__ P0, cons
 }
 
 // out[i] = sum_z partial[z][i], z ascending (fixed order => run-to-run identical results)
-__global__ void splitk_reduce(const float* __restrict__ partial, float* __restrict__ out, size_t n, int splits) {
+__global__ void splitk_reduce(const float* __restrict__ partial, float* __restrict__ out, size_t n, int splits, bool accum) {
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     float s = 0.f;
     for (int z = 0; z < splits; ++z) s += partial[(size_t)z * n + i];
-    out[i] = s;
+    out[i] = accum ? out[i] + s : s;
 }
 
-void splitk_reduce_launch(const float* partial, float* out, size_t n, int splits, cudaStream_t s) {
+void splitk_reduce_launch(const float* partial, float* out, size_t n, int splits, bool accum, cudaStream_t s) {
     Scope sc(KC_SPLITK, 0.0, 4.0 * n * (splits + 1), s);
-    splitk_reduce<<<cdiv(n, 256), 256, 0, s>>>(partial, out, n, splits);
+    splitk_reduce<<<cdiv(n, 256), 256, 0, s>>>(partial, out, n, splits, accum);
 }
 
 int wgrad_splits(const ConvGeom& g) {
@@ -297,7 +297,7 @@ void conv_dgrad(int dt, const void* dy, const void* w, void* dx, const ConvGeom&
 }
 
 template <typename T>
-static void conv_wgrad_t(const void* x, const void* dy, float* dw, float* ws, const ConvGeom& g, cudaStream_t s) {
+static void conv_wgrad_t(const void* x, const void* dy, float* dw, float* ws, const ConvGeom& g, bool accum, cudaStream_t s) {
     int Mg = g.Co, Ng = g.R * g.R * g.C, Kg = g.N * g.Ho * g.Wo;
     int splits = wgrad_splits(g);
     int kps = ((Kg + splits - 1) / splits + BK - 1) / BK * BK;
@@ -306,15 +306,16 @@ static void conv_wgrad_t(const void* x, const void* dy, float* dw, float* ws, co
     double flops = 2.0 * Mg * Ng * Kg, bytes = sizeof(T) * ((double)g.N * g.H * g.W * g.C + (double)Kg * Mg) + 4.0 * Mg * Ng;
     if (splits == 1) {
         Scope sc(KC_FMA_WGRAD, flops, bytes, s);
-        igemm_simt<T, M_WGRAD><<<grid, 256, 0, s>>>((const T*)dy, (const T*)x, dw, nullptr, nullptr, g, Mg, Ng, Kg, kps, EPI_OUT_F32);
+        igemm_simt<T, M_WGRAD><<<grid, 256, 0, s>>>((const T*)dy, (const T*)x, dw, nullptr, nullptr, g, Mg, Ng, Kg, kps,
+                                                   EPI_OUT_F32 | (accum ? EPI_ACCUM : 0));
     } else {
         { Scope sc(KC_FMA_WGRAD, flops, bytes, s);
           igemm_simt<T, M_WGRAD><<<grid, 256, 0, s>>>((const T*)dy, (const T*)x, dw, nullptr, ws, g, Mg, Ng, Kg, kps, EPI_OUT_F32); }
-        splitk_reduce_launch(ws, dw, (size_t)Mg * Ng, splits, s);
+        splitk_reduce_launch(ws, dw, (size_t)Mg * Ng, splits, accum, s);
     }
 }
-void conv_wgrad(int dt, const void* x, const void* dy, float* dw, float* ws, const ConvGeom& g, cudaStream_t s) {
-    if (dt) conv_wgrad_t<bf16>(x, dy, dw, ws, g, s); else conv_wgrad_t<float>(x, dy, dw, ws, g, s);
+void conv_wgrad(int dt, const void* x, const void* dy, float* dw, float* ws, const ConvGeom& g, bool accum, cudaStream_t s) {
+    if (dt) conv_wgrad_t<bf16>(x, dy, dw, ws, g, accum, s); else conv_wgrad_t<float>(x, dy, dw, ws, g, accum, s);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -338,21 +339,21 @@ __global__ void colsum_partial(const T* __restrict__ dy, float* __restrict__ par
         part[(size_t)blockIdx.y * C + c] = t;
     }
 }
-__global__ void colsum_final(const float* __restrict__ part, float* __restrict__ out, int chunks, int C) {
+__global__ void colsum_final(const float* __restrict__ part, float* __restrict__ out, int chunks, int C, bool accum) {
     int c = blockIdx.x * blockDim.x + threadIdx.x;
     if (c >= C) return;
     float s = 0.f;
     for (int i = 0; i < chunks; ++i) s += part[(size_t)i * C + c];
-    out[c] = s;
+    out[c] = accum ? out[c] + s : s;
 }
-void bias_grad(int dt, const void* dy, float* db, float* scratch, long rows, int C, cudaStream_t s) {
+void bias_grad(int dt, const void* dy, float* db, float* scratch, long rows, int C, bool accum, cudaStream_t s) {
     int chunks = (int)(rows < RED_CHUNKS ? rows : RED_CHUNKS);
     dim3 grid(cdiv(C, 32), chunks), blk(32, 8);
     { Scope sc(KC_BIAS_GRAD, 0.0, (dt ? 2.0 : 4.0) * rows * C, s);
       if (dt) colsum_partial<bf16><<<grid, blk, 0, s>>>((const bf16*)dy, scratch, rows, C);
       else colsum_partial<float><<<grid, blk, 0, s>>>((const float*)dy, scratch, rows, C); }
     Scope sc(KC_BIAS_GRAD, 0.0, 4.0 * chunks * C, s);
-    colsum_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, db, chunks, C);
+    colsum_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, db, chunks, C, accum);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -534,7 +535,7 @@ __global__ void bn_stats_final(const float* __restrict__ part, const T* __restri
 }
 // backward: red[w][c] = (sum dy, sum dy xhat); dgamma[c] = sum_w red[w][c].y; dbeta[c] = sum_w red[w][c].x
 __global__ void bn_bwd_final(const float* __restrict__ part, float* __restrict__ red, float* __restrict__ dgamma,
-                             float* __restrict__ dbeta, int chunks, int nw, int C) {
+                             float* __restrict__ dbeta, int chunks, int nw, int C, bool accum) {
     int c = blockIdx.x * blockDim.x + threadIdx.x;
     if (c >= C) return;
     float g = 0.f, b = 0.f;
@@ -544,7 +545,7 @@ __global__ void bn_bwd_final(const float* __restrict__ part, float* __restrict__
         red[((size_t)w * C + c) * 2] = s1; red[((size_t)w * C + c) * 2 + 1] = s2;
         b += s1; g += s2;
     }
-    dgamma[c] = g; dbeta[c] = b;
+    dgamma[c] = accum ? dgamma[c] + g : g; dbeta[c] = accum ? dbeta[c] + b : b;
 }
 template <typename T>
 __global__ void bn_apply_k(const T* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
@@ -837,7 +838,7 @@ __global__ void __launch_bounds__(128) bnv_stats_final_tiles(const float* __rest
 // block = one channel, one warp per worker (nw <= 32): red[w][c] = (sum dy, sum dy xhat); warp 0 then adds the
 // workers in ascending order into dgamma / dbeta
 __global__ void bnv_bwd_final(const float* __restrict__ part, float* __restrict__ red, float* __restrict__ dgamma,
-                              float* __restrict__ dbeta, int chunks, int nw, int C) {
+                              float* __restrict__ dbeta, int chunks, int nw, int C, bool accum) {
     __shared__ float2 sh[32];
     const int c = blockIdx.x, w = threadIdx.x >> 5, lane = threadIdx.x & 31;
     float2 a = make_float2(0.f, 0.f);
@@ -848,7 +849,7 @@ __global__ void bnv_bwd_final(const float* __restrict__ part, float* __restrict_
     if (threadIdx.x == 0) {
         float g = 0.f, b = 0.f;
         for (int i = 0; i < nw; ++i) { b += sh[i].x; g += sh[i].y; }
-        dgamma[c] = g; dbeta[c] = b;
+        dgamma[c] = accum ? dgamma[c] + g : g; dbeta[c] = accum ? dbeta[c] + b : b;
     }
 }
 
@@ -907,7 +908,7 @@ void bn_forward(int dt, const void* x, const float* gamma, const float* beta, co
 
 void bn_backward(int dt, const void* x, const void* out, const void* dout, const float* gamma, const float* beta,
                  const float* stats, void* dx, bool accum_dx, void* dres, bool accum_dres, float* dgamma, float* dbeta, float* red,
-                 float* scratch, int nw, long rpw, int C, bool relu, bool has_res, cudaStream_t s) {
+                 float* scratch, int nw, long rpw, int C, bool relu, bool has_res, bool accum_params, cudaStream_t s) {
     if (bnv_ok(dt, C)) {
         const int chunks = bnv_chunks(bnv_reduce<1>, 2, nw, rpw, C);
         const int chunks_a = bnv_chunks(bnv_bwd_apply, 3, nw, rpw, C);
@@ -919,8 +920,8 @@ void bn_backward(int dt, const void* x, const void* out, const void* dout, const
           bnv_reduce<1><<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, gamma, beta, stats, scratch, rpw, C,
                                                       relu, mask_from_x); }
         { Scope sc(KC_BN_BWD_REDUCE, 0.0, 8.0 * chunks * nw * C, s);
-          if (nw <= 32) bnv_bwd_final<<<C, 32 * nw, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C);
-          else bn_bwd_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C); }
+          if (nw <= 32) bnv_bwd_final<<<C, 32 * nw, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C, accum_params);
+          else bn_bwd_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C, accum_params); }
         Scope sc(KC_BN_BWD_APPLY, 0.0, 2.0 * total * (reads + 1 + (accum_dx ? 1 : 0) + (dres ? (accum_dres ? 2 : 1) : 0)), s);
         bnv_bwd_apply<<<dim3(chunks_a, nw), BNV_THREADS, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, gamma, beta, stats, red, (bf16*)dx,
                                                    accum_dx, (bf16*)dres, accum_dres, rpw, C, relu, mask_from_x);
@@ -934,7 +935,7 @@ void bn_backward(int dt, const void* x, const void* out, const void* dout, const
       if (dt) bn_reduce_partial<bf16, true><<<grid, blk, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, stats, scratch, rpw, C, relu);
       else bn_reduce_partial<float, true><<<grid, blk, 0, s>>>((const float*)x, (const float*)out, (const float*)dout, stats, scratch, rpw, C, relu); }
     { Scope sc(KC_BN_BWD_REDUCE, 0.0, 8.0 * chunks * nw * C, s);
-      bn_bwd_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C); }
+      bn_bwd_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C, accum_params); }
     Scope sc(KC_BN_BWD_APPLY, 0.0, esz_ * total * ((relu ? 3 : 2) + 1 + (dres ? (accum_dres ? 2 : 1) : 0) + (accum_dx ? 1 : 0)), s);
     if (dt) bn_bwd_apply_k<bf16><<<cdiv(total, 256), 256, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, gamma, stats, red,
                                                                   (bf16*)dx, accum_dx, (bf16*)dres, accum_dres, rpw, C, total, relu);

@@ -24,15 +24,16 @@ void conv_forward(int dt, const void* x, const void* w, const float* bias, void*
 void conv_dgrad(int dt, const void* dy, const void* w, void* dx, const ConvGeom& g, int epi, cudaStream_t st);
 // dW = sum over all N*Ho*Wo rows of dy^T (x) patches(x), fp32 out; the reduction runs over the
 // worker x batch axis, which is the worker average of Eq. dl_update (b) for P = 11^T/N.
-void conv_wgrad(int dt, const void* x, const void* dy, float* dw, float* workspace, const ConvGeom& g, cudaStream_t st);
+// accum: dw += (a second group of workers adds to the first group's result)
+void conv_wgrad(int dt, const void* x, const void* dy, float* dw, float* workspace, const ConvGeom& g, bool accum, cudaStream_t st);
 // db[c] = sum over rows of dy[row][c]; scratch: fp32 [64 * C]
-void bias_grad(int dt, const void* dy, float* db, float* scratch, long rows, int C, cudaStream_t st);
+void bias_grad(int dt, const void* dy, float* db, float* scratch, long rows, int C, bool accum, cudaStream_t st);
 
 // First-layer convolution (3x3, stride 1, <= 4 input channels, bf16): dedicated kernels (stem.cu).
 bool   stem_supported(int dt, const ConvGeom& g);
 size_t stem_wgrad_workspace_elems(const ConvGeom& g);
 void   stem_forward(const void* x, const void* w, const float* bias, void* y, const ConvGeom& g, bool relu, cudaStream_t st);
-void   stem_wgrad(const void* x, const void* dy, float* dw, float* workspace, const ConvGeom& g, cudaStream_t st);
+void   stem_wgrad(const void* x, const void* dy, float* dw, float* workspace, const ConvGeom& g, bool accum, cudaStream_t st);
 
 void relu_forward(int dt, const void* x, void* y, size_t n, cudaStream_t st);
 // dx (+)= dy * (y > 0)
@@ -57,7 +58,8 @@ bool bn_accepts_conv_partials(int dt, int C);
 // dgamma, dbeta (fp32) = sums over all workers.  red: fp32 [n_workers][C][2] scratch for (sum dy, sum dy xhat).
 void bn_backward(int dt, const void* x, const void* out, const void* dout, const float* gamma, const float* beta,
                  const float* stats, void* dx, bool accum_dx, void* dres_or_null, bool accum_dres, float* dgamma, float* dbeta,
-                 float* red, float* scratch, int n_workers, long rows_per_worker, int C, bool relu, bool has_res, cudaStream_t st);
+                 float* red, float* scratch, int n_workers, long rows_per_worker, int C, bool relu, bool has_res, bool accum_params,
+                 cudaStream_t st);
 
 // Softmax cross-entropy over fp32 logits [M, classes]: dlogits (storage dtype) = (softmax - onehot) / M,
 // *loss_out = mean loss.  Deterministic single-block reduction.
@@ -78,7 +80,7 @@ struct TagOps {
 void tags_step(const TagOps& ops, cudaStream_t st);
 
 void fill_f32(float* p, float v, size_t n, cudaStream_t st);
-void splitk_reduce_launch(const float* partial, float* out, size_t n, int splits, cudaStream_t st);
+void splitk_reduce_launch(const float* partial, float* out, size_t n, int splits, bool accum, cudaStream_t st);
 uint64_t launches();     // kernels launched so far through this interface
 
 // Kernel classes for launch counting and optional device timing.

@@ -157,7 +157,7 @@ __global__ void __launch_bounds__(ST_THREADS) stem_wgrad_kernel(const bf16* __re
 }
 
 // dw[co][k] = sum over CTAs (ascending) of partial[cz][b][co % 64][k]
-__global__ void stem_wgrad_reduce(const float* __restrict__ partial, float* __restrict__ dw, int blocks, int K, int Co) {
+__global__ void stem_wgrad_reduce(const float* __restrict__ partial, float* __restrict__ dw, int blocks, int K, int Co, bool accum) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= Co * K) return;
     const int co = i / K, k = i - co * K, cz = co >> 6;
@@ -165,7 +165,7 @@ __global__ void stem_wgrad_reduce(const float* __restrict__ partial, float* __re
     float s = 0.f;
 #pragma unroll 8
     for (int b = 0; b < blocks; ++b) s += p[(size_t)b * 64 * K];
-    dw[i] = s;
+    dw[i] = accum ? dw[i] + s : s;
 }
 
 void stem_forward(const void* x, const void* w, const float* bias, void* y, const ConvGeom& g, bool relu, cudaStream_t s) {
@@ -177,7 +177,7 @@ void stem_forward(const void* x, const void* w, const float* bias, void* y, cons
     stem_fwd_kernel<<<grid, ST_THREADS, smem, s>>>((const bf16*)x, (const bf16*)w, bias, (bf16*)y, g.H, g.W, g.C, g.Co, relu);
 }
 
-void stem_wgrad(const void* x, const void* dy, float* dw, float* workspace, const ConvGeom& g, cudaStream_t s) {
+void stem_wgrad(const void* x, const void* dy, float* dw, float* workspace, const ConvGeom& g, bool accum, cudaStream_t s) {
     const int TH = ST_THREADS / g.W, K = 9 * g.C;
     const size_t smem = ((size_t)(TH + 2) * (g.W + 2) * g.C + 8) * sizeof(float) + 16 + (size_t)ST_THREADS * 64 * 2 + 64 * 28 * sizeof(float);
     static bool attr = false;
@@ -188,7 +188,7 @@ void stem_wgrad(const void* x, const void* dy, float* dw, float* workspace, cons
     { Scope sc(KC_FMA_WGRAD, 2.0 * pix * g.Co * K, 2.0 * pix * (g.C + g.Co), s);
       stem_wgrad_kernel<<<dim3(blocks, 1, g.Co / 64), ST_THREADS, smem, s>>>((const bf16*)x, (const bf16*)dy, workspace, g.N, g.H, g.W, g.C, g.Co); }
     Scope sc(KC_SPLITK, 0.0, 4.0 * blocks * g.Co * K, s);
-    stem_wgrad_reduce<<<(g.Co * K + 127) / 128, 128, 0, s>>>(workspace, dw, blocks, K, g.Co);
+    stem_wgrad_reduce<<<(g.Co * K + 127) / 128, 128, 0, s>>>(workspace, dw, blocks, K, g.Co, accum);
 }
 
 }  // namespace fdg

@@ -181,7 +181,7 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 int tm = tl / tiles_c; const int co0 = (tl - tm * tiles_c) * N_TILE;
                 const int tw = tm % p.tiles_w; tm /= p.tiles_w;
                 const int th = tm % p.tiles_h; const int tn = tm / p.tiles_h;
-                const int w0 = tw * p.Wt, h0 = th * p.Ht, n0 = tn * p.Nt;
+                const int w0 = tw * p.Wt, h0 = th * p.Ht, n0 = p.n_base + tn * p.Nt;
                 const int tap0 = p.cls_tap0[cls], num_kb = (p.cls_tap0[cls + 1] - tap0) * p.kchunks;
                 for (int kb = 0; kb < num_kb; ++kb, ++kbg) {
                     const int s = kbg % STAGES, it = kbg / STAGES;
@@ -229,13 +229,13 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             const int buf = ti & 1, use = ti >> 1;
             const int cls = tile / per_cls, tl = tile - cls * per_cls;
             int tm = tl / tiles_c; const int co0 = (tl - tm * tiles_c) * N_TILE;
-            const int tmi = tm;
+            const int tmi = tm + (p.n_base / p.Nt) * (p.tiles_h * p.tiles_w);      // tile index within the whole tensor
             const int tw = tm % p.tiles_w; tm /= p.tiles_w;
             const int th = tm % p.tiles_h; const int tn = tm / p.tiles_h;
             // this lane's row of the tile -> output address (0 = row outside the tensor)
             const int row = q * 32 + lane;
             const int pw = row % p.Wt, ph = (row / p.Wt) % p.Ht, pn = row / (p.Wt * p.Ht);
-            const int n = tn * p.Nt + pn, h = th * p.Ht + ph, w = tw * p.Wt + pw;
+            const int n = p.n_base + tn * p.Nt + pn, h = th * p.Ht + ph, w = tw * p.Wt + pw;
             const bool valid = n < p.N && h < p.Hd && w < p.Wd;
             const unsigned long long rowptr = valid ? (unsigned long long)((bf16*)p.out + (((size_t)n * p.Ho + (h * p.os + p.cls_oph[cls])) * p.Wo +
                                                                                                 (w * p.os + p.cls_opw[cls])) * p.Co + co0) : 0ull;
@@ -347,7 +347,7 @@ wg_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUten
                 int pt = pt_begin + kb;
                 const int tw = pt % p.tiles_w; pt /= p.tiles_w;
                 const int th = pt % p.tiles_h; const int tn = pt / p.tiles_h;
-                const int w0 = tw * p.Wt, h0 = th * p.Ht, n0 = tn * p.Nt;
+                const int w0 = tw * p.Wt, h0 = th * p.Ht, n0 = p.n_base + tn * p.Nt;
                 uint8_t* a = smem + s * STAGE_BYTES;
                 mbar_expect_tx(&full[s], STAGE_BYTES);
                 tma_load_4d(a, &tmX, &full[s], cc0 * 64, w0 * p.xs + p.dw[tap0], h0 * p.xs + p.dh[tap0], n0);
@@ -403,7 +403,8 @@ wg_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUten
 
 // dW[co][tap][ci] = sum_z partial[z][(tap, cc)][ci % 64][co], z ascending.  32x32 transposing tiles; a thread owns
 // one (row, column) per pass and keeps eight independent loads in flight along z.
-__global__ void __launch_bounds__(1024) wg_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dw, int splits, int row_blocks, int Co) {
+__global__ void __launch_bounds__(1024) wg_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dw, int splits, int row_blocks, int Co,
+                                                         bool accum) {
     __shared__ float t[32][33];
     const int R = row_blocks * 64;                       // = taps * Cin
     const int r0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
@@ -421,7 +422,8 @@ __global__ void __launch_bounds__(1024) wg_reduce_kernel(const float* __restrict
     for (; z < splits; ++z) s += __ldg(partial + (size_t)z * zs + o);
     t[ty][tx] = s;
     __syncthreads();
-    dw[(size_t)(c0 + ty) * R + r0 + tx] = t[tx][ty];
+    float* d = dw + (size_t)(c0 + ty) * R + r0 + tx;
+    *d = accum ? *d + t[tx][ty] : t[tx][ty];
 }
 
 // Wt[ci][R*R-1-tap][co] = W[co][tap][ci]: the weights of the transposed convolution, K-major for km_kernel.
@@ -526,7 +528,7 @@ static cudaError_t launch_wg(const TensorMap& x, const TensorMap& dy, const WgPa
     return cudaGetLastError();
 }
 
-cudaError_t run_wg(const TensorMap& x, const TensorMap& dy, const WgParams& p, int n_tile, int splits, float* dw, cudaStream_t s) {
+cudaError_t run_wg(const TensorMap& x, const TensorMap& dy, const WgParams& p, int n_tile, int splits, float* dw, bool accum, cudaStream_t s) {
     dim3 grid((p.row_blocks + 1) / 2, p.Co / n_tile, splits);
     cudaError_t e;
     if (n_tile == 64) e = launch_wg<64, 4>(x, dy, p, grid, s);      // 96 KB of stages: two CTAs per SM
@@ -535,7 +537,7 @@ cudaError_t run_wg(const TensorMap& x, const TensorMap& dy, const WgParams& p, i
     else return cudaErrorInvalidValue;
     if (e != cudaSuccess) return e;
     dim3 rgrid(p.row_blocks * 2, p.Co / 32), rblk(32, 32);
-    wg_reduce_kernel<<<rgrid, rblk, 0, s>>>(p.partial, dw, splits, p.row_blocks, p.Co);
+    wg_reduce_kernel<<<rgrid, rblk, 0, s>>>(p.partial, dw, splits, p.row_blocks, p.Co, accum);
     return cudaGetLastError();
 }
 

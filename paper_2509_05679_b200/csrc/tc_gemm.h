@@ -20,6 +20,8 @@ struct KmParams {
     int cls_tap0[5];                             // class c uses taps [cls_tap0[c], cls_tap0[c+1])
     int cls_oph[4], cls_opw[4];                  // class c writes domain pixel (h, w) to (h*os + cls_oph[c], w*os + cls_opw[c])
     int N, Hd, Wd;                               // extents of the tile domain (rows outside are not stored)
+    int n_base;                                  // first sample of the group of workers this launch covers (a multiple of Nt);
+                                                 // tiles_n counts the group's tiles, N is the end of the group
     int Ho, Wo, Co, os;                          // output tensor [N,Ho,Wo,Co] and the output stride of a domain pixel
     int Cn;                                      // output channels computed (multiple of the column tile)
     int epi;                                     // EPI_RELU | EPI_ACCUM
@@ -33,6 +35,7 @@ struct KmParams {
 struct WgParams {
     int Wt, Ht, Nt, tiles_w, tiles_h, tiles_n;   // 64-pixel tile of the dY pixel grid
     int ptiles, ptiles_per_split;
+    int n_base;                                  // first sample of the group of workers this launch covers (multiple of Nt)
     int kchunks, row_blocks, xs;                 // 64-channel chunks of c_in; row blocks = taps * kchunks
     int dh[9], dw[9];
     int Co;
@@ -48,7 +51,8 @@ bool make_map_2d(TensorMap* out, const void* base, long inner, long outer, int b
 bool pixel_tile(int H, int W, int pixels, int* Wt, int* Ht, int* Nt);
 
 cudaError_t run_km(const TensorMap& a, const TensorMap& b, const KmParams& p, int n_tile, cudaStream_t s);
-cudaError_t run_wg(const TensorMap& x, const TensorMap& dy, const WgParams& p, int n_tile, int splits, float* dw, cudaStream_t s);
+// accum: dw += the result (second and later groups of workers)
+cudaError_t run_wg(const TensorMap& x, const TensorMap& dy, const WgParams& p, int n_tile, int splits, float* dw, bool accum, cudaStream_t s);
 cudaError_t run_flip_transpose(const void* w, void* wt, int Co, int taps, int Ci, cudaStream_t s);
 
 }  // namespace tc

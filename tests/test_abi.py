@@ -47,7 +47,7 @@ def test_create_without_a_device_reports_an_error_instead_of_falling_back(libpat
     # straight through the C ABI: FDG_ERR_ARCH and a message, no crash
     L = binding.lib()
     layers = (binding.fdg_layer * 1)(binding.fdg_layer(0, 8, 3, 1, 1))
-    opt = binding.fdg_options(0, 1, 1, 8, 3, 0, 0, None)
+    opt = binding.fdg_options(0, 1, 1, 8, 3, 0, 0, 0, None)
     h = ctypes.c_void_p()
     st = L.fdg_create(layers, 1, None, 1, 1, 2, 0.1, ctypes.byref(opt), None, ctypes.byref(h))
     assert st == 4 and not h.value
