@@ -160,7 +160,7 @@ def main():
     ap.add_argument("--config", type=int, default=3, help="0..4 = the five configurations; 3 = ResNet-18-shaped K=4, 8 workers x 128")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--worker-groups", type=int, default=0, help="0: chosen by the library; n: every module but the last runs its layers once per n-th of the workers")
-    ap.add_argument("--kernel-path", type=int, default=0, help="0: tensor-core kernels where shapes allow, 1: plain FMA kernels only")
+    ap.add_argument("--kernel-path", type=int, default=0, help="0: tensor-core kernels where shapes allow (CTA pairs for the 256-column tile), 1: plain FMA kernels only, 2: tensor-core kernels without CTA pairs")
     ap.add_argument("--batch", type=int, default=None, help="per-worker batch override (testing only; changes the workload name)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-uncontended", action="store_true", help="skip the extra one-stream pass that times kernels alone")

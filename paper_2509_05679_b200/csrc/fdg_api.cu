@@ -70,6 +70,7 @@ struct Op {
     tc::WgParams kw;
     std::vector<char*> a_ptrs, dy_ptrs;                      // the buffers the A / dY maps below were built for
     std::vector<tc::TensorMap> fa, fb, da, db, wx, wdy;      // fwd A, fwd B (per weight slot), dgrad A, dgrad B, wgrad X, wgrad dY
+    std::vector<tc::TensorMap> fbh, dbh;                     // fwd / dgrad B with half-height boxes (CTA-pair kernels); empty: not used
 };
 
 struct Segment { size_t canon, internal, count; bool big; };
@@ -173,10 +174,10 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
         if (bias) o.b_off = seg(cout, false);
         o.out = add_tensor(g.Ho, g.Wo, cout);
         std::snprintf(o.shape, sizeof o.shape, "%dx%d %d->%d k%d s%d", g.H, g.W, g.C, g.Co, g.R, g.stride);
-        o.stem = ctx->kernel_path == 0 && kind == FDG_CONV3X3 && stem_supported(ctx->dt, g);
+        o.stem = ctx->kernel_path != 1 && kind == FDG_CONV3X3 && stem_supported(ctx->dt, g);
         // tensor-core eligibility
         int wt, ht, nt;
-        o.tc = ctx->dt == 1 && ctx->kernel_path == 0 && g.C % 64 == 0 && g.Co % 64 == 0 &&
+        o.tc = ctx->dt == 1 && ctx->kernel_path != 1 && g.C % 64 == 0 && g.Co % 64 == 0 &&
                tc::pixel_tile(g.Ho, g.Wo, 128, &wt, &ht, &nt) && g.Ho % ht == 0 && 2 * wt <= 256 && tc::init();
         if (o.tc) {
             o.n_tile_f = g.Co % 256 == 0 ? 256 : (g.Co % 128 == 0 ? 128 : 64);
@@ -378,7 +379,7 @@ bool tc_forward(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* y_base, 
     const ConvGeom& g = o.g;
     double rows = (double)wn.n * g.Ho * g.Wo;
     Scope sc(KC_TC_FWD, 2.0 * rows * g.Co * g.R * g.R * g.C, 2.0 * ((double)wn.n * g.H * g.W * g.C + (double)g.Co * g.R * g.R * g.C + rows * g.Co), s);
-    const bool ok = tc::run_km(o.fa[ia], o.fb[version % m.D], p, o.n_tile_f, s) == cudaSuccess;
+    const bool ok = tc::run_km(o.fa[ia], o.fb[version % m.D], o.fbh.empty() ? nullptr : &o.fbh[version % m.D], p, o.n_tile_f, s) == cudaSuccess;
     if (ok && o.stat_chunks) { m.fused_stats_tensor = o.out; m.fused_stats_chunks = o.stat_chunks; }
     return ok;
 }
@@ -397,7 +398,7 @@ bool tc_dgrad(fdg_ctx* c, Module& m, const Op& o, char* dy_base, char* dx_base, 
     const double crows = (double)wn.n * p.Hd * p.Wd;         // pixels of one class; every tap belongs to exactly one class
     Scope sc(KC_TC_DGRAD, 2.0 * crows * g.C * p.ntaps * g.Co,
              2.0 * ((double)wn.n * g.Ho * g.Wo * g.Co + (double)g.Co * p.ntaps * g.C + crows * p.ncls * g.C * (accum ? 2 : 1)), s);
-    return tc::run_km(o.da[ia], o.db[version % m.D], p, o.n_tile_d, s) == cudaSuccess;
+    return tc::run_km(o.da[ia], o.db[version % m.D], o.dbh.empty() ? nullptr : &o.dbh[version % m.D], p, o.n_tile_d, s) == cudaSuccess;
 }
 bool tc_wgrad(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* dy_base, float* dw, const Win& wn, cudaStream_t s) {
     int ix = find_buf(o.a_ptrs, x_base), id = find_buf(o.dy_ptrs, dy_base);
@@ -561,6 +562,11 @@ bool build_tc_plans(fdg_ctx* c) {
             for (size_t i = 0; i < o.a_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.fa[i], o.a_ptrs[i], g.C, g.W, g.H, g.N, 64, wt, ht, nt, g.stride);
             o.fb.resize(m.D);
             for (int v = 0; v < m.D; ++v) ok = ok && tc::make_map_2d(&o.fb[v], wbig(c, m, v, o.w_off), Ktot, g.Co, 64, o.n_tile_f);
+            const bool pairs = c->kernel_path == 0;          // CTA-pair kernels for the 256-column tile (kernel_path 2: none)
+            if (pairs && o.n_tile_f >= 256) {
+                o.fbh.resize(m.D);
+                for (int v = 0; v < m.D; ++v) ok = ok && tc::make_map_2d(&o.fbh[v], wbig(c, m, v, o.w_off), Ktot, g.Co, 64, o.n_tile_f / 2);
+            }
             // ---- input gradient: dx[n, h, w, :] = sum over taps (r, s) with (h + pad - r), (w + pad - s) divisible by
             // the stride of dy[n, (h + pad - r) / stride, (w + pad - s) / stride, :] . W[:, r, s, :].
             // One launch per parity class (h mod stride, w mod stride); the class's pixels form a dense grid of the
@@ -586,6 +592,10 @@ bool build_tc_plans(fdg_ctx* c) {
             for (size_t i = 0; i < o.dy_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.da[i], o.dy_ptrs[i], g.Co, g.Wo, g.Ho, g.N, 64, wt, ht, nt, 1);
             o.db.resize(m.D);
             for (int v = 0; v < m.D; ++v) ok = ok && tc::make_map_2d(&o.db[v], wtslot(m, v, o.w_off), (long)taps * g.Co, g.C, 64, o.n_tile_d);
+            if (pairs && o.n_tile_d >= 256) {
+                o.dbh.resize(m.D);
+                for (int v = 0; v < m.D; ++v) ok = ok && tc::make_map_2d(&o.dbh[v], wtslot(m, v, o.w_off), (long)taps * g.Co, g.C, 64, o.n_tile_d / 2);
+            }
             // ---- weight gradient: 64-pixel boxes of x (shifted per tap) and of dy
             tc::pixel_tile(g.Ho, g.Wo, 64, &wt, &ht, &nt);
             tc::WgParams& w = o.kw; w = tc::WgParams{};

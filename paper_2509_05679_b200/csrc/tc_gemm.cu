@@ -58,6 +58,17 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* e
     }
     return true;
 }
+// The same for whole warps that wait long (the epilogue warps wait for a tile's MMAs): sleeping between polls keeps
+// them out of the issue slots and the barrier unit that the single producer and MMA threads depend on.
+__device__ __forceinline__ bool mbar_wait_sleep(uint64_t* bar, uint32_t parity, int* err, int code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        __nanosleep(200);
+        if (clock64() - t0 > WAIT_CYCLES) { atomicCAS(err, 0, code); return false; }
+    }
+    return true;
+}
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -90,6 +101,95 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
 // the mbarrier receives one arrival when all previously issued MMAs of this thread have completed
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// ---- forms that take 32-bit shared-memory addresses.  The TMA-producer and MMA-issuer loops run in ONE thread each, so
+// every instruction in them is on the critical path (measured: a k-block of four 128x256x16 MMAs is 512 cycles of
+// tensor-pipe work, and a loop body that rebuilt descriptors and divided by the stage count took about 900): the
+// loops keep running addresses and phases and add constants to descriptor words instead.
+__device__ __forceinline__ bool mbar_wait_a(uint32_t bar, uint32_t parity, int* err, int code) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    if (ok) return true;
+    long long t0 = clock64();
+    for (;;) {
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+        if (clock64() - t0 > WAIT_CYCLES) { atomicCAS(err, 0, code); return false; }
+    }
+}
+__device__ __forceinline__ void mbar_expect_tx_a(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_a(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+                 ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_a(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+// descriptors given as (low word, shared high word): only the address field in the low word changes between MMAs
+template <bool PAIR>
+__device__ __forceinline__ void umma_bf16_w(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t accumulate) {
+    if (PAIR)
+        asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+                     "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t}"
+                     ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate) : "memory");
+    else
+        asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+                     "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+                     ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+template <bool PAIR>
+__device__ __forceinline__ void umma_commit_a(uint32_t bar) {
+    if (PAIR)
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar), "h"((uint16_t)3) : "memory");
+    else
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// ---- CTA pairs (cluster of two, tcgen05 cta_group::2): one MMA of 256 rows, each CTA holds its 128 rows of A and of
+// the accumulator and half of B's rows, so every SM reads only half of B from its shared memory.
+__device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+// address of the same shared-memory object in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+    uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank)); return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA loads whose completion is signalled on an mbarrier of either CTA of the pair (`bar` is a cluster address)
+__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+                 ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+// executed by the same warp of both CTAs of the pair
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* slot, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// issued by one thread of the pair's first CTA; descriptors address the same offsets in both CTAs' shared memory
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// one arrival on the mbarrier at this offset in BOTH CTAs once all MMAs issued so far have completed
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"((uint16_t)3) : "memory");
 }
 // 32 lanes x 32 consecutive fp32 columns -> 32 registers per thread (thread = lane)
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
@@ -138,12 +238,21 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 constexpr int EPI_ROW_WORDS = 36;                 // 32 fp32 + 4 padding: conflict-free 128-bit rows
 
 // EPI_WARPS = 4 or 8: with 8, two warps share each quarter of the tensor-memory lanes and take alternate 32-column slices.
-template <int N_TILE, int STAGES, int EPI_WARPS>
+// PAIR: launched as clusters of two CTAs.  A pair computes two neighbouring pixel tiles against the same column tile
+// with one 256-row MMA per step, issued by the pair's first CTA; each CTA loads its own pixel tile and half of the
+// weight rows, drains its own half of the accumulator, and the tmem_empty / full barriers of the first CTA collect
+// both CTAs' arrivals.  The number of pixel tiles must be even.
+// KSUB: 64-wide K sub-blocks per pipeline stage.  One full / empty barrier round trip costs the issuing threads
+// several hundred cycles whatever the stage holds, so narrow tiles (little MMA work per sub-block) put more sub-blocks
+// behind each barrier; a tile's last stage may hold fewer.
+template <int N_TILE, int STAGES, int EPI_WARPS, bool PAIR, int KSUB>
 __global__ void __launch_bounds__(64 + 32 * EPI_WARPS, 1)
 km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, KmParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
-    constexpr int A_BYTES = BLOCK_M * BLOCK_K * 2, B_BYTES = N_TILE * BLOCK_K * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+    constexpr int B_ROWS = PAIR ? N_TILE / 2 : N_TILE;
+    constexpr int A_BYTES = BLOCK_M * BLOCK_K * 2, B_BYTES = B_ROWS * BLOCK_K * 2, SUB_BYTES = A_BYTES + B_BYTES;
+    constexpr int STAGE_BYTES = KSUB * SUB_BYTES;
     constexpr int EPI_BYTES = EPI_WARPS * 32 * EPI_ROW_WORDS * 4;
     constexpr int COL_STEP = 32 * (EPI_WARPS / 4);
     constexpr uint32_t TMEM_COLS = 2 * N_TILE;
@@ -155,68 +264,108 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     uint32_t* tmem_slot = (uint32_t*)(tmem_empty + 2);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tiles_m = p.tiles_w * p.tiles_h * p.tiles_n;
+    const uint32_t rank = PAIR ? cluster_rank() : 0u;
+    const int walker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x, walkers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const int tiles_m = p.tiles_w * p.tiles_h * p.tiles_n / (PAIR ? 2 : 1);     // pixel tiles, or pairs of them
     const int tiles_c = p.Cn / N_TILE;
     const int per_cls = tiles_m * tiles_c;
-    const int total = per_cls * p.ncls;                 // tile index = (class, pixel tile, column tile), column tile fastest
+    const int total = per_cls * p.ncls;                 // tile index = (class, pixel tile (pair), column tile), column tile fastest
 
     if (threadIdx.x == 0) {
         tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB);
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], EPI_WARPS); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], PAIR ? 2 * EPI_WARPS : EPI_WARPS); }
         fence_barrier_init();
     }
-    if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);
+    __syncwarp();
+    if (warp == 1) { if (PAIR) tmem_alloc_pair(tmem_slot, TMEM_COLS); else tmem_alloc(tmem_slot, TMEM_COLS); }
     tc_fence_before();
-    __syncthreads();
+    if (PAIR) cluster_sync_all(); else __syncthreads();       // the pair's barriers are initialised before either CTA signals one
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
         if (lane == 0) {
-            int kbg = 0;                                              // k-blocks issued so far, over all tiles
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+            const uint32_t smem0 = smem_u32(smem), full_l0 = smem_u32(full), empty0 = smem_u32(empty);
+            const uint32_t full_s0 = PAIR ? map_to_cta(full_l0, 0) : full_l0;      // where loads signal: the pair's first CTA
+            // stage cursor: destination, barriers, and the parity this thread waits for on `empty` (a fresh barrier
+            // passes a wait for parity 1, so the first round finds every stage free)
+            uint32_t st = 0, ph = 1, dst = smem0, fb = full_s0, fl = full_l0, eb = empty0;
+            for (int tile = walker; tile < total && ok; tile += walkers) {
                 const int cls = tile / per_cls, tl = tile - cls * per_cls;
                 int tm = tl / tiles_c; const int co0 = (tl - tm * tiles_c) * N_TILE;
+                if (PAIR) tm = 2 * tm + (int)rank;
                 const int tw = tm % p.tiles_w; tm /= p.tiles_w;
                 const int th = tm % p.tiles_h; const int tn = tm / p.tiles_h;
-                const int w0 = tw * p.Wt, h0 = th * p.Ht, n0 = p.n_base + tn * p.Nt;
-                const int tap0 = p.cls_tap0[cls], num_kb = (p.cls_tap0[cls + 1] - tap0) * p.kchunks;
-                for (int kb = 0; kb < num_kb; ++kb, ++kbg) {
-                    const int s = kbg % STAGES, it = kbg / STAGES;
-                    if (it > 0 && !mbar_wait(&empty[s], (it - 1) & 1, p.err, 1)) { ok = false; break; }
-                    const int tq = kb / p.kchunks, kc = kb - tq * p.kchunks, tap = tap0 + tq;
-                    uint8_t* a = smem + s * STAGE_BYTES;
-                    mbar_expect_tx(&full[s], STAGE_BYTES);
-                    tma_load_4d(a, &tmA, &full[s], kc * BLOCK_K, w0 * p.xs + p.dw[tap], h0 * p.xs + p.dh[tap], n0);
-                    tma_load_2d(a + A_BYTES, &tmB, &full[s], p.koff[tap] + kc * BLOCK_K, co0);
+                const int w0 = tw * p.Wt * p.xs, h0 = th * p.Ht * p.xs, n0 = p.n_base + tn * p.Nt;
+                const int brow = co0 + (PAIR ? (int)rank * B_ROWS : 0);
+                const int tap_end = p.cls_tap0[cls + 1];
+                int left = (tap_end - p.cls_tap0[cls]) * p.kchunks;      // sub-blocks of this tile still to load
+                int sub = 0;                                               // sub-block slot inside the current stage
+                for (int tap = p.cls_tap0[cls]; tap < tap_end && ok; ++tap) {
+                    const int cw = w0 + p.dw[tap], chh = h0 + p.dh[tap], kcol = p.koff[tap];
+                    for (int kc = 0; kc < p.kchunks; ++kc) {
+                        if (sub == 0) {
+                            if (!mbar_wait_a(eb, ph, p.err, 1)) { ok = false; break; }
+                            // the stage's loads (both CTAs' for a pair) complete on one barrier that expects all their bytes
+                            const int cnt = left < KSUB ? left : KSUB;
+                            if (!PAIR || rank == 0) mbar_expect_tx_a(fl, (PAIR ? 2 : 1) * cnt * SUB_BYTES);
+                        }
+                        const uint32_t da = dst + sub * SUB_BYTES;
+                        if (PAIR) {
+                            tma_load_4d_pair(da, &tmA, fb, kc * BLOCK_K, cw, chh, n0);
+                            tma_load_2d_pair(da + A_BYTES, &tmB, fb, kcol + kc * BLOCK_K, brow);
+                        } else {
+                            tma_load_4d_a(da, &tmA, fb, kc * BLOCK_K, cw, chh, n0);
+                            tma_load_2d_a(da + A_BYTES, &tmB, fb, kcol + kc * BLOCK_K, brow);
+                        }
+                        --left;
+                        if (++sub == KSUB || left == 0) {
+                            sub = 0;
+                            if (++st == STAGES) { st = 0; ph ^= 1u; dst = smem0; fb = full_s0; fl = full_l0; eb = empty0; }
+                            else { dst += STAGE_BYTES; fb += 8; fl += 8; eb += 8; }
+                        }
+                    }
                 }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc(BLOCK_M, N_TILE, 0, 0);
-            int kbg = 0, ti = 0;
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = make_idesc(PAIR ? 2 * BLOCK_M : BLOCK_M, N_TILE, 0, 0);
+            const uint64_t dconst = make_desc(0, 16, 1024);                     // address field left empty
+            const uint32_t d_hi = (uint32_t)(dconst >> 32), d_lo = (uint32_t)dconst;
+            const uint32_t a16_0 = smem_u32(smem) >> 4, full0 = smem_u32(full), empty0 = smem_u32(empty);
+            uint32_t st = 0, ph = 0, a16 = a16_0, fb = full0, eb = empty0;
+            int ti = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++ti) {
+            for (int tile = walker; tile < total && ok; tile += walkers, ++ti) {
                 const int buf = ti & 1, use = ti >> 1;
                 const int cls = tile / per_cls;
                 const int num_kb = (p.cls_tap0[cls + 1] - p.cls_tap0[cls]) * p.kchunks;
                 if (use > 0 && !mbar_wait(&tmem_empty[buf], (use - 1) & 1, p.err, 7)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d = tmem_base + buf * N_TILE;
-                for (int kb = 0; kb < num_kb; ++kb, ++kbg) {
-                    const int s = kbg % STAGES, it = kbg / STAGES;
-                    if (!mbar_wait(&full[s], it & 1, p.err, 2)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t a = smem_u32(smem + s * STAGE_BYTES), b = a + A_BYTES;
+                uint32_t acc = 0;
+                for (int left = num_kb; left > 0; left -= KSUB) {
+                    if (!mbar_wait_a(fb, ph, p.err, 2)) { ok = false; break; }
+                    const uint32_t a_lo = d_lo + a16, b_lo = a_lo + (A_BYTES >> 4);
 #pragma unroll
-                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                        umma_bf16(d, make_desc(a + k * UMMA_K * 2, 16, 1024), make_desc(b + k * UMMA_K * 2, 16, 1024), idesc, (kb | k) != 0);
-                    umma_commit(&empty[s]);
+                    for (int j = 0; j < KSUB; ++j) {
+                        if (j < left) {
+#pragma unroll
+                            for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {        // 16 columns of K = 32 bytes = 2 address units
+                                umma_bf16_w<PAIR>(d, a_lo + j * (SUB_BYTES >> 4) + 2 * k, b_lo + j * (SUB_BYTES >> 4) + 2 * k, d_hi, idesc, acc);
+                                acc = 1;
+                            }
+                        }
+                    }
+                    umma_commit_a<PAIR>(eb);
+                    if (++st == STAGES) { st = 0; ph ^= 1u; a16 = a16_0; fb = full0; eb = empty0; }
+                    else { a16 += STAGE_BYTES >> 4; fb += 8; eb += 8; }
                 }
-                umma_commit(&tmem_full[buf]);      // arrives once every MMA of this tile has finished
+                // arrives once every MMA of this tile has finished (in both CTAs of a pair)
+                umma_commit_a<PAIR>(smem_u32(&tmem_full[buf]));
             }
         }
     } else {
@@ -225,10 +374,12 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         float* stage = epi_smem + (warp - 2) * 32 * EPI_ROW_WORDS;
         int ti = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++ti) {
+        const uint32_t tmem_empty0 = PAIR ? map_to_cta(smem_u32(&tmem_empty[0]), 0) : 0u;
+        for (int tile = walker; tile < total && ok; tile += walkers, ++ti) {
             const int buf = ti & 1, use = ti >> 1;
             const int cls = tile / per_cls, tl = tile - cls * per_cls;
             int tm = tl / tiles_c; const int co0 = (tl - tm * tiles_c) * N_TILE;
+            if (PAIR) tm = 2 * tm + (int)rank;
             const int tmi = tm + (p.n_base / p.Nt) * (p.tiles_h * p.tiles_w);      // tile index within the whole tensor
             const int tw = tm % p.tiles_w; tm /= p.tiles_w;
             const int th = tm % p.tiles_h; const int tn = tm / p.tiles_h;
@@ -240,7 +391,7 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             const unsigned long long rowptr = valid ? (unsigned long long)((bf16*)p.out + (((size_t)n * p.Ho + (h * p.os + p.cls_oph[cls])) * p.Wo +
                                                                                                 (w * p.os + p.cls_opw[cls])) * p.Co + co0) : 0ull;
             const unsigned vmask = __ballot_sync(0xffffffffu, rowptr != 0ull);
-            ok = mbar_wait(&tmem_full[buf], use & 1, p.err, 3);
+            ok = mbar_wait_sleep(&tmem_full[buf], use & 1, p.err, 3);
             tc_fence_after();
 #pragma unroll 1
             for (int c = half * 32; c < N_TILE; c += COL_STEP) {
@@ -249,7 +400,7 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 if (c + COL_STEP >= N_TILE) {      // this warp's last read of the accumulator: hand the buffer back to the MMA warp
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&tmem_empty[buf]);
+                    if (lane == 0) { if (PAIR) mbar_arrive_cluster(tmem_empty0 + 8 * buf); else mbar_arrive(&tmem_empty[buf]); }
                 }
                 // bias / ReLU on this lane's row, then into the staging rows
 #pragma unroll
@@ -298,8 +449,9 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         }
     }
     tc_fence_before();
-    __syncthreads();
-    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, TMEM_COLS); }
+    __syncwarp();
+    if (PAIR) cluster_sync_all(); else __syncthreads();       // neither CTA of a pair leaves while the other may still signal it
+    if (warp == 1) { tc_fence_after(); if (PAIR) tmem_dealloc_pair(tmem_base, TMEM_COLS); else tmem_dealloc(tmem_base, TMEM_COLS); }
 }
 
 // ------------------------------------------------------------------------------------------ weight gradient
@@ -339,44 +491,56 @@ wg_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUten
 
     if (warp == 0) {
         if (lane == 0) {
-            const int tap0 = rb0 / p.kchunks, cc0 = rb0 - tap0 * p.kchunks;
-            const int tap1 = rb1 / p.kchunks, cc1 = rb1 - tap1 * p.kchunks;
+            const int tap0 = rb0 / p.kchunks, cc0 = (rb0 - tap0 * p.kchunks) * 64;
+            const int tap1 = rb1 / p.kchunks, cc1 = (rb1 - tap1 * p.kchunks) * 64;
+            const int dw0 = p.dw[tap0], dh0 = p.dh[tap0], dw1 = p.dw[tap1], dh1 = p.dh[tap1];
+            const uint32_t smem0 = smem_u32(smem), full0 = smem_u32(full), empty0 = smem_u32(empty);
+            uint32_t st = 0, ph = 1, dst = smem0, fb = full0, eb = empty0;
+            // pixel-tile cursor (tw fastest, then th, then tn), advanced without divisions
+            int pt = pt_begin;
+            int tw = pt % p.tiles_w; pt /= p.tiles_w;
+            int th = pt % p.tiles_h; int tn = pt / p.tiles_h;
+            const int wstep = p.Wt * p.xs, hstep = p.Ht * p.xs;
             for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % STAGES, it = kb / STAGES;
-                if (it > 0 && !mbar_wait(&empty[s], (it - 1) & 1, p.err, 4)) break;
-                int pt = pt_begin + kb;
-                const int tw = pt % p.tiles_w; pt /= p.tiles_w;
-                const int th = pt % p.tiles_h; const int tn = pt / p.tiles_h;
+                if (!mbar_wait_a(eb, ph, p.err, 4)) break;
                 const int w0 = tw * p.Wt, h0 = th * p.Ht, n0 = p.n_base + tn * p.Nt;
-                uint8_t* a = smem + s * STAGE_BYTES;
-                mbar_expect_tx(&full[s], STAGE_BYTES);
-                tma_load_4d(a, &tmX, &full[s], cc0 * 64, w0 * p.xs + p.dw[tap0], h0 * p.xs + p.dh[tap0], n0);
-                tma_load_4d(a + BOX_BYTES, &tmX, &full[s], cc1 * 64, w0 * p.xs + p.dw[tap1], h0 * p.xs + p.dh[tap1], n0);
+                const int xw = tw * wstep, xh = th * hstep;
+                mbar_expect_tx_a(fb, STAGE_BYTES);
+                tma_load_4d_a(dst, &tmX, fb, cc0, xw + dw0, xh + dh0, n0);
+                tma_load_4d_a(dst + BOX_BYTES, &tmX, fb, cc1, xw + dw1, xh + dh1, n0);
 #pragma unroll
                 for (int j = 0; j < N_TILE / 64; ++j)
-                    tma_load_4d(a + A_BYTES + j * BOX_BYTES, &tmDY, &full[s], co0 + j * 64, w0, h0, n0);
+                    tma_load_4d_a(dst + A_BYTES + j * BOX_BYTES, &tmDY, fb, co0 + j * 64, w0, h0, n0);
+                if (++tw == p.tiles_w) { tw = 0; if (++th == p.tiles_h) { th = 0; ++tn; } }
+                if (++st == STAGES) { st = 0; ph ^= 1u; dst = smem0; fb = full0; eb = empty0; }
+                else { dst += STAGE_BYTES; fb += 8; eb += 8; }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = make_idesc(BLOCK_M, N_TILE, 1, 1);
+            const uint64_t dconst = make_desc(0, BOX_BYTES, 1024);
+            const uint32_t d_hi = (uint32_t)(dconst >> 32), d_lo = (uint32_t)dconst;
+            const uint32_t a16_0 = smem_u32(smem) >> 4, full0 = smem_u32(full), empty0 = smem_u32(empty);
+            uint32_t st = 0, ph = 0, a16 = a16_0, fb = full0, eb = empty0, acc = 0;
             for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % STAGES, it = kb / STAGES;
-                if (!mbar_wait(&full[s], it & 1, p.err, 5)) break;
-                tc_fence_after();
-                const uint32_t a = smem_u32(smem + s * STAGE_BYTES), b = a + A_BYTES;
+                if (!mbar_wait_a(fb, ph, p.err, 5)) break;
+                const uint32_t a_lo = d_lo + a16, b_lo = a_lo + (A_BYTES >> 4);
 #pragma unroll
-                for (int k = 0; k < 64 / UMMA_K; ++k)      // 16 pixels = 16 rows of 128 bytes per MMA
-                    umma_bf16(tmem_base, make_desc(a + k * UMMA_K * 128, BOX_BYTES, 1024), make_desc(b + k * UMMA_K * 128, BOX_BYTES, 1024),
-                              idesc, (kb | k) != 0);
-                umma_commit(&empty[s]);
+                for (int k = 0; k < 64 / UMMA_K; ++k) {    // 16 pixels = 16 rows of 128 bytes per MMA = 128 address units
+                    umma_bf16_w<false>(tmem_base, a_lo + k * (UMMA_K * 128 >> 4), b_lo + k * (UMMA_K * 128 >> 4), d_hi, idesc, acc);
+                    acc = 1;
+                }
+                umma_commit_a<false>(eb);
+                if (++st == STAGES) { st = 0; ph ^= 1u; a16 = a16_0; fb = full0; eb = empty0; }
+                else { a16 += STAGE_BYTES >> 4; fb += 8; eb += 8; }
             }
             umma_commit(accum_bar);
         }
     } else {
         const int q = warp & 3;
         const int row = q * 32 + lane;
-        const bool ok = num_kb > 0 ? mbar_wait(accum_bar, 0, p.err, 6) : true;
+        const bool ok = num_kb > 0 ? mbar_wait_sleep(accum_bar, 0, p.err, 6) : true;
         tc_fence_after();
         const int rb = rb0 + (row >> 6);
         const bool valid = ok && rb < p.row_blocks;
@@ -492,26 +656,60 @@ static int sm_count() {
     return n;
 }
 
-template <int N_TILE, int STAGES, int EPI_WARPS>
+template <int N_TILE, int STAGES, int EPI_WARPS, int KSUB>
 static cudaError_t launch_km(const TensorMap& a, const TensorMap& b, const KmParams& p, cudaStream_t s) {
-    constexpr int smem = STAGES * (BLOCK_M * BLOCK_K * 2 + N_TILE * BLOCK_K * 2) + EPI_WARPS * 32 * EPI_ROW_WORDS * 4 + 1024 + 256;
+    constexpr int smem = STAGES * KSUB * (BLOCK_M * BLOCK_K * 2 + N_TILE * BLOCK_K * 2) + EPI_WARPS * 32 * EPI_ROW_WORDS * 4 + 1024 + 256;
+    static_assert(smem <= 232448, "shared memory");
+    auto kernel = km_kernel<N_TILE, STAGES, EPI_WARPS, false, KSUB>;
     static bool attr = false;
     if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(km_kernel<N_TILE, STAGES, EPI_WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         attr = true;
     }
     const int total = p.tiles_w * p.tiles_h * p.tiles_n * (p.Cn / N_TILE) * p.ncls;
-    const int slots = sm_count() * (smem <= 113 * 1024 ? 2 : 1);       // the 64-column variant fits twice on an SM
+    // CTAs of this variant that fit on an SM: shared memory (227 KB, 1 KB reserved per CTA) and 512 tensor-memory columns
+    constexpr int by_smem = (227 * 1024) / (smem + 1024), by_tmem = 512 / (2 * N_TILE);
+    constexpr int per_sm = by_smem < by_tmem ? by_smem : by_tmem;
+    const int slots = sm_count() * per_sm;
     const int grid = total < slots ? total : slots;
-    km_kernel<N_TILE, STAGES, EPI_WARPS><<<grid, 64 + 32 * EPI_WARPS, smem, s>>>(*(const CUtensorMap*)&a, *(const CUtensorMap*)&b, p);
+    kernel<<<grid, 64 + 32 * EPI_WARPS, smem, s>>>(*(const CUtensorMap*)&a, *(const CUtensorMap*)&b, p);
     return cudaGetLastError();
 }
 
-cudaError_t run_km(const TensorMap& a, const TensorMap& b, const KmParams& p, int n_tile, cudaStream_t s) {
-    if (n_tile == 64) return launch_km<64, 3, 4>(a, b, p, s);
-    if (n_tile == 128) return launch_km<128, 5, 8>(a, b, p, s);
-    if (n_tile == 256) return launch_km<256, 4, 4>(a, b, p, s);
+// CTA pairs: `b` is a tensor map whose box holds N_TILE / 2 weight rows.
+template <int N_TILE, int STAGES, int EPI_WARPS, int KSUB>
+static cudaError_t launch_km_pair(const TensorMap& a, const TensorMap& b, const KmParams& p, cudaStream_t s) {
+    constexpr int smem = STAGES * KSUB * (BLOCK_M * BLOCK_K * 2 + (N_TILE / 2) * BLOCK_K * 2) + EPI_WARPS * 32 * EPI_ROW_WORDS * 4 + 1024 + 256;
+    static_assert(smem <= 232448, "shared memory");
+    auto kernel = km_kernel<N_TILE, STAGES, EPI_WARPS, true, KSUB>;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(64 + 32 * EPI_WARPS); cfg.dynamicSmemBytes = smem; cfg.stream = s; cfg.attrs = at; cfg.numAttrs = 1;
+    static int max_pairs = 0;                   // pairs that can be resident at once
+    if (!max_pairs) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        cfg.gridDim = dim3(sm_count());
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n <= 0) { cudaGetLastError(); n = sm_count() / 2; }
+        max_pairs = n < sm_count() / 2 ? n : sm_count() / 2;
+    }
+    const int total = (p.tiles_w * p.tiles_h * p.tiles_n / 2) * (p.Cn / N_TILE) * p.ncls;
+    cfg.gridDim = dim3(2 * (total < max_pairs ? total : max_pairs));
+    return cudaLaunchKernelEx(&cfg, kernel, *(const CUtensorMap*)&a, *(const CUtensorMap*)&b, p);
+}
+
+cudaError_t run_km(const TensorMap& a, const TensorMap& b, const TensorMap* b_half, const KmParams& p, int n_tile, cudaStream_t s) {
+    const bool pair = b_half && n_tile == 256 && (p.tiles_w * p.tiles_h * p.tiles_n) % 2 == 0;
+    // measured on a B200: the narrow tiles run best with two CTAs per SM and short pipelines (3 x 24 KB, 2 x 32 KB stages);
+    // the 256-column tile as a CTA pair with six 32 KB stages; more sub-blocks per stage changed nothing
+    if (pair && n_tile == 256) return launch_km_pair<256, 6, 4, 1>(a, *b_half, p, s);
+    if (n_tile == 64) return launch_km<64, 3, 4, 1>(a, b, p, s);
+    if (n_tile == 128) return launch_km<128, 2, 4, 1>(a, b, p, s);
+    if (n_tile == 256) return launch_km<256, 4, 4, 1>(a, b, p, s);
     return cudaErrorInvalidValue;
 }
 

@@ -50,7 +50,9 @@ bool make_map_2d(TensorMap* out, const void* base, long inner, long outer, int b
 // Wt x Ht x Nt = pixels, Wt = min(W, pixels) ...; false unless H and W are powers of two
 bool pixel_tile(int H, int W, int pixels, int* Wt, int* Ht, int* Nt);
 
-cudaError_t run_km(const TensorMap& a, const TensorMap& b, const KmParams& p, int n_tile, cudaStream_t s);
+// b_half: nullptr, or a map of the same matrix whose box holds n_tile / 2 rows: the kernel then runs as CTA pairs
+// (two SMs share one 256-row MMA and each loads half of B) when n_tile is 256 and the number of pixel tiles is even.
+cudaError_t run_km(const TensorMap& a, const TensorMap& b, const TensorMap* b_half, const KmParams& p, int n_tile, cudaStream_t s);
 // accum: dw += the result (second and later groups of workers)
 cudaError_t run_wg(const TensorMap& x, const TensorMap& dy, const WgParams& p, int n_tile, int splits, float* dw, bool accum, cudaStream_t s);
 cudaError_t run_flip_transpose(const void* w, void* wt, int Co, int taps, int Ci, cudaStream_t s);

@@ -51,6 +51,12 @@ SINGLE_MODULE_NETS = {
                               (sy.CONV3X3, 2 * C, 2 * C, 1, 0), (sy.BATCHNORM, 2 * C, 2 * C, 1, 0), (sy.RES_ADD, C, 2 * C, 2, 1),
                               (sy.RELU, 2 * C, 2 * C, 1, 0), (sy.GLOBAL_AVGPOOL, 2 * C, 2 * C, 1, 0), (sy.LINEAR, 2 * C, 10, 1, 1)],
     "mlp": sy.mlp_layers([48, 40, 24, 10]),
+    # 64 / 128 / 256 channels without batch-norm: the tensor-core kernels with their 64-, 128- and 256-column tiles
+    # (the two wider ones as CTA pairs) where nothing amplifies a rounding difference
+    "tensor-core-conv-64-128-256": [(sy.CONV3X3, 3, 64, 1, 1), (sy.RELU, 64, 64, 1, 0), (sy.CONV3X3, 64, 128, 1, 1), (sy.RELU, 128, 128, 1, 0),
+                                    (sy.MAXPOOL2, 128, 128, 2, 0), (sy.CONV3X3, 128, 256, 1, 1), (sy.RELU, 256, 256, 1, 0),
+                                    (sy.CONV3X3, 256, 256, 1, 1), (sy.RELU, 256, 256, 1, 0), (sy.GLOBAL_AVGPOOL, 256, 256, 1, 0),
+                                    (sy.LINEAR, 256, 10, 1, 1)],
 }
 
 
@@ -59,7 +65,11 @@ def test_single_module_nets_match_the_storage_model_tightly(orc, name):
     layers = SINGLE_MODULE_NETS[name]
     shape = (1, 1, 48) if name == "mlp" else (16, 16, 3)
     net = sy.Net(name, layers, [], *shape, 10, 2, 4, 0.05, "bf16")
-    rec = run_parity(orc, net, 1, grad_tol=2e-3, loss_tol=1e-5)
+    # the tensor-core net sums up to 2304 products per output in fp32 (the others at most 144, compensated): more of its
+    # stored bf16 values land on the other side of a rounding boundary than in the fp64 oracle
+    tc = name.startswith("tensor-core")
+    rec = run_parity(orc, net, 1, grad_tol=2e-2 if tc else 2e-3, loss_tol=1e-3 if tc else 1e-5)
+    print(name, rec[0])
     assert rec[0]["grad_err"] > 0
 
 
@@ -71,3 +81,33 @@ def test_config4_shaped_resnet(orc):
 def test_config5_shaped_resnet_eight_modules(orc):
     net = sy.config(4, n_workers=2, batch=2, width_div=8)
     run_parity(orc, net, 2 * net.K + 2, grad_tol=GRAD_TOL, grad_steps=2 * net.K - 1, grad_tail=2, loss_tol=LOSS_TOL)
+
+
+@pytest.mark.parametrize("widths", [(64, 128), (64, 256)])
+def test_cta_pair_kernels_equal_single_cta_kernels_bitwise(orc, widths):
+    """Residual blocks at 128 / 256 channels (3x3, stride 2, 1x1 projection): the CTA-pair tensor-core kernels
+    (kernel_path 0) and the single-CTA ones (kernel_path 2) run the same MMAs in the same order, so gradients and
+    weights must be identical; against the oracle the first step holds the usual bf16 gradient tolerance."""
+    import torch
+    from paper_2509_05679_b200 import binding
+    from harness import make_ctx, make_oracle, grad_rel_l2
+    net = sy.Net("blocks", sy.resnet_layers(widths=widths, blocks=1)[0], [], 16, 16, 3, 10, 2, 4, 0.05, "bf16")
+    p0 = sy.perturb_params(sy.init_params(net.layers, 0, bf16=True), net.layers, 7, 0.1)
+    out = {}
+    for kp in (0, 2):
+        ctx = make_ctx(net, p0, kernel_path=kp)
+        grads = []
+        for t in range(3):
+            ctx.step(binding.to_device("bf16", sy.batch_inputs(net, t)), torch.from_numpy(sy.batch_labels(net, t)).cuda())
+            ctx.wait_ingest()
+            grads.append(ctx.grads())
+        out[kp] = (grads, ctx.params())
+        ctx.close()
+    for a, b in zip(out[0][0], out[2][0]):
+        assert np.array_equal(a, b)
+    assert np.array_equal(out[0][1], out[2][1])
+    o = make_oracle(orc, net, p0)
+    o.step(sy.batch_inputs(net, 0), sy.batch_labels(net, 0), net.lr)
+    g_avg = np.mean([o.grads(s) for s in range(net.n_workers)], axis=0)
+    err, where, _ = grad_rel_l2(out[0][0][0], g_avg, net.layers)
+    assert err <= 5e-2, (err, where)
