@@ -69,6 +69,8 @@ struct Op {
                                                              //      (this many per worker) for the batch-norm that follows
     tc::WgParams kw;
     std::vector<char*> a_ptrs, dy_ptrs;                      // the buffers the A / dY maps below were built for
+    std::vector<char*> y_ptrs, dx_ptrs;                      // where the forward output / the input gradient can be written
+    std::vector<tc::TensorMap> fo, dox;                      // output maps of the forward / input-gradient kernel, per buffer
     std::vector<tc::TensorMap> fa, fb, da, db, wx, wdy;      // fwd A, fwd B (per weight slot), dgrad A, dgrad B, wgrad X, wgrad dY
     std::vector<tc::TensorMap> fbh, dbh;                     // fwd / dgrad B with half-height boxes (CTA-pair kernels); empty: not used
 };
@@ -379,7 +381,9 @@ bool tc_forward(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* y_base, 
     const ConvGeom& g = o.g;
     double rows = (double)wn.n * g.Ho * g.Wo;
     Scope sc(KC_TC_FWD, 2.0 * rows * g.Co * g.R * g.R * g.C, 2.0 * ((double)wn.n * g.H * g.W * g.C + (double)g.Co * g.R * g.R * g.C + rows * g.Co), s);
-    const bool ok = tc::run_km(o.fa[ia], o.fb[version % m.D], o.fbh.empty() ? nullptr : &o.fbh[version % m.D], p, o.n_tile_f, s) == cudaSuccess;
+    const int io = find_buf(o.y_ptrs, y_base);
+    const bool ok = tc::run_km(o.fa[ia], o.fb[version % m.D], o.fbh.empty() ? nullptr : &o.fbh[version % m.D], io >= 0 ? &o.fo[io] : nullptr, p,
+                               o.n_tile_f, s) == cudaSuccess;
     if (ok && o.stat_chunks) { m.fused_stats_tensor = o.out; m.fused_stats_chunks = o.stat_chunks; }
     return ok;
 }
@@ -398,7 +402,9 @@ bool tc_dgrad(fdg_ctx* c, Module& m, const Op& o, char* dy_base, char* dx_base, 
     const double crows = (double)wn.n * p.Hd * p.Wd;         // pixels of one class; every tap belongs to exactly one class
     Scope sc(KC_TC_DGRAD, 2.0 * crows * g.C * p.ntaps * g.Co,
              2.0 * ((double)wn.n * g.Ho * g.Wo * g.Co + (double)g.Co * p.ntaps * g.C + crows * p.ncls * g.C * (accum ? 2 : 1)), s);
-    return tc::run_km(o.da[ia], o.db[version % m.D], o.dbh.empty() ? nullptr : &o.dbh[version % m.D], p, o.n_tile_d, s) == cudaSuccess;
+    const int io = find_buf(o.dx_ptrs, dx_base);
+    return tc::run_km(o.da[ia], o.db[version % m.D], o.dbh.empty() ? nullptr : &o.dbh[version % m.D], io >= 0 ? &o.dox[io] : nullptr, p, o.n_tile_d,
+                      s) == cudaSuccess;
 }
 bool tc_wgrad(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* dy_base, float* dw, const Win& wn, cudaStream_t s) {
     int ix = find_buf(o.a_ptrs, x_base), id = find_buf(o.dy_ptrs, dy_base);
@@ -562,6 +568,13 @@ bool build_tc_plans(fdg_ctx* c) {
             for (size_t i = 0; i < o.a_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.fa[i], o.a_ptrs[i], g.C, g.W, g.H, g.N, 64, wt, ht, nt, g.stride);
             o.fb.resize(m.D);
             for (int v = 0; v < m.D; ++v) ok = ok && tc::make_map_2d(&o.fb[v], wbig(c, m, v, o.w_off), Ktot, g.Co, 64, o.n_tile_f);
+            f.Nfull = g.N;
+            // the forward output: a stash slot, or a slot of the next module's input ring
+            if (to.loc == LOC_STASH) for (int i = 0; i < m.D; ++i) o.y_ptrs.push_back(m.stash + (size_t)i * m.stash_slot_bytes + to.off);
+            else if (to.loc == LOC_NEXT) { Module& n = c->mod[kk + 1]; for (int i = 0; i < n.in_depth; ++i) o.y_ptrs.push_back(n.in_ring + (size_t)i * n.in_slot_bytes); }
+            if (g.Co % 64 != 0) o.y_ptrs.clear();
+            o.fo.resize(o.y_ptrs.size());
+            for (size_t i = 0; i < o.y_ptrs.size(); ++i) ok = ok && tc::make_map_out(&o.fo[i], o.y_ptrs[i], g.Co, g.Wo, g.Ho, g.N, wt, ht);
             const bool pairs = c->kernel_path == 0;          // CTA-pair kernels for the 256-column tile (kernel_path 2: none)
             if (pairs && o.n_tile_f >= 256) {
                 o.fbh.resize(m.D);
@@ -590,6 +603,14 @@ bool build_tc_plans(fdg_ctx* c) {
             }
             o.da.resize(o.dy_ptrs.size());
             for (size_t i = 0; i < o.dy_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.da[i], o.dy_ptrs[i], g.Co, g.Wo, g.Ho, g.N, 64, wt, ht, nt, 1);
+            // the input gradient: the tensor's own gradient buffer, or a slot of the hand-off to the previous module;
+            // only a stride-1 layer writes it densely (tile geometry of dy = tile geometry of dx)
+            if (g.stride == 1 && g.C % 64 == 0) {
+                if (ti.own_grad) o.dx_ptrs.push_back(m.gradpool + ti.goff);
+                else if (o.in == 0 && kk > 0) for (int i = 0; i < 2; ++i) o.dx_ptrs.push_back(m.d2 + (size_t)i * m.in_slot_bytes);
+            }
+            o.dox.resize(o.dx_ptrs.size());
+            for (size_t i = 0; i < o.dx_ptrs.size(); ++i) ok = ok && tc::make_map_out(&o.dox[i], o.dx_ptrs[i], g.C, g.W, g.H, g.N, wt, ht);
             o.db.resize(m.D);
             for (int v = 0; v < m.D; ++v) ok = ok && tc::make_map_2d(&o.db[v], wtslot(m, v, o.w_off), (long)taps * g.Co, g.C, 64, o.n_tile_d);
             if (pairs && o.n_tile_d >= 256) {

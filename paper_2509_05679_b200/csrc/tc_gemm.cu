@@ -1,9 +1,9 @@
 // Tensor-core kernels for sm_100a: implicit-GEMM convolution / linear layers on tcgen05.mma with
 // accumulators in tensor memory, operands staged in shared memory by TMA (cp.async.bulk.tensor,
 // 128-byte swizzle), a 3-4 stage mbarrier pipeline, and warp-specialised roles:
-//   warp 0 : TMA producer (one elected thread)
-//   warp 1 : tensor-memory allocation, MMA issue (one elected thread), deallocation
-//   warps 2-5 : epilogue (tcgen05.ld -> registers -> global)
+//   warp 0 : TMA producer (the whole warp runs the loop, one elected lane issues the copies)
+//   warp 1 : tensor-memory allocation, MMA issue (same scheme), deallocation
+//   warps 2-5 (or 2-9) : epilogue (tcgen05.ld -> registers -> bf16 tile in shared memory -> TMA store)
 //
 // Two kernels:
 //   km_kernel  (forward and input-gradient): D[pixel][c_out] = sum_{tap, c} A[pixel + tap][c] * B[c_out][tap, c]
@@ -151,6 +151,22 @@ __device__ __forceinline__ void umma_commit_a(uint32_t bar) {
         asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// One lane of a converged warp.  The producer and MMA loops are executed by all 32 lanes, so that loop state stays
+// warp-uniform, and only the asynchronous instructions themselves sit behind this predicate.
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P1;\n\t.reg .b32 dummy;\n\telect.sync dummy|P1, 0xffffffff;\n\tselp.u32 %0, 1, 0, P1;\n\t}" : "=r"(pred));
+    return pred;
+}
+// shared -> global tile store (bulk async group of the issuing thread)
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* tm, uint32_t src, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                 ::"l"(tm), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 // ---- CTA pairs (cluster of two, tcgen05 cta_group::2): one MMA of 256 rows, each CTA holds its 128 rows of A and of
 // the accumulator and half of B's rows, so every SM reads only half of B from its shared memory.
 __device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
@@ -204,6 +220,19 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// the same without the wait: two of these fetch 64 columns, then tmem_ld_wait()
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t* v) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                   "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                   "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 // Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
 //   K-major operand  [rows][64 bf16]: 8-row groups are `sbo` bytes apart (1024); lbo unused.
 //   MN-major operand [k rows][64 bf16 of the M/N axis]: groups of 8 k-rows are `sbo` bytes apart (1024),
@@ -235,28 +264,35 @@ __device__ __forceinline__ uint8_t* align1024(uint8_t* p) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-constexpr int EPI_ROW_WORDS = 36;                 // 32 fp32 + 4 padding: conflict-free 128-bit rows
+constexpr int EPI_SLICE = 64;                     // accumulator columns an epilogue warp handles at a time
+constexpr int EPI_BUF_BYTES = 32 * EPI_SLICE * 2; // one staged slice: 32 rows x 64 bf16 = 32 rows of 128 bytes (128-byte swizzle)
 
-// EPI_WARPS = 4 or 8: with 8, two warps share each quarter of the tensor-memory lanes and take alternate 32-column slices.
+// EPI_WARPS = 4 or 8: with 8, two warps share each quarter of the tensor-memory lanes and take alternate 64-column slices.
 // PAIR: launched as clusters of two CTAs.  A pair computes two neighbouring pixel tiles against the same column tile
 // with one 256-row MMA per step, issued by the pair's first CTA; each CTA loads its own pixel tile and half of the
 // weight rows, drains its own half of the accumulator, and the tmem_empty / full barriers of the first CTA collect
 // both CTAs' arrivals.  The number of pixel tiles must be even.
-// KSUB: 64-wide K sub-blocks per pipeline stage.  One full / empty barrier round trip costs the issuing threads
-// several hundred cycles whatever the stage holds, so narrow tiles (little MMA work per sub-block) put more sub-blocks
-// behind each barrier; a tile's last stage may hold fewer.
-template <int N_TILE, int STAGES, int EPI_WARPS, bool PAIR, int KSUB>
-__global__ void __launch_bounds__(64 + 32 * EPI_WARPS, 1)
-km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, KmParams p) {
+// KSUB: 64-wide K sub-blocks per pipeline stage; a tile's last stage may hold fewer.
+// MIN_CTAS: CTAs per SM the register allocation must allow.
+//
+// Epilogue.  A warp owns 32 rows (pixels) of the tile.  Per 64-column slice it reads the accumulator, applies
+// bias / ReLU / accumulation into the old gradient, rounds to bf16 and writes the 32 x 64 block into a swizzled
+// staging buffer (two per warp).  If the launch has an output tensor map (p.tma_out) one elected lane hands the
+// block to a TMA store, whose box is exactly the warp's 32 pixels x 64 channels; otherwise the warp copies the
+// block out row by row (strided outputs of a stride-2 input gradient, partial tiles).  When a batch-norm follows, the
+// per-channel sum and sum of squares over the warp's rows are taken from the staged (rounded) values.
+template <int N_TILE, int STAGES, int EPI_WARPS, bool PAIR, int KSUB, int MIN_CTAS>
+__global__ void __launch_bounds__(64 + 32 * EPI_WARPS, MIN_CTAS)
+km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmO, KmParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
     constexpr int B_ROWS = PAIR ? N_TILE / 2 : N_TILE;
     constexpr int A_BYTES = BLOCK_M * BLOCK_K * 2, B_BYTES = B_ROWS * BLOCK_K * 2, SUB_BYTES = A_BYTES + B_BYTES;
     constexpr int STAGE_BYTES = KSUB * SUB_BYTES;
-    constexpr int EPI_BYTES = EPI_WARPS * 32 * EPI_ROW_WORDS * 4;
-    constexpr int COL_STEP = 32 * (EPI_WARPS / 4);
+    constexpr int EPI_BYTES = EPI_WARPS * 2 * EPI_BUF_BYTES;
+    constexpr int COL_STEP = EPI_SLICE * (EPI_WARPS / 4);
     constexpr uint32_t TMEM_COLS = 2 * N_TILE;
-    float* epi_smem = (float*)(smem + STAGES * STAGE_BYTES);
+    uint8_t* epi_smem = smem + STAGES * STAGE_BYTES;
     uint64_t* full = (uint64_t*)(smem + STAGES * STAGE_BYTES + EPI_BYTES);
     uint64_t* empty = full + STAGES;
     uint64_t* tmem_full = empty + STAGES;        // [2]
@@ -273,6 +309,7 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
 
     if (threadIdx.x == 0) {
         tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB);
+        if (p.tma_out) tma_prefetch_desc(&tmO);
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], PAIR ? 2 * EPI_WARPS : EPI_WARPS); }
         fence_barrier_init();
@@ -285,34 +322,35 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        if (lane == 0) {
-            bool ok = true;
-            const uint32_t smem0 = smem_u32(smem), full_l0 = smem_u32(full), empty0 = smem_u32(empty);
-            const uint32_t full_s0 = PAIR ? map_to_cta(full_l0, 0) : full_l0;      // where loads signal: the pair's first CTA
-            // stage cursor: destination, barriers, and the parity this thread waits for on `empty` (a fresh barrier
-            // passes a wait for parity 1, so the first round finds every stage free)
-            uint32_t st = 0, ph = 1, dst = smem0, fb = full_s0, fl = full_l0, eb = empty0;
-            for (int tile = walker; tile < total && ok; tile += walkers) {
-                const int cls = tile / per_cls, tl = tile - cls * per_cls;
-                int tm = tl / tiles_c; const int co0 = (tl - tm * tiles_c) * N_TILE;
-                if (PAIR) tm = 2 * tm + (int)rank;
-                const int tw = tm % p.tiles_w; tm /= p.tiles_w;
-                const int th = tm % p.tiles_h; const int tn = tm / p.tiles_h;
-                const int w0 = tw * p.Wt * p.xs, h0 = th * p.Ht * p.xs, n0 = p.n_base + tn * p.Nt;
-                const int brow = co0 + (PAIR ? (int)rank * B_ROWS : 0);
-                const int tap_end = p.cls_tap0[cls + 1];
-                int left = (tap_end - p.cls_tap0[cls]) * p.kchunks;      // sub-blocks of this tile still to load
-                int sub = 0;                                               // sub-block slot inside the current stage
-                for (int tap = p.cls_tap0[cls]; tap < tap_end && ok; ++tap) {
-                    const int cw = w0 + p.dw[tap], chh = h0 + p.dh[tap], kcol = p.koff[tap];
-                    for (int kc = 0; kc < p.kchunks; ++kc) {
+        // ---- producer (all lanes walk the loop; one elected lane issues)
+        bool ok = true;
+        const uint32_t smem0 = smem_u32(smem), full_l0 = smem_u32(full), empty0 = smem_u32(empty);
+        const uint32_t full_s0 = PAIR ? map_to_cta(full_l0, 0) : full_l0;      // where loads signal: the pair's first CTA
+        // stage cursor: destination, barriers, and the parity waited for on `empty` (a fresh barrier
+        // passes a wait for parity 1, so the first round finds every stage free)
+        uint32_t st = 0, ph = 1, dst = smem0, fb = full_s0, fl = full_l0, eb = empty0;
+        for (int tile = walker; tile < total && ok; tile += walkers) {
+            const int cls = tile / per_cls, tl = tile - cls * per_cls;
+            int tm = tl / tiles_c; const int co0 = (tl - tm * tiles_c) * N_TILE;
+            if (PAIR) tm = 2 * tm + (int)rank;
+            const int tw = tm % p.tiles_w; tm /= p.tiles_w;
+            const int th = tm % p.tiles_h; const int tn = tm / p.tiles_h;
+            const int w0 = tw * p.Wt * p.xs, h0 = th * p.Ht * p.xs, n0 = p.n_base + tn * p.Nt;
+            const int brow = co0 + (PAIR ? (int)rank * B_ROWS : 0);
+            const int tap_end = p.cls_tap0[cls + 1];
+            int left = (tap_end - p.cls_tap0[cls]) * p.kchunks;      // sub-blocks of this tile still to load
+            int sub = 0;                                               // sub-block slot inside the current stage
+            for (int tap = p.cls_tap0[cls]; tap < tap_end && ok; ++tap) {
+                const int cw = w0 + p.dw[tap], chh = h0 + p.dh[tap], kcol = p.koff[tap];
+                for (int kc = 0; kc < p.kchunks; ++kc) {
+                    if (sub == 0 && !mbar_wait_a(eb, ph, p.err, 1)) { ok = false; break; }
+                    const uint32_t da = dst + sub * SUB_BYTES;
+                    if (elect_one()) {
                         if (sub == 0) {
-                            if (!mbar_wait_a(eb, ph, p.err, 1)) { ok = false; break; }
                             // the stage's loads (both CTAs' for a pair) complete on one barrier that expects all their bytes
                             const int cnt = left < KSUB ? left : KSUB;
                             if (!PAIR || rank == 0) mbar_expect_tx_a(fl, (PAIR ? 2 : 1) * cnt * SUB_BYTES);
                         }
-                        const uint32_t da = dst + sub * SUB_BYTES;
                         if (PAIR) {
                             tma_load_4d_pair(da, &tmA, fb, kc * BLOCK_K, cw, chh, n0);
                             tma_load_2d_pair(da + A_BYTES, &tmB, fb, kcol + kc * BLOCK_K, brow);
@@ -320,18 +358,21 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                             tma_load_4d_a(da, &tmA, fb, kc * BLOCK_K, cw, chh, n0);
                             tma_load_2d_a(da + A_BYTES, &tmB, fb, kcol + kc * BLOCK_K, brow);
                         }
-                        --left;
-                        if (++sub == KSUB || left == 0) {
-                            sub = 0;
-                            if (++st == STAGES) { st = 0; ph ^= 1u; dst = smem0; fb = full_s0; fl = full_l0; eb = empty0; }
-                            else { dst += STAGE_BYTES; fb += 8; fl += 8; eb += 8; }
-                        }
+                    }
+                    __syncwarp();
+                    --left;
+                    if (++sub == KSUB || left == 0) {
+                        sub = 0;
+                        if (++st == STAGES) { st = 0; ph ^= 1u; dst = smem0; fb = full_s0; fl = full_l0; eb = empty0; }
+                        else { dst += STAGE_BYTES; fb += 8; fl += 8; eb += 8; }
                     }
                 }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0 && rank == 0) {
+        // ---- MMA issue (first CTA of a pair only; the elected lane is the same one every time, so the commits
+        // track the MMAs it issued)
+        if (rank == 0) {
             const uint32_t idesc = make_idesc(PAIR ? 2 * BLOCK_M : BLOCK_M, N_TILE, 0, 0);
             const uint64_t dconst = make_desc(0, 16, 1024);                     // address field left empty
             const uint32_t d_hi = (uint32_t)(dconst >> 32), d_lo = (uint32_t)dconst;
@@ -349,32 +390,43 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 uint32_t acc = 0;
                 for (int left = num_kb; left > 0; left -= KSUB) {
                     if (!mbar_wait_a(fb, ph, p.err, 2)) { ok = false; break; }
+                    tc_fence_after();
                     const uint32_t a_lo = d_lo + a16, b_lo = a_lo + (A_BYTES >> 4);
+                    if (elect_one()) {
 #pragma unroll
-                    for (int j = 0; j < KSUB; ++j) {
-                        if (j < left) {
+                        for (int j = 0; j < KSUB; ++j) {
+                            if (j < left) {
 #pragma unroll
-                            for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {        // 16 columns of K = 32 bytes = 2 address units
-                                umma_bf16_w<PAIR>(d, a_lo + j * (SUB_BYTES >> 4) + 2 * k, b_lo + j * (SUB_BYTES >> 4) + 2 * k, d_hi, idesc, acc);
-                                acc = 1;
+                                for (int k = 0; k < BLOCK_K / UMMA_K; ++k)        // 16 columns of K = 32 bytes = 2 address units
+                                    umma_bf16_w<PAIR>(d, a_lo + j * (SUB_BYTES >> 4) + 2 * k, b_lo + j * (SUB_BYTES >> 4) + 2 * k, d_hi, idesc,
+                                                      (j == 0 && k == 0) ? acc : 1u);
                             }
                         }
+                        umma_commit_a<PAIR>(eb);
+                        // the tile's last stage: arrives once every MMA of this tile has finished (in both CTAs of a pair)
+                        if (left <= KSUB) umma_commit_a<PAIR>(smem_u32(&tmem_full[buf]));
                     }
-                    umma_commit_a<PAIR>(eb);
+                    __syncwarp();
+                    acc = 1;
                     if (++st == STAGES) { st = 0; ph ^= 1u; a16 = a16_0; fb = full0; eb = empty0; }
                     else { a16 += STAGE_BYTES >> 4; fb += 8; eb += 8; }
                 }
-                // arrives once every MMA of this tile has finished (in both CTAs of a pair)
-                umma_commit_a<PAIR>(smem_u32(&tmem_full[buf]));
             }
         }
     } else {
         // ---- epilogue: warp q = warp % 4 owns tensor-memory lanes 32q .. 32q+31 (= tile rows)
         const int q = warp & 3, half = (warp - 2) >> 2;
-        float* stage = epi_smem + (warp - 2) * 32 * EPI_ROW_WORDS;
+        const uint32_t stg0 = smem_u32(epi_smem + (warp - 2) * 2 * EPI_BUF_BYTES);
+        uint32_t sbuf = 0;
         int ti = 0;
         bool ok = true;
+        const bool tma_out = p.tma_out != 0;
         const uint32_t tmem_empty0 = PAIR ? map_to_cta(smem_u32(&tmem_empty[0]), 0) : 0u;
+        // this lane's row of the tile, and the first row of the warp, as (pixel column, pixel row, sample) inside the tile
+        const int row = q * 32 + lane;
+        const int pw = row % p.Wt, ph = (row / p.Wt) % p.Ht, pn = row / (p.Wt * p.Ht);
+        const int bw0 = (q * 32) % p.Wt, bh0 = ((q * 32) / p.Wt) % p.Ht, bn0 = (q * 32) / (p.Wt * p.Ht);
+        const uint32_t swz = (uint32_t)(lane & 7);
         for (int tile = walker; tile < total && ok; tile += walkers, ++ti) {
             const int buf = ti & 1, use = ti >> 1;
             const int cls = tile / per_cls, tl = tile - cls * per_cls;
@@ -384,8 +436,6 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             const int tw = tm % p.tiles_w; tm /= p.tiles_w;
             const int th = tm % p.tiles_h; const int tn = tm / p.tiles_h;
             // this lane's row of the tile -> output address (0 = row outside the tensor)
-            const int row = q * 32 + lane;
-            const int pw = row % p.Wt, ph = (row / p.Wt) % p.Ht, pn = row / (p.Wt * p.Ht);
             const int n = p.n_base + tn * p.Nt + pn, h = th * p.Ht + ph, w = tw * p.Wt + pw;
             const bool valid = n < p.N && h < p.Hd && w < p.Wd;
             const unsigned long long rowptr = valid ? (unsigned long long)((bf16*)p.out + (((size_t)n * p.Ho + (h * p.os + p.cls_oph[cls])) * p.Wo +
@@ -394,59 +444,102 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             ok = mbar_wait_sleep(&tmem_full[buf], use & 1, p.err, 3);
             tc_fence_after();
 #pragma unroll 1
-            for (int c = half * 32; c < N_TILE; c += COL_STEP) {
-                uint32_t v[32];
-                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * N_TILE + c, v);
+            for (int c = half * EPI_SLICE; c < N_TILE; c += COL_STEP) {
+                uint32_t v[EPI_SLICE];
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * N_TILE + c;
+                tmem_ld32_nowait(taddr, v);
+                tmem_ld32_nowait(taddr + 32, v + 32);
+                tmem_ld_wait();
                 if (c + COL_STEP >= N_TILE) {      // this warp's last read of the accumulator: hand the buffer back to the MMA warp
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) { if (PAIR) mbar_arrive_cluster(tmem_empty0 + 8 * buf); else mbar_arrive(&tmem_empty[buf]); }
                 }
-                // bias / ReLU on this lane's row, then into the staging rows
+                if (p.bias) {
 #pragma unroll
-                for (int j = 0; j < 32; j += 4) {
-                    float4 f = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-                    if (p.bias) { const float4 bb = __ldg((const float4*)(p.bias + co0 + c + j)); f.x += bb.x; f.y += bb.y; f.z += bb.z; f.w += bb.w; }
-                    if (p.epi & EPI_RELU) { f.x = fmaxf(f.x, 0.f); f.y = fmaxf(f.y, 0.f); f.z = fmaxf(f.z, 0.f); f.w = fmaxf(f.w, 0.f); }
-                    *(float4*)(stage + lane * EPI_ROW_WORDS + j) = f;
+                    for (int j = 0; j < EPI_SLICE; j += 4) {
+                        const float4 bb = __ldg((const float4*)(p.bias + co0 + c + j));
+                        v[j] = __float_as_uint(__uint_as_float(v[j]) + bb.x); v[j + 1] = __float_as_uint(__uint_as_float(v[j + 1]) + bb.y);
+                        v[j + 2] = __float_as_uint(__uint_as_float(v[j + 2]) + bb.z); v[j + 3] = __float_as_uint(__uint_as_float(v[j + 3]) + bb.w);
+                    }
                 }
+                if (p.epi & EPI_RELU) {
+#pragma unroll
+                    for (int j = 0; j < EPI_SLICE; ++j) v[j] = __float_as_uint(fmaxf(__uint_as_float(v[j]), 0.f));
+                }
+                if ((p.epi & EPI_ACCUM) && rowptr) {
+                    // add the gradient already stored for this row (rounded once, after the addition)
+                    const uint4* o = (const uint4*)((const bf16*)rowptr + c);
+#pragma unroll
+                    for (int g = 0; g < EPI_SLICE / 8; ++g) {
+                        const uint4 old = o[g];
+                        const uint32_t w4[4] = {old.x, old.y, old.z, old.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            v[8 * g + 2 * j] = __float_as_uint(__uint_as_float(v[8 * g + 2 * j]) + __uint_as_float(w4[j] << 16));
+                            v[8 * g + 2 * j + 1] = __float_as_uint(__uint_as_float(v[8 * g + 2 * j + 1]) + __uint_as_float(w4[j] & 0xffff0000u));
+                        }
+                    }
+                }
+                // the staging buffer used two slices ago must have been read by its TMA store (the elected lane issued it)
+                const uint32_t stg = stg0 + sbuf * EPI_BUF_BYTES;
+                if (tma_out) { if (elect_one()) bulk_wait_read<1>(); }
                 __syncwarp();
+                // row `lane`, 16-byte chunk g goes to chunk position g ^ (lane % 8): the 128-byte swizzle of the store's tensor map
+#pragma unroll
+                for (int g = 0; g < EPI_SLICE / 8; ++g) {
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const __nv_bfloat162 t = __floats2bfloat162_rn(__uint_as_float(v[8 * g + 2 * j]), __uint_as_float(v[8 * g + 2 * j + 1]));
+                        pk[j] = *(const uint32_t*)&t;
+                    }
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + (((uint32_t)g ^ swz) << 4)),
+                                 "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
+                }
+                if (tma_out) {
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (elect_one()) {
+                        tma_store_4d(&tmO, stg, co0 + c, tw * p.Wt + bw0, th * p.Ht + bh0, p.n_base + tn * p.Nt + bn0);
+                        bulk_commit();
+                    }
+                } else {
+                    __syncwarp();
+                    // 8 lanes cover one row's 128 bytes, 4 rows per pass
+#pragma unroll
+                    for (int pass = 0; pass < 8; ++pass) {
+                        const int r = pass * 4 + (lane >> 3);
+                        const uint32_t g = (uint32_t)(lane & 7);
+                        const unsigned long long rp = __shfl_sync(0xffffffffu, rowptr, r);
+                        uint4 t;
+                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(t.x), "=r"(t.y), "=r"(t.z), "=r"(t.w)
+                                     : "r"(stg + r * 128 + ((g ^ (uint32_t)(r & 7)) << 4)) : "memory");
+                        if (rp && ok) *(uint4*)((bf16*)rp + c + g * 8) = t;
+                    }
+                }
                 if (p.stat_part) {
-                    // batch-norm statistics of the layer's output, fused: lane j adds column j over this warp's rows
-                    float s1 = 0.f, s2 = 0.f;
+                    // batch-norm statistics of the layer's output, fused: this lane sums columns 2*lane and 2*lane+1 of the
+                    // slice over the warp's valid rows, from the values as stored
+                    float s1a = 0.f, s2a = 0.f, s1b = 0.f, s2b = 0.f;
+                    const uint32_t cbase = stg + (uint32_t)(lane & 3) * 4, cg = (uint32_t)(lane >> 2);
 #pragma unroll 8
                     for (int r = 0; r < 32; ++r) {
-                        const float vr = __bfloat162float(__float2bfloat16_rn(stage[r * EPI_ROW_WORDS + lane]));
-                        if ((vmask >> r) & 1u) { s1 += vr; s2 = fmaf(vr, vr, s2); }
-                    }
-                    *(float2*)(p.stat_part + (((size_t)tmi * 4 + q) * p.Cn + co0 + c + lane) * 2) = make_float2(s1, s2);
-                }
-                // transposed read-out: 4 lanes cover one row's 32 columns (64 bytes of bf16), 8 rows per pass
-#pragma unroll
-                for (int pass = 0; pass < 4; ++pass) {
-                    const int r = pass * 8 + (lane >> 2), piece = lane & 3;
-                    const unsigned long long rp = __shfl_sync(0xffffffffu, rowptr, r);
-                    const float4 f0 = *(const float4*)(stage + r * EPI_ROW_WORDS + piece * 8);
-                    const float4 f1 = *(const float4*)(stage + r * EPI_ROW_WORDS + piece * 8 + 4);
-                    if (rp && ok) {
-                        float f[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
-                        uint4* o = (uint4*)((bf16*)rp + c + piece * 8);
-                        if (p.epi & EPI_ACCUM) {
-                            const uint4 old = *o;
-                            const __nv_bfloat162* ob = (const __nv_bfloat162*)&old;
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) { const float2 t = __bfloat1622float2(ob[j]); f[2 * j] += t.x; f[2 * j + 1] += t.y; }
+                        uint32_t t;
+                        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(t) : "r"(cbase + r * 128 + ((cg ^ (uint32_t)(r & 7)) << 4)) : "memory");
+                        if ((vmask >> r) & 1u) {
+                            const float x0 = __uint_as_float(t << 16), x1 = __uint_as_float(t & 0xffff0000u);
+                            s1a += x0; s2a = fmaf(x0, x0, s2a); s1b += x1; s2b = fmaf(x1, x1, s2b);
                         }
-                        uint4 pk;
-                        __nv_bfloat162 t0 = __floats2bfloat162_rn(f[0], f[1]), t1 = __floats2bfloat162_rn(f[2], f[3]);
-                        __nv_bfloat162 t2 = __floats2bfloat162_rn(f[4], f[5]), t3 = __floats2bfloat162_rn(f[6], f[7]);
-                        pk.x = *(uint32_t*)&t0; pk.y = *(uint32_t*)&t1; pk.z = *(uint32_t*)&t2; pk.w = *(uint32_t*)&t3;
-                        *o = pk;
                     }
+                    *(float4*)(p.stat_part + (((size_t)tmi * 4 + q) * p.Cn + co0 + c + 2 * lane) * 2) = make_float4(s1a, s2a, s1b, s2b);
                 }
-                __syncwarp();
+                sbuf ^= 1u;
             }
         }
+        // the staging buffers must outlive the stores that read them
+        if (tma_out) { if (elect_one()) bulk_wait_all(); }
+        __syncwarp();
     }
     tc_fence_before();
     __syncwarp();
@@ -629,6 +722,12 @@ bool make_map_4d(TensorMap* out, const void* base, int C, int W, int H, int N, i
     return r == CUDA_SUCCESS;
 }
 
+bool make_map_out(TensorMap* out, const void* base, int C, int W, int H, int N, int Wt, int Ht) {
+    // the 32 pixels an epilogue warp owns inside a 128-pixel tile of Wt x Ht x Nt pixels
+    const int bw = Wt < 32 ? Wt : 32, bh = Ht < 32 / bw ? Ht : 32 / bw, bn = 32 / (bw * bh);
+    return make_map_4d(out, base, C, W, H, N, EPI_SLICE, bw, bh, bn, 1);
+}
+
 bool make_map_2d(TensorMap* out, const void* base, long inner, long outer, int box_inner, int box_outer) {
     if (!init()) return false;
     cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
@@ -657,10 +756,14 @@ static int sm_count() {
 }
 
 template <int N_TILE, int STAGES, int EPI_WARPS, int KSUB>
-static cudaError_t launch_km(const TensorMap& a, const TensorMap& b, const KmParams& p, cudaStream_t s) {
-    constexpr int smem = STAGES * KSUB * (BLOCK_M * BLOCK_K * 2 + N_TILE * BLOCK_K * 2) + EPI_WARPS * 32 * EPI_ROW_WORDS * 4 + 1024 + 256;
+static cudaError_t launch_km(const TensorMap& a, const TensorMap& b, const TensorMap& o, const KmParams& p, cudaStream_t s) {
+    constexpr int smem = STAGES * KSUB * (BLOCK_M * BLOCK_K * 2 + N_TILE * BLOCK_K * 2) + EPI_WARPS * 2 * EPI_BUF_BYTES + 1024 + 256;
     static_assert(smem <= 232448, "shared memory");
-    auto kernel = km_kernel<N_TILE, STAGES, EPI_WARPS, false, KSUB>;
+    // CTAs of this variant that fit on an SM: shared memory (227 KB, 1 KB reserved per CTA) and 512 tensor-memory columns
+    constexpr int by_smem = (227 * 1024) / (smem + 1024), by_tmem = 512 / (2 * N_TILE);
+    constexpr int per_sm = by_smem < by_tmem ? by_smem : by_tmem;
+    static_assert(per_sm >= 1 && per_sm <= 2, "CTAs per SM");
+    auto kernel = km_kernel<N_TILE, STAGES, EPI_WARPS, false, KSUB, per_sm>;
     static bool attr = false;
     if (!attr) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -668,21 +771,18 @@ static cudaError_t launch_km(const TensorMap& a, const TensorMap& b, const KmPar
         attr = true;
     }
     const int total = p.tiles_w * p.tiles_h * p.tiles_n * (p.Cn / N_TILE) * p.ncls;
-    // CTAs of this variant that fit on an SM: shared memory (227 KB, 1 KB reserved per CTA) and 512 tensor-memory columns
-    constexpr int by_smem = (227 * 1024) / (smem + 1024), by_tmem = 512 / (2 * N_TILE);
-    constexpr int per_sm = by_smem < by_tmem ? by_smem : by_tmem;
     const int slots = sm_count() * per_sm;
     const int grid = total < slots ? total : slots;
-    kernel<<<grid, 64 + 32 * EPI_WARPS, smem, s>>>(*(const CUtensorMap*)&a, *(const CUtensorMap*)&b, p);
+    kernel<<<grid, 64 + 32 * EPI_WARPS, smem, s>>>(*(const CUtensorMap*)&a, *(const CUtensorMap*)&b, *(const CUtensorMap*)&o, p);
     return cudaGetLastError();
 }
 
 // CTA pairs: `b` is a tensor map whose box holds N_TILE / 2 weight rows.
 template <int N_TILE, int STAGES, int EPI_WARPS, int KSUB>
-static cudaError_t launch_km_pair(const TensorMap& a, const TensorMap& b, const KmParams& p, cudaStream_t s) {
-    constexpr int smem = STAGES * KSUB * (BLOCK_M * BLOCK_K * 2 + (N_TILE / 2) * BLOCK_K * 2) + EPI_WARPS * 32 * EPI_ROW_WORDS * 4 + 1024 + 256;
+static cudaError_t launch_km_pair(const TensorMap& a, const TensorMap& b, const TensorMap& o, const KmParams& p, cudaStream_t s) {
+    constexpr int smem = STAGES * KSUB * (BLOCK_M * BLOCK_K * 2 + (N_TILE / 2) * BLOCK_K * 2) + EPI_WARPS * 2 * EPI_BUF_BYTES + 1024 + 256;
     static_assert(smem <= 232448, "shared memory");
-    auto kernel = km_kernel<N_TILE, STAGES, EPI_WARPS, true, KSUB>;
+    auto kernel = km_kernel<N_TILE, STAGES, EPI_WARPS, true, KSUB, 1>;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
@@ -699,17 +799,21 @@ static cudaError_t launch_km_pair(const TensorMap& a, const TensorMap& b, const 
     }
     const int total = (p.tiles_w * p.tiles_h * p.tiles_n / 2) * (p.Cn / N_TILE) * p.ncls;
     cfg.gridDim = dim3(2 * (total < max_pairs ? total : max_pairs));
-    return cudaLaunchKernelEx(&cfg, kernel, *(const CUtensorMap*)&a, *(const CUtensorMap*)&b, p);
+    return cudaLaunchKernelEx(&cfg, kernel, *(const CUtensorMap*)&a, *(const CUtensorMap*)&b, *(const CUtensorMap*)&o, p);
 }
 
-cudaError_t run_km(const TensorMap& a, const TensorMap& b, const TensorMap* b_half, const KmParams& p, int n_tile, cudaStream_t s) {
+cudaError_t run_km(const TensorMap& a, const TensorMap& b, const TensorMap* b_half, const TensorMap* out_map, const KmParams& p_in, int n_tile,
+                   cudaStream_t s) {
+    KmParams p = p_in;
+    // the store through the output map covers whole 32-pixel boxes and clips only at the tensor's edge: it needs a dense
+    // output (stride 1) and a sample range that ends where the tiles end or where the tensor ends
+    p.tma_out = out_map && p.os == 1 && p.ncls == 1 && (p.n_base + p.tiles_n * p.Nt <= p.N || p.N == p.Nfull) ? 1 : 0;
+    const TensorMap& o = p.tma_out ? *out_map : a;       // unused by the kernel without tma_out
     const bool pair = b_half && n_tile == 256 && (p.tiles_w * p.tiles_h * p.tiles_n) % 2 == 0;
-    // measured on a B200: the narrow tiles run best with two CTAs per SM and short pipelines (3 x 24 KB, 2 x 32 KB stages);
-    // the 256-column tile as a CTA pair with six 32 KB stages; more sub-blocks per stage changed nothing
-    if (pair && n_tile == 256) return launch_km_pair<256, 6, 4, 1>(a, *b_half, p, s);
-    if (n_tile == 64) return launch_km<64, 3, 4, 1>(a, b, p, s);
-    if (n_tile == 128) return launch_km<128, 2, 4, 1>(a, b, p, s);
-    if (n_tile == 256) return launch_km<256, 4, 4, 1>(a, b, p, s);
+    if (pair) return launch_km_pair<256, 6, 4, 1>(a, *b_half, o, p, s);
+    if (n_tile == 64) return launch_km<64, 3, 4, 1>(a, b, o, p, s);
+    if (n_tile == 128) return launch_km<128, 2, 4, 1>(a, b, o, p, s);
+    if (n_tile == 256) return launch_km<256, 4, 4, 1>(a, b, o, p, s);
     return cudaErrorInvalidValue;
 }
 

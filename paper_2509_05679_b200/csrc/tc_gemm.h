@@ -20,6 +20,8 @@ struct KmParams {
     int cls_tap0[5];                             // class c uses taps [cls_tap0[c], cls_tap0[c+1])
     int cls_oph[4], cls_opw[4];                  // class c writes domain pixel (h, w) to (h*os + cls_oph[c], w*os + cls_opw[c])
     int N, Hd, Wd;                               // extents of the tile domain (rows outside are not stored)
+    int Nfull;                                   // samples in the whole output tensor (N is the end of this launch's group)
+    int tma_out;                                 // set by run_km: the epilogue stores through the output tensor map
     int n_base;                                  // first sample of the group of workers this launch covers (a multiple of Nt);
                                                  // tiles_n counts the group's tiles, N is the end of the group
     int Ho, Wo, Co, os;                          // output tensor [N,Ho,Wo,Co] and the output stride of a domain pixel
@@ -50,9 +52,15 @@ bool make_map_2d(TensorMap* out, const void* base, long inner, long outer, int b
 // Wt x Ht x Nt = pixels, Wt = min(W, pixels) ...; false unless H and W are powers of two
 bool pixel_tile(int H, int W, int pixels, int* Wt, int* Ht, int* Nt);
 
+// Output map of run_km: the [N,H,W,C] output tensor with a box of 64 channels x the 32 pixels one epilogue warp owns
+// inside a 128-pixel tile of Wt x Ht x Nt pixels.  C must be a multiple of 64.
+bool make_map_out(TensorMap* out, const void* base, int C, int W, int H, int N, int Wt, int Ht);
+
 // b_half: nullptr, or a map of the same matrix whose box holds n_tile / 2 rows: the kernel then runs as CTA pairs
 // (two SMs share one 256-row MMA and each loads half of B) when n_tile is 256 and the number of pixel tiles is even.
-cudaError_t run_km(const TensorMap& a, const TensorMap& b, const TensorMap* b_half, const KmParams& p, int n_tile, cudaStream_t s);
+// out_map: nullptr, or the output tensor's map from make_map_out: dense outputs are then written by TMA stores.
+cudaError_t run_km(const TensorMap& a, const TensorMap& b, const TensorMap* b_half, const TensorMap* out_map, const KmParams& p, int n_tile,
+                   cudaStream_t s);
 // accum: dw += the result (second and later groups of workers)
 cudaError_t run_wg(const TensorMap& x, const TensorMap& dy, const WgParams& p, int n_tile, int splits, float* dw, bool accum, cudaStream_t s);
 cudaError_t run_flip_transpose(const void* w, void* wt, int Co, int taps, int Ci, cudaStream_t s);
