@@ -329,7 +329,8 @@ def main():
                             "gbs": round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1) if v["ms"] > 0 else None}
                         for k, v in sorted(kstats.items(), key=lambda kv: -kv[1]["ms"])},
             "kernel_shapes": {k: {"launches": v["launches"], "ms": round(v["ms"], 4),
-                                  "tflops": round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 1) if v["ms"] > 0 else None}
+                                  "tflops": round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 1) if v["ms"] > 0 else None,
+                                  "gbs": round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1) if v["ms"] > 0 else None}
                               for k, v in sorted(kshapes.items(), key=lambda kv: -kv[1]["ms"])},
             "module_ms_last_step": mod_ms,
             "gpu_launches": int(launches1 - launches0),

@@ -454,11 +454,15 @@ void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int grou
                 profile_detail(nullptr);
                 break; }
             case OP_BN: {
+                char tag[40];
+                std::snprintf(tag, sizeof tag, "%dx%dx%d%s%s", ti.h, ti.w, ti.c, o.has_res ? " +res" : "", o.relu ? " relu" : "");
+                profile_detail(tag);
                 const bool fused = m.fused_stats_tensor == o.in;
                 const float* part = fused ? m.cstat + (size_t)wn.w0 * m.fused_stats_chunks * ti.c * 2 : nullptr;
                 bn_forward(dt, T(o.in), wsmall(c, m, version, o.gamma_off), wsmall(c, m, version, o.beta_off),
                            o.has_res ? T(o.in2) : nullptr, T(o.out), P.stats(o) + (size_t)wn.w0 * ti.c * 2, m.scratch_f, wn.nw,
-                           (long)c->B * ti.h * ti.w, ti.c, o.relu, part, fused ? m.fused_stats_chunks : 0, s);
+                           (long)c->B * ti.h * ti.w, ti.c, o.relu, part, fused ? m.fused_stats_chunks : 0, c->tc_err, s);
+                profile_detail(nullptr);
                 m.fused_stats_tensor = -1;
                 break; }
             case OP_RELU: relu_forward(dt, T(o.in), T(o.out), n_out, s); break;
@@ -511,10 +515,14 @@ void backward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int64_t
                 profile_detail(nullptr);
                 break; }
             case OP_BN: {
+                char tag[40];
+                std::snprintf(tag, sizeof tag, "%dx%dx%d%s%s", ti.h, ti.w, ti.c, o.has_res ? " +res" : "", o.relu ? " relu" : "");
+                profile_detail(tag);
                 char* gres = o.has_res ? G(o.in2) : nullptr;
                 bn_backward(dt, T(o.in), T(o.out), gout, wsmall(c, m, version, o.gamma_off), wsmall(c, m, version, o.beta_off),
                             P.stats(o) + (size_t)wn.w0 * ti.c * 2, gin, o.acc_in, gres, o.acc_in2, m.grad + m.n_big + o.gamma_off,
-                            m.grad + m.n_big + o.beta_off, m.red, m.scratch, wn.nw, (long)c->B * ti.h * ti.w, ti.c, o.relu, o.has_res, acc_p, s);
+                            m.grad + m.n_big + o.beta_off, m.red, m.scratch, wn.nw, (long)c->B * ti.h * ti.w, ti.c, o.relu, o.has_res, acc_p, c->tc_err, s);
+                profile_detail(nullptr);
                 break; }
             case OP_RELU: if (gin) relu_backward(dt, T(o.out), gout, gin, n_out, o.acc_in, s); break;
             case OP_POOL: if (gin) maxpool_backward(dt, T(o.in), gout, gin, wn.n, ti.h, ti.w, ti.c, o.acc_in, s); break;
@@ -656,10 +664,10 @@ fdg_status reset_state(fdg_ctx* ctx) {
 
 // Reads the device error word (the caller has synchronised the stream it cares about).
 fdg_status check_device_error(fdg_ctx* ctx) {
-    if (!ctx->any_tc) return FDG_OK;
+    if (!ctx->any_tc && ctx->dt != 1) return FDG_OK;
     int e = 0;
     CK(cudaMemcpy(&e, ctx->tc_err, sizeof(int), cudaMemcpyDeviceToHost));
-    if (e) return fail(ctx, FDG_ERR_TIMEOUT, "a tensor-core kernel gave up waiting on an mbarrier (code %d)", e);
+    if (e) return fail(ctx, FDG_ERR_TIMEOUT, "a kernel gave up waiting on an mbarrier (code %d)", e);
     return FDG_OK;
 }
 

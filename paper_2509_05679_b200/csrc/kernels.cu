@@ -581,209 +581,192 @@ __global__ void bn_bwd_apply_k(const T* __restrict__ x, const T* __restrict__ ou
 }
 
 // ------------------------------------------------------------------------------------------
-// batch-norm, bf16 storage, 64-bit accesses: a thread owns 4 consecutive channels and walks down
-// the rows of one worker, four rows in flight; grid = (row chunks, workers).  Used when C/4 is a
-// power of two <= 256.
+// Batch-norm, bf16 storage, streamed: a CTA owns a contiguous range of one worker's rows, which is one
+// contiguous range of memory (NHWC).  One thread feeds a ring of shared-memory stages with bulk asynchronous
+// copies (cp.async.bulk, completion on an mbarrier), 8 KB per input tensor and stage, so that about 90 KB per
+// CTA are in flight whatever the registers hold; all 256 threads read 16-byte vectors (8 channels) from the
+// stage, and results go straight to global memory.  A thread keeps the same 8 channels for every row.
+// grid = (row chunks, workers).  Used when C/8 is a power of two <= 256.
 // ------------------------------------------------------------------------------------------
 constexpr int BNV_THREADS = 256;
 constexpr int BNV_MAX_CHUNKS = 128;
-constexpr int BV = 4;                               // channels per thread (one 64-bit access)
+constexpr int BV = 8;                               // channels per thread (one 128-bit access)
+constexpr int BNS_TILE = 8192;                      // bytes per input tensor and stage
+constexpr int BNS_RING = 12 * BNS_TILE;             // shared memory of the ring (stages = 12 / input tensors, at most 8)
+constexpr long long BNS_WAIT_CYCLES = 4000000000LL; // ~2 s
 
-__device__ __forceinline__ void unpack4(const uint2& v, float (&f)[BV]) {
-    const float2 a = __bfloat1622float2(*(const __nv_bfloat162*)&v.x), b = __bfloat1622float2(*(const __nv_bfloat162*)&v.y);
-    f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y;
+__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[BV]) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { f[2 * j] = __uint_as_float(w[j] << 16); f[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u); }
 }
-__device__ __forceinline__ uint2 pack4(const float (&f)[BV]) {
-    uint2 v;
-    __nv_bfloat162 a = __floats2bfloat162_rn(f[0], f[1]), b = __floats2bfloat162_rn(f[2], f[3]);
-    v.x = *(uint32_t*)&a; v.y = *(uint32_t*)&b;
-    return v;
+__device__ __forceinline__ uint4 pack8(const float (&f)[BV]) {
+    uint32_t w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { const __nv_bfloat162 t = __floats2bfloat162_rn(f[2 * j], f[2 * j + 1]); w[j] = *(const uint32_t*)&t; }
+    return make_uint4(w[0], w[1], w[2], w[3]);
 }
-__device__ __forceinline__ uint2 ldg8(const bf16* p) { return __ldg((const uint2*)p); }
 // the one expression both passes use for the normalised value, so that the backward pass can
 // recompute the sign of the forward output from x alone
 __device__ __forceinline__ float bn_value(float x, float mean, float istd, float g, float b) {
     return __fmaf_rn(g, (x - mean) * istd, b);
 }
 
+__device__ __forceinline__ uint32_t bns_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool bns_wait(uint32_t bar, uint32_t parity, int* err) {
+    uint32_t ok;
+    long long t0 = 0;
+    for (;;) {
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+        if (t0 == 0) t0 = clock64();
+        else if (clock64() - t0 > BNS_WAIT_CYCLES) { atomicCAS(err, 0, 20); return false; }
+    }
+}
+
+struct BnsArgs {
+    const bf16* in[3];          // input tensors streamed through the ring: x, then dout, then the forward output (as the mode needs)
+    int n_in;
+    const float* gamma; const float* beta; const float* stats; const float* red; const bf16* res;
+    float* part;                // modes 0, 1: partial sums [chunk][worker][C][2]
+    bf16* y;                    // mode 2: output; mode 3: dx
+    bf16* dres;                 // mode 3: gradient of the residual input, or nullptr
+    long rpw; int C; int relu; int mask_from_x; int accum_dx; int accum_dres;
+    int* err;
+};
+
 // MODE 0: (sum x, sum x^2).  MODE 1: (sum dy, sum dy * xhat) with dy = dout * [forward output > 0] if relu.
+// MODE 2: y = bn(x) (+ res) (relu).  MODE 3: dx (+)= BN backward of dy, dres (+)= dy.
 // mask_from_x: the forward output had no residual, so its sign is the sign of bn_value(x).
 template <int MODE>
-__global__ void __launch_bounds__(BNV_THREADS, 3) bnv_reduce(const bf16* __restrict__ x, const bf16* __restrict__ out,
-                                                             const bf16* __restrict__ dout, const float* __restrict__ gamma,
-                                                             const float* __restrict__ beta, const float* __restrict__ stats,
-                                                             float* __restrict__ part, long rpw, int C, int relu, int mask_from_x) {
-    __shared__ float sh[BNV_THREADS][2 * BV + 1];
-    const int cgs = C / BV, rows_it = BNV_THREADS / cgs;
-    const int cg = threadIdx.x % cgs, r = threadIdx.x / cgs;
+__global__ void __launch_bounds__(BNV_THREADS, 2) bns_kernel(const BnsArgs a) {
+    extern __shared__ __align__(128) uint8_t bns_sm[];
+    const int C = a.C, cgs = C / BV, rows_it = BNV_THREADS / cgs;
+    const int tid = threadIdx.x, cg = tid % cgs, rl = tid / cgs;
     const int w = blockIdx.y, nw = gridDim.y;
-    const long per = (rpw + gridDim.x - 1) / gridDim.x;
-    const long r0 = (long)blockIdx.x * per, r1 = min(rpw, r0 + per);
-    float s1[BV], s2[BV], mean[BV], istd[BV], g[BV], b[BV];
-#pragma unroll
-    for (int j = 0; j < BV; ++j) {
-        s1[j] = 0.f; s2[j] = 0.f;
-        if (MODE == 1) {
-            const int c = cg * BV + j;
-            mean[j] = stats[((size_t)w * C + c) * 2]; istd[j] = stats[((size_t)w * C + c) * 2 + 1];
-            g[j] = gamma[c]; b[j] = beta[c];
-        }
+    const int n_in = a.n_in, stages = 12 / n_in < 8 ? 12 / n_in : 8;
+    const int tile_rows = BNS_TILE / (C * 2);
+    long per = (a.rpw + gridDim.x - 1) / gridDim.x;
+    per = (per + tile_rows - 1) / tile_rows * tile_rows;
+    const long r0 = (long)blockIdx.x * per, r1 = min(a.rpw, r0 + per);
+    const int ntiles = r1 > r0 ? (int)((r1 - r0 + tile_rows - 1) / tile_rows) : 0;
+    uint64_t* full = (uint64_t*)(bns_sm + BNS_RING);
+    const uint32_t full0 = bns_smem(full), ring0 = bns_smem(bns_sm);
+    if (tid == 0) {
+        for (int s = 0; s < stages; ++s) asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full0 + 8 * s), "r"(1) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    const size_t base = (size_t)w * rpw * C + (size_t)cg * BV;
-    const bool need_out = MODE == 1 && relu && !mask_from_x;
-    constexpr int U = 4;
-    for (long row = r0 + r; row < r1; row += (long)rows_it * U) {
-        uint2 xr[U], dr[U], orr[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const long rr = row + (long)u * rows_it;
-            if (rr < r1) {
-                const size_t o = base + (size_t)rr * C;
-                xr[u] = ldg8(x + o);
-                if (MODE == 1) dr[u] = ldg8(dout + o);
-                if (need_out) orr[u] = ldg8(out + o);
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            if (row + (long)u * rows_it >= r1) break;
-            float xv[BV];
-            unpack4(xr[u], xv);
-            if (MODE == 0) {
-#pragma unroll
-                for (int j = 0; j < BV; ++j) { s1[j] += xv[j]; s2[j] = fmaf(xv[j], xv[j], s2[j]); }
-            } else {
-                float dv[BV], ov[BV];
-                unpack4(dr[u], dv);
-                if (need_out) unpack4(orr[u], ov);
-#pragma unroll
-                for (int j = 0; j < BV; ++j) {
-                    float dy = dv[j];
-                    if (relu) { float f = mask_from_x ? bn_value(xv[j], mean[j], istd[j], g[j], b[j]) : ov[j]; if (!(f > 0.f)) dy = 0.f; }
-                    s1[j] += dy; s2[j] = fmaf(dy, (xv[j] - mean[j]) * istd[j], s2[j]);
-                }
-            }
-        }
-    }
-#pragma unroll
-    for (int j = 0; j < BV; ++j) { sh[threadIdx.x][j] = s1[j]; sh[threadIdx.x][BV + j] = s2[j]; }
     __syncthreads();
-    // thread t < 2*BV*cgs sums one (channel group, value) column over the rows_it row lanes, in a fixed order
-    for (int t = threadIdx.x; t < cgs * 2 * BV; t += BNV_THREADS) {
-        const int q = t / (2 * BV), k = t % (2 * BV);
-        float acc = 0.f;
-        for (int rr = 0; rr < rows_it; ++rr) acc += sh[rr * cgs + q][k];
-        const int c = q * BV + (k % BV);
-        part[(((size_t)blockIdx.x * nw + w) * C + c) * 2 + (k / BV)] = acc;
-    }
-}
+    const size_t wbase = (size_t)w * a.rpw * C;           // first element of this worker
+    auto issue = [&](int i) {                             // thread 0: fill stage i % stages with tile i
+        const int st = i % stages;
+        const long row = r0 + (long)i * tile_rows;
+        const long rows = r1 - row < tile_rows ? r1 - row : tile_rows;
+        const uint32_t bytes = (uint32_t)(rows * C * 2), bar = full0 + 8 * st;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes * n_in) : "memory");
+        for (int k = 0; k < n_in; ++k)
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(ring0 + (st * n_in + k) * BNS_TILE), "l"(a.in[k] + wbase + (size_t)row * C), "r"(bytes), "r"(bar) : "memory");
+    };
+    if (tid == 0) for (int i = 0; i < stages - 1 && i < ntiles; ++i) issue(i);
 
-__global__ void __launch_bounds__(BNV_THREADS, 4) bnv_apply(const bf16* __restrict__ x, const float* __restrict__ gamma,
-                                                            const float* __restrict__ beta, const bf16* __restrict__ res,
-                                                            bf16* __restrict__ y, const float* __restrict__ stats, long rpw, int C, int relu) {
-    const int cgs = C / BV, rows_it = BNV_THREADS / cgs;
-    const int cg = threadIdx.x % cgs, r = threadIdx.x / cgs;
-    const int w = blockIdx.y;
-    const long per = (rpw + gridDim.x - 1) / gridDim.x;
-    const long r0 = (long)blockIdx.x * per, r1 = min(rpw, r0 + per);
-    float mean[BV], istd[BV], g[BV], b[BV];
-#pragma unroll
-    for (int j = 0; j < BV; ++j) {
-        const int c = cg * BV + j;
-        mean[j] = stats[((size_t)w * C + c) * 2]; istd[j] = stats[((size_t)w * C + c) * 2 + 1];
-        g[j] = gamma[c]; b[j] = beta[c];
-    }
-    const size_t base = (size_t)w * rpw * C + (size_t)cg * BV;
-    constexpr int U = 4;
-    for (long row = r0 + r; row < r1; row += (long)rows_it * U) {
-        uint2 xr[U], rr_[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const long rr = row + (long)u * rows_it;
-            if (rr < r1) { const size_t o = base + (size_t)rr * C; xr[u] = ldg8(x + o); if (res) rr_[u] = ldg8(res + o); }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const long rr = row + (long)u * rows_it;
-            if (rr >= r1) break;
-            float xv[BV], rv[BV];
-            unpack4(xr[u], xv);
-            if (res) unpack4(rr_[u], rv);
-#pragma unroll
-            for (int j = 0; j < BV; ++j) {
-                float v = bn_value(xv[j], mean[j], istd[j], g[j], b[j]);
-                if (res) v += rv[j];
-                if (relu) v = fmaxf(v, 0.f);
-                xv[j] = v;
-            }
-            *(uint2*)(y + base + (size_t)rr * C) = pack4(xv);
-        }
-    }
-}
-
-__global__ void __launch_bounds__(BNV_THREADS, 3) bnv_bwd_apply(const bf16* __restrict__ x, const bf16* __restrict__ out,
-                                                                const bf16* __restrict__ dout, const float* __restrict__ gamma,
-                                                                const float* __restrict__ beta, const float* __restrict__ stats,
-                                                                const float* __restrict__ red, bf16* __restrict__ dx, int accum_dx,
-                                                                bf16* __restrict__ dres, int accum_dres, long rpw, int C, int relu,
-                                                                int mask_from_x) {
-    const int cgs = C / BV, rows_it = BNV_THREADS / cgs;
-    const int cg = threadIdx.x % cgs, r = threadIdx.x / cgs;
-    const int w = blockIdx.y;
-    const long per = (rpw + gridDim.x - 1) / gridDim.x;
-    const long r0 = (long)blockIdx.x * per, r1 = min(rpw, r0 + per);
-    const float inv_n = 1.f / (float)rpw;
-    float mean[BV], istd[BV], g[BV], b[BV], c1[BV], c2[BV];
+    float s1[BV], s2[BV], mean[BV], istd[BV], g[BV], b[BV], c1[BV], c2[BV];
+    const float inv_n = 1.f / (float)a.rpw;
 #pragma unroll
     for (int j = 0; j < BV; ++j) {
         const int c = cg * BV + j;
         const size_t so = ((size_t)w * C + c) * 2;
-        mean[j] = stats[so]; istd[j] = stats[so + 1];
-        g[j] = gamma[c]; b[j] = beta[c];
-        c1[j] = red[so] * inv_n; c2[j] = red[so + 1] * inv_n;
+        s1[j] = 0.f; s2[j] = 0.f;
+        if (MODE != 0) { mean[j] = a.stats[so]; istd[j] = a.stats[so + 1]; g[j] = a.gamma[c]; b[j] = a.beta[c]; }
+        if (MODE == 3) { c1[j] = a.red[so] * inv_n; c2[j] = a.red[so + 1] * inv_n; }
     }
-    const size_t base = (size_t)w * rpw * C + (size_t)cg * BV;
-    const bool need_out = relu && !mask_from_x;
-    constexpr int U = 2;
-    for (long row = r0 + r; row < r1; row += (long)rows_it * U) {
-        uint2 xr[U], dr[U], orr[U];
+    const bool need_out = (MODE == 1 || MODE == 3) && a.relu && !a.mask_from_x;
+    bool ok = true;
+    for (int i = 0; i < ntiles; ++i) {
+        // every thread left tile i - 1 at the barrier below, so its stage can take tile i + stages - 1
+        if (tid == 0 && i + stages - 1 < ntiles) issue(i + stages - 1);
+        const int st = i % stages;
+        if (ok && !bns_wait(full0 + 8 * st, (uint32_t)(i / stages) & 1u, a.err)) ok = false;
+        const uint8_t* sx = bns_sm + (size_t)(st * n_in) * BNS_TILE;
+        const long trow = r0 + (long)i * tile_rows;
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const long rr = row + (long)u * rows_it;
-            if (rr < r1) {
-                const size_t o = base + (size_t)rr * C;
-                xr[u] = ldg8(x + o); dr[u] = ldg8(dout + o);
-                if (need_out) orr[u] = ldg8(out + o);
+        for (int k = 0; k < 2; ++k) {
+            const int lr = rl + k * rows_it;                 // row inside the tile
+            const long row = trow + lr;
+            if (row >= r1 || !ok) continue;
+            const int so = (lr * cgs + cg) * 16;
+            float xv[BV];
+            unpack8(*(const uint4*)(sx + so), xv);
+            if (MODE == 0) {
+#pragma unroll
+                for (int j = 0; j < BV; ++j) { s1[j] += xv[j]; s2[j] = fmaf(xv[j], xv[j], s2[j]); }
+            } else if (MODE == 2) {
+                float rv[BV];
+                const size_t o = wbase + (size_t)row * C + (size_t)cg * BV;
+                if (a.res) { if (n_in > 1) unpack8(*(const uint4*)(sx + BNS_TILE + so), rv); else unpack8(__ldg((const uint4*)(a.res + o)), rv); }
+#pragma unroll
+                for (int j = 0; j < BV; ++j) {
+                    float v = bn_value(xv[j], mean[j], istd[j], g[j], b[j]);
+                    if (a.res) v += rv[j];
+                    if (a.relu) v = fmaxf(v, 0.f);
+                    xv[j] = v;
+                }
+                *(uint4*)(a.y + o) = pack8(xv);
+            } else {
+                float dv[BV], ov[BV];
+                unpack8(*(const uint4*)(sx + BNS_TILE + so), dv);
+                if (need_out) unpack8(*(const uint4*)(sx + 2 * BNS_TILE + so), ov);
+                if (a.relu) {
+#pragma unroll
+                    for (int j = 0; j < BV; ++j) {
+                        const float f = a.mask_from_x ? bn_value(xv[j], mean[j], istd[j], g[j], b[j]) : ov[j];
+                        if (!(f > 0.f)) dv[j] = 0.f;
+                    }
+                }
+                if (MODE == 1) {
+#pragma unroll
+                    for (int j = 0; j < BV; ++j) { s1[j] += dv[j]; s2[j] = fmaf(dv[j], (xv[j] - mean[j]) * istd[j], s2[j]); }
+                } else {
+                    const size_t o = wbase + (size_t)row * C + (size_t)cg * BV;
+                    float t[BV];
+#pragma unroll
+                    for (int j = 0; j < BV; ++j) {
+                        const float xh = (xv[j] - mean[j]) * istd[j];
+                        t[j] = g[j] * istd[j] * (dv[j] - c1[j] - xh * c2[j]);
+                    }
+                    if (a.accum_dx) {
+                        float old[BV]; unpack8(*(const uint4*)(a.y + o), old);
+#pragma unroll
+                        for (int j = 0; j < BV; ++j) t[j] += old[j];
+                    }
+                    *(uint4*)(a.y + o) = pack8(t);
+                    if (a.dres) {
+                        if (a.accum_dres) {
+                            float old[BV]; unpack8(*(const uint4*)(a.dres + o), old);
+#pragma unroll
+                            for (int j = 0; j < BV; ++j) dv[j] += old[j];
+                        }
+                        *(uint4*)(a.dres + o) = pack8(dv);
+                    }
+                }
             }
         }
+        __syncthreads();
+    }
+    if (MODE == 0 || MODE == 1) {
+        // the ring is idle now (every issued tile was waited for): reuse it for the reduction over the row lanes
+        float (*sh)[2 * BV + 1] = (float (*)[2 * BV + 1])bns_sm;
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const long rr = row + (long)u * rows_it;
-            if (rr >= r1) break;
-            const size_t o = base + (size_t)rr * C;
-            float xv[BV], dv[BV], ov[BV], t[BV];
-            unpack4(xr[u], xv); unpack4(dr[u], dv);
-            if (need_out) unpack4(orr[u], ov);
-#pragma unroll
-            for (int j = 0; j < BV; ++j) {
-                if (relu) { float f = mask_from_x ? bn_value(xv[j], mean[j], istd[j], g[j], b[j]) : ov[j]; if (!(f > 0.f)) dv[j] = 0.f; }
-                const float xh = (xv[j] - mean[j]) * istd[j];
-                t[j] = g[j] * istd[j] * (dv[j] - c1[j] - xh * c2[j]);
-            }
-            if (accum_dx) {
-                float old[BV]; unpack4(*(const uint2*)(dx + o), old);
-#pragma unroll
-                for (int j = 0; j < BV; ++j) t[j] += old[j];
-            }
-            *(uint2*)(dx + o) = pack4(t);
-            if (dres) {
-                if (accum_dres) {
-                    float old[BV]; unpack4(*(const uint2*)(dres + o), old);
-#pragma unroll
-                    for (int j = 0; j < BV; ++j) dv[j] += old[j];
-                }
-                *(uint2*)(dres + o) = pack4(dv);
-            }
+        for (int j = 0; j < BV; ++j) { sh[tid][j] = s1[j]; sh[tid][BV + j] = s2[j]; }
+        __syncthreads();
+        // thread t < 2*BV*cgs sums one (channel group, value) column over the rows_it row lanes, in a fixed order
+        for (int t = tid; t < cgs * 2 * BV; t += BNV_THREADS) {
+            const int q = t / (2 * BV), k = t % (2 * BV);
+            float acc = 0.f;
+            for (int rr = 0; rr < rows_it; ++rr) acc += sh[rr * cgs + q][k];
+            const int c = q * BV + (k % BV);
+            a.part[(((size_t)blockIdx.x * nw + w) * C + c) * 2 + (k / BV)] = acc;
         }
     }
 }
@@ -808,31 +791,33 @@ __global__ void bnv_stats_final(const float* __restrict__ part, float* __restric
         *(float2*)(stats + (size_t)i * 2) = make_float2((float)mean, (float)(1.0 / sqrt(var + 1e-5)));
     }
 }
-// same, from the partials a convolution epilogue left: [w * cpw + k][C][2], k < cpw.  One block of 128 threads per
-// (worker, channel): strided partial sums, then a fixed-order tree in shared memory.
-__global__ void __launch_bounds__(128) bnv_stats_final_tiles(const float* __restrict__ part, float* __restrict__ stats, int cpw, int nw, int C, long rpw) {
-    __shared__ float2 sh[128];
-    const int i = blockIdx.x, w = i / C, c = i - w * C, tid = threadIdx.x;
+// same, from the partials a convolution epilogue left: [w * cpw + k][C][2], k < cpw.  One block of 256 threads per
+// (worker, 4 channels): a thread owns one channel and every 64th partial, so that a warp's loads cover whole
+// 32-byte sectors; then a fixed-order tree over the 64 partial lanes in shared memory.
+__global__ void __launch_bounds__(256) bnv_stats_final_tiles(const float* __restrict__ part, float* __restrict__ stats, int cpw, int nw, int C, long rpw) {
+    __shared__ float2 sh[64][5];
+    const int w = blockIdx.y, tid = threadIdx.x, cl = tid & 3, kl = tid >> 2;
+    const int c = blockIdx.x * 4 + cl;
     const float* p = part + ((size_t)w * cpw * C + c) * 2;
     float2 a = make_float2(0.f, 0.f);
-    int k = tid;
-    for (; k + 384 < cpw; k += 512) {                      // four independent loads in flight
-        const float2 v0 = *(const float2*)(p + (size_t)k * C * 2), v1 = *(const float2*)(p + (size_t)(k + 128) * C * 2);
-        const float2 v2 = *(const float2*)(p + (size_t)(k + 256) * C * 2), v3 = *(const float2*)(p + (size_t)(k + 384) * C * 2);
+    int k = kl;
+    for (; k + 192 < cpw; k += 256) {                      // four independent loads in flight
+        const float2 v0 = *(const float2*)(p + (size_t)k * C * 2), v1 = *(const float2*)(p + (size_t)(k + 64) * C * 2);
+        const float2 v2 = *(const float2*)(p + (size_t)(k + 128) * C * 2), v3 = *(const float2*)(p + (size_t)(k + 192) * C * 2);
         a.x += (v0.x + v1.x) + (v2.x + v3.x); a.y += (v0.y + v1.y) + (v2.y + v3.y);
     }
-    for (; k < cpw; k += 128) { const float2 v = *(const float2*)(p + (size_t)k * C * 2); a.x += v.x; a.y += v.y; }
-    sh[tid] = a;
+    for (; k < cpw; k += 64) { const float2 v = *(const float2*)(p + (size_t)k * C * 2); a.x += v.x; a.y += v.y; }
+    sh[kl][cl] = a;
     __syncthreads();
-    for (int d = 64; d > 0; d >>= 1) {
-        if (tid < d) { sh[tid].x += sh[tid + d].x; sh[tid].y += sh[tid + d].y; }
+    for (int d = 32; d > 0; d >>= 1) {
+        if (kl < d) { sh[kl][cl].x += sh[kl + d][cl].x; sh[kl][cl].y += sh[kl + d][cl].y; }
         __syncthreads();
     }
-    if (tid == 0) {
-        const double mean = (double)sh[0].x / (double)rpw;
-        double var = (double)sh[0].y / (double)rpw - mean * mean;
+    if (kl == 0) {
+        const double mean = (double)sh[0][cl].x / (double)rpw;
+        double var = (double)sh[0][cl].y / (double)rpw - mean * mean;
         if (var < 0.0) var = 0.0;
-        *(float2*)(stats + (size_t)i * 2) = make_float2((float)mean, (float)(1.0 / sqrt(var + 1e-5)));
+        *(float2*)(stats + ((size_t)w * C + c) * 2) = make_float2((float)mean, (float)(1.0 / sqrt(var + 1e-5)));
     }
 }
 // block = one channel, one warp per worker (nw <= 32): red[w][c] = (sum dy, sum dy xhat); warp 0 then adds the
@@ -854,41 +839,47 @@ __global__ void bnv_bwd_final(const float* __restrict__ part, float* __restrict_
 }
 
 static bool bnv_ok(int dt, int C) { int cgs = C / BV; return dt == 1 && C % BV == 0 && cgs <= BNV_THREADS && (cgs & (cgs - 1)) == 0; }
-// Row chunks per worker such that chunks * nw CTAs fill the GPU exactly once (no partial second wave).
-template <typename K>
-static int bnv_chunks(K kernel, int which, int nw, long rpw, int C) {
-    static int occ_cache[4] = {0, 0, 0, 0}, sms = 0;
+constexpr int BNS_SMEM = BNS_RING + 8 * 8;
+// Row chunks per worker such that chunks * nw CTAs fill the GPU once (two CTAs per SM), each with at least four tiles.
+static int bns_chunks(int nw, long rpw, int C) {
+    static int sms = 0;
     if (!sms) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); if (sms <= 0) sms = 148; }
-    if (!occ_cache[which] && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_cache[which], kernel, BNV_THREADS, 0) != cudaSuccess || occ_cache[which] < 1))
-        occ_cache[which] = 2;
-    const int occ = occ_cache[which];
-    long rows_it = BNV_THREADS / (C / BV);
-    long want = ((long)sms * occ) / nw, maxc = (rpw + rows_it * 4 - 1) / (rows_it * 4);
+    const long tile_rows = BNS_TILE / (C * 2);
+    long want = ((long)sms * 2) / nw, maxc = (rpw + tile_rows * 4 - 1) / (tile_rows * 4);
     long c = want < maxc ? want : maxc;
     if (c > BNV_MAX_CHUNKS) c = BNV_MAX_CHUNKS;
     return (int)(c < 1 ? 1 : c);
+}
+template <int MODE>
+static void bns_launch(const BnsArgs& a, int chunks, int nw, cudaStream_t s) {
+    static bool attr = false;
+    if (!attr) { cudaFuncSetAttribute(bns_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, BNS_SMEM); attr = true; }
+    bns_kernel<MODE><<<dim3(chunks, nw), BNV_THREADS, BNS_SMEM, s>>>(a);
 }
 
 bool bn_accepts_conv_partials(int dt, int C) { return bnv_ok(dt, C); }
 
 void bn_forward(int dt, const void* x, const float* gamma, const float* beta, const void* res, void* y, float* stats,
-                float* scratch, int nw, long rpw, int C, bool relu, const float* conv_part, int conv_chunks, cudaStream_t s) {
-    if (bnv_ok(dt, C)) {
-        const int chunks = bnv_chunks(bnv_reduce<0>, 0, nw, rpw, C);
-        const int chunks_a = bnv_chunks(bnv_apply, 1, nw, rpw, C);
+                float* scratch, int nw, long rpw, int C, bool relu, const float* conv_part, int conv_chunks, int* err, cudaStream_t s) {
+    if (bnv_ok(dt, C) && err) {
+        const int chunks = bns_chunks(nw, rpw, C);
         const double total = (double)nw * rpw * C;
-        dim3 grid(chunks, nw), grid_a(chunks_a, nw);
+        BnsArgs a{};
+        a.in[0] = (const bf16*)x; a.n_in = 1; a.gamma = gamma; a.beta = beta; a.stats = stats; a.rpw = rpw; a.C = C; a.relu = relu; a.err = err;
         if (conv_part) {
             Scope sc(KC_BN_FWD_STATS, 0.0, 8.0 * conv_chunks * nw * C, s);
-            bnv_stats_final_tiles<<<nw * C, 128, 0, s>>>(conv_part, stats, conv_chunks, nw, C, rpw);
+            bnv_stats_final_tiles<<<dim3(C / 4, nw), 256, 0, s>>>(conv_part, stats, conv_chunks, nw, C, rpw);
         } else {
             { Scope sc(KC_BN_FWD_STATS, 0.0, 2.0 * total, s);
-              bnv_reduce<0><<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, nullptr, nullptr, nullptr, nullptr, nullptr, scratch, rpw, C, 0, 0); }
+              BnsArgs r = a; r.part = scratch;
+              bns_launch<0>(r, chunks, nw, s); }
             { Scope sc(KC_BN_FWD_STATS, 0.0, 8.0 * chunks * nw * C, s);
               bnv_stats_final<<<cdiv((size_t)nw * C * 32, 256), 256, 0, s>>>(scratch, stats, chunks, nw * C, rpw); }
         }
         Scope sc(KC_BN_FWD_APPLY, 0.0, 2.0 * total * (res ? 3 : 2), s);
-        bnv_apply<<<grid_a, BNV_THREADS, 0, s>>>((const bf16*)x, gamma, beta, (const bf16*)res, (bf16*)y, stats, rpw, C, relu);
+        a.y = (bf16*)y; a.res = (const bf16*)res;
+        if (res) { a.in[1] = (const bf16*)res; a.n_in = 2; }
+        bns_launch<2>(a, chunks, nw, s);
         return;
     }
     int chunks = (int)(rpw < RED_CHUNKS ? rpw : RED_CHUNKS);
@@ -908,23 +899,25 @@ void bn_forward(int dt, const void* x, const float* gamma, const float* beta, co
 
 void bn_backward(int dt, const void* x, const void* out, const void* dout, const float* gamma, const float* beta,
                  const float* stats, void* dx, bool accum_dx, void* dres, bool accum_dres, float* dgamma, float* dbeta, float* red,
-                 float* scratch, int nw, long rpw, int C, bool relu, bool has_res, bool accum_params, cudaStream_t s) {
-    if (bnv_ok(dt, C)) {
-        const int chunks = bnv_chunks(bnv_reduce<1>, 2, nw, rpw, C);
-        const int chunks_a = bnv_chunks(bnv_bwd_apply, 3, nw, rpw, C);
+                 float* scratch, int nw, long rpw, int C, bool relu, bool has_res, bool accum_params, int* err, cudaStream_t s) {
+    if (bnv_ok(dt, C) && err) {
+        const int chunks = bns_chunks(nw, rpw, C);
         const double total = (double)nw * rpw * C;
         const int mask_from_x = relu && !has_res;
-        const int reads = 2 + ((relu && !mask_from_x) ? 1 : 0);
-        dim3 grid(chunks, nw);
+        const bool need_out = relu && !mask_from_x;
+        const int reads = 2 + (need_out ? 1 : 0);
+        BnsArgs a{};
+        a.in[0] = (const bf16*)x; a.in[1] = (const bf16*)dout; a.in[2] = (const bf16*)out; a.n_in = reads;
+        a.gamma = gamma; a.beta = beta; a.stats = stats; a.red = red; a.rpw = rpw; a.C = C; a.relu = relu; a.mask_from_x = mask_from_x; a.err = err;
         { Scope sc(KC_BN_BWD_REDUCE, 0.0, 2.0 * total * reads, s);
-          bnv_reduce<1><<<grid, BNV_THREADS, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, gamma, beta, stats, scratch, rpw, C,
-                                                      relu, mask_from_x); }
+          BnsArgs r = a; r.part = scratch;
+          bns_launch<1>(r, chunks, nw, s); }
         { Scope sc(KC_BN_BWD_REDUCE, 0.0, 8.0 * chunks * nw * C, s);
           if (nw <= 32) bnv_bwd_final<<<C, 32 * nw, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C, accum_params);
           else bn_bwd_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C, accum_params); }
         Scope sc(KC_BN_BWD_APPLY, 0.0, 2.0 * total * (reads + 1 + (accum_dx ? 1 : 0) + (dres ? (accum_dres ? 2 : 1) : 0)), s);
-        bnv_bwd_apply<<<dim3(chunks_a, nw), BNV_THREADS, 0, s>>>((const bf16*)x, (const bf16*)out, (const bf16*)dout, gamma, beta, stats, red, (bf16*)dx,
-                                                   accum_dx, (bf16*)dres, accum_dres, rpw, C, relu, mask_from_x);
+        a.y = (bf16*)dx; a.accum_dx = accum_dx; a.dres = (bf16*)dres; a.accum_dres = accum_dres;
+        bns_launch<3>(a, chunks, nw, s);
         return;
     }
     int chunks = (int)(rpw < RED_CHUNKS ? rpw : RED_CHUNKS);
