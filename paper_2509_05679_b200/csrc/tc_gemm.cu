@@ -583,52 +583,56 @@ wg_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUten
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        if (lane == 0) {
-            const int tap0 = rb0 / p.kchunks, cc0 = (rb0 - tap0 * p.kchunks) * 64;
-            const int tap1 = rb1 / p.kchunks, cc1 = (rb1 - tap1 * p.kchunks) * 64;
-            const int dw0 = p.dw[tap0], dh0 = p.dh[tap0], dw1 = p.dw[tap1], dh1 = p.dh[tap1];
-            const uint32_t smem0 = smem_u32(smem), full0 = smem_u32(full), empty0 = smem_u32(empty);
-            uint32_t st = 0, ph = 1, dst = smem0, fb = full0, eb = empty0;
-            // pixel-tile cursor (tw fastest, then th, then tn), advanced without divisions
-            int pt = pt_begin;
-            int tw = pt % p.tiles_w; pt /= p.tiles_w;
-            int th = pt % p.tiles_h; int tn = pt / p.tiles_h;
-            const int wstep = p.Wt * p.xs, hstep = p.Ht * p.xs;
-            for (int kb = 0; kb < num_kb; ++kb) {
-                if (!mbar_wait_a(eb, ph, p.err, 4)) break;
-                const int w0 = tw * p.Wt, h0 = th * p.Ht, n0 = p.n_base + tn * p.Nt;
-                const int xw = tw * wstep, xh = th * hstep;
+        // ---- producer: all lanes walk the loop, one elected lane issues
+        const int tap0 = rb0 / p.kchunks, cc0 = (rb0 - tap0 * p.kchunks) * 64;
+        const int tap1 = rb1 / p.kchunks, cc1 = (rb1 - tap1 * p.kchunks) * 64;
+        const int dw0 = p.dw[tap0], dh0 = p.dh[tap0], dw1 = p.dw[tap1], dh1 = p.dh[tap1];
+        const uint32_t smem0 = smem_u32(smem), full0 = smem_u32(full), empty0 = smem_u32(empty);
+        uint32_t st = 0, ph = 1, dst = smem0, fb = full0, eb = empty0;
+        // pixel-tile cursor (tw fastest, then th, then tn), advanced without divisions
+        int pt = pt_begin;
+        int tw = pt % p.tiles_w; pt /= p.tiles_w;
+        int th = pt % p.tiles_h; int tn = pt / p.tiles_h;
+        const int wstep = p.Wt * p.xs, hstep = p.Ht * p.xs;
+        for (int kb = 0; kb < num_kb; ++kb) {
+            if (!mbar_wait_a(eb, ph, p.err, 4)) break;
+            const int w0 = tw * p.Wt, h0 = th * p.Ht, n0 = p.n_base + tn * p.Nt;
+            const int xw = tw * wstep, xh = th * hstep;
+            if (elect_one()) {
                 mbar_expect_tx_a(fb, STAGE_BYTES);
                 tma_load_4d_a(dst, &tmX, fb, cc0, xw + dw0, xh + dh0, n0);
                 tma_load_4d_a(dst + BOX_BYTES, &tmX, fb, cc1, xw + dw1, xh + dh1, n0);
 #pragma unroll
                 for (int j = 0; j < N_TILE / 64; ++j)
                     tma_load_4d_a(dst + A_BYTES + j * BOX_BYTES, &tmDY, fb, co0 + j * 64, w0, h0, n0);
-                if (++tw == p.tiles_w) { tw = 0; if (++th == p.tiles_h) { th = 0; ++tn; } }
-                if (++st == STAGES) { st = 0; ph ^= 1u; dst = smem0; fb = full0; eb = empty0; }
-                else { dst += STAGE_BYTES; fb += 8; eb += 8; }
             }
+            __syncwarp();
+            if (++tw == p.tiles_w) { tw = 0; if (++th == p.tiles_h) { th = 0; ++tn; } }
+            if (++st == STAGES) { st = 0; ph ^= 1u; dst = smem0; fb = full0; eb = empty0; }
+            else { dst += STAGE_BYTES; fb += 8; eb += 8; }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc(BLOCK_M, N_TILE, 1, 1);
-            const uint64_t dconst = make_desc(0, BOX_BYTES, 1024);
-            const uint32_t d_hi = (uint32_t)(dconst >> 32), d_lo = (uint32_t)dconst;
-            const uint32_t a16_0 = smem_u32(smem) >> 4, full0 = smem_u32(full), empty0 = smem_u32(empty);
-            uint32_t st = 0, ph = 0, a16 = a16_0, fb = full0, eb = empty0, acc = 0;
-            for (int kb = 0; kb < num_kb; ++kb) {
-                if (!mbar_wait_a(fb, ph, p.err, 5)) break;
-                const uint32_t a_lo = d_lo + a16, b_lo = a_lo + (A_BYTES >> 4);
+        // ---- MMA issue (the elected lane is the same one every time, so the commits track the MMAs it issued)
+        const uint32_t idesc = make_idesc(BLOCK_M, N_TILE, 1, 1);
+        const uint64_t dconst = make_desc(0, BOX_BYTES, 1024);
+        const uint32_t d_hi = (uint32_t)(dconst >> 32), d_lo = (uint32_t)dconst;
+        const uint32_t a16_0 = smem_u32(smem) >> 4, full0 = smem_u32(full), empty0 = smem_u32(empty);
+        uint32_t st = 0, ph = 0, a16 = a16_0, fb = full0, eb = empty0, acc = 0;
+        for (int kb = 0; kb < num_kb; ++kb) {
+            if (!mbar_wait_a(fb, ph, p.err, 5)) break;
+            tc_fence_after();
+            const uint32_t a_lo = d_lo + a16, b_lo = a_lo + (A_BYTES >> 4);
+            if (elect_one()) {
 #pragma unroll
-                for (int k = 0; k < 64 / UMMA_K; ++k) {    // 16 pixels = 16 rows of 128 bytes per MMA = 128 address units
-                    umma_bf16_w<false>(tmem_base, a_lo + k * (UMMA_K * 128 >> 4), b_lo + k * (UMMA_K * 128 >> 4), d_hi, idesc, acc);
-                    acc = 1;
-                }
+                for (int k = 0; k < 64 / UMMA_K; ++k)      // 16 pixels = 16 rows of 128 bytes per MMA = 128 address units
+                    umma_bf16_w<false>(tmem_base, a_lo + k * (UMMA_K * 128 >> 4), b_lo + k * (UMMA_K * 128 >> 4), d_hi, idesc, k == 0 ? acc : 1u);
                 umma_commit_a<false>(eb);
-                if (++st == STAGES) { st = 0; ph ^= 1u; a16 = a16_0; fb = full0; eb = empty0; }
-                else { a16 += STAGE_BYTES >> 4; fb += 8; eb += 8; }
+                if (kb == num_kb - 1) umma_commit(accum_bar);
             }
-            umma_commit(accum_bar);
+            __syncwarp();
+            acc = 1;
+            if (++st == STAGES) { st = 0; ph ^= 1u; a16 = a16_0; fb = full0; eb = empty0; }
+            else { a16 += STAGE_BYTES >> 4; fb += 8; eb += 8; }
         }
     } else {
         const int q = warp & 3;
