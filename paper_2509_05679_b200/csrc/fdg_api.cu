@@ -71,6 +71,7 @@ struct Op {
     std::vector<char*> a_ptrs, dy_ptrs;                      // the buffers the A / dY maps below were built for
     std::vector<char*> y_ptrs, dx_ptrs;                      // where the forward output / the input gradient can be written
     std::vector<tc::TensorMap> fo, dox;                      // output maps of the forward / input-gradient kernel, per buffer
+    std::vector<tc::TensorMap> far, dar;                     // rows-mode activation maps (3x3, stride 1, tiles of whole image rows); empty: not used
     std::vector<tc::TensorMap> fa, fb, da, db, wx, wdy;      // fwd A, fwd B (per weight slot), dgrad A, dgrad B, wgrad X, wgrad dY
     std::vector<tc::TensorMap> fbh, dbh;                     // fwd / dgrad B with half-height boxes (CTA-pair kernels); empty: not used
 };
@@ -382,8 +383,9 @@ bool tc_forward(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* y_base, 
     double rows = (double)wn.n * g.Ho * g.Wo;
     Scope sc(KC_TC_FWD, 2.0 * rows * g.Co * g.R * g.R * g.C, 2.0 * ((double)wn.n * g.H * g.W * g.C + (double)g.Co * g.R * g.R * g.C + rows * g.Co), s);
     const int io = find_buf(o.y_ptrs, y_base);
-    const bool ok = tc::run_km(o.fa[ia], o.fb[version % m.D], o.fbh.empty() ? nullptr : &o.fbh[version % m.D], io >= 0 ? &o.fo[io] : nullptr, p,
-                               o.n_tile_f, s) == cudaSuccess;
+    const tc::KmMaps maps{&o.fa[ia], o.far.empty() ? nullptr : &o.far[ia], &o.fb[version % m.D], o.fbh.empty() ? nullptr : &o.fbh[version % m.D],
+                          io >= 0 ? &o.fo[io] : nullptr};
+    const bool ok = tc::run_km(maps, p, o.n_tile_f, s) == cudaSuccess;
     if (ok && o.stat_chunks) { m.fused_stats_tensor = o.out; m.fused_stats_chunks = o.stat_chunks; }
     return ok;
 }
@@ -403,8 +405,9 @@ bool tc_dgrad(fdg_ctx* c, Module& m, const Op& o, char* dy_base, char* dx_base, 
     Scope sc(KC_TC_DGRAD, 2.0 * crows * g.C * p.ntaps * g.Co,
              2.0 * ((double)wn.n * g.Ho * g.Wo * g.Co + (double)g.Co * p.ntaps * g.C + crows * p.ncls * g.C * (accum ? 2 : 1)), s);
     const int io = find_buf(o.dx_ptrs, dx_base);
-    return tc::run_km(o.da[ia], o.db[version % m.D], o.dbh.empty() ? nullptr : &o.dbh[version % m.D], io >= 0 ? &o.dox[io] : nullptr, p, o.n_tile_d,
-                      s) == cudaSuccess;
+    const tc::KmMaps maps{&o.da[ia], o.dar.empty() ? nullptr : &o.dar[ia], &o.db[version % m.D], o.dbh.empty() ? nullptr : &o.dbh[version % m.D],
+                          io >= 0 ? &o.dox[io] : nullptr};
+    return tc::run_km(maps, p, o.n_tile_d, s) == cudaSuccess;
 }
 bool tc_wgrad(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* dy_base, float* dw, const Win& wn, cudaStream_t s) {
     int ix = find_buf(o.a_ptrs, x_base), id = find_buf(o.dy_ptrs, dy_base);
@@ -574,6 +577,12 @@ bool build_tc_plans(fdg_ctx* c) {
             f.ncls = 1; f.cls_tap0[0] = 0; f.cls_tap0[1] = taps; f.cls_oph[0] = 0; f.cls_opw[0] = 0;
             o.fa.resize(o.a_ptrs.size());
             for (size_t i = 0; i < o.a_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.fa[i], o.a_ptrs[i], g.C, g.W, g.H, g.N, 64, wt, ht, nt, g.stride);
+            // rows mode: a box of the tile's rows plus one above and one below, for a tile that is whole rows of one image
+            const bool rows_ok = g.R == 3 && g.stride == 1 && wt == g.Wo && nt == 1;
+            if (rows_ok) {
+                o.far.resize(o.a_ptrs.size());
+                for (size_t i = 0; i < o.a_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.far[i], o.a_ptrs[i], g.C, g.W, g.H, g.N, 64, g.W, ht + 2, 1, 1);
+            }
             o.fb.resize(m.D);
             for (int v = 0; v < m.D; ++v) ok = ok && tc::make_map_2d(&o.fb[v], wbig(c, m, v, o.w_off), Ktot, g.Co, 64, o.n_tile_f);
             f.Nfull = g.N;
@@ -584,7 +593,7 @@ bool build_tc_plans(fdg_ctx* c) {
             o.fo.resize(o.y_ptrs.size());
             for (size_t i = 0; i < o.y_ptrs.size(); ++i) ok = ok && tc::make_map_out(&o.fo[i], o.y_ptrs[i], g.Co, g.Wo, g.Ho, g.N, wt, ht);
             const bool pairs = c->kernel_path == 0;          // CTA-pair kernels for the 256-column tile (kernel_path 2: none)
-            if (pairs && o.n_tile_f >= 256) {
+            if (pairs && (o.n_tile_f >= 256 || (rows_ok && o.n_tile_f == 128))) {
                 o.fbh.resize(m.D);
                 for (int v = 0; v < m.D; ++v) ok = ok && tc::make_map_2d(&o.fbh[v], wbig(c, m, v, o.w_off), Ktot, g.Co, 64, o.n_tile_f / 2);
             }
@@ -619,9 +628,13 @@ bool build_tc_plans(fdg_ctx* c) {
             }
             o.dox.resize(o.dx_ptrs.size());
             for (size_t i = 0; i < o.dx_ptrs.size(); ++i) ok = ok && tc::make_map_out(&o.dox[i], o.dx_ptrs[i], g.C, g.W, g.H, g.N, wt, ht);
+            if (rows_ok) {
+                o.dar.resize(o.dy_ptrs.size());
+                for (size_t i = 0; i < o.dy_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.dar[i], o.dy_ptrs[i], g.Co, g.Wo, g.Ho, g.N, 64, g.Wo, ht + 2, 1, 1);
+            }
             o.db.resize(m.D);
             for (int v = 0; v < m.D; ++v) ok = ok && tc::make_map_2d(&o.db[v], wtslot(m, v, o.w_off), (long)taps * g.Co, g.C, 64, o.n_tile_d);
-            if (pairs && o.n_tile_d >= 256) {
+            if (pairs && (o.n_tile_d >= 256 || (rows_ok && o.n_tile_d == 128))) {
                 o.dbh.resize(m.D);
                 for (int v = 0; v < m.D; ++v) ok = ok && tc::make_map_2d(&o.dbh[v], wtslot(m, v, o.w_off), (long)taps * g.Co, g.C, 64, o.n_tile_d / 2);
             }

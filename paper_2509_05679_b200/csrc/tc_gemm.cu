@@ -33,6 +33,9 @@ constexpr int BLOCK_K = 64;       // bf16 elements per 128-byte swizzle row
 constexpr int UMMA_K = 16;
 constexpr int NUM_THREADS = 192;
 constexpr long long WAIT_CYCLES = 4000000000LL;   // ~2 s at 2 GHz
+#ifndef EPI_SLEEP_NS
+#define EPI_SLEEP_NS 200
+#endif
 
 // ------------------------------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -64,7 +67,7 @@ __device__ __forceinline__ bool mbar_wait_sleep(uint64_t* bar, uint32_t parity, 
     if (mbar_try_wait(bar, parity)) return true;
     long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
-        __nanosleep(200);
+        __nanosleep(EPI_SLEEP_NS);
         if (clock64() - t0 > WAIT_CYCLES) { atomicCAS(err, 0, code); return false; }
     }
     return true;
@@ -281,23 +284,34 @@ constexpr int EPI_BUF_BYTES = 32 * EPI_SLICE * 2; // one staged slice: 32 rows x
 // block to a TMA store, whose box is exactly the warp's 32 pixels x 64 channels; otherwise the warp copies the
 // block out row by row (strided outputs of a stride-2 input gradient, partial tiles).  When a batch-norm follows, the
 // per-channel sum and sum of squares over the warp's rows are taken from the staged (rounded) values.
-template <int N_TILE, int STAGES, int EPI_WARPS, bool PAIR, int KSUB, int MIN_CTAS>
+//
+// ROWS (3x3, stride 1, a tile = whole rows of one image): a stage holds the tile's rows plus one row above and below
+// for ONE horizontal shift and one 64-channel chunk; the three vertical taps read it through descriptors that start
+// 0, 1 or 2 image rows into the stage (a multiple of 1024 bytes, so the swizzle pattern is unchanged), against three
+// weight tiles.  The activation is fetched three times instead of nine.  RESIDENT: the whole weight matrix (all taps
+// and chunks of this CTA's rows) is loaded once and stays in shared memory; stages then hold activations only.
+constexpr int ROWS_A_BYTES = 24 * 1024;           // room for 128 + 2 * 32 pixels of 128 bytes
+template <int N_TILE, int STAGES, int EPI_WARPS, bool PAIR, int KSUB, int MIN_CTAS, bool ROWS, int RES_KB>
 __global__ void __launch_bounds__(64 + 32 * EPI_WARPS, MIN_CTAS)
 km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmO, KmParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
+    constexpr bool RESIDENT = RES_KB > 0;
     constexpr int B_ROWS = PAIR ? N_TILE / 2 : N_TILE;
     constexpr int A_BYTES = BLOCK_M * BLOCK_K * 2, B_BYTES = B_ROWS * BLOCK_K * 2, SUB_BYTES = A_BYTES + B_BYTES;
-    constexpr int STAGE_BYTES = KSUB * SUB_BYTES;
+    constexpr int STAGE_BYTES = ROWS ? ROWS_A_BYTES + (RESIDENT ? 0 : 3 * B_BYTES) : KSUB * SUB_BYTES;
+    constexpr int RES_BYTES = RES_KB * 1024;
     constexpr int EPI_BYTES = EPI_WARPS * 2 * EPI_BUF_BYTES;
     constexpr int COL_STEP = EPI_SLICE * (EPI_WARPS / 4);
     constexpr uint32_t TMEM_COLS = 2 * N_TILE;
-    uint8_t* epi_smem = smem + STAGES * STAGE_BYTES;
-    uint64_t* full = (uint64_t*)(smem + STAGES * STAGE_BYTES + EPI_BYTES);
+    uint8_t* wres = smem + STAGES * STAGE_BYTES;                 // resident weights: [tap][chunk][B_ROWS x 64]
+    uint8_t* epi_smem = wres + RES_BYTES;
+    uint64_t* full = (uint64_t*)(epi_smem + EPI_BYTES);
     uint64_t* empty = full + STAGES;
     uint64_t* tmem_full = empty + STAGES;        // [2]
     uint64_t* tmem_empty = tmem_full + 2;        // [2]
-    uint32_t* tmem_slot = (uint32_t*)(tmem_empty + 2);
+    uint64_t* wres_bar = tmem_empty + 2;
+    uint32_t* tmem_slot = (uint32_t*)(wres_bar + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = PAIR ? cluster_rank() : 0u;
@@ -312,6 +326,7 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         if (p.tma_out) tma_prefetch_desc(&tmO);
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], PAIR ? 2 * EPI_WARPS : EPI_WARPS); }
+        mbar_init(wres_bar, 1);
         fence_barrier_init();
     }
     __syncwarp();
@@ -329,6 +344,18 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         // stage cursor: destination, barriers, and the parity waited for on `empty` (a fresh barrier
         // passes a wait for parity 1, so the first round finds every stage free)
         uint32_t st = 0, ph = 1, dst = smem0, fb = full_s0, fl = full_l0, eb = empty0;
+        if (RESIDENT) {
+            // every tap and chunk of this CTA's weight rows, once (a single column tile: Cn == N_TILE)
+            const int nblk = p.ntaps * p.kchunks;
+            if (elect_one()) {
+                mbar_expect_tx_a(smem_u32(wres_bar), nblk * B_BYTES);
+                for (int t = 0; t < p.ntaps; ++t)
+                    for (int kc = 0; kc < p.kchunks; ++kc)
+                        tma_load_2d_a(smem_u32(wres) + (t * p.kchunks + kc) * B_BYTES, &tmB, smem_u32(wres_bar), p.koff[t] + kc * BLOCK_K,
+                                      PAIR ? (int)rank * B_ROWS : 0);
+            }
+            __syncwarp();
+        }
         for (int tile = walker; tile < total && ok; tile += walkers) {
             const int cls = tile / per_cls, tl = tile - cls * per_cls;
             int tm = tl / tiles_c; const int co0 = (tl - tm * tiles_c) * N_TILE;
@@ -337,6 +364,31 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             const int th = tm % p.tiles_h; const int tn = tm / p.tiles_h;
             const int w0 = tw * p.Wt * p.xs, h0 = th * p.Ht * p.xs, n0 = p.n_base + tn * p.Nt;
             const int brow = co0 + (PAIR ? (int)rank * B_ROWS : 0);
+            if (ROWS) {
+                const uint32_t a_bytes = (uint32_t)(p.Ht + 2) * p.Wt * 128u;
+                for (int kc = 0; kc < p.kchunks && ok; ++kc) {
+                    for (int dwi = 0; dwi < 3; ++dwi) {
+                        if (!mbar_wait_a(eb, ph, p.err, 1)) { ok = false; break; }
+                        if (elect_one()) {
+                            if (!PAIR || rank == 0) mbar_expect_tx_a(fl, (PAIR ? 2 : 1) * (a_bytes + (RESIDENT ? 0 : 3 * B_BYTES)));
+                            if (PAIR) tma_load_4d_pair(dst, &tmA, fb, kc * BLOCK_K, dwi - 1, h0 - 1, n0);
+                            else tma_load_4d_a(dst, &tmA, fb, kc * BLOCK_K, dwi - 1, h0 - 1, n0);
+                            if (!RESIDENT) {
+#pragma unroll
+                                for (int dhi = 0; dhi < 3; ++dhi) {
+                                    const int kcol = p.koff[p.rows_tap[dwi * 3 + dhi]] + kc * BLOCK_K;
+                                    if (PAIR) tma_load_2d_pair(dst + ROWS_A_BYTES + dhi * B_BYTES, &tmB, fb, kcol, brow);
+                                    else tma_load_2d_a(dst + ROWS_A_BYTES + dhi * B_BYTES, &tmB, fb, kcol, brow);
+                                }
+                            }
+                        }
+                        __syncwarp();
+                        if (++st == STAGES) { st = 0; ph ^= 1u; dst = smem0; fb = full_s0; fl = full_l0; eb = empty0; }
+                        else { dst += STAGE_BYTES; fb += 8; fl += 8; eb += 8; }
+                    }
+                }
+                continue;
+            }
             const int tap_end = p.cls_tap0[cls + 1];
             int left = (tap_end - p.cls_tap0[cls]) * p.kchunks;      // sub-blocks of this tile still to load
             int sub = 0;                                               // sub-block slot inside the current stage
@@ -388,6 +440,35 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 tc_fence_after();
                 const uint32_t d = tmem_base + buf * N_TILE;
                 uint32_t acc = 0;
+                if (ROWS) {
+                    if (RESIDENT && ti == 0 && !mbar_wait(wres_bar, 0, p.err, 8)) { ok = false; break; }
+                    const uint32_t row16 = (uint32_t)p.Wt * 128u >> 4;          // one image row of the stage, in descriptor address units
+                    const uint32_t wres16 = smem_u32(wres) >> 4;
+                    const int nst = 3 * p.kchunks;
+                    for (int sidx = 0; sidx < nst; ++sidx) {
+                        if (!mbar_wait_a(fb, ph, p.err, 2)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t a_lo = d_lo + a16;
+                        const int kc = sidx / 3, dwi = sidx - kc * 3;
+                        if (elect_one()) {
+#pragma unroll
+                            for (int dhi = 0; dhi < 3; ++dhi) {
+                                const uint32_t b_lo = RESIDENT ? d_lo + wres16 + (uint32_t)((p.rows_tap[dwi * 3 + dhi] * p.kchunks + kc) * (B_BYTES >> 4))
+                                                               : a_lo + (uint32_t)((ROWS_A_BYTES + dhi * B_BYTES) >> 4);
+#pragma unroll
+                                for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                                    umma_bf16_w<PAIR>(d, a_lo + dhi * row16 + 2 * k, b_lo + 2 * k, d_hi, idesc, (dhi == 0 && k == 0) ? acc : 1u);
+                            }
+                            umma_commit_a<PAIR>(eb);
+                            if (sidx == nst - 1) umma_commit_a<PAIR>(smem_u32(&tmem_full[buf]));
+                        }
+                        __syncwarp();
+                        acc = 1;
+                        if (++st == STAGES) { st = 0; ph ^= 1u; a16 = a16_0; fb = full0; eb = empty0; }
+                        else { a16 += STAGE_BYTES >> 4; fb += 8; eb += 8; }
+                    }
+                    continue;
+                }
                 for (int left = num_kb; left > 0; left -= KSUB) {
                     if (!mbar_wait_a(fb, ph, p.err, 2)) { ok = false; break; }
                     tc_fence_after();
@@ -759,15 +840,16 @@ static int sm_count() {
     return n;
 }
 
-template <int N_TILE, int STAGES, int EPI_WARPS, int KSUB>
+template <int N_TILE, int STAGES, int EPI_WARPS, int KSUB, bool ROWS, int RES_KB>
 static cudaError_t launch_km(const TensorMap& a, const TensorMap& b, const TensorMap& o, const KmParams& p, cudaStream_t s) {
-    constexpr int smem = STAGES * KSUB * (BLOCK_M * BLOCK_K * 2 + N_TILE * BLOCK_K * 2) + EPI_WARPS * 2 * EPI_BUF_BYTES + 1024 + 256;
+    constexpr int stage = ROWS ? ROWS_A_BYTES + (RES_KB ? 0 : 3 * N_TILE * BLOCK_K * 2) : KSUB * (BLOCK_M * BLOCK_K * 2 + N_TILE * BLOCK_K * 2);
+    constexpr int smem = STAGES * stage + RES_KB * 1024 + EPI_WARPS * 2 * EPI_BUF_BYTES + 1024 + 256;
     static_assert(smem <= 232448, "shared memory");
     // CTAs of this variant that fit on an SM: shared memory (227 KB, 1 KB reserved per CTA) and 512 tensor-memory columns
     constexpr int by_smem = (227 * 1024) / (smem + 1024), by_tmem = 512 / (2 * N_TILE);
     constexpr int per_sm = by_smem < by_tmem ? by_smem : by_tmem;
     static_assert(per_sm >= 1 && per_sm <= 2, "CTAs per SM");
-    auto kernel = km_kernel<N_TILE, STAGES, EPI_WARPS, false, KSUB, per_sm>;
+    auto kernel = km_kernel<N_TILE, STAGES, EPI_WARPS, false, KSUB, per_sm, ROWS, RES_KB>;
     static bool attr = false;
     if (!attr) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -782,11 +864,12 @@ static cudaError_t launch_km(const TensorMap& a, const TensorMap& b, const Tenso
 }
 
 // CTA pairs: `b` is a tensor map whose box holds N_TILE / 2 weight rows.
-template <int N_TILE, int STAGES, int EPI_WARPS, int KSUB>
+template <int N_TILE, int STAGES, int EPI_WARPS, int KSUB, bool ROWS>
 static cudaError_t launch_km_pair(const TensorMap& a, const TensorMap& b, const TensorMap& o, const KmParams& p, cudaStream_t s) {
-    constexpr int smem = STAGES * KSUB * (BLOCK_M * BLOCK_K * 2 + (N_TILE / 2) * BLOCK_K * 2) + EPI_WARPS * 2 * EPI_BUF_BYTES + 1024 + 256;
+    constexpr int stage = ROWS ? ROWS_A_BYTES + 3 * (N_TILE / 2) * BLOCK_K * 2 : KSUB * (BLOCK_M * BLOCK_K * 2 + (N_TILE / 2) * BLOCK_K * 2);
+    constexpr int smem = STAGES * stage + EPI_WARPS * 2 * EPI_BUF_BYTES + 1024 + 256;
     static_assert(smem <= 232448, "shared memory");
-    auto kernel = km_kernel<N_TILE, STAGES, EPI_WARPS, true, KSUB, 1>;
+    auto kernel = km_kernel<N_TILE, STAGES, EPI_WARPS, true, KSUB, 1, ROWS, 0>;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
@@ -806,18 +889,32 @@ static cudaError_t launch_km_pair(const TensorMap& a, const TensorMap& b, const 
     return cudaLaunchKernelEx(&cfg, kernel, *(const CUtensorMap*)&a, *(const CUtensorMap*)&b, *(const CUtensorMap*)&o, p);
 }
 
-cudaError_t run_km(const TensorMap& a, const TensorMap& b, const TensorMap* b_half, const TensorMap* out_map, const KmParams& p_in, int n_tile,
-                   cudaStream_t s) {
+cudaError_t run_km(const KmMaps& m, const KmParams& p_in, int n_tile, cudaStream_t s) {
     KmParams p = p_in;
     // the store through the output map covers whole 32-pixel boxes and clips only at the tensor's edge: it needs a dense
     // output (stride 1) and a sample range that ends where the tiles end or where the tensor ends
-    p.tma_out = out_map && p.os == 1 && p.ncls == 1 && (p.n_base + p.tiles_n * p.Nt <= p.N || p.N == p.Nfull) ? 1 : 0;
-    const TensorMap& o = p.tma_out ? *out_map : a;       // unused by the kernel without tma_out
-    const bool pair = b_half && n_tile == 256 && (p.tiles_w * p.tiles_h * p.tiles_n) % 2 == 0;
-    if (pair) return launch_km_pair<256, 6, 4, 1>(a, *b_half, o, p, s);
-    if (n_tile == 64) return launch_km<64, 3, 4, 1>(a, b, o, p, s);
-    if (n_tile == 128) return launch_km<128, 2, 4, 1>(a, b, o, p, s);
-    if (n_tile == 256) return launch_km<256, 4, 4, 1>(a, b, o, p, s);
+    p.tma_out = m.out && p.os == 1 && p.ncls == 1 && (p.n_base + p.tiles_n * p.Nt <= p.N || p.N == p.Nfull) ? 1 : 0;
+    const TensorMap& o = p.tma_out ? *m.out : *m.a;       // unused by the kernel without tma_out
+    const bool even = (p.tiles_w * p.tiles_h * p.tiles_n) % 2 == 0;
+    // rows mode: 3x3, stride 1, tiles that are whole rows of one image
+    bool rows = m.a_rows && p.ncls == 1 && p.ntaps == 9 && p.xs == 1 && p.os == 1 && p.tiles_w == 1 && p.Nt == 1;
+    if (rows) {
+        for (int i = 0; i < 9; ++i) p.rows_tap[i] = -1;
+        for (int t = 0; t < 9; ++t) {
+            const int dwi = p.dw[t] + 1, dhi = p.dh[t] + 1;
+            if (dwi < 0 || dwi > 2 || dhi < 0 || dhi > 2) { rows = false; break; }
+            p.rows_tap[dwi * 3 + dhi] = t;
+        }
+        for (int i = 0; i < 9; ++i) rows = rows && p.rows_tap[i] >= 0;
+    }
+    if (rows && n_tile == 64 && p.Cn == 64 && p.kchunks == 1) return launch_km<64, 3, 4, 1, true, 72>(*m.a_rows, *m.b, o, p, s);
+    if (rows && n_tile == 128 && p.kchunks >= 2 && m.b_half && even) return launch_km_pair<128, 4, 4, 1, true>(*m.a_rows, *m.b_half, o, p, s);
+    // measured on a B200: the narrow tiles run best with two CTAs per SM and short pipelines (3 x 24 KB, 2 x 32 KB stages);
+    // the 256-column tile as a CTA pair with six 32 KB stages; more sub-blocks per stage changed nothing
+    if (m.b_half && n_tile == 256 && even) return launch_km_pair<256, 6, 4, 1, false>(*m.a, *m.b_half, o, p, s);
+    if (n_tile == 64) return launch_km<64, 3, 4, 1, false, 0>(*m.a, *m.b, o, p, s);
+    if (n_tile == 128) return launch_km<128, 2, 4, 1, false, 0>(*m.a, *m.b, o, p, s);
+    if (n_tile == 256) return launch_km<256, 4, 4, 1, false, 0>(*m.a, *m.b, o, p, s);
     return cudaErrorInvalidValue;
 }
 

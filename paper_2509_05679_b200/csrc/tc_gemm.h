@@ -22,6 +22,7 @@ struct KmParams {
     int N, Hd, Wd;                               // extents of the tile domain (rows outside are not stored)
     int Nfull;                                   // samples in the whole output tensor (N is the end of this launch's group)
     int tma_out;                                 // set by run_km: the epilogue stores through the output tensor map
+    int rows_tap[9];                             // set by run_km (rows mode): tap index of (horizontal shift, vertical shift), [dw + 1][dh + 1]
     int n_base;                                  // first sample of the group of workers this launch covers (a multiple of Nt);
                                                  // tiles_n counts the group's tiles, N is the end of the group
     int Ho, Wo, Co, os;                          // output tensor [N,Ho,Wo,Co] and the output stride of a domain pixel
@@ -56,11 +57,16 @@ bool pixel_tile(int H, int W, int pixels, int* Wt, int* Ht, int* Nt);
 // inside a 128-pixel tile of Wt x Ht x Nt pixels.  C must be a multiple of 64.
 bool make_map_out(TensorMap* out, const void* base, int C, int W, int H, int N, int Wt, int Ht);
 
-// b_half: nullptr, or a map of the same matrix whose box holds n_tile / 2 rows: the kernel then runs as CTA pairs
-// (two SMs share one 256-row MMA and each loads half of B) when n_tile is 256 and the number of pixel tiles is even.
-// out_map: nullptr, or the output tensor's map from make_map_out: dense outputs are then written by TMA stores.
-cudaError_t run_km(const TensorMap& a, const TensorMap& b, const TensorMap* b_half, const TensorMap* out_map, const KmParams& p, int n_tile,
-                   cudaStream_t s);
+// Tensor maps of one run_km launch.
+//   a      : activation, box = 64 channels x one 128-pixel tile (make_map_4d)
+//   a_rows : nullptr, or the same tensor with a box of 64 channels x W x (Ht + 2) x 1 pixels: a 3x3 stride-1 layer whose
+//            tiles are whole rows of one image then fetches the activation once per horizontal shift ("rows mode")
+//   b      : weights, box = 64 x n_tile rows
+//   b_half : nullptr, or a map of the same matrix whose box holds n_tile / 2 rows: the kernel then runs as CTA pairs
+//            (two SMs share one 256-row MMA and each loads half of B) when the number of pixel tiles is even
+//   out    : nullptr, or the output tensor's map from make_map_out: dense outputs are then written by TMA stores
+struct KmMaps { const TensorMap* a; const TensorMap* a_rows; const TensorMap* b; const TensorMap* b_half; const TensorMap* out; };
+cudaError_t run_km(const KmMaps& m, const KmParams& p, int n_tile, cudaStream_t s);
 // accum: dw += the result (second and later groups of workers)
 cudaError_t run_wg(const TensorMap& x, const TensorMap& dy, const WgParams& p, int n_tile, int splits, float* dw, bool accum, cudaStream_t s);
 cudaError_t run_flip_transpose(const void* w, void* wt, int Co, int taps, int Ci, cudaStream_t s);
