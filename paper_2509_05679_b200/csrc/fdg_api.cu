@@ -71,6 +71,9 @@ struct Op {
     std::vector<char*> a_ptrs, dy_ptrs;                      // the buffers the A / dY maps below were built for
     std::vector<char*> y_ptrs, dx_ptrs;                      // where the forward output / the input gradient can be written
     std::vector<tc::TensorMap> fo, dox;                      // output maps of the forward / input-gradient kernel, per buffer
+    int wgr_variant, wgr_splits;                             // rows-mode weight gradient: kernel variant (0: not used) and splits
+    std::vector<tc::TensorMap> wxr;                          // x with a rows-mode box of 128-pixel steps (weight gradient)
+    tc::WgRowsParams kwr;
     std::vector<tc::TensorMap> far, dar;                     // rows-mode activation maps (3x3, stride 1, tiles of whole image rows); empty: not used
     std::vector<tc::TensorMap> fa, fb, da, db, wx, wdy;      // fwd A, fwd B (per weight slot), dgrad A, dgrad B, wgrad X, wgrad dY
     std::vector<tc::TensorMap> fbh, dbh;                     // fwd / dgrad B with half-height boxes (CTA-pair kernels); empty: not used
@@ -195,6 +198,11 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
             if (splits > ptiles) splits = ptiles;
             long pps = (ptiles + splits - 1) / splits;
             o.wg_splits = (int)((ptiles + pps - 1) / pps);
+            o.wgr_variant = (g.R == 3 && g.stride == 1) ? tc::wg_rows_variant(g.H, g.W, g.C, g.Co) : 0;
+            if (o.wgr_variant) {
+                tc::pixel_tile(g.Ho, g.Wo, 128, &wt, &ht, &nt);
+                o.wgr_splits = tc::wg_rows_splits(o.wgr_variant, g.C, g.Co, (long)(g.Ho / ht) * ((g.N + nt - 1) / nt));
+            }
         }
         m.ops.push_back(o);
         return "";
@@ -299,7 +307,7 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
             m.red_elems = std::max(m.red_elems, (size_t)ctx->n_workers * o.g.C * 2);
         }
         if (o.type == OP_CONV) {
-            if (o.tc) m.ws_elems = std::max(m.ws_elems, (size_t)o.wg_splits * o.g.R * o.g.R * o.g.C * o.g.Co);
+            if (o.tc) m.ws_elems = std::max(m.ws_elems, (size_t)std::max(o.wg_splits, o.wgr_variant ? o.wgr_splits : 0) * o.g.R * o.g.R * o.g.C * o.g.Co);
             if (o.stem) m.ws_elems = std::max(m.ws_elems, stem_wgrad_workspace_elems(o.g));
             m.ws_elems = std::max(m.ws_elems, wgrad_workspace_elems(o.g));
             m.scratch_elems = std::max(m.scratch_elems, (size_t)64 * o.g.Co);
@@ -412,6 +420,16 @@ bool tc_dgrad(fdg_ctx* c, Module& m, const Op& o, char* dy_base, char* dx_base, 
 bool tc_wgrad(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* dy_base, float* dw, const Win& wn, cudaStream_t s) {
     int ix = find_buf(o.a_ptrs, x_base), id = find_buf(o.dy_ptrs, dy_base);
     if (ix < 0 || id < 0) return false;
+    const ConvGeom& g = o.g;
+    if (o.wgr_variant && wn.n % o.kwr.Nt == 0) {
+        tc::WgRowsParams q = o.kwr;
+        q.partial = m.ws; q.err = c->tc_err; q.n_base = wn.n0; q.tiles_n = wn.n / q.Nt;
+        const long steps = (long)q.tiles_h * q.tiles_n;
+        const int splits = o.wgr_splits < steps ? o.wgr_splits : (int)steps;
+        double rows = (double)wn.n * g.Ho * g.Wo, R = (double)g.R * g.R * g.C;
+        Scope sc(KC_TC_WGRAD, 2.0 * rows * g.Co * R, 2.0 * ((double)wn.n * g.H * g.W * g.C + rows * g.Co) + 4.0 * R * g.Co, s);
+        return tc::run_wg_rows(o.wxr[ix], o.da[id], q, o.wgr_variant, splits, dw, !wn.first, s) == cudaSuccess;
+    }
     tc::WgParams p = o.kw;
     p.partial = m.ws; p.err = c->tc_err;
     p.n_base = wn.n0; p.tiles_n = (wn.n + p.Nt - 1) / p.Nt;
@@ -419,7 +437,6 @@ bool tc_wgrad(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* dy_base, f
     int splits = o.wg_splits < p.ptiles ? o.wg_splits : p.ptiles;
     p.ptiles_per_split = (p.ptiles + splits - 1) / splits;
     splits = (p.ptiles + p.ptiles_per_split - 1) / p.ptiles_per_split;
-    const ConvGeom& g = o.g;
     double rows = (double)wn.n * g.Ho * g.Wo, R = (double)g.R * g.R * g.C;
     Scope sc(KC_TC_WGRAD, 2.0 * rows * g.Co * R, 2.0 * ((double)wn.n * g.H * g.W * g.C + rows * g.Co) + 4.0 * R * g.Co, s);
     return tc::run_wg(o.wx[ix], o.wdy[id], p, o.n_tile_w, splits, dw, !wn.first, s) == cudaSuccess;
@@ -650,6 +667,14 @@ bool build_tc_plans(fdg_ctx* c) {
             for (size_t i = 0; i < o.a_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.wx[i], o.a_ptrs[i], g.C, g.W, g.H, g.N, 64, wt, ht, nt, g.stride);
             o.wdy.resize(o.dy_ptrs.size());
             for (size_t i = 0; i < o.dy_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.wdy[i], o.dy_ptrs[i], g.Co, g.Wo, g.Ho, g.N, 64, wt, ht, nt, 1);
+            if (o.wgr_variant) {
+                // contraction steps of 128 pixels: dy through the input-gradient kernel's activation map (o.da), x with two extra rows
+                tc::pixel_tile(g.Ho, g.Wo, 128, &wt, &ht, &nt);
+                tc::WgRowsParams& q = o.kwr; q = tc::WgRowsParams{};
+                q.W = g.W; q.Ht = ht; q.Nt = nt; q.tiles_h = g.Ho / ht; q.tiles_n = (g.N + nt - 1) / nt; q.C = g.C; q.Co = g.Co;
+                o.wxr.resize(o.a_ptrs.size());
+                for (size_t i = 0; i < o.a_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.wxr[i], o.a_ptrs[i], g.C, g.W, g.H, g.N, 64, g.W, ht + 2, nt, 1);
+            }
             if (!ok) return false;
             c->any_tc = true;
         }

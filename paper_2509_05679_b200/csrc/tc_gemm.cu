@@ -743,6 +743,155 @@ wg_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUten
     if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, N_TILE < 32 ? 32 : N_TILE); }
 }
 
+// ------------------------------------------------------------------------------------------ weight gradient, rows mode
+// 3x3, stride 1, pad 1, with a contraction step of 128 pixels = whole rows of one or two images (W >= 8).  A stage holds
+// NX sub-tiles of x, each the step's rows plus one above and one below for one (horizontal shift, 64-channel chunk),
+// and the step's dy.  The three vertical taps of a sub-tile are views that start 0, 1 or 2 image rows into it, so one
+// fetch of x serves three taps, and dy is fetched once for all 3 * NX (tap, chunk) row blocks the CTA accumulates:
+// row blocks 2g and 2g+1 form the two 64-row halves of accumulator g (the descriptor's leading-dimension offset is
+// the distance between the two views).  NX = 3: the three shifts of a 64-channel input (all nine taps in one CTA);
+// NX = 2: one shift, two chunks (blockIdx.x = shift + 3 * chunk pair).
+struct Wg2Params {
+    int W, Ht, Nt, tiles_h, tiles_n;          // contraction step = W x Ht x Nt = 128 pixels
+    int ptiles, ptiles_per_split, n_base;
+    int kchunks, row_blocks, Co;
+    float* partial;                           // [splits][row_blocks * 64][Co]
+    int* err;
+};
+template <int N_TILE, int NX, int XSUB_KB, int STAGES>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+wg2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmDY, Wg2Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align1024(smem_raw);
+    constexpr int XSUB = XSUB_KB * 1024, DYBOX = 128 * 128, NB = N_TILE / 64;
+    constexpr int STAGE_BYTES = NX * XSUB + NB * DYBOX;
+    constexpr int RB = 3 * NX, G = (RB + 1) / 2;
+    constexpr uint32_t TMEM_COLS = 512;
+    static_assert(G * N_TILE <= 512, "tensor memory");
+    uint64_t* full = (uint64_t*)(smem + STAGES * STAGE_BYTES);
+    uint64_t* empty = full + STAGES;
+    uint64_t* accum_bar = empty + STAGES;
+    uint32_t* tmem_slot = (uint32_t*)(accum_bar + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int dw_fixed = NX == 3 ? 0 : (int)blockIdx.x % 3, chunk0 = NX == 3 ? 0 : 2 * ((int)blockIdx.x / 3);
+    const int co0 = blockIdx.y * N_TILE;
+    const int pt_begin = blockIdx.z * p.ptiles_per_split;
+    const int pt_end = min(p.ptiles, pt_begin + p.ptiles_per_split);
+    const int num_kb = pt_end - pt_begin;
+
+    if (threadIdx.x == 0) {
+        tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmDY);
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        mbar_init(accum_bar, 1);
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t xsub_bytes = (uint32_t)(p.Ht + 2) * p.W * p.Nt * 128u;
+
+    if (warp == 0) {
+        const uint32_t smem0 = smem_u32(smem), full0 = smem_u32(full), empty0 = smem_u32(empty);
+        uint32_t st = 0, ph = 1, dst = smem0, fb = full0, eb = empty0;
+        int th = pt_begin % p.tiles_h, tn = pt_begin / p.tiles_h;
+        for (int kb = 0; kb < num_kb; ++kb) {
+            if (!mbar_wait_a(eb, ph, p.err, 4)) break;
+            const int h0 = th * p.Ht, n0 = p.n_base + tn * p.Nt;
+            if (elect_one()) {
+                mbar_expect_tx_a(fb, NX * xsub_bytes + NB * DYBOX);
+#pragma unroll
+                for (int sx = 0; sx < NX; ++sx)
+                    tma_load_4d_a(dst + sx * XSUB, &tmX, fb, (NX == 3 ? 0 : chunk0 + sx) * 64, (NX == 3 ? sx : dw_fixed) - 1, h0 - 1, n0);
+#pragma unroll
+                for (int j = 0; j < NB; ++j) tma_load_4d_a(dst + NX * XSUB + j * DYBOX, &tmDY, fb, co0 + j * 64, 0, h0, n0);
+            }
+            __syncwarp();
+            if (++th == p.tiles_h) { th = 0; ++tn; }
+            if (++st == STAGES) { st = 0; ph ^= 1u; dst = smem0; fb = full0; eb = empty0; }
+            else { dst += STAGE_BYTES; fb += 8; eb += 8; }
+        }
+    } else if (warp == 1) {
+        const uint32_t idesc = make_idesc(BLOCK_M, N_TILE, 1, 1);
+        const uint32_t d_hi = (uint32_t)(make_desc(0, 0, 1024) >> 32);
+        const uint32_t row16 = (uint32_t)p.W * 128u >> 4;                   // one image row, in descriptor address units
+        // low descriptor word of accumulator g's x operand, without the stage address: view of row block 2g, and the
+        // distance to the view of row block 2g+1 as the leading-dimension offset
+        uint32_t xlo[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            const int ra = 2 * g, rb = 2 * g + 1 < RB ? 2 * g + 1 : 2 * g;
+            const uint32_t oa = (uint32_t)(ra / 3) * (XSUB >> 4) + (uint32_t)(ra % 3) * row16;
+            const uint32_t ob = (uint32_t)(rb / 3) * (XSUB >> 4) + (uint32_t)(rb % 3) * row16;
+            xlo[g] = oa | ((ob - oa) << 16);
+        }
+        const uint32_t dylo = (uint32_t)((NX * XSUB) >> 4) | ((uint32_t)(DYBOX >> 4) << 16);
+        // x rows of the step's 16-pixel slices (the sub-tile keeps two extra rows per image)
+        uint32_t koff[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int pix = 16 * k, ni = pix / (p.W * p.Ht), hi = (pix / p.W) % p.Ht, wi = pix % p.W;
+            koff[k] = (uint32_t)((ni * (p.Ht + 2) + hi) * p.W + wi) * 8u;
+        }
+        const uint32_t a16_0 = smem_u32(smem) >> 4, full0 = smem_u32(full), empty0 = smem_u32(empty);
+        uint32_t st = 0, ph = 0, a16 = a16_0, fb = full0, eb = empty0, acc = 0;
+        for (int kb = 0; kb < num_kb; ++kb) {
+            if (!mbar_wait_a(fb, ph, p.err, 5)) break;
+            tc_fence_after();
+            if (elect_one()) {
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+                                     "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+                                     ::"r"(tmem_base + g * N_TILE), "r"(xlo[g] + a16 + koff[k]), "r"(dylo + a16 + (uint32_t)k * 128u), "r"(d_hi), "r"(idesc),
+                                       "r"(k == 0 ? acc : 1u) : "memory");
+                    }
+                }
+                umma_commit_a<false>(eb);
+                if (kb == num_kb - 1) umma_commit(accum_bar);
+            }
+            __syncwarp();
+            acc = 1;
+            if (++st == STAGES) { st = 0; ph ^= 1u; a16 = a16_0; fb = full0; eb = empty0; }
+            else { a16 += STAGE_BYTES >> 4; fb += 8; eb += 8; }
+        }
+    } else {
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const bool ok = num_kb > 0 ? mbar_wait_sleep(accum_bar, 0, p.err, 6) : true;
+        tc_fence_after();
+#pragma unroll 1
+        for (int g = 0; g < G; ++g) {
+            const int rb = 2 * g + (row >> 6);                       // local row block -> (sub-tile, vertical tap)
+            const bool valid = ok && rb < RB;
+            const int sx = rb / 3, dhi = rb % 3;
+            const int dwi = NX == 3 ? sx : dw_fixed, chunk = NX == 3 ? 0 : chunk0 + sx;
+            const int grb = (dhi * 3 + dwi) * p.kchunks + chunk;     // row block of the whole matrix: (tap, chunk)
+            float* out = p.partial + (((size_t)blockIdx.z * p.row_blocks + grb) * 64 + (row & 63)) * p.Co + co0;
+#pragma unroll 1
+            for (int c = 0; c < N_TILE; c += 32) {
+                uint32_t v[32];
+                if (num_kb > 0) tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + g * N_TILE + c, v);
+                else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0u;
+                }
+                if (!valid) continue;
+                uint4* o4 = (uint4*)(out + c);
+#pragma unroll
+                for (int gq = 0; gq < 8; ++gq) o4[gq] = make_uint4(v[4 * gq], v[4 * gq + 1], v[4 * gq + 2], v[4 * gq + 3]);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, TMEM_COLS); }
+}
+
 // dW[co][tap][ci] = sum_z partial[z][(tap, cc)][ci % 64][co], z ascending.  32x32 transposing tiles; a thread owns
 // one (row, column) per pass and keeps eight independent loads in flight along z.
 __global__ void __launch_bounds__(1024) wg_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dw, int splits, int row_blocks, int Co,
@@ -941,6 +1090,52 @@ cudaError_t run_wg(const TensorMap& x, const TensorMap& dy, const WgParams& p, i
     if (e != cudaSuccess) return e;
     dim3 rgrid(p.row_blocks * 2, p.Co / 32), rblk(32, 32);
     wg_reduce_kernel<<<rgrid, rblk, 0, s>>>(p.partial, dw, splits, p.row_blocks, p.Co, accum);
+    return cudaGetLastError();
+}
+
+template <int N_TILE, int NX, int XSUB_KB, int STAGES>
+static cudaError_t launch_wg2(const TensorMap& x, const TensorMap& dy, const Wg2Params& p, dim3 grid, cudaStream_t s) {
+    constexpr int smem = STAGES * (NX * XSUB_KB * 1024 + (N_TILE / 64) * 128 * 128) + 1024 + 256;
+    static_assert(smem <= 232448, "shared memory");
+    static bool attr = false;
+    if (!attr) {
+        cudaError_t e = cudaFuncSetAttribute(wg2_kernel<N_TILE, NX, XSUB_KB, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        attr = true;
+    }
+    wg2_kernel<N_TILE, NX, XSUB_KB, STAGES><<<grid, NUM_THREADS, smem, s>>>(*(const CUtensorMap*)&x, *(const CUtensorMap*)&dy, p);
+    return cudaGetLastError();
+}
+
+int wg_rows_variant(int H, int W, int C, int Co) {
+    if (C == 64 && Co % 64 == 0 && W == 32 && H % 4 == 0) return 1;                               // nine taps of a 64-channel input, 64 columns
+    if (C % 128 == 0 && Co % 128 == 0 && ((W == 16 && H % 8 == 0) || (W == 8 && H == 8))) return 2;  // one shift, two chunks, 128 columns
+    return 0;
+}
+
+int wg_rows_splits(int variant, int C, int Co, long steps) {
+    const int tiles = variant == 1 ? Co / 64 : 3 * (C / 128) * (Co / 128);
+    long s = sm_count() / tiles;
+    if (s < 1) s = 1;
+    if (s > steps) s = steps;
+    const long per = (steps + s - 1) / s;
+    return (int)((steps + per - 1) / per);
+}
+
+cudaError_t run_wg_rows(const TensorMap& x_rows, const TensorMap& dy128, const WgRowsParams& q, int variant, int splits, float* dw, bool accum,
+                        cudaStream_t s) {
+    Wg2Params p{};
+    p.W = q.W; p.Ht = q.Ht; p.Nt = q.Nt; p.tiles_h = q.tiles_h; p.tiles_n = q.tiles_n; p.n_base = q.n_base;
+    p.ptiles = q.tiles_h * q.tiles_n; p.ptiles_per_split = (p.ptiles + splits - 1) / splits;
+    p.kchunks = q.C / 64; p.row_blocks = 9 * p.kchunks; p.Co = q.Co; p.partial = q.partial; p.err = q.err;
+    const int z = (p.ptiles + p.ptiles_per_split - 1) / p.ptiles_per_split;
+    cudaError_t e;
+    if (variant == 1) e = launch_wg2<64, 3, 24, 2>(x_rows, dy128, p, dim3(1, q.Co / 64, z), s);
+    else if (variant == 2) e = launch_wg2<128, 2, 20, 3>(x_rows, dy128, p, dim3(3 * (q.C / 128), q.Co / 128, z), s);
+    else return cudaErrorInvalidValue;
+    if (e != cudaSuccess) return e;
+    dim3 rgrid(p.row_blocks * 2, p.Co / 32), rblk(32, 32);
+    wg_reduce_kernel<<<rgrid, rblk, 0, s>>>(p.partial, dw, z, p.row_blocks, p.Co, accum);
     return cudaGetLastError();
 }
 

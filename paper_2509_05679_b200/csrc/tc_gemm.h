@@ -69,6 +69,22 @@ struct KmMaps { const TensorMap* a; const TensorMap* a_rows; const TensorMap* b;
 cudaError_t run_km(const KmMaps& m, const KmParams& p, int n_tile, cudaStream_t s);
 // accum: dw += the result (second and later groups of workers)
 cudaError_t run_wg(const TensorMap& x, const TensorMap& dy, const WgParams& p, int n_tile, int splits, float* dw, bool accum, cudaStream_t s);
+// Weight gradient of a 3x3, stride-1, pad-1 layer in rows mode (x is fetched once per horizontal shift and 64-channel
+// chunk, dy once per contraction step of 128 pixels).
+//   wg_rows_variant: 0 = not supported for this geometry (use run_wg), else the kernel variant
+//   wg_rows_splits : CTAs along the contraction for `steps` = 128-pixel steps; the workspace holds that many partial matrices
+//   x_rows : x with a box of 64 channels x W x (Ht + 2) x Nt pixels, dy128 : dy with a box of 64 channels x W x Ht x Nt,
+//            W x Ht x Nt = 128 pixels
+struct WgRowsParams {
+    int W, Ht, Nt, tiles_h, tiles_n, n_base;
+    int C, Co;
+    float* partial;                              // [splits][9 * C][Co]
+    int* err;
+};
+int wg_rows_variant(int H, int W, int C, int Co);
+int wg_rows_splits(int variant, int C, int Co, long steps);
+cudaError_t run_wg_rows(const TensorMap& x_rows, const TensorMap& dy128, const WgRowsParams& p, int variant, int splits, float* dw, bool accum,
+                        cudaStream_t s);
 cudaError_t run_flip_transpose(const void* w, void* wt, int Co, int taps, int Ci, cudaStream_t s);
 
 }  // namespace tc
