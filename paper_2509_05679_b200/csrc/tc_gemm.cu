@@ -356,6 +356,10 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             }
             __syncwarp();
         }
+        int ktab[9];                                   // rows mode: weight column of (shift, vertical tap), chunk 0
+#pragma unroll
+        for (int i = 0; i < 9; ++i) ktab[i] = ROWS ? p.koff[p.rows_tap[i]] : 0;
+        const uint32_t a_bytes = ROWS ? (uint32_t)(p.Ht + 2) * p.Wt * 128u : 0u;
         for (int tile = walker; tile < total && ok; tile += walkers) {
             const int cls = tile / per_cls, tl = tile - cls * per_cls;
             int tm = tl / tiles_c; const int co0 = (tl - tm * tiles_c) * N_TILE;
@@ -365,8 +369,8 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             const int w0 = tw * p.Wt * p.xs, h0 = th * p.Ht * p.xs, n0 = p.n_base + tn * p.Nt;
             const int brow = co0 + (PAIR ? (int)rank * B_ROWS : 0);
             if (ROWS) {
-                const uint32_t a_bytes = (uint32_t)(p.Ht + 2) * p.Wt * 128u;
                 for (int kc = 0; kc < p.kchunks && ok; ++kc) {
+#pragma unroll
                     for (int dwi = 0; dwi < 3; ++dwi) {
                         if (!mbar_wait_a(eb, ph, p.err, 1)) { ok = false; break; }
                         if (elect_one()) {
@@ -376,7 +380,7 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                             if (!RESIDENT) {
 #pragma unroll
                                 for (int dhi = 0; dhi < 3; ++dhi) {
-                                    const int kcol = p.koff[p.rows_tap[dwi * 3 + dhi]] + kc * BLOCK_K;
+                                    const int kcol = ktab[dwi * 3 + dhi] + kc * BLOCK_K;
                                     if (PAIR) tma_load_2d_pair(dst + ROWS_A_BYTES + dhi * B_BYTES, &tmB, fb, kcol, brow);
                                     else tma_load_2d_a(dst + ROWS_A_BYTES + dhi * B_BYTES, &tmB, fb, kcol, brow);
                                 }
@@ -432,6 +436,10 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             uint32_t st = 0, ph = 0, a16 = a16_0, fb = full0, eb = empty0;
             int ti = 0;
             bool ok = true;
+            const uint32_t row16 = ROWS ? (uint32_t)p.Wt * 128u >> 4 : 0u;      // one image row of a rows-mode stage, in descriptor address units
+            uint32_t btab[9];                                                  // resident weights: descriptor word of (shift, vertical tap), chunk 0
+#pragma unroll
+            for (int i = 0; i < 9; ++i) btab[i] = RESIDENT ? d_lo + (smem_u32(wres) >> 4) + (uint32_t)(p.rows_tap[i] * p.kchunks * (B_BYTES >> 4)) : 0u;
             for (int tile = walker; tile < total && ok; tile += walkers, ++ti) {
                 const int buf = ti & 1, use = ti >> 1;
                 const int cls = tile / per_cls;
@@ -442,30 +450,31 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 uint32_t acc = 0;
                 if (ROWS) {
                     if (RESIDENT && ti == 0 && !mbar_wait(wres_bar, 0, p.err, 8)) { ok = false; break; }
-                    const uint32_t row16 = (uint32_t)p.Wt * 128u >> 4;          // one image row of the stage, in descriptor address units
-                    const uint32_t wres16 = smem_u32(wres) >> 4;
-                    const int nst = 3 * p.kchunks;
-                    for (int sidx = 0; sidx < nst; ++sidx) {
-                        if (!mbar_wait_a(fb, ph, p.err, 2)) { ok = false; break; }
-                        tc_fence_after();
-                        const uint32_t a_lo = d_lo + a16;
-                        const int kc = sidx / 3, dwi = sidx - kc * 3;
-                        if (elect_one()) {
+                    // one stage = one (chunk, horizontal shift); the loop over shifts is unrolled and every table
+                    // look-up happens before the tile loop, because the tensor pipe drains while this warp computes
+                    for (int kc = 0; kc < p.kchunks && ok; ++kc) {
 #pragma unroll
-                            for (int dhi = 0; dhi < 3; ++dhi) {
-                                const uint32_t b_lo = RESIDENT ? d_lo + wres16 + (uint32_t)((p.rows_tap[dwi * 3 + dhi] * p.kchunks + kc) * (B_BYTES >> 4))
-                                                               : a_lo + (uint32_t)((ROWS_A_BYTES + dhi * B_BYTES) >> 4);
+                        for (int dwi = 0; dwi < 3; ++dwi) {
+                            if (!mbar_wait_a(fb, ph, p.err, 2)) { ok = false; break; }
+                            tc_fence_after();
+                            const uint32_t a_lo = d_lo + a16;
+                            if (elect_one()) {
 #pragma unroll
-                                for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                                    umma_bf16_w<PAIR>(d, a_lo + dhi * row16 + 2 * k, b_lo + 2 * k, d_hi, idesc, (dhi == 0 && k == 0) ? acc : 1u);
+                                for (int dhi = 0; dhi < 3; ++dhi) {
+                                    const uint32_t b_lo = RESIDENT ? btab[dwi * 3 + dhi] + (uint32_t)kc * (B_BYTES >> 4)
+                                                                   : a_lo + (uint32_t)((ROWS_A_BYTES + dhi * B_BYTES) >> 4);
+#pragma unroll
+                                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                                        umma_bf16_w<PAIR>(d, a_lo + dhi * row16 + 2 * k, b_lo + 2 * k, d_hi, idesc, (dhi == 0 && k == 0) ? acc : 1u);
+                                }
+                                umma_commit_a<PAIR>(eb);
+                                if (dwi == 2 && kc == p.kchunks - 1) umma_commit_a<PAIR>(smem_u32(&tmem_full[buf]));
                             }
-                            umma_commit_a<PAIR>(eb);
-                            if (sidx == nst - 1) umma_commit_a<PAIR>(smem_u32(&tmem_full[buf]));
+                            __syncwarp();
+                            acc = 1;
+                            if (++st == STAGES) { st = 0; ph ^= 1u; a16 = a16_0; fb = full0; eb = empty0; }
+                            else { a16 += STAGE_BYTES >> 4; fb += 8; eb += 8; }
                         }
-                        __syncwarp();
-                        acc = 1;
-                        if (++st == STAGES) { st = 0; ph ^= 1u; a16 = a16_0; fb = full0; eb = empty0; }
-                        else { a16 += STAGE_BYTES >> 4; fb += 8; eb += 8; }
                     }
                     continue;
                 }
