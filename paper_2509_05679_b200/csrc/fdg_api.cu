@@ -71,6 +71,8 @@ struct Op {
     std::vector<char*> a_ptrs, dy_ptrs;                      // the buffers the A / dY maps below were built for
     std::vector<char*> y_ptrs, dx_ptrs;                      // where the forward output / the input gradient can be written
     std::vector<tc::TensorMap> fo, dox;                      // output maps of the forward / input-gradient kernel, per buffer
+    bool stem_tc;                                            // first layer: weight gradient on the tensor cores
+    std::vector<tc::TensorMap> sxr, sdy;                     // its raw-row map of x per input buffer, its dy map
     int wgr_variant, wgr_splits;                             // rows-mode weight gradient: kernel variant (0: not used) and splits
     std::vector<tc::TensorMap> wxr;                          // x with a rows-mode box of 128-pixel steps (weight gradient)
     tc::WgRowsParams kwr;
@@ -181,6 +183,7 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
         o.out = add_tensor(g.Ho, g.Wo, cout);
         std::snprintf(o.shape, sizeof o.shape, "%dx%d %d->%d k%d s%d", g.H, g.W, g.C, g.Co, g.R, g.stride);
         o.stem = ctx->kernel_path != 1 && kind == FDG_CONV3X3 && stem_supported(ctx->dt, g);
+        o.stem_tc = o.stem && tc::stem_wg_supported(g.H, g.W, g.C, g.Co) && tc::init();
         // tensor-core eligibility
         int wt, ht, nt;
         o.tc = ctx->dt == 1 && ctx->kernel_path != 1 && g.C % 64 == 0 && g.Co % 64 == 0 &&
@@ -309,6 +312,7 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
         if (o.type == OP_CONV) {
             if (o.tc) m.ws_elems = std::max(m.ws_elems, (size_t)std::max(o.wg_splits, o.wgr_variant ? o.wgr_splits : 0) * o.g.R * o.g.R * o.g.C * o.g.Co);
             if (o.stem) m.ws_elems = std::max(m.ws_elems, stem_wgrad_workspace_elems(o.g));
+            if (o.stem_tc) m.ws_elems = std::max(m.ws_elems, tc::stem_wg_workspace_elems(o.g.Co, (long)o.g.N * o.g.H));
             m.ws_elems = std::max(m.ws_elems, wgrad_workspace_elems(o.g));
             m.scratch_elems = std::max(m.scratch_elems, (size_t)64 * o.g.Co);
         }
@@ -442,6 +446,17 @@ bool tc_wgrad(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* dy_base, f
     return tc::run_wg(o.wx[ix], o.wdy[id], p, o.n_tile_w, splits, dw, !wn.first, s) == cudaSuccess;
 }
 
+// first-layer weight gradient on the tensor cores (whole batch only)
+bool tc_stem_wgrad(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* dy_base, float* dw, const Win& wn, cudaStream_t s) {
+    if (!o.stem_tc || wn.n != c->M) return false;
+    const int ix = find_buf(o.a_ptrs, x_base), id = find_buf(o.dy_ptrs, dy_base);
+    if (ix < 0 || id < 0) return false;
+    const ConvGeom& g = o.g;
+    const double pix = (double)g.N * g.H * g.W;
+    Scope sc(KC_FMA_WGRAD, 2.0 * pix * g.Co * 9 * g.C, 2.0 * pix * (g.C + g.Co), s);
+    return tc::run_stem_wg(o.sxr[ix], o.sdy[id], g.H, g.W, g.N, g.Co, m.ws, dw, false, c->tc_err, s) == cudaSuccess;
+}
+
 // byte offset of the group's first sample inside a tensor of the module
 size_t row_off(const fdg_ctx* c, const TensorDesc& d, const Win& wn) {
     return (size_t)wn.n0 * d.elems() * (d.loc == LOC_LOGITS ? sizeof(float) : (size_t)c->esz);
@@ -526,7 +541,8 @@ void backward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int64_t
                 ConvGeom g = o.g; g.N = wn.n;
                 if (o.relu) relu_backward(dt, T(o.out), gout, gout, n_out, false, s);       // in place: dZ = dA * (A > 0)
                 profile_detail(o.shape);
-                if (o.stem) stem_wgrad(T(o.in), gout, m.grad + o.w_off, m.ws, g, acc_p, s);
+                if (o.stem && tc_stem_wgrad(c, m, o, P.tensor(o.in), grad_ptr(c, kk, o.out, t), m.grad + o.w_off, wn, s)) {}
+                else if (o.stem) stem_wgrad(T(o.in), gout, m.grad + o.w_off, m.ws, g, acc_p, s);
                 else if (!(o.tc && tc_wgrad(c, m, o, P.tensor(o.in), grad_ptr(c, kk, o.out, t), m.grad + o.w_off, wn, s)))
                     conv_wgrad(dt, T(o.in), gout, m.grad + o.w_off, m.ws, g, acc_p, s);
                 if (o.bias) bias_grad(dt, gout, m.grad + m.n_big + o.b_off, m.scratch, (long)g.N * g.Ho * g.Wo, g.Co, acc_p, s);
@@ -570,6 +586,24 @@ bool build_tc_plans(fdg_ctx* c) {
     for (int kk = 0; kk < c->K; ++kk) {
         Module& m = c->mod[kk];
         for (Op& o : m.ops) {
+            if (o.type == OP_CONV && o.stem_tc) {
+                const ConvGeom& g = o.g;
+                const TensorDesc& ti = m.t[o.in];
+                const TensorDesc& to = m.t[o.out];
+                if (ti.loc == LOC_IN) for (int i = 0; i < m.in_depth; ++i) o.a_ptrs.push_back(m.in_ring + (size_t)i * m.in_slot_bytes);
+                else for (int i = 0; i < m.D; ++i) o.a_ptrs.push_back(m.stash + (size_t)i * m.stash_slot_bytes + ti.off);
+                if (to.own_grad) o.dy_ptrs.push_back(m.gradpool + to.goff);
+                else if (to.loc == LOC_NEXT) { Module& n = c->mod[kk + 1]; for (int i = 0; i < 2; ++i) o.dy_ptrs.push_back(n.d2 + (size_t)i * n.in_slot_bytes); }
+                int wt, ht, nt;
+                tc::pixel_tile(g.Ho, g.Wo, 128, &wt, &ht, &nt);
+                bool ok = true;
+                o.sxr.resize(o.a_ptrs.size()); o.sdy.resize(o.dy_ptrs.size());
+                for (size_t i = 0; i < o.a_ptrs.size(); ++i) ok = ok && tc::make_map_raw_rows(&o.sxr[i], o.a_ptrs[i], g.C, g.W, g.H, g.N, ht + 2);
+                for (size_t i = 0; i < o.dy_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.sdy[i], o.dy_ptrs[i], g.Co, g.Wo, g.Ho, g.N, 64, wt, ht, nt, 1);
+                if (!ok || o.dy_ptrs.empty()) { o.stem_tc = false; continue; }
+                c->any_tc = true;
+                continue;
+            }
             if (o.type != OP_CONV || !o.tc) continue;
             const ConvGeom& g = o.g;
             const TensorDesc& ti = m.t[o.in];

@@ -901,6 +901,172 @@ wg2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, TMEM_COLS); }
 }
 
+// ------------------------------------------------------------------------------------------ first layer, weight gradient
+// 3x3, stride 1, pad 1, 3 input channels (K = 27 of the weight matrix's columns).  The 27 columns of the im2col
+// matrix are built in shared memory: the producer fetches the step's image rows (plus one above and below) as raw
+// rows of W * 3 elements, four builder warps write one 128-byte line per pixel, [pixel][k] with k = (row tap, column tap,
+// channel), zero beyond 27, in the 128-byte-swizzled layout the MMA reads (MN-major: M = k, contraction = pixels).
+// D[k][c_out] accumulates over all steps of the CTA in tensor memory; rows 64..127 of the accumulator repeat rows 0..63
+// (leading-dimension offset 0) and are dropped.  Partials per CTA, reduced in a fixed order by stem_wg_reduce_kernel.
+struct StemWgParams {
+    int W, Ht, tiles_h;                 // contraction step = W x Ht = 128 pixels of one image
+    int steps, steps_per_cta;           // steps = N * tiles_h
+    float* partial;                     // [Co / 64][CTAs][64 k][64 c_out]
+    int* err;
+};
+constexpr int STEM_RAW_BYTES = 2048;    // room for (Ht + 2) raw rows of W * 3 bf16
+template <int STAGES>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+stem_wg_kernel(const __grid_constant__ CUtensorMap tmRaw, const __grid_constant__ CUtensorMap tmDY, StemWgParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align1024(smem_raw);
+    constexpr int TILE = 128 * 128;                                  // im2col tile and dy tile: 128 pixels x 128 bytes
+    uint8_t* im = smem;                                              // [STAGES][TILE]
+    uint8_t* dyt = smem + STAGES * TILE;                             // [STAGES][TILE]
+    uint8_t* raw = smem + 2 * STAGES * TILE;                         // [STAGES][STEM_RAW_BYTES]
+    uint64_t* tma_full = (uint64_t*)(raw + STAGES * STEM_RAW_BYTES);
+    uint64_t* im_full = tma_full + STAGES;
+    uint64_t* empty = im_full + STAGES;
+    uint64_t* accum_bar = empty + STAGES;
+    uint32_t* tmem_slot = (uint32_t*)(accum_bar + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int co0 = blockIdx.y * 64;
+    const int s_begin = blockIdx.x * p.steps_per_cta;
+    const int s_end = min(p.steps, s_begin + p.steps_per_cta);
+    const int num_kb = s_end > s_begin ? s_end - s_begin : 0;
+    const uint32_t raw_bytes = (uint32_t)(p.Ht + 2) * p.W * 6u;
+
+    if (threadIdx.x == 0) {
+        tma_prefetch_desc(&tmRaw); tma_prefetch_desc(&tmDY);
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&tma_full[s], 1); mbar_init(&im_full[s], 4); mbar_init(&empty[s], 1); }
+        mbar_init(accum_bar, 1);
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, 64);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        uint32_t st = 0, ph = 1;
+        int th = s_begin % p.tiles_h, n = s_begin / p.tiles_h;
+        for (int kb = 0; kb < num_kb; ++kb) {
+            if (!mbar_wait(&empty[st], ph, p.err, 11)) break;
+            if (elect_one()) {
+                const uint32_t bar = smem_u32(&tma_full[st]);
+                mbar_expect_tx_a(bar, raw_bytes + TILE);
+                asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+                             ::"r"(smem_u32(raw + st * STEM_RAW_BYTES)), "l"(&tmRaw), "r"(bar), "r"(0), "r"(th * p.Ht - 1), "r"(n) : "memory");
+                tma_load_4d_a(smem_u32(dyt + st * TILE), &tmDY, bar, co0, 0, th * p.Ht, n);
+            }
+            __syncwarp();
+            if (++th == p.tiles_h) { th = 0; ++n; }
+            if (++st == STAGES) { st = 0; ph ^= 1u; }
+        }
+    } else if (warp == 1) {
+        const uint32_t idesc = make_idesc(BLOCK_M, 64, 1, 1);
+        const uint64_t dA = make_desc(0, 0, 1024), dB = make_desc(0, TILE, 1024);
+        const uint32_t d_hi = (uint32_t)(dA >> 32), a_lo0 = (uint32_t)dA, b_lo0 = (uint32_t)dB;
+        uint32_t st = 0, ph = 0, acc = 0;
+        for (int kb = 0; kb < num_kb; ++kb) {
+            if (!mbar_wait(&tma_full[st], ph, p.err, 12)) break;      // dy has landed
+            if (!mbar_wait(&im_full[st], ph, p.err, 13)) break;       // the im2col lines are written
+            tc_fence_after();
+            const uint32_t a_lo = a_lo0 + (smem_u32(im + st * TILE) >> 4), b_lo = b_lo0 + (smem_u32(dyt + st * TILE) >> 4);
+            if (elect_one()) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k)               // 16 pixels = 16 lines of 128 bytes per MMA
+                    umma_bf16_w<false>(tmem_base, a_lo + k * 128, b_lo + k * 128, d_hi, idesc, k == 0 ? acc : 1u);
+                umma_commit(&empty[st]);
+                if (kb == num_kb - 1) umma_commit(accum_bar);
+            }
+            __syncwarp();
+            acc = 1;
+            if (++st == STAGES) { st = 0; ph ^= 1u; }
+        }
+    } else {
+        // ---- builders: thread = one pixel of the step
+        const int pix = (warp - 2) * 32 + lane;
+        const int r = pix / p.W, c = pix - r * p.W;
+        const bool left = c > 0, right = c < p.W - 1;
+        const uint32_t line = (uint32_t)pix * 128u, swz = (uint32_t)(pix & 7);
+        uint32_t st = 0, ph = 0;
+        bool ok = true;
+        // columns 32..63 of every line are never written below: clear them once (their accumulator rows are dropped)
+        for (int s2 = 0; s2 < STAGES; ++s2)
+#pragma unroll
+            for (int ch = 4; ch < 8; ++ch)
+                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(smem_u32(im + s2 * TILE) + line + (((uint32_t)ch ^ swz) << 4)), "r"(0u) : "memory");
+        for (int kb = 0; kb < num_kb && ok; ++kb) {
+            ok = mbar_wait(&tma_full[st], ph, p.err, 14);
+            const uint32_t rb = smem_u32(raw + st * STEM_RAW_BYTES) + (uint32_t)(r * p.W + c - 1) * 6u;
+            uint32_t h[28];
+#pragma unroll
+            for (int dr = 0; dr < 3; ++dr) {
+#pragma unroll
+                for (int j = 0; j < 9; ++j) {
+                    uint32_t v = 0;
+                    const bool in = j < 3 ? left : (j < 6 ? true : right);
+                    if (in) { uint16_t t; asm volatile("ld.shared.u16 %0, [%1];" : "=h"(t) : "r"(rb + (uint32_t)(dr * p.W * 6 + 2 * j)) : "memory"); v = t; }
+                    h[dr * 9 + j] = v;
+                }
+            }
+            h[27] = 0;
+            const uint32_t dst = smem_u32(im + st * TILE) + line;
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+                uint32_t w4[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { const int i = 8 * ch + 2 * j; w4[j] = i + 1 < 28 ? (h[i] | (h[i + 1] << 16)) : 0u; }
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (((uint32_t)ch ^ swz) << 4)), "r"(w4[0]), "r"(w4[1]), "r"(w4[2]), "r"(w4[3]) : "memory");
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&im_full[st]);
+            if (++st == STAGES) { st = 0; ph ^= 1u; }
+        }
+        // ---- epilogue: accumulator rows 0..63 (warps of lane quarters 0 and 1) are the im2col columns k
+        const int q = warp & 3;
+        if (q < 2) {
+            const bool done = num_kb > 0 ? mbar_wait_sleep(accum_bar, 0, p.err, 15) : true;
+            tc_fence_after();
+            const int k = q * 32 + lane;
+            float* out = p.partial + (((size_t)blockIdx.y * gridDim.x + blockIdx.x) * 64 + k) * 64;
+#pragma unroll 1
+            for (int cc = 0; cc < 64; cc += 32) {
+                uint32_t v[32];
+                if (num_kb > 0) tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + cc, v);
+                else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0u;
+                }
+                if (!done || k >= 27) continue;
+                uint4* o4 = (uint4*)(out + cc);
+#pragma unroll
+                for (int g = 0; g < 8; ++g) o4[g] = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 64); }
+}
+
+// dw[co][k] = sum over CTAs (ascending) of partial[co / 64][cta][k][co % 64], k < 27
+__global__ void stem_wg_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dw, int ctas, int Co, bool accum) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= Co * 27) return;
+    const int k = i / Co, co = i - k * Co;                 // consecutive threads: consecutive c_out (coalesced reads)
+    const float* ptr = partial + ((size_t)(co >> 6) * ctas * 64 + k) * 64 + (co & 63);
+    float s = 0.f;
+#pragma unroll 4
+    for (int b = 0; b < ctas; ++b) s += ptr[(size_t)b * 64 * 64];
+    float* d = dw + (size_t)co * 27 + k;
+    *d = accum ? *d + s : s;
+}
+
 // dW[co][tap][ci] = sum_z partial[z][(tap, cc)][ci % 64][co], z ascending.  32x32 transposing tiles; a thread owns
 // one (row, column) per pass and keeps eight independent loads in flight along z.
 __global__ void __launch_bounds__(1024) wg_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dw, int splits, int row_blocks, int Co,
@@ -1145,6 +1311,46 @@ cudaError_t run_wg_rows(const TensorMap& x_rows, const TensorMap& dy128, const W
     if (e != cudaSuccess) return e;
     dim3 rgrid(p.row_blocks * 2, p.Co / 32), rblk(32, 32);
     wg_reduce_kernel<<<rgrid, rblk, 0, s>>>(p.partial, dw, z, p.row_blocks, p.Co, accum);
+    return cudaGetLastError();
+}
+
+bool make_map_raw_rows(TensorMap* out, const void* base, int C, int W, int H, int N, int box_rows) {
+    if (!init()) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)W * C, (cuuint64_t)H, (cuuint64_t)N};
+    cuuint64_t strides[2] = {(cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+    cuuint32_t box[3] = {(cuuint32_t)(W * C), (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode((CUtensorMap*)out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+bool stem_wg_supported(int H, int W, int C, int Co) {
+    return C == 3 && Co % 64 == 0 && (W == 32 || W == 16) && H % (128 / W) == 0 && (W * C * 2) % 16 == 0 && (128 / W + 2) * W * 6 <= STEM_RAW_BYTES;
+}
+int stem_wg_ctas(long steps) { const long n = sm_count(); return (int)(steps < n ? steps : n); }
+size_t stem_wg_workspace_elems(int Co, long steps) { return (size_t)(Co / 64) * stem_wg_ctas(steps) * 64 * 64; }
+
+cudaError_t run_stem_wg(const TensorMap& x_raw, const TensorMap& dy128, int H, int W, int N, int Co, float* partial, float* dw, bool accum, int* err,
+                        cudaStream_t s) {
+    constexpr int STAGES = 4;
+    constexpr int smem = STAGES * (2 * 128 * 128 + STEM_RAW_BYTES) + 1024 + 256;
+    static bool attr = false;
+    if (!attr) {
+        cudaError_t e = cudaFuncSetAttribute(stem_wg_kernel<STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        attr = true;
+    }
+    StemWgParams p{};
+    p.W = W; p.Ht = 128 / W; p.tiles_h = H / p.Ht; p.steps = N * p.tiles_h;
+    const int ctas = stem_wg_ctas(p.steps);
+    p.steps_per_cta = (p.steps + ctas - 1) / ctas;
+    p.partial = partial; p.err = err;
+    stem_wg_kernel<STAGES><<<dim3(ctas, Co / 64), NUM_THREADS, smem, s>>>(*(const CUtensorMap*)&x_raw, *(const CUtensorMap*)&dy128, p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    stem_wg_reduce_kernel<<<(Co * 27 + 127) / 128, 128, 0, s>>>(partial, dw, ctas, Co, accum);
     return cudaGetLastError();
 }
 

@@ -85,6 +85,14 @@ int wg_rows_variant(int H, int W, int C, int Co);
 int wg_rows_splits(int variant, int C, int Co, long steps);
 cudaError_t run_wg_rows(const TensorMap& x_rows, const TensorMap& dy128, const WgRowsParams& p, int variant, int splits, float* dw, bool accum,
                         cudaStream_t s);
+// Weight gradient of the first layer (3x3, stride 1, pad 1, 3 input channels) on the tensor cores; the im2col lines are
+// built in shared memory.  x_raw: x as rows of W * 3 elements with a box of (128 / W + 2) rows (make_map_raw_rows);
+// dy128: dy with a box of 64 channels x 128 pixels (make_map_4d).  All N samples; partial: stem_wg_workspace_elems floats.
+bool make_map_raw_rows(TensorMap* out, const void* base, int C, int W, int H, int N, int box_rows);
+bool stem_wg_supported(int H, int W, int C, int Co);
+size_t stem_wg_workspace_elems(int Co, long steps);
+cudaError_t run_stem_wg(const TensorMap& x_raw, const TensorMap& dy128, int H, int W, int N, int Co, float* partial, float* dw, bool accum, int* err,
+                        cudaStream_t s);
 cudaError_t run_flip_transpose(const void* w, void* wt, int Co, int taps, int Ci, cudaStream_t s);
 
 }  // namespace tc
