@@ -324,7 +324,7 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
         Op& o = m.ops[i];
         const Op& nx = m.ops[i + 1];
         o.stat_chunks = 0;
-        if (o.type != OP_CONV || !o.tc || nx.type != OP_BN || nx.in != o.out || !bn_accepts_conv_partials(ctx->dt, o.g.Co)) continue;
+        if (o.type != OP_CONV || !(o.tc || o.stem_tc) || nx.type != OP_BN || nx.in != o.out || !bn_accepts_conv_partials(ctx->dt, o.g.Co)) continue;
         int wt, ht, nt;
         tc::pixel_tile(o.g.Ho, o.g.Wo, 128, &wt, &ht, &nt);
         if (ctx->B % nt != 0) continue;
@@ -446,6 +446,20 @@ bool tc_wgrad(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* dy_base, f
     return tc::run_wg(o.wx[ix], o.wdy[id], p, o.n_tile_w, splits, dw, !wn.first, s) == cudaSuccess;
 }
 
+// first-layer forward on the tensor cores (whole batch only)
+bool tc_stem_forward(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* y_base, int64_t version, const Win& wn, cudaStream_t s) {
+    if (!o.stem_tc || wn.n != c->M) return false;
+    const int ix = find_buf(o.a_ptrs, x_base), io = find_buf(o.y_ptrs, y_base);
+    if (ix < 0 || io < 0) return false;
+    const ConvGeom& g = o.g;
+    const double pix = (double)g.N * g.H * g.W;
+    Scope sc(KC_FMA_FWD, 2.0 * pix * g.Co * 9 * g.C, 2.0 * pix * (g.C + g.Co), s);
+    const bool ok = tc::run_stem_fw(o.sxr[ix], o.fo[io], g.H, g.W, g.N, g.Co, wbig(c, m, version, o.w_off), o.bias ? wsmall(c, m, version, o.b_off) : nullptr,
+                                    o.relu, o.stat_chunks ? m.cstat : nullptr, c->tc_err, s) == cudaSuccess;
+    if (ok && o.stat_chunks) { m.fused_stats_tensor = o.out; m.fused_stats_chunks = o.stat_chunks; }
+    return ok;
+}
+
 // first-layer weight gradient on the tensor cores (whole batch only)
 bool tc_stem_wgrad(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* dy_base, float* dw, const Win& wn, cudaStream_t s) {
     if (!o.stem_tc || wn.n != c->M) return false;
@@ -480,6 +494,7 @@ void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int grou
                 ConvGeom g = o.g; g.N = wn.n;
                 profile_detail(o.shape);
                 if (o.tc && tc_forward(c, m, o, P.tensor(o.in), P.tensor(o.out), version, wn, s)) { profile_detail(nullptr); break; }
+                if (o.stem && tc_stem_forward(c, m, o, P.tensor(o.in), P.tensor(o.out), version, wn, s)) { profile_detail(nullptr); break; }
                 if (o.stem) {
                     stem_forward(T(o.in), wbig(c, m, version, o.w_off), o.bias ? wsmall(c, m, version, o.b_off) : nullptr, T(o.out), g, o.relu, s);
                     profile_detail(nullptr);
@@ -600,7 +615,11 @@ bool build_tc_plans(fdg_ctx* c) {
                 o.sxr.resize(o.a_ptrs.size()); o.sdy.resize(o.dy_ptrs.size());
                 for (size_t i = 0; i < o.a_ptrs.size(); ++i) ok = ok && tc::make_map_raw_rows(&o.sxr[i], o.a_ptrs[i], g.C, g.W, g.H, g.N, ht + 2);
                 for (size_t i = 0; i < o.dy_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.sdy[i], o.dy_ptrs[i], g.Co, g.Wo, g.Ho, g.N, 64, wt, ht, nt, 1);
-                if (!ok || o.dy_ptrs.empty()) { o.stem_tc = false; continue; }
+                if (to.loc == LOC_STASH) for (int i = 0; i < m.D; ++i) o.y_ptrs.push_back(m.stash + (size_t)i * m.stash_slot_bytes + to.off);
+                else if (to.loc == LOC_NEXT) { Module& n = c->mod[kk + 1]; for (int i = 0; i < n.in_depth; ++i) o.y_ptrs.push_back(n.in_ring + (size_t)i * n.in_slot_bytes); }
+                o.fo.resize(o.y_ptrs.size());
+                for (size_t i = 0; i < o.y_ptrs.size(); ++i) ok = ok && tc::make_map_out(&o.fo[i], o.y_ptrs[i], g.Co, g.Wo, g.Ho, g.N, wt, ht);
+                if (!ok || o.dy_ptrs.empty() || o.y_ptrs.empty()) { o.stem_tc = false; o.stat_chunks = 0; continue; }
                 c->any_tc = true;
                 continue;
             }

@@ -270,6 +270,95 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 constexpr int EPI_SLICE = 64;                     // accumulator columns an epilogue warp handles at a time
 constexpr int EPI_BUF_BYTES = 32 * EPI_SLICE * 2; // one staged slice: 32 rows x 64 bf16 = 32 rows of 128 bytes (128-byte swizzle)
 
+// One 64-column slice of a warp's 32 accumulator rows (v: this lane's row): bias / ReLU / accumulation into the stored
+// gradient, rounding to bf16, the staged copy in shared memory (stg: one EPI_BUF_BYTES buffer), the store (a TMA store of
+// the box at (cx, cw, chh, cn) of tmO, or row by row through rowptr), and the per-column sums for a following batch-norm.
+// bias, rowptr and stat_dst already point at the slice's first column (or are null).
+__device__ __forceinline__ void epi_slice(uint32_t (&v)[EPI_SLICE], const float* bias, int epi, unsigned long long rowptr, unsigned vmask, bool ok,
+                                          bool tma_out, const CUtensorMap* tmO, int cx, int cw, int chh, int cn, uint32_t stg, int lane,
+                                          float* stat_dst) {
+    const uint32_t swz = (uint32_t)(lane & 7);
+    if (bias) {
+#pragma unroll
+        for (int j = 0; j < EPI_SLICE; j += 4) {
+            const float4 bb = __ldg((const float4*)(bias + j));
+            v[j] = __float_as_uint(__uint_as_float(v[j]) + bb.x); v[j + 1] = __float_as_uint(__uint_as_float(v[j + 1]) + bb.y);
+            v[j + 2] = __float_as_uint(__uint_as_float(v[j + 2]) + bb.z); v[j + 3] = __float_as_uint(__uint_as_float(v[j + 3]) + bb.w);
+        }
+    }
+    if (epi & EPI_RELU) {
+#pragma unroll
+        for (int j = 0; j < EPI_SLICE; ++j) v[j] = __float_as_uint(fmaxf(__uint_as_float(v[j]), 0.f));
+    }
+    if ((epi & EPI_ACCUM) && rowptr) {
+        // add the gradient already stored for this row (rounded once, after the addition)
+        const uint4* o = (const uint4*)((const bf16*)rowptr);
+#pragma unroll
+        for (int g = 0; g < EPI_SLICE / 8; ++g) {
+            const uint4 old = o[g];
+            const uint32_t w4[4] = {old.x, old.y, old.z, old.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                v[8 * g + 2 * j] = __float_as_uint(__uint_as_float(v[8 * g + 2 * j]) + __uint_as_float(w4[j] << 16));
+                v[8 * g + 2 * j + 1] = __float_as_uint(__uint_as_float(v[8 * g + 2 * j + 1]) + __uint_as_float(w4[j] & 0xffff0000u));
+            }
+        }
+    }
+    // the staging buffer used two slices ago must have been read by its TMA store (the elected lane issued it)
+    if (tma_out) { if (elect_one()) bulk_wait_read<1>(); }
+    __syncwarp();
+    // row `lane`, 16-byte chunk g goes to chunk position g ^ (lane % 8): the 128-byte swizzle of the store's tensor map
+#pragma unroll
+    for (int g = 0; g < EPI_SLICE / 8; ++g) {
+        uint32_t pk[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const __nv_bfloat162 t = __floats2bfloat162_rn(__uint_as_float(v[8 * g + 2 * j]), __uint_as_float(v[8 * g + 2 * j + 1]));
+            pk[j] = *(const uint32_t*)&t;
+        }
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + (((uint32_t)g ^ swz) << 4)),
+                     "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
+    }
+    if (tma_out) {
+        fence_proxy_async();
+        __syncwarp();
+        if (elect_one()) {
+            tma_store_4d(tmO, stg, cx, cw, chh, cn);
+            bulk_commit();
+        }
+    } else {
+        __syncwarp();
+        // 8 lanes cover one row's 128 bytes, 4 rows per pass
+#pragma unroll
+        for (int pass = 0; pass < 8; ++pass) {
+            const int r = pass * 4 + (lane >> 3);
+            const uint32_t g = (uint32_t)(lane & 7);
+            const unsigned long long rp = __shfl_sync(0xffffffffu, rowptr, r);
+            uint4 t;
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(t.x), "=r"(t.y), "=r"(t.z), "=r"(t.w)
+                         : "r"(stg + r * 128 + ((g ^ (uint32_t)(r & 7)) << 4)) : "memory");
+            if (rp && ok) *(uint4*)((bf16*)rp + g * 8) = t;
+        }
+    }
+    if (stat_dst) {
+        // batch-norm statistics of the layer's output, fused: this lane sums columns 2*lane and 2*lane+1 of the
+        // slice over the warp's valid rows, from the values as stored
+        float s1a = 0.f, s2a = 0.f, s1b = 0.f, s2b = 0.f;
+        const uint32_t cbase = stg + (uint32_t)(lane & 3) * 4, cg = (uint32_t)(lane >> 2);
+#pragma unroll 8
+        for (int r = 0; r < 32; ++r) {
+            uint32_t t;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(t) : "r"(cbase + r * 128 + ((cg ^ (uint32_t)(r & 7)) << 4)) : "memory");
+            if ((vmask >> r) & 1u) {
+                const float x0 = __uint_as_float(t << 16), x1 = __uint_as_float(t & 0xffff0000u);
+                s1a += x0; s2a = fmaf(x0, x0, s2a); s1b += x1; s2b = fmaf(x1, x1, s2b);
+            }
+        }
+        *(float4*)(stat_dst + 4 * lane) = make_float4(s1a, s2a, s1b, s2b);
+    }
+}
+
+
 // EPI_WARPS = 4 or 8: with 8, two warps share each quarter of the tensor-memory lanes and take alternate 64-column slices.
 // PAIR: launched as clusters of two CTAs.  A pair computes two neighbouring pixel tiles against the same column tile
 // with one 256-row MMA per step, issued by the pair's first CTA; each CTA loads its own pixel tile and half of the
@@ -516,7 +605,6 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         const int row = q * 32 + lane;
         const int pw = row % p.Wt, ph = (row / p.Wt) % p.Ht, pn = row / (p.Wt * p.Ht);
         const int bw0 = (q * 32) % p.Wt, bh0 = ((q * 32) / p.Wt) % p.Ht, bn0 = (q * 32) / (p.Wt * p.Ht);
-        const uint32_t swz = (uint32_t)(lane & 7);
         for (int tile = walker; tile < total && ok; tile += walkers, ++ti) {
             const int buf = ti & 1, use = ti >> 1;
             const int cls = tile / per_cls, tl = tile - cls * per_cls;
@@ -545,85 +633,9 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     __syncwarp();
                     if (lane == 0) { if (PAIR) mbar_arrive_cluster(tmem_empty0 + 8 * buf); else mbar_arrive(&tmem_empty[buf]); }
                 }
-                if (p.bias) {
-#pragma unroll
-                    for (int j = 0; j < EPI_SLICE; j += 4) {
-                        const float4 bb = __ldg((const float4*)(p.bias + co0 + c + j));
-                        v[j] = __float_as_uint(__uint_as_float(v[j]) + bb.x); v[j + 1] = __float_as_uint(__uint_as_float(v[j + 1]) + bb.y);
-                        v[j + 2] = __float_as_uint(__uint_as_float(v[j + 2]) + bb.z); v[j + 3] = __float_as_uint(__uint_as_float(v[j + 3]) + bb.w);
-                    }
-                }
-                if (p.epi & EPI_RELU) {
-#pragma unroll
-                    for (int j = 0; j < EPI_SLICE; ++j) v[j] = __float_as_uint(fmaxf(__uint_as_float(v[j]), 0.f));
-                }
-                if ((p.epi & EPI_ACCUM) && rowptr) {
-                    // add the gradient already stored for this row (rounded once, after the addition)
-                    const uint4* o = (const uint4*)((const bf16*)rowptr + c);
-#pragma unroll
-                    for (int g = 0; g < EPI_SLICE / 8; ++g) {
-                        const uint4 old = o[g];
-                        const uint32_t w4[4] = {old.x, old.y, old.z, old.w};
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            v[8 * g + 2 * j] = __float_as_uint(__uint_as_float(v[8 * g + 2 * j]) + __uint_as_float(w4[j] << 16));
-                            v[8 * g + 2 * j + 1] = __float_as_uint(__uint_as_float(v[8 * g + 2 * j + 1]) + __uint_as_float(w4[j] & 0xffff0000u));
-                        }
-                    }
-                }
-                // the staging buffer used two slices ago must have been read by its TMA store (the elected lane issued it)
-                const uint32_t stg = stg0 + sbuf * EPI_BUF_BYTES;
-                if (tma_out) { if (elect_one()) bulk_wait_read<1>(); }
-                __syncwarp();
-                // row `lane`, 16-byte chunk g goes to chunk position g ^ (lane % 8): the 128-byte swizzle of the store's tensor map
-#pragma unroll
-                for (int g = 0; g < EPI_SLICE / 8; ++g) {
-                    uint32_t pk[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const __nv_bfloat162 t = __floats2bfloat162_rn(__uint_as_float(v[8 * g + 2 * j]), __uint_as_float(v[8 * g + 2 * j + 1]));
-                        pk[j] = *(const uint32_t*)&t;
-                    }
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + (((uint32_t)g ^ swz) << 4)),
-                                 "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
-                }
-                if (tma_out) {
-                    fence_proxy_async();
-                    __syncwarp();
-                    if (elect_one()) {
-                        tma_store_4d(&tmO, stg, co0 + c, tw * p.Wt + bw0, th * p.Ht + bh0, p.n_base + tn * p.Nt + bn0);
-                        bulk_commit();
-                    }
-                } else {
-                    __syncwarp();
-                    // 8 lanes cover one row's 128 bytes, 4 rows per pass
-#pragma unroll
-                    for (int pass = 0; pass < 8; ++pass) {
-                        const int r = pass * 4 + (lane >> 3);
-                        const uint32_t g = (uint32_t)(lane & 7);
-                        const unsigned long long rp = __shfl_sync(0xffffffffu, rowptr, r);
-                        uint4 t;
-                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(t.x), "=r"(t.y), "=r"(t.z), "=r"(t.w)
-                                     : "r"(stg + r * 128 + ((g ^ (uint32_t)(r & 7)) << 4)) : "memory");
-                        if (rp && ok) *(uint4*)((bf16*)rp + c + g * 8) = t;
-                    }
-                }
-                if (p.stat_part) {
-                    // batch-norm statistics of the layer's output, fused: this lane sums columns 2*lane and 2*lane+1 of the
-                    // slice over the warp's valid rows, from the values as stored
-                    float s1a = 0.f, s2a = 0.f, s1b = 0.f, s2b = 0.f;
-                    const uint32_t cbase = stg + (uint32_t)(lane & 3) * 4, cg = (uint32_t)(lane >> 2);
-#pragma unroll 8
-                    for (int r = 0; r < 32; ++r) {
-                        uint32_t t;
-                        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(t) : "r"(cbase + r * 128 + ((cg ^ (uint32_t)(r & 7)) << 4)) : "memory");
-                        if ((vmask >> r) & 1u) {
-                            const float x0 = __uint_as_float(t << 16), x1 = __uint_as_float(t & 0xffff0000u);
-                            s1a += x0; s2a = fmaf(x0, x0, s2a); s1b += x1; s2b = fmaf(x1, x1, s2b);
-                        }
-                    }
-                    *(float4*)(p.stat_part + (((size_t)tmi * 4 + q) * p.Cn + co0 + c + 2 * lane) * 2) = make_float4(s1a, s2a, s1b, s2b);
-                }
+                epi_slice(v, p.bias ? p.bias + co0 + c : nullptr, p.epi, rowptr ? rowptr + 2ull * c : 0ull, vmask, ok, tma_out, &tmO, co0 + c,
+                          tw * p.Wt + bw0, th * p.Ht + bh0, p.n_base + tn * p.Nt + bn0, stg0 + sbuf * EPI_BUF_BYTES, lane,
+                          p.stat_part ? p.stat_part + (((size_t)tmi * 4 + q) * p.Cn + co0 + c) * 2 : nullptr);
                 sbuf ^= 1u;
             }
         }
@@ -1067,6 +1079,176 @@ __global__ void stem_wg_reduce_kernel(const float* __restrict__ partial, float* 
     *d = accum ? *d + s : s;
 }
 
+// ------------------------------------------------------------------------------------------ first layer, forward
+// Same im2col lines as stem_wg_kernel, read K-major this time: D[pixel][c_out] = lines[pixel][k] * W[c_out][k], k < 32
+// (two MMAs per 128-pixel tile).  The 64 x 27 weight tile is written once per CTA.  Warps: 0 producer of raw rows,
+// 1 MMA issue, 2-5 epilogue (the one of km_kernel: bf16 tile, TMA store, batch-norm sums), 6-9 line builders.
+struct StemFwParams {
+    int W, Ht, tiles_h, tiles;          // tile = W x Ht = 128 pixels of one image; tiles = N * tiles_h
+    int Co, epi;
+    const bf16* w;                      // [Co][27]
+    const float* bias;                  // or nullptr
+    float* stat_part;                   // or nullptr: [tile * 4 + warp][Co][2]
+    int* err;
+};
+template <int STAGES>
+__global__ void __launch_bounds__(320, 2)
+stem_fw_kernel(const __grid_constant__ CUtensorMap tmRaw, const __grid_constant__ CUtensorMap tmO, StemFwParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align1024(smem_raw);
+    constexpr int TILE = 128 * 128;
+    uint8_t* im = smem;                                              // [STAGES][TILE]
+    uint8_t* wt = smem + STAGES * TILE;                              // [64 c_out][128 bytes]
+    uint8_t* epi_smem = wt + 64 * 128;                               // [4 warps][2][EPI_BUF_BYTES]
+    uint8_t* raw = epi_smem + 4 * 2 * EPI_BUF_BYTES;                 // [STAGES][STEM_RAW_BYTES]
+    uint64_t* raw_full = (uint64_t*)(raw + STAGES * STEM_RAW_BYTES);
+    uint64_t* im_full = raw_full + STAGES;
+    uint64_t* empty = im_full + STAGES;
+    uint64_t* tmem_full = empty + STAGES;                            // [2]
+    uint64_t* tmem_empty = tmem_full + 2;                            // [2]
+    uint64_t* wt_bar = tmem_empty + 2;
+    uint32_t* tmem_slot = (uint32_t*)(wt_bar + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int co0 = blockIdx.y * 64;
+    const uint32_t raw_bytes = (uint32_t)(p.Ht + 2) * p.W * 6u;
+
+    if (threadIdx.x == 0) {
+        tma_prefetch_desc(&tmRaw); tma_prefetch_desc(&tmO);
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&raw_full[s], 1); mbar_init(&im_full[s], 4); mbar_init(&empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 4); }
+        mbar_init(wt_bar, 4);
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, 128);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        uint32_t st = 0, ph = 1;
+        for (int tile = blockIdx.x; tile < p.tiles; tile += gridDim.x) {
+            if (!mbar_wait(&empty[st], ph, p.err, 21)) break;
+            const int n = tile / p.tiles_h, th = tile - n * p.tiles_h;
+            if (elect_one()) {
+                const uint32_t bar = smem_u32(&raw_full[st]);
+                mbar_expect_tx_a(bar, raw_bytes);
+                asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+                             ::"r"(smem_u32(raw + st * STEM_RAW_BYTES)), "l"(&tmRaw), "r"(bar), "r"(0), "r"(th * p.Ht - 1), "r"(n) : "memory");
+            }
+            __syncwarp();
+            if (++st == STAGES) { st = 0; ph ^= 1u; }
+        }
+    } else if (warp == 1) {
+        const uint32_t idesc = make_idesc(BLOCK_M, 64, 0, 0);
+        const uint64_t dK = make_desc(0, 16, 1024);
+        const uint32_t d_hi = (uint32_t)(dK >> 32), d_lo = (uint32_t)dK;
+        const uint32_t b_lo = d_lo + (smem_u32(wt) >> 4);
+        uint32_t st = 0, ph = 0;
+        int ti = 0;
+        bool ok = mbar_wait(wt_bar, 0, p.err, 22);
+        for (int tile = blockIdx.x; tile < p.tiles && ok; tile += gridDim.x, ++ti) {
+            const int buf = ti & 1, use = ti >> 1;
+            if (use > 0 && !mbar_wait(&tmem_empty[buf], (use - 1) & 1, p.err, 23)) break;
+            if (!mbar_wait(&im_full[st], ph, p.err, 24)) break;
+            tc_fence_after();
+            const uint32_t a_lo = d_lo + (smem_u32(im + st * TILE) >> 4);
+            if (elect_one()) {
+                umma_bf16_w<false>(tmem_base + buf * 64, a_lo, b_lo, d_hi, idesc, 0u);
+                umma_bf16_w<false>(tmem_base + buf * 64, a_lo + 2, b_lo + 2, d_hi, idesc, 1u);
+                umma_commit(&empty[st]);
+                umma_commit(&tmem_full[buf]);
+            }
+            __syncwarp();
+            if (++st == STAGES) { st = 0; ph ^= 1u; }
+        }
+    } else if (warp >= 6) {
+        // ---- builders: thread = one pixel of the tile; first the weight tile (threads 0..63: one c_out row each)
+        const int pix = (warp - 6) * 32 + lane;
+        const uint32_t line = (uint32_t)pix * 128u, swz = (uint32_t)(pix & 7);
+        if (pix < 64) {
+            const bf16* wr = p.w + (size_t)(co0 + pix) * 27;
+            uint32_t h[28];
+#pragma unroll
+            for (int j = 0; j < 27; ++j) h[j] = (uint32_t)__bfloat16_as_ushort(wr[j]);
+            h[27] = 0;
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch) {
+                uint32_t w4[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { const int i = 8 * ch + 2 * j; w4[j] = i + 1 < 28 ? (h[i] | (h[i + 1] << 16)) : 0u; }
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(wt) + line + (((uint32_t)ch ^ swz) << 4)), "r"(w4[0]), "r"(w4[1]), "r"(w4[2]), "r"(w4[3]) : "memory");
+            }
+        }
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(wt_bar);
+        const int r = pix / p.W, c = pix - r * p.W;
+        const bool left = c > 0, right = c < p.W - 1;
+        uint32_t st = 0, ph = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < p.tiles && ok; tile += gridDim.x) {
+            ok = mbar_wait(&raw_full[st], ph, p.err, 25);
+            const uint32_t rb = smem_u32(raw + st * STEM_RAW_BYTES) + (uint32_t)(r * p.W + c - 1) * 6u;
+            uint32_t h[28];
+#pragma unroll
+            for (int dr = 0; dr < 3; ++dr) {
+#pragma unroll
+                for (int j = 0; j < 9; ++j) {
+                    uint32_t v = 0;
+                    const bool in = j < 3 ? left : (j < 6 ? true : right);
+                    if (in) { uint16_t t; asm volatile("ld.shared.u16 %0, [%1];" : "=h"(t) : "r"(rb + (uint32_t)(dr * p.W * 6 + 2 * j)) : "memory"); v = t; }
+                    h[dr * 9 + j] = v;
+                }
+            }
+            h[27] = 0;
+            const uint32_t dst = smem_u32(im + st * TILE) + line;
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+                uint32_t w4[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { const int i = 8 * ch + 2 * j; w4[j] = i + 1 < 28 ? (h[i] | (h[i + 1] << 16)) : 0u; }
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (((uint32_t)ch ^ swz) << 4)), "r"(w4[0]), "r"(w4[1]), "r"(w4[2]), "r"(w4[3]) : "memory");
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&im_full[st]);
+            if (++st == STAGES) { st = 0; ph ^= 1u; }
+        }
+    } else {
+        // ---- epilogue: warp q = warp % 4 owns tensor-memory lanes 32q .. 32q+31 = 32 consecutive pixels of the tile
+        const int q = warp & 3;
+        const uint32_t stg0 = smem_u32(epi_smem + (warp - 2) * 2 * EPI_BUF_BYTES);
+        uint32_t sbuf = 0;
+        int ti = 0;
+        bool ok = true;
+        const int bw0 = (q * 32) % p.W, bh0 = (q * 32) / p.W;
+        for (int tile = blockIdx.x; tile < p.tiles && ok; tile += gridDim.x, ++ti) {
+            const int buf = ti & 1, use = ti >> 1;
+            const int n = tile / p.tiles_h, th = tile - n * p.tiles_h;
+            ok = mbar_wait_sleep(&tmem_full[buf], use & 1, p.err, 26);
+            tc_fence_after();
+            uint32_t v[EPI_SLICE];
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * 64;
+            tmem_ld32_nowait(taddr, v);
+            tmem_ld32_nowait(taddr + 32, v + 32);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tmem_empty[buf]);
+            epi_slice(v, p.bias ? p.bias + co0 : nullptr, p.epi, 0ull, 0xffffffffu, ok, true, &tmO, co0, bw0, th * p.Ht + bh0, n,
+                      stg0 + sbuf * EPI_BUF_BYTES, lane, p.stat_part ? p.stat_part + (((size_t)tile * 4 + q) * p.Co + co0) * 2 : nullptr);
+            sbuf ^= 1u;
+        }
+        if (elect_one()) bulk_wait_all();
+        __syncwarp();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 128); }
+}
+
 // dW[co][tap][ci] = sum_z partial[z][(tap, cc)][ci % 64][co], z ascending.  32x32 transposing tiles; a thread owns
 // one (row, column) per pass and keeps eight independent loads in flight along z.
 __global__ void __launch_bounds__(1024) wg_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dw, int splits, int row_blocks, int Co,
@@ -1351,6 +1533,24 @@ cudaError_t run_stem_wg(const TensorMap& x_raw, const TensorMap& dy128, int H, i
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     stem_wg_reduce_kernel<<<(Co * 27 + 127) / 128, 128, 0, s>>>(partial, dw, ctas, Co, accum);
+    return cudaGetLastError();
+}
+
+cudaError_t run_stem_fw(const TensorMap& x_raw, const TensorMap& out_map, int H, int W, int N, int Co, const void* w, const float* bias, bool relu,
+                        float* stat_part, int* err, cudaStream_t s) {
+    constexpr int STAGES = 3;
+    constexpr int smem = STAGES * (128 * 128 + STEM_RAW_BYTES) + 64 * 128 + 4 * 2 * EPI_BUF_BYTES + 1024 + 256;
+    static bool attr = false;
+    if (!attr) {
+        cudaError_t e = cudaFuncSetAttribute(stem_fw_kernel<STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        attr = true;
+    }
+    StemFwParams p{};
+    p.W = W; p.Ht = 128 / W; p.tiles_h = H / p.Ht; p.tiles = N * p.tiles_h; p.Co = Co; p.epi = relu ? EPI_RELU : 0;
+    p.w = (const bf16*)w; p.bias = bias; p.stat_part = stat_part; p.err = err;
+    const int slots = 2 * sm_count();
+    stem_fw_kernel<STAGES><<<dim3(p.tiles < slots ? p.tiles : slots, Co / 64), 320, smem, s>>>(*(const CUtensorMap*)&x_raw, *(const CUtensorMap*)&out_map, p);
     return cudaGetLastError();
 }
 

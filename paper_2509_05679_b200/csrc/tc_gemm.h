@@ -93,6 +93,10 @@ bool stem_wg_supported(int H, int W, int C, int Co);
 size_t stem_wg_workspace_elems(int Co, long steps);
 cudaError_t run_stem_wg(const TensorMap& x_raw, const TensorMap& dy128, int H, int W, int N, int Co, float* partial, float* dw, bool accum, int* err,
                         cudaStream_t s);
+// Forward pass of the first layer on the tensor cores (same geometry as run_stem_wg).  out_map: the output's map from
+// make_map_out with the tile geometry W x (128 / W) x 1.  w: [Co][27] bf16.  stat_part as in KmParams.
+cudaError_t run_stem_fw(const TensorMap& x_raw, const TensorMap& out_map, int H, int W, int N, int Co, const void* w, const float* bias, bool relu,
+                        float* stat_part, int* err, cudaStream_t s);
 cudaError_t run_flip_transpose(const void* w, void* wt, int Co, int taps, int Ci, cudaStream_t s);
 
 }  // namespace tc
