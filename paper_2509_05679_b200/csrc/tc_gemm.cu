@@ -565,8 +565,7 @@ km_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                             else { a16 += STAGE_BYTES >> 4; fb += 8; eb += 8; }
                         }
                     }
-                    continue;
-                }
+                } else
                 for (int left = num_kb; left > 0; left -= KSUB) {
                     if (!mbar_wait_a(fb, ph, p.err, 2)) { ok = false; break; }
                     tc_fence_after();
