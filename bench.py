@@ -34,11 +34,11 @@ FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 148 SMs x 128 fp32 FMA l
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel classes, from the ncu
 # capture summarised under profiles/.  Valid only for the kernel source it was taken from: a changed source gives null.
-NCU_SHA1 = "68072dbb385993dd7289f8470a575a07c2bfc997"   # sha1 of csrc/tc_gemm.cu when the counters were taken
+NCU_SHA1 = "60fe7d81444287362298e7c2facd7fe16e66c71a"   # sha1 of csrc/tc_gemm.cu when the counters were taken
 NCU_TRAFFIC = {          # profiles/ncu_dram_bytes_C4_full_size.md: single-pass capture at the bench's own size (M = 1024)
-    "tc_gemm_fwd": {"bytes_per_launch": 111.0e6, "sha1": NCU_SHA1},      # km_kernel, average over the 76 forward + input-gradient launches
-    "tc_gemm_dgrad": {"bytes_per_launch": 111.0e6, "sha1": NCU_SHA1},
-    "tc_gemm_wgrad": {"bytes_per_launch": 125.6e6, "sha1": NCU_SHA1},    # wg_kernel, average over its 38 launches (wg_reduce_kernel not included)
+    "tc_gemm_fwd": {"bytes_per_launch": 110.8e6, "sha1": NCU_SHA1},      # km_kernel, average over 74 forward + input-gradient launches
+    "tc_gemm_dgrad": {"bytes_per_launch": 110.8e6, "sha1": NCU_SHA1},
+    "tc_gemm_wgrad": {"bytes_per_launch": 122.8e6, "sha1": NCU_SHA1},    # wg_kernel + wg2_kernel, average over 36 launches (wg_reduce_kernel not included)
 }
 
 
