@@ -57,13 +57,22 @@ SINGLE_MODULE_NETS = {
                                     (sy.MAXPOOL2, 128, 128, 2, 0), (sy.CONV3X3, 128, 256, 1, 1), (sy.RELU, 256, 256, 1, 0),
                                     (sy.CONV3X3, 256, 256, 1, 1), (sy.RELU, 256, 256, 1, 0), (sy.GLOBAL_AVGPOOL, 256, 256, 1, 0),
                                     (sy.LINEAR, 256, 10, 1, 1)],
+    # 32x32 input: the first layer on the tensor cores (im2col lines built in shared memory), 64->64 at 32x32 and 128->128 at
+    # 16x16 in rows mode (resident weights / CTA pairs) with their rows-mode weight gradients
+    "tensor-core-rows-32x32": [(sy.CONV3X3, 3, 64, 1, 1), (sy.RELU, 64, 64, 1, 0), (sy.CONV3X3, 64, 64, 1, 1), (sy.RELU, 64, 64, 1, 0),
+                               (sy.MAXPOOL2, 64, 64, 2, 0), (sy.CONV3X3, 64, 128, 1, 1), (sy.RELU, 128, 128, 1, 0),
+                               (sy.CONV3X3, 128, 128, 1, 1), (sy.RELU, 128, 128, 1, 0), (sy.GLOBAL_AVGPOOL, 128, 128, 1, 0),
+                               (sy.LINEAR, 128, 10, 1, 1)],
+    # the same kernels with batch-norm sums taken in their epilogues: first layer + one identity block of 64 channels at 32x32
+    "tensor-core-bn-block-32x32": sy.resnet_layers(widths=(64,), blocks=1)[0],
 }
+INPUT_SHAPE = {"mlp": (1, 1, 48), "tensor-core-rows-32x32": (32, 32, 3), "tensor-core-bn-block-32x32": (32, 32, 3)}
 
 
 @pytest.mark.parametrize("name", sorted(SINGLE_MODULE_NETS))
 def test_single_module_nets_match_the_storage_model_tightly(orc, name):
     layers = SINGLE_MODULE_NETS[name]
-    shape = (1, 1, 48) if name == "mlp" else (16, 16, 3)
+    shape = INPUT_SHAPE.get(name, (16, 16, 3))
     net = sy.Net(name, layers, [], *shape, 10, 2, 4, 0.05, "bf16")
     # the tensor-core net sums up to 2304 products per output in fp32 (the others at most 144, compensated): more of its
     # stored bf16 values land on the other side of a rounding boundary than in the fp64 oracle
