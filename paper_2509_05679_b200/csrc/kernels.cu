@@ -583,7 +583,7 @@ __global__ void bn_bwd_apply_k(const T* __restrict__ x, const T* __restrict__ ou
 // ------------------------------------------------------------------------------------------
 // Batch-norm, bf16 storage, streamed: a CTA owns a contiguous range of one worker's rows, which is one
 // contiguous range of memory (NHWC).  One thread feeds a ring of shared-memory stages with bulk asynchronous
-// copies (cp.async.bulk, completion on an mbarrier), 8 KB per input tensor and stage, so that about 90 KB per
+// copies (cp.async.bulk, completion on an mbarrier), 16 KB per input tensor and stage, so that about 90 KB per
 // CTA are in flight whatever the registers hold; all 256 threads read 16-byte vectors (8 channels) from the
 // stage, and results go straight to global memory.  A thread keeps the same 8 channels for every row.
 // grid = (row chunks, workers).  Used when C/8 is a power of two <= 256.
@@ -591,8 +591,12 @@ __global__ void bn_bwd_apply_k(const T* __restrict__ x, const T* __restrict__ ou
 constexpr int BNV_THREADS = 256;
 constexpr int BNV_MAX_CHUNKS = 128;
 constexpr int BV = 8;                               // channels per thread (one 128-bit access)
-constexpr int BNS_TILE = 8192;                      // bytes per input tensor and stage
-constexpr int BNS_RING = 12 * BNS_TILE;             // shared memory of the ring (stages = 12 / input tensors, at most 8)
+#ifndef BNS_TILE_BYTES
+#define BNS_TILE_BYTES 16384
+#endif
+constexpr int BNS_TILE = BNS_TILE_BYTES;            // bytes per input tensor and stage
+constexpr int BNS_RING = 96 * 1024;                 // shared memory of the ring (stages = tiles in the ring / input tensors, at most 8)
+constexpr int BNS_VPT = BNS_TILE / 16 / 256;        // 16-byte vectors per thread and tile
 constexpr long long BNS_WAIT_CYCLES = 4000000000LL; // ~2 s
 
 __device__ __forceinline__ void unpack8(const uint4& v, float (&f)[BV]) {
@@ -645,7 +649,7 @@ __global__ void __launch_bounds__(BNV_THREADS, 2) bns_kernel(const BnsArgs a) {
     const int C = a.C, cgs = C / BV, rows_it = BNV_THREADS / cgs;
     const int tid = threadIdx.x, cg = tid % cgs, rl = tid / cgs;
     const int w = blockIdx.y, nw = gridDim.y;
-    const int n_in = a.n_in, stages = 12 / n_in < 8 ? 12 / n_in : 8;
+    const int n_in = a.n_in, stages = (BNS_RING / BNS_TILE) / n_in < 8 ? (BNS_RING / BNS_TILE) / n_in : 8;
     const int tile_rows = BNS_TILE / (C * 2);
     long per = (a.rpw + gridDim.x - 1) / gridDim.x;
     per = (per + tile_rows - 1) / tile_rows * tile_rows;
@@ -691,7 +695,7 @@ __global__ void __launch_bounds__(BNV_THREADS, 2) bns_kernel(const BnsArgs a) {
         const uint8_t* sx = bns_sm + (size_t)(st * n_in) * BNS_TILE;
         const long trow = r0 + (long)i * tile_rows;
 #pragma unroll
-        for (int k = 0; k < 2; ++k) {
+        for (int k = 0; k < BNS_VPT; ++k) {
             const int lr = rl + k * rows_it;                 // row inside the tile
             const long row = trow + lr;
             if (row >= r1 || !ok) continue;
