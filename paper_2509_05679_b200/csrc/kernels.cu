@@ -595,7 +595,13 @@ constexpr int BV = 8;                               // channels per thread (one 
 #define BNS_TILE_BYTES 16384
 #endif
 constexpr int BNS_TILE = BNS_TILE_BYTES;            // bytes per input tensor and stage
-constexpr int BNS_RING = 96 * 1024;                 // shared memory of the ring (stages = tiles in the ring / input tensors, at most 8)
+#ifndef BNS_RING_KB
+#define BNS_RING_KB 96
+#endif
+#ifndef BNS_CTAS
+#define BNS_CTAS 2                                  // CTAs per SM the ring size allows
+#endif
+constexpr int BNS_RING = BNS_RING_KB * 1024;                 // shared memory of the ring (stages = tiles in the ring / input tensors, at most 8)
 constexpr int BNS_VPT = BNS_TILE / 16 / 256;        // 16-byte vectors per thread and tile
 constexpr long long BNS_WAIT_CYCLES = 4000000000LL; // ~2 s
 
@@ -644,7 +650,7 @@ struct BnsArgs {
 // MODE 2: y = bn(x) (+ res) (relu).  MODE 3: dx (+)= BN backward of dy, dres (+)= dy.
 // mask_from_x: the forward output had no residual, so its sign is the sign of bn_value(x).
 template <int MODE>
-__global__ void __launch_bounds__(BNV_THREADS, 2) bns_kernel(const BnsArgs a) {
+__global__ void __launch_bounds__(BNV_THREADS, BNS_CTAS) bns_kernel(const BnsArgs a) {
     extern __shared__ __align__(128) uint8_t bns_sm[];
     const int C = a.C, cgs = C / BV, rows_it = BNV_THREADS / cgs;
     const int tid = threadIdx.x, cg = tid % cgs, rl = tid / cgs;
@@ -849,7 +855,7 @@ static int bns_chunks(int nw, long rpw, int C) {
     static int sms = 0;
     if (!sms) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); if (sms <= 0) sms = 148; }
     const long tile_rows = BNS_TILE / (C * 2);
-    long want = ((long)sms * 2) / nw, maxc = (rpw + tile_rows * 4 - 1) / (tile_rows * 4);
+    long want = ((long)sms * BNS_CTAS) / nw, maxc = (rpw + tile_rows * 4 - 1) / (tile_rows * 4);
     long c = want < maxc ? want : maxc;
     if (c > BNV_MAX_CHUNKS) c = BNV_MAX_CHUNKS;
     return (int)(c < 1 ? 1 : c);
