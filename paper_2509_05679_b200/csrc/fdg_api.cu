@@ -100,6 +100,8 @@ struct Module {
     int64_t *tag_in, *tag_stash, *tag_d2, *tag_w, *trace;
     cudaStream_t stream;           // backward pass, loss, update (and everything in serial mode)
     cudaStream_t fstream;          // forward pass: independent of the backward pass of the same iteration (other batch)
+    cudaStream_t wstream;          // weight gradients: off the chain input gradient -> batch-norm backward -> input gradient
+    cudaEvent_t wev, wdone;        // dy ready for the weight-gradient stream / its work of this iteration finished
     cudaEvent_t done, fdone, ev0, ev1;
     float* scratch_f;              // reduction scratch of the forward stream
     bool had_bwd;
@@ -556,10 +558,13 @@ void backward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int64_t
                 ConvGeom g = o.g; g.N = wn.n;
                 if (o.relu) relu_backward(dt, T(o.out), gout, gout, n_out, false, s);       // in place: dZ = dA * (A > 0)
                 profile_detail(o.shape);
-                if (o.stem && tc_stem_wgrad(c, m, o, P.tensor(o.in), grad_ptr(c, kk, o.out, t), m.grad + o.w_off, wn, s)) {}
-                else if (o.stem) stem_wgrad(T(o.in), gout, m.grad + o.w_off, m.ws, g, acc_p, s);
-                else if (!(o.tc && tc_wgrad(c, m, o, P.tensor(o.in), grad_ptr(c, kk, o.out, t), m.grad + o.w_off, wn, s)))
-                    conv_wgrad(dt, T(o.in), gout, m.grad + o.w_off, m.ws, g, acc_p, s);
+                // the weight gradient needs dy as it stands now and is needed only by the update: it goes to its own stream
+                cudaStream_t ws = m.wstream;
+                if (ws != s) { cudaEventRecord(m.wev, s); cudaStreamWaitEvent(ws, m.wev, 0); }
+                if (o.stem && tc_stem_wgrad(c, m, o, P.tensor(o.in), grad_ptr(c, kk, o.out, t), m.grad + o.w_off, wn, ws)) {}
+                else if (o.stem) stem_wgrad(T(o.in), gout, m.grad + o.w_off, m.ws, g, acc_p, ws);
+                else if (!(o.tc && tc_wgrad(c, m, o, P.tensor(o.in), grad_ptr(c, kk, o.out, t), m.grad + o.w_off, wn, ws)))
+                    conv_wgrad(dt, T(o.in), gout, m.grad + o.w_off, m.ws, g, acc_p, ws);
                 if (o.bias) bias_grad(dt, gout, m.grad + m.n_big + o.b_off, m.scratch, (long)g.N * g.Ho * g.Wo, g.Co, acc_p, s);
                 if (gin && !(o.tc && tc_dgrad(c, m, o, grad_ptr(c, kk, o.out, t), grad_ptr(c, kk, o.in, t), version, o.acc_in, wn, s)))
                     conv_dgrad(dt, gout, wbig(c, m, version, o.w_off), gin, g, o.acc_in ? EPI_ACCUM : 0, s);
@@ -827,6 +832,7 @@ fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, boo
         // Eq. dl_update with P = 11^T/N: w(t+1) = w(t) - lr * averaged gradient; also emits version t+1
         // (after the forward pass has read version t: with a one-slot ring the update overwrites it)
         if (!lastm && m.fstream != m.stream) CK(cudaStreamWaitEvent(m.stream, m.fdone, 0));
+        if (tau_b >= 0 && m.wstream != m.stream) { CK(cudaEventRecord(m.wdone, m.wstream)); CK(cudaStreamWaitEvent(m.stream, m.wdone, 0)); }
         sgd_update(ctx->dt, m.master, tau_b >= 0 ? m.grad : nullptr, wslot(ctx, m, t + 1), m.n_big, ctx->lr, m.stream);
         if (m.n_small)
             sgd_update(0, m.master + m.n_big, tau_b >= 0 ? m.grad + m.n_big : nullptr,
@@ -861,6 +867,8 @@ void fdg_destroy(fdg_ctx* ctx) {
     for (Module& m : ctx->mod) {
         if (m.done) cudaEventDestroy(m.done);
         if (m.fdone) cudaEventDestroy(m.fdone);
+        if (m.wev) cudaEventDestroy(m.wev);
+        if (m.wdone) cudaEventDestroy(m.wdone);
         if (m.ev0) cudaEventDestroy(m.ev0);
         if (m.ev1) cudaEventDestroy(m.ev1);
     }
@@ -980,6 +988,10 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
         else { e = cudaStreamCreateWithFlags(&m.stream, cudaStreamNonBlocking); if (e == cudaSuccess) ctx->owned.push_back(m.stream); }
         m.fstream = m.stream;
         if (e == cudaSuccess && !ctx->serial) { e = cudaStreamCreateWithFlags(&m.fstream, cudaStreamNonBlocking); if (e == cudaSuccess) ctx->owned.push_back(m.fstream); }
+        m.wstream = m.stream;
+        if (e == cudaSuccess && !ctx->serial) { e = cudaStreamCreateWithFlags(&m.wstream, cudaStreamNonBlocking); if (e == cudaSuccess) ctx->owned.push_back(m.wstream); }
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.wev, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.wdone, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.done, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.fdone, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreate(&m.ev0);
