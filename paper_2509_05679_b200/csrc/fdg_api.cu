@@ -653,7 +653,7 @@ bool build_tc_plans(fdg_ctx* c) {
             o.fa.resize(o.a_ptrs.size());
             for (size_t i = 0; i < o.a_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.fa[i], o.a_ptrs[i], g.C, g.W, g.H, g.N, 64, wt, ht, nt, g.stride);
             // rows mode: a box of the tile's rows plus one above and one below, for a tile that is whole rows of one image
-            const bool rows_ok = g.R == 3 && g.stride == 1 && wt == g.Wo && nt == 1;
+            const bool rows_ok = g.R == 3 && g.stride == 1 && wt == g.Wo && nt == 1 && (ht + 2) * g.Wo * 128 <= 24 * 1024;   // the stage holds ht + 2 rows of 128-byte pixels in 24 KB
             if (rows_ok) {
                 o.far.resize(o.a_ptrs.size());
                 for (size_t i = 0; i < o.a_ptrs.size(); ++i) ok = ok && tc::make_map_4d(&o.far[i], o.a_ptrs[i], g.C, g.W, g.H, g.N, 64, g.W, ht + 2, 1, 1);

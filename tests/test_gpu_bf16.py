@@ -63,17 +63,21 @@ SINGLE_MODULE_NETS = {
                                (sy.MAXPOOL2, 64, 64, 2, 0), (sy.CONV3X3, 64, 128, 1, 1), (sy.RELU, 128, 128, 1, 0),
                                (sy.CONV3X3, 128, 128, 1, 1), (sy.RELU, 128, 128, 1, 0), (sy.GLOBAL_AVGPOOL, 128, 128, 1, 0),
                                (sy.LINEAR, 128, 10, 1, 1)],
+    # 64-pixel-wide images: tiles of two image rows, too tall a halo for rows mode (tap-by-tap kernels, 64-pixel boxes)
+    "tensor-core-64x64": [(sy.CONV3X3, 3, 64, 1, 1), (sy.RELU, 64, 64, 1, 0), (sy.CONV3X3, 64, 64, 1, 1), (sy.RELU, 64, 64, 1, 0),
+                          (sy.MAXPOOL2, 64, 64, 2, 0), (sy.GLOBAL_AVGPOOL, 64, 64, 1, 0), (sy.LINEAR, 64, 10, 1, 1)],
     # the same kernels with batch-norm sums taken in their epilogues: first layer + one identity block of 64 channels at 32x32
     "tensor-core-bn-block-32x32": sy.resnet_layers(widths=(64,), blocks=1)[0],
 }
-INPUT_SHAPE = {"mlp": (1, 1, 48), "tensor-core-rows-32x32": (32, 32, 3), "tensor-core-bn-block-32x32": (32, 32, 3)}
+INPUT_SHAPE = {"mlp": (1, 1, 48), "tensor-core-rows-32x32": (32, 32, 3), "tensor-core-bn-block-32x32": (32, 32, 3),
+               "tensor-core-64x64": (64, 64, 3)}
 
 
 @pytest.mark.parametrize("name", sorted(SINGLE_MODULE_NETS))
 def test_single_module_nets_match_the_storage_model_tightly(orc, name):
     layers = SINGLE_MODULE_NETS[name]
     shape = INPUT_SHAPE.get(name, (16, 16, 3))
-    net = sy.Net(name, layers, [], *shape, 10, 2, 4, 0.05, "bf16")
+    net = sy.Net(name, layers, [], *shape, 10, 2, 2 if shape[0] == 64 else 4, 0.05, "bf16")
     # the tensor-core net sums up to 2304 products per output in fp32 (the others at most 144, compensated): more of its
     # stored bf16 values land on the other side of a rounding boundary than in the fp64 oracle
     tc = name.startswith("tensor-core")
