@@ -90,9 +90,11 @@ typedef struct {
     int32_t serial;            /* 1: run every module on one stream (results are bit-identical
                                   to the concurrent mode; used to test the event wiring)        */
     int32_t kernel_path;       /* 0: tensor-core kernels where shapes allow (bf16 only), the 256-column
-                                     tile as pairs of CTAs on two SMs (tcgen05 cta_group::2);
+                                     tile (and the 128-column tile of 3x3 stride-1 layers on 16x16 images) as
+                                     pairs of CTAs on two SMs (tcgen05 cta_group::2);
                                   1: plain FMA kernels only;
-                                  2: tensor-core kernels, no CTA pairs (bit-identical results to 0) */
+                                  2: tensor-core kernels, no CTA pairs (bit-identical results to 0 wherever
+                                     both run the same loop order: everything but those 128-column layers) */
     int32_t worker_groups;     /* 0 or 1: every kernel covers all workers.  n > 1: every module but the last runs
                                   its layers once per group of n_workers / n workers (n rounded down to a power
                                   of two that divides n_workers; ignored where a group would cut a tensor-core
