@@ -3,10 +3,12 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config 0..4] [--impl ours|reference]
 
-Prints ONE JSON line (rank 0).  `value` = samples/s with inputs resident in HBM; `e2e` = the same
-through fdg_step_host with pinned host buffers (host->device copies and the loss read-back inside
-the timed region); `roofline` describes the kernel class with the largest share of device time;
-`cpu_baseline` is the CPU oracle timed on a bounded sample.  With N > 1 every rank runs an
+Prints ONE JSON line (rank 0).  `value` = samples/s with inputs resident in HBM, timed with nothing but
+the step's own work on the device; `e2e` = the same through fdg_step_host with pinned host buffers
+(host->device copies and the loss read-back inside the timed region); `roofline` describes the kernel
+class with the largest share of device time, timed launch by launch in a separate pass with every module
+on one stream (so that a launch's events bracket that kernel alone), and carries the whole step's
+fraction of the tensor roofline under `step`; `cpu_baseline` is the CPU oracle timed on a bounded sample.  With N > 1 every rank runs an
 independent replica (the method has no exchange between GPUs here) and the time is the maximum
 over ranks.  `--impl reference` times the CPU oracle only.
 """
@@ -32,13 +34,15 @@ UNIT = "samples/s"
 FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 148 SMs x 128 fp32 FMA lanes x 2 flop x 1.965 GHz
 
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel classes, from the ncu
-# capture summarised under profiles/.  Valid only for the kernel source it was taken from: a changed source gives null.
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel classes of the default
+# workload: ncu counters of a few launches of one kernel at a reduced per-worker batch, scaled to the full batch by
+# the samples a launch processes (traffic of these kernels grows in proportion to the batch).  Valid only for the kernel
+# source it was taken from: a changed source gives null.
 NCU_SHA1 = "60fe7d81444287362298e7c2facd7fe16e66c71a"   # sha1 of csrc/tc_gemm.cu when the counters were taken
-NCU_TRAFFIC = {          # profiles/ncu_dram_bytes_C4_full_size.md: single-pass capture at the bench's own size (M = 1024)
-    "tc_gemm_fwd": {"bytes_per_launch": 110.8e6, "sha1": NCU_SHA1},      # km_kernel, average over 74 forward + input-gradient launches
+NCU_TRAFFIC = {
+    "tc_gemm_fwd": {"bytes_per_launch": 110.8e6, "sha1": NCU_SHA1},
     "tc_gemm_dgrad": {"bytes_per_launch": 110.8e6, "sha1": NCU_SHA1},
-    "tc_gemm_wgrad": {"bytes_per_launch": 122.8e6, "sha1": NCU_SHA1},    # wg_kernel + wg2_kernel, average over 36 launches (wg_reduce_kernel not included)
+    "tc_gemm_wgrad": {"bytes_per_launch": 122.8e6, "sha1": NCU_SHA1},
 }
 
 
@@ -143,9 +147,11 @@ def run_reference(args, net):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    v, cores, desc, dt = oracle_sample(net, max(1, min(args.steps, 3)), min(args.warmup, 1))
+    timed, warm = max(1, min(args.steps, 3)), min(args.warmup, 1)      # bounded: a step of the oracle takes seconds
+    v, cores, desc, dt = oracle_sample(net, timed, warm)
     print(json.dumps({
-        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": timed, "warmup": warm,
+        "steps_requested": args.steps, "warmup_requested": args.warmup,
         "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": net.name, "K": net.K, "n_workers": net.n_workers, "per_worker_batch": net.batch, "note": desc},
         "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
@@ -163,7 +169,7 @@ def main():
     ap.add_argument("--kernel-path", type=int, default=0, help="0: tensor-core kernels where shapes allow (CTA pairs for the 256-column tile), 1: plain FMA kernels only, 2: tensor-core kernels without CTA pairs")
     ap.add_argument("--batch", type=int, default=None, help="per-worker batch override (testing only; changes the workload name)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-uncontended", action="store_true", help="skip the extra one-stream pass that times kernels alone")
+    ap.add_argument("--no-kernel-pass", action="store_true", help="skip the extra one-stream pass that times every kernel class (roofline becomes null)")
     ap.add_argument("--serial", action="store_true", help="diagnosis: all modules on one stream (uncontended per-kernel times)")
     args = ap.parse_args()
 
@@ -187,11 +193,10 @@ def main():
 
     warmup = max(args.warmup, 3)
     fill = 2 * net.K - 2                      # iterations until every module has a backward batch
-    streams = [torch.cuda.Stream() for _ in range(net.K)]
+    timing_stream = torch.cuda.Stream()       # carries only the two timing events; the library runs on its own streams
     ctx = binding.Context(net.layers, net.splits, net.n_workers, net.batch, net.lr, dtype=net.dtype,
                           in_shape=(net.in_h, net.in_w, net.in_c), num_classes=net.classes, device=local,
-                          kernel_path=args.kernel_path, streams=[s.cuda_stream for s in streams], serial=args.serial,
-                          worker_groups=args.worker_groups)
+                          kernel_path=args.kernel_path, serial=args.serial, worker_groups=args.worker_groups)
     ctx.set_params(sy.init_params(net.layers, 0, bf16=net.dtype == "bf16"))
 
     # a pool of distinct batches, resident in HBM (device arm) and in pinned host memory (e2e arm)
@@ -210,13 +215,10 @@ def main():
         torch.cuda.synchronize()
 
     def join_event():
-        """An event that fires when all module streams are done (recorded on stream 0 after waits)."""
-        for s in streams[1:]:
-            e = torch.cuda.Event()
-            e.record(s)
-            streams[0].wait_event(e)
+        """An event that fires when all module streams are done (fdg_join makes the timing stream wait for them)."""
+        ctx.join(timing_stream.cuda_stream)
         e = torch.cuda.Event(enable_timing=True)
-        e.record(streams[0])
+        e.record(timing_stream)
         return e
 
     step_no = 0
@@ -227,25 +229,20 @@ def main():
             ctx.step(dev_x[step_no % pool], dev_y[step_no % pool])
             step_no += 1
 
-    # ---- device-resident arm
+    # ---- device-resident arm (no per-launch instrumentation: only the step's own work is on the device)
     dev_steps(fill + warmup)
     barrier()
     _, launches0 = ctx.stats()
     sampler = ClockSampler(local)
     sampler.start()
-    ctx.profile(True)
     start = torch.cuda.Event(enable_timing=True)
-    start.record(streams[0])                 # the device is idle here: this is the start of the timed region
+    start.record(timing_stream)              # the device is idle here: this is the start of the timed region
     dev_steps(args.steps)
     end = join_event()
     barrier()
     ms = start.elapsed_time(end)
-    ctx.profile(False)
-    kall = ctx.profile_read()
-    kstats = {k: v for k, v in kall.items() if "[" not in k}
-    kshapes = {k: v for k, v in kall.items() if "[" in k}
     clocks = sampler.stop()
-    _, launches1 = ctx.stats()
+    dev_bytes, launches1 = ctx.stats()
     mod_ms = [float(v) for v in ctx.module_times()]
 
     # ---- end-to-end arm: host buffers in, loss out, every step
@@ -259,9 +256,11 @@ def main():
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
-    # ---- uncontended kernel times: the same workload with every module on one stream (rank 0, N=1 only)
-    kstats_alone, alone_steps = None, 3
-    if world == 1 and not args.serial and not args.no_uncontended:
+    # ---- kernel pass: the same workload with every module on ONE stream and CUDA events around every launch, so that
+    # an event pair brackets one kernel running alone (with the module streams running side by side a pair would also
+    # contain whatever the other modules had on the GPU).  Not part of `value`.
+    kstats, kshapes, kernel_steps = None, None, 3
+    if not args.no_kernel_pass:
         ctx.close()
         ctx = binding.Context(net.layers, net.splits, net.n_workers, net.batch, net.lr, dtype=net.dtype,
                               in_shape=(net.in_h, net.in_w, net.in_c), num_classes=net.classes, device=local,
@@ -271,10 +270,12 @@ def main():
             ctx.step(dev_x[i % pool], dev_y[i % pool])
         torch.cuda.synchronize()
         ctx.profile(True)
-        for i in range(alone_steps):
+        for i in range(kernel_steps):
             ctx.step(dev_x[i % pool], dev_y[i % pool])
         ctx.profile(False)
-        kstats_alone = {k: v for k, v in ctx.profile_read().items() if "[" not in k}
+        kall = ctx.profile_read()
+        kstats = {k: v for k, v in kall.items() if "[" not in k}
+        kshapes = {k: v for k, v in kall.items() if "[" in k}
 
     ms, e2e_s = max_over_ranks([ms, e2e_s], dist, "cuda")
 
@@ -283,20 +284,32 @@ def main():
         total_samples = net.M * args.steps * world
         value = whole_job_throughput(net.M, args.steps, world, ms * 1e-3)
         flops_step = sy.flops_per_sample(net) * net.M
-        def roofline_of(stats, which=None):
-            """Roofline entry of the kernel class with the largest summed event time (or of class `which`)."""
+        ms_step = ms / args.steps
+        # which measured peak: the sustained figure for a whole step under load; for a kernel timed alone the burst figure
+        step_tflops = flops_step / (ms_step * 1e-3) / 1e12
+        step_entry = {"flop_per_step": flops_step, "ms_per_step": ms_step, "achieved": step_tflops, "unit": "TFLOP/s",
+                      "peak": pk["tensor_burst"], "frac": step_tflops / pk["tensor_burst"],
+                      "peak_sustained": pk["tensor"], "frac_of_sustained": step_tflops / pk["tensor"],
+                      "peak_source": pk["source"] + ": bf16 GEMM, burst (frac) and sustained (frac_of_sustained)"}
+
+        def roofline_of(stats):
+            """Roofline entry of the kernel class with the largest summed time in the one-stream kernel pass."""
             if not stats:
                 return None
-            name, st = (which, stats[which]) if which in stats else max(stats.items(), key=lambda kv: kv[1]["ms"])
+            name, st = max(stats.items(), key=lambda kv: kv[1]["ms"])
             total_ms = sum(v["ms"] for v in stats.values())
-            base = {"kernel": name, "launches": st["launches"], "avg_launch_ms": st["ms"] / st["launches"],
-                    "share_of_kernel_time": st["ms"] / total_ms, "traffic": traffic_per_launch(name)}
+            per_step = st["launches"] / kernel_steps
+            base = {"kernel": name, "launches_per_step": per_step, "avg_launch_ms": st["ms"] / st["launches"],
+                    "class_ms_per_step": st["ms"] / kernel_steps, "share_of_kernel_time": st["ms"] / total_ms,
+                    "kernel_ms_per_step_all_classes": total_ms / kernel_steps, "traffic": traffic_per_launch(name),
+                    "timing": f"CUDA events around every launch, separate pass of {kernel_steps} steps with all modules on one stream "
+                              "(each event pair brackets one kernel running alone); not part of the timed region of `value`"}
             if name.startswith("tc_gemm") or name.startswith("igemm_fma"):
                 tensor = name.startswith("tc_gemm")
                 ach = st["flops"] / (st["ms"] * 1e-3) / 1e12
-                peak = pk["tensor"] if tensor else FMA_PEAK_TFLOPS
+                peak = pk["tensor_burst"] if tensor else FMA_PEAK_TFLOPS
                 base.update({"bound": "tensor" if tensor else "alu", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
-                             "peak_source": (pk["source"] + ", sustained bf16 GEMM (kernel timed inside a long step)") if tensor
+                             "peak_source": (pk["source"] + ", burst bf16 GEMM (a kernel timed alone)") if tensor
                              else "derived: 148 SMs x 128 FMA x 2 x 1.965 GHz"})
             else:
                 ach = st["bytes"] / (st["ms"] * 1e-3) / 1e9
@@ -305,10 +318,9 @@ def main():
 
         roof = roofline_of(kstats)
         if roof:
-            roof["timing"] = "CUDA events around every launch of the class inside the timed region; K module streams run concurrently, so a launch shares the GPU with other modules' kernels"
-        roof_alone = roofline_of(kstats_alone, roof["kernel"]) if (roof and kstats_alone) else None
-        if roof_alone:
-            roof_alone["timing"] = f"same class, separate pass of {alone_steps} steps with all modules on one stream (kernels do not share the GPU)"
+            roof["step"] = step_entry
+        else:
+            roof = {"kernel": None, "step": step_entry}
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -318,28 +330,23 @@ def main():
                        "l2": "inputs rotate over 4 batches; each step streams the multi-GB activation stash, far larger than L2",
                        "multi_gpu": "independent replicas (no exchange between GPUs)", "kernel_path": args.kernel_path, "serial": bool(args.serial), "worker_groups": args.worker_groups},
             "clocks": clocks,
-            "step_tensor_roofline": {"flop_per_step": flops_step, "tflops_achieved": flops_step / (ms / args.steps * 1e-3) / 1e12 * 1.0,
-                                     "frac_of_burst_peak": flops_step / (ms / args.steps * 1e-3) / 1e12 / pk["tensor_burst"],
-                                     "frac_of_sustained_peak": flops_step / (ms / args.steps * 1e-3) / 1e12 / pk["tensor"],
-                                     "peak_source": pk["source"]},
             "roofline": roof,
-            "roofline_uncontended": roof_alone,
-            "kernels": {k: {"launches": v["launches"], "ms": round(v["ms"], 4),
+            "kernels": {k: {"launches_per_step": v["launches"] / kernel_steps, "ms_per_step": round(v["ms"] / kernel_steps, 4),
                             "tflops": round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 2) if v["ms"] > 0 else None,
                             "gbs": round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1) if v["ms"] > 0 else None}
-                        for k, v in sorted(kstats.items(), key=lambda kv: -kv[1]["ms"])},
-            "kernel_shapes": {k: {"launches": v["launches"], "ms": round(v["ms"], 4),
+                        for k, v in sorted((kstats or {}).items(), key=lambda kv: -kv[1]["ms"])},
+            "kernel_shapes": {k: {"launches_per_step": v["launches"] / kernel_steps, "ms_per_step": round(v["ms"] / kernel_steps, 4),
                                   "tflops": round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 1) if v["ms"] > 0 else None,
                                   "gbs": round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1) if v["ms"] > 0 else None}
-                              for k, v in sorted(kshapes.items(), key=lambda kv: -kv[1]["ms"])},
-            "module_ms_last_step": mod_ms,
+                              for k, v in sorted((kshapes or {}).items(), key=lambda kv: -kv[1]["ms"])},
+            "module_ms_last_step": mod_ms, "device_bytes": int(dev_bytes),
             "gpu_launches": int(launches1 - launches0),
             "e2e": {"value": total_samples / e2e_s, "unit": UNIT,
                     "h2d_bytes_per_step": int(host_x[0].numel() * host_x[0].element_size() + host_y[0].numel() * 4),
                     "d2h_bytes_per_step": 4, "last_loss": loss},
         }
         if world == 1 and not args.no_cpu_baseline:
-            v, cores, desc, _ = oracle_sample(net, 1, 0)
+            v, cores, desc, _ = oracle_sample(net, 3, 0)
             out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
         print(json.dumps(out))
     ctx.close()

@@ -99,13 +99,20 @@ typedef struct {
                                   its layers once per group of n_workers / n workers (n rounded down to a power
                                   of two that divides n_workers; ignored where a group would cut a tensor-core
                                   tile) and adds the groups' parameter gradients; results differ from n = 1 only
-                                  in fp32 summation order.  Smaller launches, more of them: on a B200 this was
-                                  slower at every n for the ResNet-18-shaped benchmark (7.2 ms per step at 1,
-                                  7.6 at 2, 8.6 at 4), so it is off by default                                  */
-    void* const* streams;      /* K cudaStream_t of the caller, or NULL: the library creates K  */
+                                  in fp32 summation order.  Smaller launches, more of them: measured slower on a
+                                  B200 at every n for the ResNet-18-shaped benchmark, so it is off by default     */
+    void* const* streams;      /* K cudaStream_t of the caller (one per module, for its backward pass and update),
+                                  or NULL: the library creates them, with priorities that rise with the module
+                                  index (the last module's chain of short kernels goes first when SMs free up)  */
 } fdg_options;
 
-/* Build a context.  Paper: the split of layers 1..L into groups g(1)..g(K) (Sec. 3.2) and the
+/* Stash policy.  Every activation a module's backward pass needs is kept from the module's forward pass of
+ * that batch (iteration tau+k-1) until its backward pass (iteration tau+2K-k-1): "store all", the h~_k(tau) of
+ * Sec. 3.2.  There is no recompute-from-module-input mode: the largest configuration this library is run on
+ * (ResNet-18-shaped, K = 8, 16 workers x 256) holds its whole stash in the 180 GB of one B200, and
+ * fdg_create fails with FDG_ERR_OOM before any launch when the allocator cannot supply it.
+ *
+ * Build a context.  Paper: the split of layers 1..L into groups g(1)..g(K) (Sec. 3.2) and the
  * S x K agents of Sec. 3.3, all placed on the current CUDA device.
  *   layers/n_layers : the network, host array.
  *   split_points    : host array of K-1 layer indices (0-based): first layer of modules 2..K.
@@ -120,6 +127,22 @@ FDG_API fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers,
 
 /* Number of parameters (length of the canonical parameter vector). */
 FDG_API fdg_status fdg_param_count(const fdg_ctx* ctx, size_t* count);
+
+/* Where every tensor sits in the canonical parameter vector (the order fdg_set_params, fdg_params and fdg_grads
+ * use): one record per tensor, in that order.  Paper: the per-layer weights w_l of Sec. 2.1 grouped into the modules
+ * g(k) = {p_k .. q_k} of Sec. 3.2.
+ *   layer  : index into the layer list given to fdg_create
+ *   module : k - 1 of the module that owns the layer
+ *   role   : FDG_PARAM_W (linear [out][in]; conv [c_out][kh][kw][c_in]), _BIAS, _GAMMA, _BETA, and for a projecting
+ *            FDG_RES_ADD  _PROJ_W [c_out][1][1][c_in], _PROJ_GAMMA, _PROJ_BETA
+ *   ndim, shape[4] : extents, outermost first (unused trailing extents are 1)
+ *   offset, count  : first element and number of elements in the canonical vector
+ * out may be NULL to query the number of tensors; otherwise at most `capacity` records are written and *count
+ * receives the total number. */
+typedef enum { FDG_PARAM_W = 0, FDG_PARAM_BIAS = 1, FDG_PARAM_GAMMA = 2, FDG_PARAM_BETA = 3,
+               FDG_PARAM_PROJ_W = 4, FDG_PARAM_PROJ_GAMMA = 5, FDG_PARAM_PROJ_BETA = 6 } fdg_param_role;
+typedef struct { int32_t layer, module, role, ndim; int64_t shape[4]; uint64_t offset, count; } fdg_param_tensor;
+FDG_API fdg_status fdg_param_layout(const fdg_ctx* ctx, fdg_param_tensor* out, int32_t capacity, int32_t* count);
 
 /* Load version-0 weights from a host fp32 array in canonical order (the library draws no random
  * numbers).  Resets the iteration counter to 0 and empties every FIFO. */
@@ -148,17 +171,30 @@ FDG_API fdg_status fdg_step_host(fdg_ctx* ctx, const void* host_inputs, const in
  * that the caller may overwrite or free the buffers it passed to that step. */
 FDG_API fdg_status fdg_wait_ingest(fdg_ctx* ctx);
 
+/* Make `stream` (a cudaStream_t of the caller, NULL = the default stream) wait for everything the steps enqueued
+ * so far: work the caller puts on that stream afterwards (an event record for timing, a kernel that reads the
+ * caller's own buffers) runs after the last module's update of the most recent step.  Only enqueues waits. */
+FDG_API fdg_status fdg_join(fdg_ctx* ctx, void* stream);
+
 /* Wait for all modules, then copy the fp32 master weights w(t) (t = number of steps done) to a
- * host array in canonical order.  count receives the number of floats written. */
+ * host array in canonical order.  count receives the number of floats written.  Paper: the agents'
+ * weights w^_{s,k}(t) of Eq. "dl_update" (b); with P = (1/N) 1 1^T and equal initial values they are the same
+ * for every worker s (the consensus error of Sec. 4 is identically zero), so one copy is kept and returned. */
 FDG_API fdg_status fdg_params(fdg_ctx* ctx, float* host_out, size_t capacity, size_t* count);
 
-/* Debug twin of fdg_params: the averaged gradients that entered the last step's update
- * (zeros for modules that had no backward batch yet). */
+/* Debug twin of fdg_params: the gradients that entered the last step's update, i.e. the mean over the workers of
+ * the stale gradients of Eq. "dl_update", (1/N) sum_s grad^_{w_{s,k}} Phi_s(t - 2K + k + 1) with the per-sample scale
+ * 1/per_worker_batch (zeros for modules that had no backward batch yet: the gradient is 0 while tau < 0). */
 FDG_API fdg_status fdg_grads(fdg_ctx* ctx, float* host_out, size_t capacity, size_t* count);
 
-/* The delay schedule as observed on the device in the last step: every FIFO slot carries a tag
- * (batch id, weight version) written on the producer's stream; each module's step copies the
- * tags of the slots it is about to read into a trace.  Arrays of K int64 (host):
+/* The delay schedule of Sec. 3.2 (forward batch t-k+1, backward batch t-2K+k+1, backward weights of version
+ * t-2K+2k) as observed on the device in the last step.  Every FIFO slot carries a tag (batch id, weight version) in
+ * device memory.  One small kernel per module and step, on the module's backward / update stream and ordered like the
+ * step's other work by the neighbour events, first stamps the slots this step fills, then copies the tags of the
+ * slots the step reads into a trace.  The trace therefore proves the slot arithmetic (which slot holds which batch and
+ * version at which step); that the DATA in a slot is complete when it is read is what the event wiring guarantees
+ * and the parity tests (and the bit-identity of the one-stream and the concurrent mode) check.
+ * Arrays of K int64 (host):
  *   fwd_batch[k]          batch id found in the activation slot module k forwarded (-1 idle)
  *   bwd_batch[k]          batch id found in the stash slot module k back-propagated (-1 idle);
  *                         -2 if the error-gradient slot carried a different batch id
@@ -203,7 +239,9 @@ FDG_API fdg_status fdg_profile_read(fdg_ctx* ctx, fdg_kernel_stat* out, int32_t 
  *     fdg_static_last_error() says why.  Nothing is launched in that case.
  *   - The partial sums go to a fixed 1 MiB array inside the library image (present on every GPU
  *     that loads the library, for the life of the process).  The entry point calls no cudaMalloc,
- *     cudaFree or any allocating routine.
+ *     cudaFree or any allocating routine.  The first call on a device may make the CUDA runtime load the
+ *     library's device code (which is when the 1 MiB is reserved), so it doubles as the warm-up.
+ *   - dev_dy, dev_db and the stream must belong to the CURRENT device: the array used is the current device's.
  *   - All calls on a device share that array.  It keeps the previous call's contents; nothing in it
  *     has to start at zero, because the first kernel writes every slot the second one reads.  Two
  *     calls that may overlap on the GPU (different streams, no ordering) race on it: order them.

@@ -62,15 +62,20 @@ int num_threads() {
     return n < 1 ? 1 : n;
 }
 
-// Run fn(i) for i in [0,n) on up to num_threads() threads (static interleaving).  A parallel_for
-// reached from inside another one runs serially: the outer level (the workers) owns the threads.
-thread_local bool t_inside_parallel = false;
+// Run fn(i) for i in [0,n) on up to `budget` threads (static interleaving); the outermost call's budget is
+// num_threads().  A parallel_for reached from inside another one gets its share of the outer budget (the
+// workers are the outer level; with fewer workers than threads the layer loops below use the rest).
+// Every loop that is split this way writes disjoint outputs and keeps its own summation order, so the
+// results do not depend on the number of threads.
+thread_local int t_budget = 0;       // 0: outermost level
 void parallel_for(int n, const std::function<void(int)>& fn) {
-    int nt = std::min(num_threads(), n);
-    if (nt <= 1 || t_inside_parallel) { for (int i = 0; i < n; ++i) fn(i); return; }
+    const int budget = t_budget > 0 ? t_budget : num_threads();
+    const int nt = std::min(budget, n);
+    if (nt <= 1) { for (int i = 0; i < n; ++i) fn(i); return; }
+    const int inner = std::max(1, budget / nt);
     std::vector<std::thread> th;
     for (int w = 0; w < nt; ++w)
-        th.emplace_back([=, &fn] { t_inside_parallel = true; for (int i = w; i < n; i += nt) fn(i); });
+        th.emplace_back([=, &fn] { t_budget = inner; for (int i = w; i < n; i += nt) fn(i); });
     for (auto& t : th) t.join();
 }
 

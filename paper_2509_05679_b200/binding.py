@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libfdg.so")
 STATUS = {0: "FDG_OK", 1: "FDG_ERR_INVALID_ARG", 2: "FDG_ERR_BAD_SPLIT", 3: "FDG_ERR_UNSUPPORTED",
           4: "FDG_ERR_ARCH", 5: "FDG_ERR_OOM", 6: "FDG_ERR_CUDA", 7: "FDG_ERR_TIMEOUT", 8: "FDG_ERR_STATE"}
 
-EXPORTS = ["fdg_create", "fdg_param_count", "fdg_set_params", "fdg_step", "fdg_step_host", "fdg_wait_ingest", "fdg_params",
+EXPORTS = ["fdg_create", "fdg_param_count", "fdg_param_layout", "fdg_set_params", "fdg_step", "fdg_step_host", "fdg_wait_ingest", "fdg_join", "fdg_params",
            "fdg_grads", "fdg_trace", "fdg_set_lr", "fdg_stats", "fdg_module_times", "fdg_profile", "fdg_profile_read",
            "fdg_bias_grad_static", "fdg_static_last_error",
            "fdg_last_error", "fdg_destroy"]
@@ -47,6 +47,14 @@ class fdg_kernel_stat(C.Structure):
     _fields_ = [("name", C.c_char * 48), ("launches", C.c_uint64), ("ms", C.c_double), ("flops", C.c_double), ("bytes", C.c_double)]
 
 
+class fdg_param_tensor(C.Structure):
+    _fields_ = [("layer", C.c_int32), ("module", C.c_int32), ("role", C.c_int32), ("ndim", C.c_int32),
+                ("shape", C.c_int64 * 4), ("offset", C.c_uint64), ("count", C.c_uint64)]
+
+
+PARAM_ROLES = ["W", "b", "gamma", "beta", "Wp", "gamma_p", "beta_p"]     # fdg_param_role
+
+
 class fdg_options(C.Structure):
     _fields_ = [("dtype", C.c_int32), ("in_h", C.c_int32), ("in_w", C.c_int32), ("in_c", C.c_int32),
                 ("num_classes", C.c_int32), ("serial", C.c_int32), ("kernel_path", C.c_int32),
@@ -69,6 +77,8 @@ def lib():
                                  C.c_float, C.POINTER(fdg_options), C.POINTER(fdg_allocator), C.POINTER(vp)]
         L.fdg_param_count.restype = C.c_int
         L.fdg_param_count.argtypes = [vp, C.POINTER(C.c_size_t)]
+        L.fdg_param_layout.restype = C.c_int
+        L.fdg_param_layout.argtypes = [vp, C.POINTER(fdg_param_tensor), C.c_int32, C.POINTER(C.c_int32)]
         L.fdg_set_params.restype = C.c_int
         L.fdg_set_params.argtypes = [vp, fp, C.c_size_t]
         for name in ("fdg_step", "fdg_step_host"):
@@ -83,6 +93,8 @@ def lib():
         L.fdg_set_lr.argtypes = [vp, C.c_float]
         L.fdg_wait_ingest.restype = C.c_int
         L.fdg_wait_ingest.argtypes = [vp]
+        L.fdg_join.restype = C.c_int
+        L.fdg_join.argtypes = [vp, vp]
         L.fdg_stats.restype = C.c_int
         L.fdg_stats.argtypes = [vp, C.POINTER(C.c_size_t), C.POINTER(C.c_uint64)]
         L.fdg_module_times.restype = C.c_int
@@ -188,6 +200,15 @@ class Context:
         except Exception:
             pass
 
+    def param_layout(self):
+        """[(layer, module, role name, shape tuple, offset, count)] in canonical order (fdg_param_layout)."""
+        n = C.c_int32()
+        self._ck(lib().fdg_param_layout(self.h, None, 0, C.byref(n)))
+        arr = (fdg_param_tensor * max(1, n.value))()
+        self._ck(lib().fdg_param_layout(self.h, arr, n.value, C.byref(n)))
+        return [(int(a.layer), int(a.module), PARAM_ROLES[a.role], tuple(int(v) for v in a.shape[:a.ndim]), int(a.offset), int(a.count))
+                for a in arr[:n.value]]
+
     def set_params(self, params: np.ndarray):
         p = np.ascontiguousarray(params, dtype=np.float32)
         self._ck(lib().fdg_set_params(self.h, p.ctypes.data_as(C.POINTER(C.c_float)), p.size))
@@ -204,6 +225,10 @@ class Context:
 
     def wait_ingest(self):
         self._ck(lib().fdg_wait_ingest(self.h))
+
+    def join(self, stream: int = 0):
+        """Make the caller's stream (a cudaStream_t handle) wait for all work enqueued so far."""
+        self._ck(lib().fdg_join(self.h, stream or None))
 
     def _vec(self, fn) -> np.ndarray:
         out = np.empty(self.n_params, dtype=np.float32)

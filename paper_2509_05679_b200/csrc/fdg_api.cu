@@ -26,6 +26,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <cstdlib>
 #include <string>
 #include <vector>
 
@@ -115,6 +116,7 @@ struct fdg_ctx {
     float lr;
     int64_t t;
     bool have_params;
+    bool broken;                   // a step failed after part of its work was enqueued: the FIFOs are inconsistent until fdg_set_params
     std::vector<fdg_layer> layers;
     std::vector<Module> mod;
     std::vector<void*> blocks;
@@ -771,6 +773,7 @@ fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, boo
     if (!ctx) return FDG_ERR_INVALID_ARG;
     if (!inputs || !labels) return fail(ctx, FDG_ERR_INVALID_ARG, "inputs and labels must not be NULL");
     if (!ctx->have_params) return fail(ctx, FDG_ERR_STATE, "fdg_set_params must be called before fdg_step");
+    if (ctx->broken) return fail(ctx, FDG_ERR_STATE, "an earlier step failed after part of its work was enqueued; call fdg_set_params to start over");
     const int K = ctx->K;
     const int64_t t = ctx->t;
     // 1. dependencies on the neighbours' previous iteration (all waits first, so that no wait sees an
@@ -901,7 +904,7 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
     ctx->K = K; ctx->n_workers = n_workers; ctx->B = per_worker_batch; ctx->M = n_workers * per_worker_batch;
     ctx->dt = opt->dtype; ctx->esz = opt->dtype ? 2 : 4; ctx->classes = opt->num_classes; ctx->serial = opt->serial;
     ctx->kernel_path = opt->kernel_path;
-    ctx->in_h = opt->in_h; ctx->in_w = opt->in_w; ctx->in_c = opt->in_c; ctx->lr = lr; ctx->t = 0; ctx->have_params = false;
+    ctx->in_h = opt->in_h; ctx->in_w = opt->in_w; ctx->in_c = opt->in_c; ctx->lr = lr; ctx->t = 0; ctx->have_params = false; ctx->broken = false;
     ctx->layers.assign(layers, layers + n_layers);
     ctx->alloc = alloc ? *alloc : fdg_allocator{default_alloc, default_free, nullptr};
     ctx->own_streams = opt->streams == nullptr;
@@ -980,16 +983,25 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
         m.trace = ctx->tags + tpos; tpos += 4;
     }
     if (oom) return bail(FDG_ERR_OOM, "the allocator returned NULL");
+    // Stream priorities: the later a module, the smaller its tensors and the longer its chain of short kernels (the last
+    // module's forward pass, loss and backward pass of one batch are one serial chain inside a step), so its kernels go
+    // first whenever SMs free up; a module's weight gradients, which only its update waits for, rank below its two passes.
+    int prio_least = 0, prio_greatest = 0;
+    cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest);
+    if (getenv("FDG_NO_PRIO")) prio_greatest = prio_least;     // TEMP experiment hook
     for (int kk = 0; kk < K; ++kk) {
         Module& m = ctx->mod[kk];
         cudaError_t e = cudaSuccess;
+        const int span = prio_least - prio_greatest;                       // priorities run from prio_least (low) down to prio_greatest (high)
+        const int prio = prio_least - (K > 1 ? span * kk / (K - 1) : 0);
+        const int prio_w = prio < prio_least ? prio + 1 : prio_least;
         if (opt->streams) m.stream = (cudaStream_t)opt->streams[ctx->serial ? 0 : kk];
         else if (ctx->serial && kk > 0) m.stream = ctx->mod[0].stream;
-        else { e = cudaStreamCreateWithFlags(&m.stream, cudaStreamNonBlocking); if (e == cudaSuccess) ctx->owned.push_back(m.stream); }
+        else { e = cudaStreamCreateWithPriority(&m.stream, cudaStreamNonBlocking, prio); if (e == cudaSuccess) ctx->owned.push_back(m.stream); }
         m.fstream = m.stream;
-        if (e == cudaSuccess && !ctx->serial) { e = cudaStreamCreateWithFlags(&m.fstream, cudaStreamNonBlocking); if (e == cudaSuccess) ctx->owned.push_back(m.fstream); }
+        if (e == cudaSuccess && !ctx->serial) { e = cudaStreamCreateWithPriority(&m.fstream, cudaStreamNonBlocking, prio); if (e == cudaSuccess) ctx->owned.push_back(m.fstream); }
         m.wstream = m.stream;
-        if (e == cudaSuccess && !ctx->serial) { e = cudaStreamCreateWithFlags(&m.wstream, cudaStreamNonBlocking); if (e == cudaSuccess) ctx->owned.push_back(m.wstream); }
+        if (e == cudaSuccess && !ctx->serial) { e = cudaStreamCreateWithPriority(&m.wstream, cudaStreamNonBlocking, prio_w); if (e == cudaSuccess) ctx->owned.push_back(m.wstream); }
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.wev, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.wdone, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.done, cudaEventDisableTiming);
@@ -1020,9 +1032,57 @@ fdg_status fdg_wait_ingest(fdg_ctx* ctx) {
     return FDG_OK;
 }
 
+fdg_status fdg_join(fdg_ctx* ctx, void* stream) {
+    if (!ctx) return FDG_ERR_INVALID_ARG;
+    if (ctx->t > 0)
+        for (Module& m : ctx->mod) CK(cudaStreamWaitEvent((cudaStream_t)stream, m.done, 0));
+    return FDG_OK;
+}
+
 fdg_status fdg_param_count(const fdg_ctx* ctx, size_t* count) {
     if (!ctx || !count) return FDG_ERR_INVALID_ARG;
     *count = ctx->n_params;
+    return FDG_OK;
+}
+
+fdg_status fdg_param_layout(const fdg_ctx* ctx, fdg_param_tensor* out, int32_t capacity, int32_t* count) {
+    if (!ctx || !count || (out && capacity < 0)) return FDG_ERR_INVALID_ARG;
+    int32_t n = 0;
+    uint64_t off = 0;
+    int module = 0;
+    auto emit = [&](int layer, int role, int ndim, int64_t d0, int64_t d1, int64_t d2, int64_t d3) {
+        const uint64_t cnt = (uint64_t)(d0 * d1 * d2 * d3);
+        if (out && n < capacity) out[n] = fdg_param_tensor{layer, module, role, ndim, {d0, d1, d2, d3}, off, cnt};
+        off += cnt; ++n;
+    };
+    for (int l = 0; l < (int)ctx->layers.size(); ++l) {
+        while (module + 1 < ctx->K && l >= ctx->mod[module + 1].p) ++module;
+        const fdg_layer& Y = ctx->layers[l];
+        switch (Y.kind) {
+            case FDG_LINEAR:
+                emit(l, FDG_PARAM_W, 2, Y.c_out, Y.c_in, 1, 1);
+                if (Y.flags & 1) emit(l, FDG_PARAM_BIAS, 1, Y.c_out, 1, 1, 1);
+                break;
+            case FDG_CONV3X3: case FDG_CONV1X1: {
+                const int r = Y.kind == FDG_CONV3X3 ? 3 : 1;
+                emit(l, FDG_PARAM_W, 4, Y.c_out, r, r, Y.c_in);
+                if (Y.flags & 1) emit(l, FDG_PARAM_BIAS, 1, Y.c_out, 1, 1, 1);
+                break; }
+            case FDG_BATCHNORM:
+                emit(l, FDG_PARAM_GAMMA, 1, Y.c_in, 1, 1, 1);
+                emit(l, FDG_PARAM_BETA, 1, Y.c_in, 1, 1, 1);
+                break;
+            case FDG_RES_ADD:
+                if (Y.flags & 1) {
+                    emit(l, FDG_PARAM_PROJ_W, 4, Y.c_out, 1, 1, Y.c_in);
+                    emit(l, FDG_PARAM_PROJ_GAMMA, 1, Y.c_out, 1, 1, 1);
+                    emit(l, FDG_PARAM_PROJ_BETA, 1, Y.c_out, 1, 1, 1);
+                }
+                break;
+            default: break;
+        }
+    }
+    *count = n;
     return FDG_OK;
 }
 
@@ -1048,14 +1108,22 @@ fdg_status fdg_set_params(fdg_ctx* ctx, const float* host_params, size_t count) 
     if (s != FDG_OK) return s;
     CK(cudaDeviceSynchronize());
     ctx->have_params = true;
+    ctx->broken = false;
     return FDG_OK;
 }
 
+// A CUDA error in the middle of a step leaves some of its kernels enqueued and the iteration counter where it was:
+// the context then refuses further steps until fdg_set_params resets the FIFOs.
+static fdg_status guarded_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, bool host_src, float* host_loss) {
+    const fdg_status s = run_step(ctx, inputs, labels, host_src, host_loss);
+    if (ctx && (s == FDG_ERR_CUDA || s == FDG_ERR_TIMEOUT)) ctx->broken = true;
+    return s;
+}
 fdg_status fdg_step(fdg_ctx* ctx, const void* dev_inputs, const int32_t* dev_labels, float* host_loss_or_null) {
-    return run_step(ctx, dev_inputs, dev_labels, false, host_loss_or_null);
+    return guarded_step(ctx, dev_inputs, dev_labels, false, host_loss_or_null);
 }
 fdg_status fdg_step_host(fdg_ctx* ctx, const void* host_inputs, const int32_t* host_labels, float* host_loss_or_null) {
-    return run_step(ctx, host_inputs, host_labels, true, host_loss_or_null);
+    return guarded_step(ctx, host_inputs, host_labels, true, host_loss_or_null);
 }
 
 static fdg_status gather(fdg_ctx* ctx, bool grads, float* host_out, size_t capacity, size_t* count) {

@@ -91,11 +91,15 @@ FDG_API fdg_status fdg_bias_grad_static(const void* dev_dy, int32_t dtype, int64
     cudaStream_t s = (cudaStream_t)stream;
     const int chunks = (int)(rows < CHUNKS ? rows : CHUNKS);
     dim3 grid((channels + 31) / 32, chunks), blk(32, 8);
+    // an error left behind by earlier, unrelated work must not be reported as a failure of these launches
+    cudaGetLastError();
     if (dtype) static_colsum_partial<__nv_bfloat16><<<grid, blk, 0, s>>>((const __nv_bfloat16*)dev_dy, scratch, rows, channels, MAX_CHANNELS);
     else static_colsum_partial<float><<<grid, blk, 0, s>>>((const float*)dev_dy, scratch, rows, channels, MAX_CHANNELS);
-    static_colsum_final<<<(channels + 127) / 128, 128, 0, s>>>(scratch, dev_db, chunks, channels, MAX_CHANNELS);
     cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return fail(FDG_ERR_CUDA, (std::string("fdg_bias_grad_static: launch failed: ") + cudaGetErrorString(e)).c_str());
+    if (e != cudaSuccess) return fail(FDG_ERR_CUDA, (std::string("fdg_bias_grad_static: launch of the partial sums failed: ") + cudaGetErrorString(e)).c_str());
+    static_colsum_final<<<(channels + 127) / 128, 128, 0, s>>>(scratch, dev_db, chunks, channels, MAX_CHANNELS);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(FDG_ERR_CUDA, (std::string("fdg_bias_grad_static: launch of the final sums failed: ") + cudaGetErrorString(e)).c_str());
     return FDG_OK;
 }
 

@@ -16,27 +16,51 @@ def tensor_slices(layers):
     return out
 
 
+FP32_FLOOR = 5e-2          # of the tensor's rms
+
+
 def max_rel_err(a, b, layers):
-    """Per tensor: max_i |a_i - b_i| / max(|b_i|, 0.1 * rms(b)); returns the worst tensor.
-    The floor exists because an fp32 sum of terms of size s carries an absolute error of about
+    """Per tensor: max_i |a_i - b_i| / max(|b_i|, 5e-2 * rms(b)); returns the worst tensor.
+    The floor exists because an fp32 sum of terms of size s carries an absolute error of a few
     2^-24 * s however small the sum itself turns out (cancellation): an element far below the
-    tensor's scale cannot be held to a RELATIVE 1e-5 by any fp32 evaluation order."""
+    tensor's scale cannot be held to a RELATIVE 1e-5 by any fp32 evaluation order.  Measured over
+    the fp32 tests of this directory: the worst element is off by 2.2e-7 of its tensor's rms (about
+    four fp32 ulps of an rms-sized value), i.e. 2.2e-5 against a floor of 1e-2 rms and 4.4e-6 against
+    this one."""
     worst, where = 0.0, ""
     for name, sl in tensor_slices(layers):
         bb, aa = np.asarray(b[sl], np.float64), np.asarray(a[sl], np.float64)
-        floor = 0.1 * np.sqrt(np.mean(bb * bb)) + 1e-30
+        floor = FP32_FLOOR * np.sqrt(np.mean(bb * bb)) + 1e-30
         e = float(np.max(np.abs(aa - bb) / np.maximum(np.abs(bb), floor)))
         if e > worst:
             worst, where = e, name
     return worst, where
 
 
-def grad_rel_l2(a, b, layers, min_norm=1e-12):
+def gradient_groups(layers, pair_bn=False):
+    """[(name, index array)] of the tensors a gradient comparison looks at.  pair_bn: gamma and beta of one
+    batch-norm form one group (in a network without ReLU layers a shift of a batch-norm's output is removed again
+    by the next batch-norm, so the gradient of beta is what the zero padding at the image border leaves of it,
+    tens of times smaller than gamma's and no scale to measure an error against)."""
+    sl = tensor_slices(layers)
+    out, i = [], 0
+    while i < len(sl):
+        name, s = sl[i]
+        if pair_bn and name.split(".")[1].startswith("gamma") and i + 1 < len(sl):
+            out.append((name + "+beta", np.r_[s, sl[i + 1][1]]))
+            i += 2
+        else:
+            out.append((name, np.r_[s]))
+            i += 1
+    return out
+
+
+def grad_rel_l2(a, b, layers, min_norm=1e-12, pair_bn=False):
     """Per tensor ||a - b||_2 / ||b||_2 (tensors whose reference gradient is ~0 are skipped).
     Returns (worst error, its tensor, {tensor: error})."""
     worst, where, per = 0.0, "", {}
-    for name, sl in tensor_slices(layers):
-        bb, aa = np.asarray(b[sl], np.float64), np.asarray(a[sl], np.float64)
+    for name, ix in gradient_groups(layers, pair_bn):
+        bb, aa = np.asarray(b[ix], np.float64), np.asarray(a[ix], np.float64)
         nb = np.linalg.norm(bb)
         if nb < min_norm:
             continue
@@ -45,6 +69,29 @@ def grad_rel_l2(a, b, layers, min_norm=1e-12):
         if e > worst:
             worst, where = e, name
     return worst, where, per
+
+
+def grad_max_err(a, b, layers, min_norm=1e-12, pair_bn=False):
+    """Element by element: per tensor max_i |a_i - b_i| / max_i |b_i|.  Returns (worst, its tensor)."""
+    worst, where = 0.0, ""
+    for name, ix in gradient_groups(layers, pair_bn):
+        bb, aa = np.asarray(b[ix], np.float64), np.asarray(a[ix], np.float64)
+        if np.linalg.norm(bb) < min_norm:
+            continue
+        e = float(np.max(np.abs(aa - bb)) / np.max(np.abs(bb)))
+        if e > worst:
+            worst, where = e, name
+    return worst, where
+
+
+def ulp_perturbed(x, fraction=1e-3, seed=5):
+    """A copy of a bf16-representable array with `fraction` of its values moved to the next bf16 value away
+    from zero: the smallest change of the inputs a bf16 run can see."""
+    g = np.random.Generator(np.random.Philox(key=seed))
+    flat = np.ascontiguousarray(x, dtype=np.float32).reshape(-1).copy()
+    idx = g.choice(flat.size, max(1, int(fraction * flat.size)), replace=False)
+    flat[idx] = (flat[idx].view(np.uint32) + np.uint32(0x10000)).view(np.float32)
+    return flat.reshape(x.shape)
 
 
 def make_oracle(orc, net: sy.Net, params, storage_model=True):
@@ -90,22 +137,26 @@ def closed_form_trace(K, t):
 
 
 def run_parity(orc, net: sy.Net, steps: int, *, param_tol=None, grad_tol=None, grad_best_tol=None, loss_tol=None,
-               perturb=True, kink_guard=None, grad_steps=None, grad_tail=None, grad_tol_later=None, **ctx_kw):
+               perturb=True, kink_guard=None, grad_steps=None, grad_tol_later=None, elem_tol=None, pair_bn=False,
+               noise_factor=None, elem_noise_factor=None, **ctx_kw):
     """Step both implementations `steps` times; check the schedule bit-exactly after every step and
     parameters / gradients / loss within the given tolerances.  Returns the per-step records.
 
-    Gradients: every tensor must be within `grad_tol` at every step.  `grad_best_tol` is a much
+    Gradients: every tensor must be within `grad_tol` (relative L2) at every step, and, with `elem_tol`,
+    every element within `elem_tol` of the tensor's largest element.  `grad_best_tol` is a much
     tighter bound on each tensor's BEST step: a pre-activation that lands on the other side of a
     ReLU / max-pool kink in one precision but not the other legitimately changes a few terms of a
     gradient sum in that step, whereas a wrong formula is wrong at every step.
-    `grad_steps`: check gradients only while t < grad_steps (afterwards the two trajectories have
-    moved apart and a gradient comparison compares different weights).  `grad_tail`: hold only the
-    last `grad_tail` tensors to `grad_tol` and ask the whole gradient for a cosine similarity of 0.7
-    (deep batch-norm networks amplify a single rounding difference by orders of magnitude on the
-    way back to the first layers).  `grad_tol_later`: tolerance after the run's first backward pass
-    (t = K-1, held to `grad_tol`): from then on the weights of the two runs differ by their
-    earlier gradient differences."""
+    `grad_steps`: check gradients only while t < grad_steps.  `grad_tol_later`: tolerance after the run's
+    first backward pass (t = K-1, held to `grad_tol`): from then on the weights of the two runs differ by
+    their earlier gradient differences.
+    `noise_factor` (bf16 networks with ReLU layers, where two bf16 evaluations of the same gradient differ by
+    tens of percent, see tests/test_oracle_pins.py): a second oracle runs beside the first on inputs of which
+    0.1 % were moved by one bf16 ulp; a tensor may deviate from the oracle by `grad_tol` or by `noise_factor`
+    times what that twin deviates, whichever is larger (`elem_noise_factor`: the same for the element-wise
+    bound `elem_tol`)."""
     from paper_2509_05679_b200 import binding
+    import torch
     bf16 = net.dtype == "bf16"
     p0 = sy.init_params(net.layers, 0, bf16=False)
     if perturb:
@@ -113,43 +164,51 @@ def run_parity(orc, net: sy.Net, steps: int, *, param_tol=None, grad_tol=None, g
     if bf16:
         p0 = sy.round_to_bf16(p0)
     stream = pick_data_stream(orc, net, p0, steps, kink_guard) if kink_guard else 0
+    if kink_guard:
+        print(f"{net.name}: data stream {stream} keeps every pre-activation {kink_guard:g} away from the kinks")
     o = make_oracle(orc, net, p0)
+    twin = make_oracle(orc, net, p0) if noise_factor else None
     ctx = make_ctx(net, p0, **ctx_kw)
     rec, best = [], {}
     try:
         for t in range(steps):
             x, y = sy.batch_inputs(net, t, stream), sy.batch_labels(net, t, stream)
             lo, _ = o.step(x, y, net.lr)
-            import torch
             lg = ctx.step(binding.to_device(net.dtype, x), torch.from_numpy(y).cuda(), want_loss=True)
             fo, bo, vo, _ = o.trace()
             fg, bg, vg = ctx.trace()
             assert (fg == fo).all() and (bg == bo).all() and (vg == vo).all(), (t, fg, fo, bg, bo, vg, vo)
             fc, bc, vc = closed_form_trace(net.K, t)
             assert (fg == fc).all() and (bg == bc).all() and (vg == vc).all()
-            r = {"t": t, "loss_o": lo, "loss_g": lg}
+            r = {"t": t, "loss_o": lo, "loss_g": lg, "stream": stream}
             if np.isnan(lo):
                 assert np.isnan(lg)
             elif loss_tol is not None:
                 assert abs(lg - lo) <= loss_tol * max(abs(lo), 1e-6), (t, lg, lo)
+            if twin is not None:
+                twin.step(ulp_perturbed(x, 1e-3, 5 + t), y, net.lr)
             if grad_tol is not None and (grad_steps is None or t < grad_steps):
                 g_avg = np.mean([o.grads(s) for s in range(net.n_workers)], axis=0)     # P = 11^T/N averages the workers
                 g_gpu = ctx.grads()
-                r["grad_err"], r["grad_where"], per = grad_rel_l2(g_gpu, g_avg, net.layers)
+                r["grad_err"], r["grad_where"], per = grad_rel_l2(g_gpu, g_avg, net.layers, pair_bn=pair_bn)
                 for k_, e_ in per.items():
                     best[k_] = min(best.get(k_, np.inf), e_)
-                if grad_tail is None and grad_tol_later is None:
-                    assert r["grad_err"] <= grad_tol, (t, r)
-                elif grad_tail is None:
-                    first = t == net.K - 1          # the first backward pass of the run: no weight has changed yet
-                    assert r["grad_err"] <= (grad_tol if first else grad_tol_later), (t, r)
-                elif per:
-                    tail = list(per.items())[-grad_tail:]
-                    assert all(e_ <= grad_tol for _, e_ in tail), (t, tail)
-                    nz = np.abs(g_avg) > 0
-                    cos = float(np.dot(g_gpu[nz], g_avg[nz]) / (np.linalg.norm(g_gpu[nz]) * np.linalg.norm(g_avg[nz]) + 1e-300))
-                    r["grad_cos"] = cos
-                    assert cos >= 0.7, (t, cos)
+                tol = grad_tol if (grad_tol_later is None or t == net.K - 1) else grad_tol_later
+                if twin is None:
+                    assert r["grad_err"] <= tol, (t, r)
+                else:
+                    g_twin = np.mean([twin.grads(s) for s in range(net.n_workers)], axis=0)
+                    _, _, noise = grad_rel_l2(g_twin, g_avg, net.layers, pair_bn=pair_bn)
+                    bad = {k_: (e_, noise.get(k_, 0.0)) for k_, e_ in per.items() if e_ > max(tol, noise_factor * noise.get(k_, 0.0))}
+                    r["noise_max"] = max(noise.values()) if noise else 0.0
+                    assert not bad, (t, bad)
+                if elem_tol is not None:
+                    r["elem_err"], r["elem_where"] = grad_max_err(g_gpu, g_avg, net.layers, pair_bn=pair_bn)
+                    bound = elem_tol
+                    if twin is not None and elem_noise_factor:
+                        r["elem_noise"] = grad_max_err(g_twin, g_avg, net.layers, pair_bn=pair_bn)[0]
+                        bound = max(elem_tol, elem_noise_factor * r["elem_noise"])
+                    assert r["elem_err"] <= bound, (t, r)
             if param_tol is not None:
                 r["param_err"], r["param_where"] = max_rel_err(ctx.params(), o.params(0), net.layers)
                 assert r["param_err"] <= param_tol, (t, r)
@@ -157,7 +216,7 @@ def run_parity(orc, net: sy.Net, steps: int, *, param_tol=None, grad_tol=None, g
     finally:
         ctx.close()
     if grad_best_tol is not None:
-        assert best and len(best) == len(tensor_slices(net.layers)), "some tensor never received a gradient"
+        assert best and len(best) == len(gradient_groups(net.layers, pair_bn)), "some tensor never received a gradient"
         bad = {k_: e_ for k_, e_ in best.items() if e_ > grad_best_tol}
         assert not bad, bad
     return rec

@@ -1,16 +1,22 @@
 """bf16 path (bf16 activations / weight copies / error gradients, fp32 accumulation, fp32 master
 weights) against the oracle run with the same bf16 storage points: bit-exact schedule, gradients
-within 2e-2 (per tensor, relative L2), loss trajectory within 1e-2 (relative, every step).
+within 2e-2 (per tensor relative L2, and element by element against the tensor's largest element), loss
+trajectory within 1e-2 (relative, every step).
 
-What limits these checks is the problem, not the kernels: with bf16 storage, moving 0.1 % of the
-input values by one bf16 ulp changes the ORACLE's own gradients of a small batch-norm ResNet by
-5-10 % (every changed value re-draws the rounding of everything downstream).  So
-  * single-module nets are held to 2e-3 on every tensor at the first step (same rounding points,
-    nothing to amplify): this is the test of the bf16 kernels themselves;
-  * multi-module runs check the schedule, the loss trajectory, and gradients while the two
-    trajectories are still together (until every module has had its first backward pass);
-  * deep batch-norm nets hold only the last tensors to 2e-2 and ask the rest for the right
-    direction; their full-depth logic is what the fp32 tests pin to 1e-5."""
+How far a gradient comparison can go is a property of the problem, measured on the oracle alone in
+tests/test_oracle_pins.py: two bf16 evaluations of a DEEP ReLU network differ by tens of percent (ReLU masks
+flip where a stored value re-draws its rounding), while shallow networks and deep networks without ReLU layers
+reproduce to about 1 %.  So
+  * every tensor-core kernel family meets the oracle in a shallow network of its own (at most three convolutions
+    deep, full channel widths 64..512, strides 1 and 2, projections, 32x32 .. 4x4 images, even, odd and ragged batch
+    sizes): without its ReLU layers at 2e-2 on EVERY tensor and 3e-2 element by element, with them at the larger of
+    2e-2 and three times the oracle's own response to a one-ulp change of 0.1 % of the inputs (wide layers and a
+    few hundred pixels per channel already put that response at 1-3 %);
+  * the ResNet-18-shaped networks, split into 4 and 8 modules, run WITHOUT their ReLU layers at lr 0.05 with every
+    tensor of every module within 2e-2 at every step (wrong taps, batch-norm reductions and weight versions show
+    there, see test_relu_free_network_shows_a_wrong_weight_version_at_the_gpu_tests_tolerance);
+  * the same networks WITH their ReLU layers check the schedule, the loss trajectory and every tensor against
+    the larger of 2e-2 and three times the oracle's own response to a one-ulp change of 0.1 % of the inputs."""
 import numpy as np
 import pytest
 
@@ -23,20 +29,19 @@ GRAD_TOL, LOSS_TOL = 2e-2, 1e-2
 
 def test_config2_shaped_mlp_50_step_loss_trajectory(orc):
     net = sy.config(1, n_workers=4, batch=32, width_div=4)
-    rec = run_parity(orc, net, 50, grad_tol=GRAD_TOL, grad_tol_later=5e-2, grad_steps=2 * net.K - 1, loss_tol=LOSS_TOL, perturb=False)
+    rec = run_parity(orc, net, 50, grad_tol=GRAD_TOL, noise_factor=3.0, grad_steps=2 * net.K + 2, loss_tol=LOSS_TOL, perturb=False)
     assert sum(not np.isnan(r["loss_g"]) for r in rec) == 50 - (net.K - 1)
 
 
 def test_config3_shaped_vgg(orc):
     net = sy.config(2, n_workers=2, batch=4, width_div=4)
-    net.lr = 0.01          # 8 samples per step: at 0.05 this tiny run is unstable and any two precisions part ways
-    run_parity(orc, net, 2 * net.K + 2, grad_tol=GRAD_TOL, grad_steps=2 * net.K - 1, grad_tail=2, loss_tol=LOSS_TOL, perturb=False)
+    run_parity(orc, net, 2 * net.K + 2, grad_tol=GRAD_TOL, noise_factor=3.0, loss_tol=LOSS_TOL, perturb=False)
 
 
 def test_shallow_resnet_three_modules_identity_and_projection_blocks(orc):
     layers, bs = sy.resnet_layers(widths=(16, 32), blocks=1, in_c=3, classes=10)
     net = sy.Net("resnet-2-blocks", layers, [bs[0], bs[1]], 16, 16, 3, 10, 2, 4, 0.05, "bf16")
-    run_parity(orc, net, 3 * net.K, grad_tol=GRAD_TOL, grad_steps=2 * net.K - 1, grad_tail=2, loss_tol=LOSS_TOL)
+    run_parity(orc, net, 3 * net.K, grad_tol=GRAD_TOL, noise_factor=3.0, loss_tol=LOSS_TOL)
 
 
 C = 16
@@ -69,6 +74,57 @@ SINGLE_MODULE_NETS = {
     # the same kernels with batch-norm sums taken in their epilogues: first layer + one identity block of 64 channels at 32x32
     "tensor-core-bn-block-32x32": sy.resnet_layers(widths=(64,), blocks=1)[0],
 }
+
+
+def _block(c, w, stride):
+    """One basic block (conv-bn-relu-conv-bn, shortcut with a 1x1 projection where the shape changes)."""
+    proj = sy.FLAG_PROJ if (stride != 1 or c != w) else 0
+    return [(sy.RES_BEGIN, c, c, 1, 0), (sy.CONV3X3, c, w, stride, 0), (sy.BATCHNORM, w, w, 1, 0), (sy.RELU, w, w, 1, 0),
+            (sy.CONV3X3, w, w, 1, 0), (sy.BATCHNORM, w, w, 1, 0), (sy.RES_ADD, c, w, stride, proj), (sy.RELU, w, w, 1, 0)]
+
+
+def _head(c):
+    return [(sy.GLOBAL_AVGPOOL, c, c, 1, 0), (sy.LINEAR, c, 10, 1, 1)]
+
+
+# One shallow network per tensor-core kernel family at the channel widths and image sizes of the ResNet-18- and VGG-shaped
+# configurations; inputs with 64..512 channels feed the wide layers directly, so nothing is deeper than three convolutions.
+FAMILY_NETS = {
+    # 3x3 stride 2, 64 -> 128 (forward with element strides, four-parity-class input gradient, strided weight gradient)
+    "stride2-3x3-64-128": ((16, 16, 3), [(sy.CONV3X3, 3, 64, 1, 1), (sy.RELU, 64, 64, 1, 0), (sy.CONV3X3, 64, 128, 2, 1), (sy.RELU, 128, 128, 1, 0),
+                                         (sy.CONV3X3, 128, 128, 1, 1), (sy.RELU, 128, 128, 1, 0)] + _head(128)),
+    # first layer + a projecting block 64 -> 128: 1x1 stride-2 projection (input gradient with empty parity classes)
+    "projection-block-64-128": ((16, 16, 3), [(sy.CONV3X3, 3, 64, 1, 0), (sy.BATCHNORM, 64, 64, 1, 0), (sy.RELU, 64, 64, 1, 0)] + _block(64, 128, 2) + _head(128)),
+    # 128 -> 128 at 16x16 in rows mode as a CTA pair, then 128 -> 256 stride 2 and 256 -> 256 at 8x8
+    "projection-block-128-256": ((16, 16, 128), [(sy.CONV3X3, 128, 128, 1, 1), (sy.RELU, 128, 128, 1, 0)] + _block(128, 256, 2) + _head(256)),
+    # 256 -> 256 at 8x8 (256-column tile, CTA pairs, rows-mode weight gradient), then 256 -> 512 stride 2 and 512 -> 512 at 4x4
+    "projection-block-256-512": ((8, 8, 256), [(sy.CONV3X3, 256, 256, 1, 1), (sy.RELU, 256, 256, 1, 0)] + _block(256, 512, 2) + _head(512)),
+    "identity-block-256-8x8": ((8, 8, 256), [(sy.CONV3X3, 256, 256, 1, 0), (sy.BATCHNORM, 256, 256, 1, 0), (sy.RELU, 256, 256, 1, 0)] + _block(256, 256, 1) + _head(256)),
+    # 4x4 images: a 128-pixel tile spans eight samples
+    "identity-block-512-4x4": ((4, 4, 512), [(sy.CONV3X3, 512, 512, 1, 0), (sy.BATCHNORM, 512, 512, 1, 0), (sy.RELU, 512, 512, 1, 0)] + _block(512, 512, 1) + _head(512)),
+    # the VGG-shaped tail: 512-channel layers with bias and ReLU in the epilogue, max-pool in front
+    "vgg-tail-256-512": ((8, 8, 256), [(sy.CONV3X3, 256, 256, 1, 1), (sy.RELU, 256, 256, 1, 0), (sy.MAXPOOL2, 256, 256, 2, 0),
+                                      (sy.CONV3X3, 256, 512, 1, 1), (sy.RELU, 512, 512, 1, 0), (sy.CONV3X3, 512, 512, 1, 1), (sy.RELU, 512, 512, 1, 0)] + _head(512)),
+}
+
+
+@pytest.mark.parametrize("relu", [False, True])
+@pytest.mark.parametrize("workers,batch", [(2, 8), (3, 8), (3, 3)])
+@pytest.mark.parametrize("name", sorted(FAMILY_NETS))
+def test_every_tensor_core_kernel_family_matches_the_oracle_on_every_tensor(orc, name, workers, batch, relu):
+    """2 x 8 samples: even tile counts (CTA pairs) and batch-norm sums taken in the conv epilogues (a 4x4-image tile is
+    eight samples of one worker); 3 x 8: odd tile counts (no pairs); 3 x 3: ragged last tiles, tiles that straddle workers
+    (separate statistics pass), contraction splits that do not divide the number of steps."""
+    shape, layers = FAMILY_NETS[name]
+    net = sy.Net(name, layers, [], *shape, 10, workers, batch, 0.05, "bf16")
+    if relu:
+        rec = run_parity(orc, net, 1, grad_tol=GRAD_TOL, noise_factor=3.0, elem_tol=3e-2, elem_noise_factor=3.0, loss_tol=1e-3)
+    else:
+        rec = run_parity(orc, sy.without_relu(net), 1, grad_tol=GRAD_TOL, elem_tol=3e-2, pair_bn=True, loss_tol=1e-3)
+    print(name, workers, batch, relu, rec[0])
+    assert rec[0]["grad_err"] > 0
+
+
 INPUT_SHAPE = {"mlp": (1, 1, 48), "tensor-core-rows-32x32": (32, 32, 3), "tensor-core-bn-block-32x32": (32, 32, 3),
                "tensor-core-64x64": (64, 64, 3)}
 
@@ -99,12 +155,22 @@ def test_odd_worker_and_batch_counts(orc, name):
 
 def test_config4_shaped_resnet(orc):
     net = sy.config(3, n_workers=2, batch=4, width_div=4)
-    run_parity(orc, net, 2 * net.K + 2, grad_tol=GRAD_TOL, grad_steps=2 * net.K - 1, grad_tail=2, loss_tol=LOSS_TOL)
+    run_parity(orc, net, 2 * net.K + 2, grad_tol=GRAD_TOL, noise_factor=3.0, loss_tol=LOSS_TOL)
 
 
 def test_config5_shaped_resnet_eight_modules(orc):
     net = sy.config(4, n_workers=2, batch=2, width_div=8)
-    run_parity(orc, net, 2 * net.K + 2, grad_tol=GRAD_TOL, grad_steps=2 * net.K - 1, grad_tail=2, loss_tol=LOSS_TOL)
+    run_parity(orc, net, 2 * net.K + 2, grad_tol=GRAD_TOL, noise_factor=3.0, loss_tol=LOSS_TOL)
+
+
+@pytest.mark.parametrize("idx,workers,batch,width_div", [(3, 2, 4, 4), (4, 2, 2, 4)])
+def test_relu_free_resnet18_shaped_every_tensor_of_every_module_at_every_step(orc, idx, workers, batch, width_div):
+    """K = 4 and K = 8, lr 0.05: without ReLU layers two bf16 evaluations agree to about 1 %, so every convolution,
+    batch-norm and shortcut gradient of every module is held to 2e-2 (L2 and element by element) from the module's
+    first backward pass on, through several weight versions."""
+    net = sy.without_relu(sy.config(idx, n_workers=workers, batch=batch, width_div=width_div))
+    rec = run_parity(orc, net, 2 * net.K + 1, grad_tol=GRAD_TOL, elem_tol=3e-2, pair_bn=True, loss_tol=LOSS_TOL)
+    print(net.name, max(r.get("grad_err", 0) for r in rec), max(r.get("elem_err", 0) for r in rec))
 
 
 @pytest.mark.parametrize("widths", [(64, 128), (64, 256)])
@@ -112,10 +178,10 @@ def test_cta_pair_kernels_equal_single_cta_kernels_bitwise(orc, widths):
     """Residual blocks at 128 / 256 channels (3x3, stride 2, 1x1 projection): the CTA-pair tensor-core kernels
     (kernel_path 0) and the single-CTA ones (kernel_path 2) run the same MMAs in the same order, so gradients and
     weights must be identical (no layer here is wide and large enough for the paired rows-mode kernel, whose
-    accumulation order differs); against the oracle the first step holds the usual bf16 gradient tolerance."""
+    accumulation order differs).  Against the oracle these kernels are held to 2e-2 by the family networks above."""
     import torch
     from paper_2509_05679_b200 import binding
-    from harness import make_ctx, make_oracle, grad_rel_l2
+    from harness import make_ctx
     net = sy.Net("blocks", sy.resnet_layers(widths=widths, blocks=1)[0], [], 16, 16, 3, 10, 2, 4, 0.05, "bf16")
     p0 = sy.perturb_params(sy.init_params(net.layers, 0, bf16=True), net.layers, 7, 0.1)
     out = {}
@@ -131,8 +197,3 @@ def test_cta_pair_kernels_equal_single_cta_kernels_bitwise(orc, widths):
     for a, b in zip(out[0][0], out[2][0]):
         assert np.array_equal(a, b)
     assert np.array_equal(out[0][1], out[2][1])
-    o = make_oracle(orc, net, p0)
-    o.step(sy.batch_inputs(net, 0), sy.batch_labels(net, 0), net.lr)
-    g_avg = np.mean([o.grads(s) for s in range(net.n_workers)], axis=0)
-    err, where, _ = grad_rel_l2(out[0][0][0], g_avg, net.layers)
-    assert err <= 5e-2, (err, where)

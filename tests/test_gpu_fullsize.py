@@ -10,6 +10,8 @@ holds at any size:
     front of it, so <dW[c], W[c]> = 0 for every such channel (this ties the convolution's weight
     gradient, the batch-norm backward pass and the weights the backward pass read together).
 """
+import os
+
 import numpy as np
 import pytest
 
@@ -17,14 +19,72 @@ from paper_2509_05679_b200 import synth as sy
 from harness import closed_form_trace, make_ctx, run_parity
 
 pytestmark = pytest.mark.gpu
+# Runs whose oracle side takes several minutes (full-size configuration 2 for its 200 iterations, full-width configuration 3
+# for 50) are run on request: FDG_LONG_TESTS=1.  Their recorded outcome is quoted in the design document.
+long_run = pytest.mark.skipif(os.environ.get("FDG_LONG_TESTS", "0") != "1", reason="minutes of oracle time: set FDG_LONG_TESTS=1")
 
 
 def test_config2_full_size_against_the_oracle(orc):
     net = sy.config(1)                      # 3072 -> 8 x 1024 -> 10, K = 4, 4 workers x 128
-    # lr 0.05 makes this configuration's loss climb from 3 to 7 within a few iterations (an unstable run amplifies
-    # every rounding difference), so only the first backward pass is held to 2e-2; later ones to 1e-1
-    rec = run_parity(orc, net, 2 * net.K + 2, grad_tol=2e-2, grad_tol_later=1e-1, grad_steps=2 * net.K - 1, loss_tol=1e-2, perturb=False)
+    # every tensor within 2e-2 or, eight ReLU layers deep, three times the oracle's own response to a one-ulp change of 0.1 % of the inputs
+    rec = run_parity(orc, net, 2 * net.K + 2, grad_tol=2e-2, noise_factor=3.0, loss_tol=1e-2, perturb=False)
     assert not np.isnan(rec[-1]["loss_g"])
+
+
+@long_run
+def test_config2_full_size_all_200_iterations(orc):
+    """Configuration 2 as stated (lr 0.05, 200 iterations): loss within 1e-2 of the oracle's at every one of them."""
+    net = sy.config(1)
+    rec = run_parity(orc, net, net.steps, loss_tol=1e-2, perturb=False)
+    assert len(rec) == 200 and not np.isnan(rec[-1]["loss_g"])
+
+
+@pytest.mark.parametrize("idx,workers,batch", [(3, 8, 8), (4, 16, 2)])
+def test_full_width_resnet18_without_relu_every_tensor_of_every_module(orc, idx, workers, batch):
+    """Full channel widths (64 .. 512, 32x32 input), K = 4 with 8 workers x 8 samples and K = 8 with 16 workers x 2, lr
+    0.05, the networks without their ReLU layers (see tests/test_oracle_pins.py for why): every convolution,
+    batch-norm and shortcut gradient of every module within 2e-2 of the oracle (L2 and element by element) at every
+    step until the first module has had its second backward pass.  This is where the 256-column CTA-pair kernels, the
+    plain and rows-mode weight gradients of the 256- and 512-channel layers, the 4x4-image tiles (eight samples per tile;
+    with 2 samples per worker they straddle workers and the batch-norm statistics take their own pass) and the
+    stride-2 / 1x1 kernels meet the oracle inside the whole pipeline."""
+    net = sy.without_relu(sy.config(idx, n_workers=workers, batch=batch))
+    rec = run_parity(orc, net, 2 * net.K + 1, grad_tol=2e-2, elem_tol=3e-2, pair_bn=True, loss_tol=1e-2)
+    print(net.name, "worst tensor", max(r.get("grad_err", 0) for r in rec), "worst element", max(r.get("elem_err", 0) for r in rec))
+
+
+def test_full_width_resnet18_with_relu_loss_and_noise_calibrated_gradients(orc):
+    """The benchmark's own network at full width, K = 4, 8 workers x 8 samples: schedule, loss within 1e-2, and every
+    tensor within the larger of 2e-2 and three times the oracle's own one-ulp response."""
+    net = sy.config(3, n_workers=8, batch=8)
+    run_parity(orc, net, 2 * net.K, grad_tol=2e-2, noise_factor=3.0, loss_tol=1e-2)
+
+
+def test_config3_full_width_diverges_at_lr_0_05_in_the_oracle_too_and_is_stable_at_0_005(orc):
+    """The VGG-shaped network (eight convolutions, no normalisation) at full width under the stale gradients: at
+    lr 0.05 the ORACLE's loss leaves 1e3 within ten iterations (so a non-finite loss of the library at that step size
+    is the method diverging, not a kernel fault); at 0.005, the step size the configuration runs with here, both
+    stay finite and the library's loss tracks the oracle's."""
+    net = sy.config(2, n_workers=4, batch=8)
+    p0 = sy.init_params(net.layers, 0, bf16=True)
+    from harness import make_oracle
+    o = make_oracle(orc, net, p0)
+    worst = 0.0
+    for t in range(10):
+        lo, _ = o.step(sy.batch_inputs(net, t), sy.batch_labels(net, t), 0.05)
+        if not np.isnan(lo):
+            worst = max(worst, lo)
+    assert worst > 1e3, worst
+    assert net.lr == 0.005
+    rec = run_parity(orc, net, 12, loss_tol=1e-2, perturb=False)
+    assert all(r["loss_g"] < 50.0 for r in rec if not np.isnan(r["loss_g"])) and rec[-1]["loss_g"] < 3.0
+
+
+@long_run
+def test_config3_full_width_50_step_loss_trajectory(orc):
+    net = sy.config(2, n_workers=4, batch=8)
+    rec = run_parity(orc, net, 50, loss_tol=1e-2, perturb=False)
+    assert sum(not np.isnan(r["loss_g"]) for r in rec) == 50 - (net.K - 1)
 
 
 def _run(net, p0, steps, serial):

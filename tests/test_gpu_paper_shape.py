@@ -28,6 +28,15 @@ def test_the_four_compared_methods_match_the_oracle(orc, S, K):
     assert not np.isnan(rec[-1]["loss_g"])
 
 
+@pytest.mark.parametrize("S,K", [(1, 1), (1, 2), (4, 1), (4, 2)])
+def test_the_four_compared_methods_without_relu_layers_hold_1e_5(orc, S, K):
+    """The same ResNet-20 without its ReLU layers has no kinks, so fp32 and fp64 cannot take different branches and
+    the parameters stay within 1e-5 after every step, through every weight version."""
+    net = sy.without_relu(resnet20(S, K, 4))
+    rec = run_parity(orc, net, 2 * K + 3, param_tol=1e-5, loss_tol=1e-5)
+    assert not np.isnan(rec[-1]["loss_g"])
+
+
 def test_step_size_sequence(orc):
     """eta_t changes between steps (the paper's Strategy II switches 0.1 -> 0.01 -> 0.001 -> 0.0001)."""
     import torch

@@ -34,7 +34,7 @@ def test_fp32_vgg_with_biases_grouped_matches_oracle(orc):
 
 def test_bf16_tensor_core_resnet_grouped_matches_oracle(orc):
     net = _tensor_core_net()
-    run_parity(orc, net, 3 * net.K, grad_tol=2e-2, grad_steps=2 * net.K - 1, grad_tail=2, loss_tol=1e-2, worker_groups=2)
+    run_parity(orc, net, 3 * net.K, grad_tol=2e-2, noise_factor=3.0, loss_tol=1e-2, worker_groups=2)
 
 
 @pytest.mark.parametrize("groups", [2, 4])
