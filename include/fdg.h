@@ -102,8 +102,18 @@ typedef struct {
                                   in fp32 summation order.  Smaller launches, more of them: measured slower on a
                                   B200 at every n for the ResNet-18-shaped benchmark, so it is off by default     */
     void* const* streams;      /* K cudaStream_t of the caller (one per module, for its backward pass and update),
-                                  or NULL: the library creates them, with priorities that rise with the module
-                                  index (the last module's chain of short kernels goes first when SMs free up)  */
+                                  or NULL: the library creates them                                             */
+    const double* mixing;      /* NULL: P = (1/N) 1 1^T, the exact average; every worker then holds the same weights and
+                                  the library keeps ONE copy per module and takes the average inside the
+                                  weight-gradient contraction.
+                                  Otherwise: host array, N x N row-major, the weight matrix P of Sec. 2.3 (Eq.
+                                  "weight_matrix": P_ij = alpha on the edges of the model-group graph, 1 - kappa_i alpha on
+                                  the diagonal); every row must sum to 1.  The library then keeps one weight replica
+                                  w^_{s,k} per worker s and module k, runs every layer once per worker on that
+                                  worker's replica (plain FMA kernels: kernel_path is taken as 1), computes each
+                                  worker's own gradient with scale 1/per_worker_batch, and updates
+                                  u_{s,k} = w^_{s,k} - lr g_{s,k},  w^_{s,k}(t+1) = sum_r P_sr u_{r,k}  (Eq. "dl_update").
+                                  At most 32 workers.  The matrix is copied.                                     */
 } fdg_options;
 
 /* Stash policy.  Every activation a module's backward pass needs is kept from the module's forward pass of
@@ -148,6 +158,10 @@ FDG_API fdg_status fdg_param_layout(const fdg_ctx* ctx, fdg_param_tensor* out, i
  * numbers).  Resets the iteration counter to 0 and empties every FIFO. */
 FDG_API fdg_status fdg_set_params(fdg_ctx* ctx, const float* host_params, size_t count);
 
+/* Contexts created with a mixing matrix only: replace replica `worker` of the initial weights (after fdg_set_params,
+ * before the first step), so that a run can start from replicas that differ (consensus error delta(0) > 0). */
+FDG_API fdg_status fdg_set_params_worker(fdg_ctx* ctx, int32_t worker, const float* host_params, size_t count);
+
 /* One iteration t of Algorithm 1 for all modules and workers (steps listed at the top).
  *   dev_inputs : device, [M, in_h, in_w, in_c] in the context's dtype (fp32 or bf16), the
  *                batch sampled at iteration t.  Its contents must be complete before the call
@@ -186,6 +200,18 @@ FDG_API fdg_status fdg_params(fdg_ctx* ctx, float* host_out, size_t capacity, si
  * the stale gradients of Eq. "dl_update", (1/N) sum_s grad^_{w_{s,k}} Phi_s(t - 2K + k + 1) with the per-sample scale
  * 1/per_worker_batch (zeros for modules that had no backward batch yet: the gradient is 0 while tau < 0). */
 FDG_API fdg_status fdg_grads(fdg_ctx* ctx, float* host_out, size_t capacity, size_t* count);
+
+/* The weights w^_{s,k}(t) / the gradient g_{s,k} of ONE worker s.  Without a mixing matrix every worker has the same
+ * weights (fdg_params_worker returns them for any s) and only the averaged gradient exists (fdg_grads_worker fails with
+ * FDG_ERR_STATE).  With a mixing matrix fdg_params returns worker 0's weights and fdg_grads the mean over the workers. */
+FDG_API fdg_status fdg_params_worker(fdg_ctx* ctx, int32_t worker, float* host_out, size_t capacity, size_t* count);
+FDG_API fdg_status fdg_grads_worker(fdg_ctx* ctx, int32_t worker, float* host_out, size_t capacity, size_t* count);
+
+/* Maximum consensus error of Sec. 5 (Eq. "max_consensus_error"):
+ *   delta(t) = max over layers l and workers s of || w_{s,l}(t) - (1/N) sum_r w_{r,l}(t) ||_2
+ * (a layer's tensors -- W with b, gamma with beta, a projection's three tensors -- form one vector w_{s,l}).  Waits for
+ * the modules and evaluates the definition on the host in double precision.  0 without a mixing matrix. */
+FDG_API fdg_status fdg_consensus_error(fdg_ctx* ctx, double* delta);
 
 /* The delay schedule of Sec. 3.2 (forward batch t-k+1, backward batch t-2K+k+1, backward weights of version
  * t-2K+2k) as observed on the device in the last step.  Every FIFO slot carries a tag (batch id, weight version) in

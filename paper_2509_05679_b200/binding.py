@@ -19,7 +19,8 @@ LIB_PATH = os.path.join(_HERE, "libfdg.so")
 STATUS = {0: "FDG_OK", 1: "FDG_ERR_INVALID_ARG", 2: "FDG_ERR_BAD_SPLIT", 3: "FDG_ERR_UNSUPPORTED",
           4: "FDG_ERR_ARCH", 5: "FDG_ERR_OOM", 6: "FDG_ERR_CUDA", 7: "FDG_ERR_TIMEOUT", 8: "FDG_ERR_STATE"}
 
-EXPORTS = ["fdg_create", "fdg_param_count", "fdg_param_layout", "fdg_set_params", "fdg_step", "fdg_step_host", "fdg_wait_ingest", "fdg_join", "fdg_params",
+EXPORTS = ["fdg_create", "fdg_param_count", "fdg_param_layout", "fdg_set_params", "fdg_set_params_worker", "fdg_params_worker",
+           "fdg_grads_worker", "fdg_consensus_error", "fdg_step", "fdg_step_host", "fdg_wait_ingest", "fdg_join", "fdg_params",
            "fdg_grads", "fdg_trace", "fdg_set_lr", "fdg_stats", "fdg_module_times", "fdg_profile", "fdg_profile_read",
            "fdg_bias_grad_static", "fdg_static_last_error",
            "fdg_last_error", "fdg_destroy"]
@@ -58,7 +59,7 @@ PARAM_ROLES = ["W", "b", "gamma", "beta", "Wp", "gamma_p", "beta_p"]     # fdg_p
 class fdg_options(C.Structure):
     _fields_ = [("dtype", C.c_int32), ("in_h", C.c_int32), ("in_w", C.c_int32), ("in_c", C.c_int32),
                 ("num_classes", C.c_int32), ("serial", C.c_int32), ("kernel_path", C.c_int32),
-                ("worker_groups", C.c_int32), ("streams", C.POINTER(C.c_void_p))]
+                ("worker_groups", C.c_int32), ("streams", C.POINTER(C.c_void_p)), ("mixing", C.POINTER(C.c_double))]
 
 
 _lib = None
@@ -81,6 +82,13 @@ def lib():
         L.fdg_param_layout.argtypes = [vp, C.POINTER(fdg_param_tensor), C.c_int32, C.POINTER(C.c_int32)]
         L.fdg_set_params.restype = C.c_int
         L.fdg_set_params.argtypes = [vp, fp, C.c_size_t]
+        L.fdg_set_params_worker.restype = C.c_int
+        L.fdg_set_params_worker.argtypes = [vp, C.c_int32, fp, C.c_size_t]
+        for name in ("fdg_params_worker", "fdg_grads_worker"):
+            getattr(L, name).restype = C.c_int
+            getattr(L, name).argtypes = [vp, C.c_int32, fp, C.c_size_t, C.POINTER(C.c_size_t)]
+        L.fdg_consensus_error.restype = C.c_int
+        L.fdg_consensus_error.argtypes = [vp, C.POINTER(C.c_double)]
         for name in ("fdg_step", "fdg_step_host"):
             getattr(L, name).restype = C.c_int
             getattr(L, name).argtypes = [vp, vp, vp, fp]
@@ -155,7 +163,7 @@ class Context:
     def __init__(self, layers: Sequence[Sequence[int]], split_points: Sequence[int], n_workers: int,
                  per_worker_batch: int, lr: float, *, dtype: str = "bf16", in_shape=(32, 32, 3), num_classes: int = 10,
                  serial: bool = False, kernel_path: int = 0, device: int = 0, use_torch_allocator: bool = True,
-                 streams: Optional[Sequence[int]] = None, worker_groups: int = 0):
+                 streams: Optional[Sequence[int]] = None, worker_groups: int = 0, mixing=None):
         import torch
         L = lib()
         if not torch.cuda.is_available():
@@ -171,9 +179,14 @@ class Context:
         if streams is not None:          # K cudaStream_t handles owned by the caller
             assert len(streams) == self.K
             self._streams = (C.c_void_p * self.K)(*[C.c_void_p(int(h_)) for h_ in streams])
+        self._mixing = None
+        if mixing is not None:           # N x N weight matrix P (row-major doubles); the library copies it
+            self._mixing = np.ascontiguousarray(mixing, dtype=np.float64)
+            assert self._mixing.shape == (n_workers, n_workers)
         opt = fdg_options({"fp32": 0, "bf16": 1}[dtype], int(in_shape[0]), int(in_shape[1]), int(in_shape[2]),
                           int(num_classes), int(serial), int(kernel_path), int(worker_groups),
-                          C.cast(self._streams, C.POINTER(C.c_void_p)) if self._streams is not None else None)
+                          C.cast(self._streams, C.POINTER(C.c_void_p)) if self._streams is not None else None,
+                          self._mixing.ctypes.data_as(C.POINTER(C.c_double)) if self._mixing is not None else None)
         self._alloc = _TorchAllocator(torch.device("cuda", device)) if use_torch_allocator else None
         h = C.c_void_p()
         st = L.fdg_create(arr, len(layers), sp, self.K, n_workers, per_worker_batch, float(lr), C.byref(opt),
@@ -212,6 +225,27 @@ class Context:
     def set_params(self, params: np.ndarray):
         p = np.ascontiguousarray(params, dtype=np.float32)
         self._ck(lib().fdg_set_params(self.h, p.ctypes.data_as(C.POINTER(C.c_float)), p.size))
+
+    def set_params_worker(self, worker: int, params: np.ndarray):
+        p = np.ascontiguousarray(params, dtype=np.float32)
+        self._ck(lib().fdg_set_params_worker(self.h, int(worker), p.ctypes.data_as(C.POINTER(C.c_float)), p.size))
+
+    def _vec_worker(self, fn, worker: int) -> np.ndarray:
+        out = np.empty(self.n_params, dtype=np.float32)
+        n = C.c_size_t()
+        self._ck(fn(self.h, int(worker), out.ctypes.data_as(C.POINTER(C.c_float)), out.size, C.byref(n)))
+        return out
+
+    def params_worker(self, worker: int) -> np.ndarray:
+        return self._vec_worker(lib().fdg_params_worker, worker)
+
+    def grads_worker(self, worker: int) -> np.ndarray:
+        return self._vec_worker(lib().fdg_grads_worker, worker)
+
+    def consensus_error(self) -> float:
+        d = C.c_double()
+        self._ck(lib().fdg_consensus_error(self.h, C.byref(d)))
+        return d.value
 
     def step(self, dev_inputs, dev_labels, want_loss: bool = False) -> Optional[float]:
         loss = C.c_float()

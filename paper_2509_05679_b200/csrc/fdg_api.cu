@@ -26,7 +26,6 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
-#include <cstdlib>
 #include <string>
 #include <vector>
 
@@ -112,6 +111,9 @@ struct Module {
 
 struct fdg_ctx {
     int K, n_workers, B, M, dt, esz, classes, serial, kernel_path;
+    int R;                         // weight replicas per module: 1 (exact averaging, P = 11^T/N), or n_workers (general mixing matrix)
+    std::vector<double> P;         // R x R mixing matrix (row-major) when R > 1
+    float* P_dev;
     int in_h, in_w, in_c;
     float lr;
     int64_t t;
@@ -319,6 +321,7 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
             if (o.stem_tc) m.ws_elems = std::max(m.ws_elems, tc::stem_wg_workspace_elems(o.g.Co, (long)o.g.N * o.g.H));
             m.ws_elems = std::max(m.ws_elems, wgrad_workspace_elems(o.g));
             m.scratch_elems = std::max(m.scratch_elems, (size_t)64 * o.g.Co);
+            if (relu_bias_backward_supported(ctx->dt, o.g.Co)) m.scratch_elems = std::max(m.scratch_elems, relu_bias_backward_scratch_elems(o.g.Co));
         }
     }
     // a tensor-core conv whose output goes straight into a batch-norm computes that batch-norm's statistics
@@ -365,9 +368,11 @@ struct StepPtrs {            // resolved addresses for one (module, batch)
     float* stats(const Op& o) const { return (float*)(m->stash + (size_t)(batch % m->D) * m->stash_slot_bytes + o.stats_off); }
 };
 
-char* wslot(fdg_ctx* c, Module& m, int64_t version) { return m.wring + (size_t)(version % m.D) * m.wslot_bytes; }
-char* wbig(fdg_ctx* c, Module& m, int64_t version, size_t off) { return wslot(c, m, version) + off * c->esz; }
-float* wsmall(fdg_ctx* c, Module& m, int64_t version, size_t off) { return (float*)(wslot(c, m, version) + m.n_big * c->esz) + off; }
+// weight version `version` of replica r (r = 0 unless the context keeps one replica per worker)
+char* wslot(fdg_ctx* c, Module& m, int64_t version, int r = 0) { return m.wring + ((size_t)(version % m.D) * c->R + r) * m.wslot_bytes; }
+char* wbig(fdg_ctx* c, Module& m, int64_t version, size_t off, int r = 0) { return wslot(c, m, version, r) + off * c->esz; }
+float* wsmall(fdg_ctx* c, Module& m, int64_t version, size_t off, int r = 0) { return (float*)(wslot(c, m, version, r) + m.n_big * c->esz) + off; }
+size_t npar(const Module& m) { return m.n_big + m.n_small; }
 
 char* wtslot(Module& m, int64_t version, size_t off) { return m.wtring + ((size_t)(version % m.D) * m.n_big + off) * 2; }
 
@@ -484,6 +489,7 @@ void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int grou
     Module& m = c->mod[kk];
     StepPtrs P{c, &m, kk, batch};
     const Win wn = group_window(c, m, group);
+    const int rep = c->R > 1 ? group : 0;               // worker `group` runs on its own weights w_{s,k}
     cudaStream_t s = m.fstream;
     const int dt = c->dt;
     m.fused_stats_tensor = -1;
@@ -500,11 +506,11 @@ void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int grou
                 if (o.tc && tc_forward(c, m, o, P.tensor(o.in), P.tensor(o.out), version, wn, s)) { profile_detail(nullptr); break; }
                 if (o.stem && tc_stem_forward(c, m, o, P.tensor(o.in), P.tensor(o.out), version, wn, s)) { profile_detail(nullptr); break; }
                 if (o.stem) {
-                    stem_forward(T(o.in), wbig(c, m, version, o.w_off), o.bias ? wsmall(c, m, version, o.b_off) : nullptr, T(o.out), g, o.relu, s);
+                    stem_forward(T(o.in), wbig(c, m, version, o.w_off, rep), o.bias ? wsmall(c, m, version, o.b_off, rep) : nullptr, T(o.out), g, o.relu, s);
                     profile_detail(nullptr);
                     break;
                 }
-                conv_forward(dt, T(o.in), wbig(c, m, version, o.w_off), o.bias ? wsmall(c, m, version, o.b_off) : nullptr, T(o.out), g, epi, s);
+                conv_forward(dt, T(o.in), wbig(c, m, version, o.w_off, rep), o.bias ? wsmall(c, m, version, o.b_off, rep) : nullptr, T(o.out), g, epi, s);
                 profile_detail(nullptr);
                 break; }
             case OP_BN: {
@@ -513,7 +519,7 @@ void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int grou
                 profile_detail(tag);
                 const bool fused = m.fused_stats_tensor == o.in;
                 const float* part = fused ? m.cstat + (size_t)wn.w0 * m.fused_stats_chunks * ti.c * 2 : nullptr;
-                bn_forward(dt, T(o.in), wsmall(c, m, version, o.gamma_off), wsmall(c, m, version, o.beta_off),
+                bn_forward(dt, T(o.in), wsmall(c, m, version, o.gamma_off, rep), wsmall(c, m, version, o.beta_off, rep),
                            o.has_res ? T(o.in2) : nullptr, T(o.out), P.stats(o) + (size_t)wn.w0 * ti.c * 2, m.scratch_f, wn.nw,
                            (long)c->B * ti.h * ti.w, ti.c, o.relu, part, fused ? m.fused_stats_chunks : 0, c->tc_err, s);
                 profile_detail(nullptr);
@@ -544,7 +550,9 @@ void backward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int64_t
     const Win wn = group_window(c, m, group);
     cudaStream_t s = m.stream;
     const int dt = c->dt;
-    const bool acc_p = !wn.first;                       // parameter gradients of later groups add to the first group's
+    const int rep = c->R > 1 ? group : 0;
+    const bool acc_p = c->R > 1 ? false : !wn.first;    // one replica: parameter gradients of later groups add to the first group's
+    float* const mgrad = m.grad + (size_t)rep * npar(m); // g_{s,k} of this replica
     auto T = [&](int id) { return P.tensor(id) + row_off(c, m.t[id], wn); };
     // gradients are stored in the storage dtype (also the one of the logits)
     auto G = [&](int id) -> char* { char* b = grad_ptr(c, kk, id, t); return b ? b + (size_t)wn.n0 * m.t[id].elems() * c->esz : nullptr; };
@@ -558,18 +566,22 @@ void backward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int64_t
         switch (o.type) {
             case OP_CONV: {
                 ConvGeom g = o.g; g.N = wn.n;
-                if (o.relu) relu_backward(dt, T(o.out), gout, gout, n_out, false, s);       // in place: dZ = dA * (A > 0)
+                // dZ = dA * (A > 0) in place and the bias gradient, in one pass over dA where the width allows
+                const long orows = (long)g.N * g.Ho * g.Wo;
+                const bool fused_rb = (o.relu || o.bias) && relu_bias_backward_supported(dt, g.Co);
+                if (fused_rb) relu_bias_backward(dt, o.relu ? T(o.out) : nullptr, gout, o.bias ? mgrad + m.n_big + o.b_off : nullptr, m.scratch, orows, g.Co, acc_p, s);
+                else if (o.relu) relu_backward(dt, T(o.out), gout, gout, n_out, false, s);
                 profile_detail(o.shape);
                 // the weight gradient needs dy as it stands now and is needed only by the update: it goes to its own stream
                 cudaStream_t ws = m.wstream;
                 if (ws != s) { cudaEventRecord(m.wev, s); cudaStreamWaitEvent(ws, m.wev, 0); }
-                if (o.stem && tc_stem_wgrad(c, m, o, P.tensor(o.in), grad_ptr(c, kk, o.out, t), m.grad + o.w_off, wn, ws)) {}
-                else if (o.stem) stem_wgrad(T(o.in), gout, m.grad + o.w_off, m.ws, g, acc_p, ws);
-                else if (!(o.tc && tc_wgrad(c, m, o, P.tensor(o.in), grad_ptr(c, kk, o.out, t), m.grad + o.w_off, wn, ws)))
-                    conv_wgrad(dt, T(o.in), gout, m.grad + o.w_off, m.ws, g, acc_p, ws);
-                if (o.bias) bias_grad(dt, gout, m.grad + m.n_big + o.b_off, m.scratch, (long)g.N * g.Ho * g.Wo, g.Co, acc_p, s);
+                if (o.stem && tc_stem_wgrad(c, m, o, P.tensor(o.in), grad_ptr(c, kk, o.out, t), mgrad + o.w_off, wn, ws)) {}
+                else if (o.stem) stem_wgrad(T(o.in), gout, mgrad + o.w_off, m.ws, g, acc_p, ws);
+                else if (!(o.tc && tc_wgrad(c, m, o, P.tensor(o.in), grad_ptr(c, kk, o.out, t), mgrad + o.w_off, wn, ws)))
+                    conv_wgrad(dt, T(o.in), gout, mgrad + o.w_off, m.ws, g, acc_p, ws);
+                if (o.bias && !fused_rb) bias_grad(dt, gout, mgrad + m.n_big + o.b_off, m.scratch, orows, g.Co, acc_p, s);
                 if (gin && !(o.tc && tc_dgrad(c, m, o, grad_ptr(c, kk, o.out, t), grad_ptr(c, kk, o.in, t), version, o.acc_in, wn, s)))
-                    conv_dgrad(dt, gout, wbig(c, m, version, o.w_off), gin, g, o.acc_in ? EPI_ACCUM : 0, s);
+                    conv_dgrad(dt, gout, wbig(c, m, version, o.w_off, rep), gin, g, o.acc_in ? EPI_ACCUM : 0, s);
                 profile_detail(nullptr);
                 break; }
             case OP_BN: {
@@ -577,9 +589,9 @@ void backward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int64_t
                 std::snprintf(tag, sizeof tag, "%dx%dx%d%s%s", ti.h, ti.w, ti.c, o.has_res ? " +res" : "", o.relu ? " relu" : "");
                 profile_detail(tag);
                 char* gres = o.has_res ? G(o.in2) : nullptr;
-                bn_backward(dt, T(o.in), T(o.out), gout, wsmall(c, m, version, o.gamma_off), wsmall(c, m, version, o.beta_off),
-                            P.stats(o) + (size_t)wn.w0 * ti.c * 2, gin, o.acc_in, gres, o.acc_in2, m.grad + m.n_big + o.gamma_off,
-                            m.grad + m.n_big + o.beta_off, m.red, m.scratch, wn.nw, (long)c->B * ti.h * ti.w, ti.c, o.relu, o.has_res, acc_p, c->tc_err, s);
+                bn_backward(dt, T(o.in), T(o.out), gout, wsmall(c, m, version, o.gamma_off, rep), wsmall(c, m, version, o.beta_off, rep),
+                            P.stats(o) + (size_t)wn.w0 * ti.c * 2, gin, o.acc_in, gres, o.acc_in2, mgrad + m.n_big + o.gamma_off,
+                            mgrad + m.n_big + o.beta_off, m.red, m.scratch, wn.nw, (long)c->B * ti.h * ti.w, ti.c, o.relu, o.has_res, acc_p, c->tc_err, s);
                 profile_detail(nullptr);
                 break; }
             case OP_RELU: if (gin) relu_backward(dt, T(o.out), gout, gin, n_out, o.acc_in, s); break;
@@ -827,8 +839,10 @@ fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, boo
         if (lastm && m.fstream != m.stream) CK(cudaStreamWaitEvent(m.stream, m.fdone, 0));   // the last module back-propagates the batch it just forwarded
         if (lastm) {
             float* loss_slot = ctx->loss_ring + (t % 64);
+            // one replica: dphi/dlogits / M, the mean over all samples.  One replica per worker: / B, worker s's own
+            // gradient scale 1/per_worker_batch of Eq. dl_update (the mixing matrix does the averaging)
             if (tau_f >= 0) softmax_ce(ctx->dt, ctx->logits, ctx->labels + (size_t)(tau_f % ctx->label_depth) * ctx->M, ctx->dlogits,
-                                       loss_slot, ctx->M, ctx->classes, m.stream);
+                                       loss_slot, ctx->M, ctx->classes, ctx->R > 1 ? 1.f / (float)ctx->B : 1.f / (float)ctx->M, m.stream);
             else fill_f32(loss_slot, NAN, 1, m.stream);
         }
         if (tau_b >= 0) for (int g = 0; g < m.groups; ++g) backward_module(ctx, kk, tau_b, v_b, t, g);
@@ -836,11 +850,17 @@ fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, boo
         // (after the forward pass has read version t: with a one-slot ring the update overwrites it)
         if (!lastm && m.fstream != m.stream) CK(cudaStreamWaitEvent(m.stream, m.fdone, 0));
         if (tau_b >= 0 && m.wstream != m.stream) { CK(cudaEventRecord(m.wdone, m.wstream)); CK(cudaStreamWaitEvent(m.stream, m.wdone, 0)); }
-        sgd_update(ctx->dt, m.master, tau_b >= 0 ? m.grad : nullptr, wslot(ctx, m, t + 1), m.n_big, ctx->lr, m.stream);
-        if (m.n_small)
-            sgd_update(0, m.master + m.n_big, tau_b >= 0 ? m.grad + m.n_big : nullptr,
-                       wsmall(ctx, m, t + 1, 0), m.n_small, ctx->lr, m.stream);
-        emit_transposed_weights(ctx, m, t + 1);
+        if (ctx->R > 1) {
+            // Eq. dl_update (a), (b) with a general P: u_r = w_r - lr g_r, w_s(t+1) = sum_r P_sr u_r, all replicas in one pass
+            mix_update(ctx->dt, m.master, tau_b >= 0 ? m.grad : nullptr, wslot(ctx, m, t + 1, 0), m.n_big, m.n_small, m.wslot_bytes, ctx->R, ctx->P_dev,
+                       ctx->lr, m.stream);
+        } else {
+            sgd_update(ctx->dt, m.master, tau_b >= 0 ? m.grad : nullptr, wslot(ctx, m, t + 1), m.n_big, ctx->lr, m.stream);
+            if (m.n_small)
+                sgd_update(0, m.master + m.n_big, tau_b >= 0 ? m.grad + m.n_big : nullptr,
+                           wsmall(ctx, m, t + 1, 0), m.n_small, ctx->lr, m.stream);
+            emit_transposed_weights(ctx, m, t + 1);
+        }
         m.had_bwd = tau_b >= 0;
         CK(cudaEventRecord(m.ev1, m.stream));
         CK(cudaEventRecord(m.done, m.stream));
@@ -904,6 +924,18 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
     ctx->K = K; ctx->n_workers = n_workers; ctx->B = per_worker_batch; ctx->M = n_workers * per_worker_batch;
     ctx->dt = opt->dtype; ctx->esz = opt->dtype ? 2 : 4; ctx->classes = opt->num_classes; ctx->serial = opt->serial;
     ctx->kernel_path = opt->kernel_path;
+    ctx->R = 1; ctx->P_dev = nullptr;
+    if (opt->mixing) {
+        // general mixing matrix: one weight replica per worker, every layer runs once per worker on the plain FMA kernels
+        if (n_workers > mix_max_replicas()) { delete ctx; return fail(nullptr, FDG_ERR_UNSUPPORTED, "a mixing matrix is supported for at most %d workers", mix_max_replicas()); }
+        ctx->R = n_workers; ctx->kernel_path = 1;
+        ctx->P.assign(opt->mixing, opt->mixing + (size_t)n_workers * n_workers);
+        for (int i = 0; i < n_workers; ++i) {
+            double row = 0.0;
+            for (int j = 0; j < n_workers; ++j) { const double v = ctx->P[(size_t)i * n_workers + j]; if (!(v == v) || std::fabs(v) > 1e6) row = NAN; row += v; }
+            if (!(std::fabs(row - 1.0) <= 1e-6)) { delete ctx; return fail(nullptr, FDG_ERR_INVALID_ARG, "row %d of the mixing matrix does not sum to 1", i); }
+        }
+    }
     ctx->in_h = opt->in_h; ctx->in_w = opt->in_w; ctx->in_c = opt->in_c; ctx->lr = lr; ctx->t = 0; ctx->have_params = false; ctx->broken = false;
     ctx->layers.assign(layers, layers + n_layers);
     ctx->alloc = alloc ? *alloc : fdg_allocator{default_alloc, default_free, nullptr};
@@ -929,7 +961,8 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
         // worker groups (off unless asked for: measured slower on every configuration, see fdg_options.worker_groups):
         // a group is a whole number of workers; the last module of a split network stays whole
         m.groups = 1;
-        if (opt->worker_groups > 1 && (kk + 1 < K || K == 1)) {
+        if (ctx->R > 1) m.groups = n_workers;
+        else if (opt->worker_groups > 1 && (kk + 1 < K || K == 1)) {
             int g = 1;
             while (g * 2 <= opt->worker_groups && n_workers % (g * 2) == 0) g *= 2;
             m.groups = g;
@@ -959,6 +992,7 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
     ctx->dlogits = get((size_t)ctx->M * ctx->classes * ctx->esz);
     ctx->loss_ring = (float*)get(64 * sizeof(float));
     ctx->tc_err = (int*)get(256);
+    if (ctx->R > 1) ctx->P_dev = (float*)get((size_t)ctx->R * ctx->R * sizeof(float));
     size_t tpos = 0;
     for (int kk = 0; kk < K && !oom; ++kk) {
         Module& m = ctx->mod[kk];
@@ -966,10 +1000,10 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
         m.stash = get((size_t)m.D * m.stash_slot_bytes);
         m.gradpool = get(m.grad_pool_bytes);
         m.d2 = kk > 0 ? get(2 * m.in_slot_bytes) : nullptr;
-        m.wring = get((size_t)m.D * m.wslot_bytes);
-        m.wtring = ctx->dt == 1 ? get((size_t)m.D * m.n_big * 2) : nullptr;
-        m.master = (float*)get((m.n_big + m.n_small) * sizeof(float));
-        m.grad = (float*)get((m.n_big + m.n_small) * sizeof(float));
+        m.wring = get((size_t)m.D * ctx->R * m.wslot_bytes);
+        m.wtring = (ctx->dt == 1 && ctx->R == 1) ? get((size_t)m.D * m.n_big * 2) : nullptr;
+        m.master = (float*)get((size_t)ctx->R * (m.n_big + m.n_small) * sizeof(float));
+        m.grad = (float*)get((size_t)ctx->R * (m.n_big + m.n_small) * sizeof(float));
         m.ws = (float*)get(m.ws_elems * sizeof(float));
         m.scratch = (float*)get(m.scratch_elems * sizeof(float));
         m.red = (float*)get(m.red_elems * sizeof(float));
@@ -983,37 +1017,35 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
         m.trace = ctx->tags + tpos; tpos += 4;
     }
     if (oom) return bail(FDG_ERR_OOM, "the allocator returned NULL");
-    // Stream priorities: the later a module, the smaller its tensors and the longer its chain of short kernels (the last
-    // module's forward pass, loss and backward pass of one batch are one serial chain inside a step), so its kernels go
-    // first whenever SMs free up; a module's weight gradients, which only its update waits for, rank below its two passes.
-    int prio_least = 0, prio_greatest = 0;
-    cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest);
-    if (getenv("FDG_NO_PRIO")) prio_greatest = prio_least;     // TEMP experiment hook
+    // All streams have the same priority.  Measured on the ResNet-18-shaped benchmark: the step is bound by the sum of its
+    // kernels, not by one module's chain, and ranking the later modules' short kernels first lengthened the first
+    // module's step (the one with the largest tensors) by more than it saved elsewhere (5.65 against 5.50 ms per step).
     for (int kk = 0; kk < K; ++kk) {
         Module& m = ctx->mod[kk];
         cudaError_t e = cudaSuccess;
-        const int span = prio_least - prio_greatest;                       // priorities run from prio_least (low) down to prio_greatest (high)
-        const int prio = prio_least - (K > 1 ? span * kk / (K - 1) : 0);
-        const int prio_w = prio < prio_least ? prio + 1 : prio_least;
         if (opt->streams) m.stream = (cudaStream_t)opt->streams[ctx->serial ? 0 : kk];
         else if (ctx->serial && kk > 0) m.stream = ctx->mod[0].stream;
-        else { e = cudaStreamCreateWithPriority(&m.stream, cudaStreamNonBlocking, prio); if (e == cudaSuccess) ctx->owned.push_back(m.stream); }
+        else { e = cudaStreamCreateWithFlags(&m.stream, cudaStreamNonBlocking); if (e == cudaSuccess) ctx->owned.push_back(m.stream); }
         m.fstream = m.stream;
-        if (e == cudaSuccess && !ctx->serial) { e = cudaStreamCreateWithPriority(&m.fstream, cudaStreamNonBlocking, prio); if (e == cudaSuccess) ctx->owned.push_back(m.fstream); }
+        if (e == cudaSuccess && !ctx->serial) { e = cudaStreamCreateWithFlags(&m.fstream, cudaStreamNonBlocking); if (e == cudaSuccess) ctx->owned.push_back(m.fstream); }
         m.wstream = m.stream;
-        if (e == cudaSuccess && !ctx->serial) { e = cudaStreamCreateWithPriority(&m.wstream, cudaStreamNonBlocking, prio_w); if (e == cudaSuccess) ctx->owned.push_back(m.wstream); }
+        if (e == cudaSuccess && !ctx->serial) { e = cudaStreamCreateWithFlags(&m.wstream, cudaStreamNonBlocking); if (e == cudaSuccess) ctx->owned.push_back(m.wstream); }
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.wev, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.wdone, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.done, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.fdone, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreate(&m.ev0);
         if (e == cudaSuccess) e = cudaEventCreate(&m.ev1);
-        if (e == cudaSuccess) e = cudaMemset(m.grad, 0, (m.n_big + m.n_small) * sizeof(float));
-        if (e == cudaSuccess) e = cudaMemset(m.master, 0, (m.n_big + m.n_small) * sizeof(float));
+        if (e == cudaSuccess) e = cudaMemset(m.grad, 0, (size_t)ctx->R * (m.n_big + m.n_small) * sizeof(float));
+        if (e == cudaSuccess) e = cudaMemset(m.master, 0, (size_t)ctx->R * (m.n_big + m.n_small) * sizeof(float));
         if (e != cudaSuccess) return bail(FDG_ERR_CUDA, cudaGetErrorString(e));
     }
     if (cudaEventCreateWithFlags(&ctx->ingested, cudaEventDisableTiming) != cudaSuccess) return bail(FDG_ERR_CUDA, "cudaEventCreate failed");
     if (cudaMemset(ctx->tc_err, 0, 256) != cudaSuccess) return bail(FDG_ERR_CUDA, "cudaMemset failed");
+    if (ctx->R > 1) {
+        std::vector<float> pf(ctx->P.begin(), ctx->P.end());
+        if (cudaMemcpy(ctx->P_dev, pf.data(), pf.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) return bail(FDG_ERR_CUDA, "cudaMemcpy failed");
+    }
     ctx->any_tc = false;
     if (!build_tc_plans(ctx)) return bail(FDG_ERR_CUDA, "cuTensorMapEncodeTiled rejected a tensor map");
     // a group must hold whole image tiles of every tensor-core tiling: a ragged tile would reach into the next group's rows
@@ -1086,29 +1118,53 @@ fdg_status fdg_param_layout(const fdg_ctx* ctx, fdg_param_tensor* out, int32_t c
     return FDG_OK;
 }
 
+// Copy a canonical parameter vector into replica `worker` (all replicas if worker < 0) and emit its version-0 copies.
+static fdg_status load_replicas(fdg_ctx* ctx, const float* host_params, int worker) {
+    for (Module& m : ctx->mod) {
+        std::vector<float> h(npar(m), 0.f);
+        for (const Segment& s : m.segs)
+            std::memcpy(h.data() + (s.big ? 0 : m.n_big) + s.internal, host_params + s.canon, s.count * sizeof(float));
+        for (int r = 0; r < ctx->R; ++r) {
+            if (worker >= 0 && r != worker) continue;
+            float* master = m.master + (size_t)r * npar(m);
+            // in-stream copy, then wait: a plain cudaMemcpy from pageable memory may return before the DMA has
+            // landed, and the module streams are non-blocking streams that do not order behind the default stream
+            CK(cudaMemcpyAsync(master, h.data(), h.size() * sizeof(float), cudaMemcpyHostToDevice, m.stream));
+            CK(cudaStreamSynchronize(m.stream));
+            // version 0 into weight slot 0
+            sgd_update(ctx->dt, master, nullptr, wslot(ctx, m, 0, r), m.n_big, 0.f, m.stream);
+            if (m.n_small) sgd_update(0, master + m.n_big, nullptr, wsmall(ctx, m, 0, 0, r), m.n_small, 0.f, m.stream);
+        }
+        if (ctx->R == 1) emit_transposed_weights(ctx, m, 0);
+        CK(cudaMemsetAsync(m.grad, 0, (size_t)ctx->R * npar(m) * sizeof(float), m.stream));
+    }
+    return FDG_OK;
+}
+
 fdg_status fdg_set_params(fdg_ctx* ctx, const float* host_params, size_t count) {
     if (!ctx || !host_params) return FDG_ERR_INVALID_ARG;
     if (count != ctx->n_params) return fail(ctx, FDG_ERR_INVALID_ARG, "expected %zu parameters, got %zu", ctx->n_params, count);
     CK(cudaDeviceSynchronize());
-    for (Module& m : ctx->mod) {
-        std::vector<float> h(m.n_big + m.n_small, 0.f);
-        for (const Segment& s : m.segs)
-            std::memcpy(h.data() + (s.big ? 0 : m.n_big) + s.internal, host_params + s.canon, s.count * sizeof(float));
-        // in-stream copy, then wait: a plain cudaMemcpy from pageable memory may return before the DMA has
-        // landed, and the module streams are non-blocking streams that do not order behind the default stream
-        CK(cudaMemcpyAsync(m.master, h.data(), h.size() * sizeof(float), cudaMemcpyHostToDevice, m.stream));
-        CK(cudaStreamSynchronize(m.stream));
-        // version 0 into weight slot 0
-        sgd_update(ctx->dt, m.master, nullptr, wslot(ctx, m, 0), m.n_big, 0.f, m.stream);
-        if (m.n_small) sgd_update(0, m.master + m.n_big, nullptr, wsmall(ctx, m, 0, 0), m.n_small, 0.f, m.stream);
-        emit_transposed_weights(ctx, m, 0);
-        CK(cudaMemsetAsync(m.grad, 0, (m.n_big + m.n_small) * sizeof(float), m.stream));
-    }
-    fdg_status s = reset_state(ctx);
+    fdg_status s = load_replicas(ctx, host_params, -1);
+    if (s != FDG_OK) return s;
+    s = reset_state(ctx);
     if (s != FDG_OK) return s;
     CK(cudaDeviceSynchronize());
     ctx->have_params = true;
     ctx->broken = false;
+    return FDG_OK;
+}
+
+fdg_status fdg_set_params_worker(fdg_ctx* ctx, int32_t worker, const float* host_params, size_t count) {
+    if (!ctx || !host_params) return FDG_ERR_INVALID_ARG;
+    if (count != ctx->n_params) return fail(ctx, FDG_ERR_INVALID_ARG, "expected %zu parameters, got %zu", ctx->n_params, count);
+    if (ctx->R == 1) return fail(ctx, FDG_ERR_STATE, "the context keeps one weight copy for all workers (no mixing matrix was given)");
+    if (worker < 0 || worker >= ctx->R) return fail(ctx, FDG_ERR_INVALID_ARG, "worker %d out of range", worker);
+    if (!ctx->have_params || ctx->t != 0) return fail(ctx, FDG_ERR_STATE, "fdg_set_params_worker replaces one replica of the initial weights: call it after fdg_set_params and before the first step");
+    CK(cudaDeviceSynchronize());
+    fdg_status s = load_replicas(ctx, host_params, worker);
+    if (s != FDG_OK) return s;
+    CK(cudaDeviceSynchronize());
     return FDG_OK;
 }
 
@@ -1126,22 +1182,80 @@ fdg_status fdg_step_host(fdg_ctx* ctx, const void* host_inputs, const int32_t* h
     return guarded_step(ctx, host_inputs, host_labels, true, host_loss_or_null);
 }
 
-static fdg_status gather(fdg_ctx* ctx, bool grads, float* host_out, size_t capacity, size_t* count) {
+// worker < 0: the parameters of replica 0, or the gradient averaged over the replicas
+static fdg_status gather(fdg_ctx* ctx, bool grads, int worker, float* host_out, size_t capacity, size_t* count) {
     if (!ctx || !host_out) return FDG_ERR_INVALID_ARG;
     if (capacity < ctx->n_params) return fail(ctx, FDG_ERR_INVALID_ARG, "capacity %zu < %zu parameters", capacity, ctx->n_params);
+    if (worker >= ctx->n_workers) return fail(ctx, FDG_ERR_INVALID_ARG, "worker %d out of range", worker);
     CK(cudaDeviceSynchronize());
     { fdg_status es = check_device_error(ctx); if (es != FDG_OK) return es; }
     for (Module& m : ctx->mod) {
-        std::vector<float> h(m.n_big + m.n_small, 0.f);
-        if (!grads || m.had_bwd) CK(cudaMemcpy(h.data(), grads ? m.grad : m.master, h.size() * sizeof(float), cudaMemcpyDeviceToHost));
+        const size_t n = npar(m);
+        std::vector<float> h(n, 0.f);
+        if (!grads || m.had_bwd) {
+            if (grads && worker < 0 && ctx->R > 1) {
+                // (1/N) sum_s g_{s,k}, accumulated in double
+                std::vector<float> one(n);
+                std::vector<double> acc(n, 0.0);
+                for (int r = 0; r < ctx->R; ++r) {
+                    CK(cudaMemcpy(one.data(), m.grad + (size_t)r * n, n * sizeof(float), cudaMemcpyDeviceToHost));
+                    for (size_t i = 0; i < n; ++i) acc[i] += one[i];
+                }
+                for (size_t i = 0; i < n; ++i) h[i] = (float)(acc[i] / ctx->R);
+            } else {
+                const int r = (ctx->R > 1 && worker > 0) ? worker : 0;       // one copy: every worker has the same
+                CK(cudaMemcpy(h.data(), (grads ? m.grad : m.master) + (size_t)r * n, n * sizeof(float), cudaMemcpyDeviceToHost));
+            }
+        }
         for (const Segment& s : m.segs)
             std::memcpy(host_out + s.canon, h.data() + (s.big ? 0 : m.n_big) + s.internal, s.count * sizeof(float));
     }
     if (count) *count = ctx->n_params;
     return FDG_OK;
 }
-fdg_status fdg_params(fdg_ctx* ctx, float* host_out, size_t capacity, size_t* count) { return gather(ctx, false, host_out, capacity, count); }
-fdg_status fdg_grads(fdg_ctx* ctx, float* host_out, size_t capacity, size_t* count) { return gather(ctx, true, host_out, capacity, count); }
+fdg_status fdg_params(fdg_ctx* ctx, float* host_out, size_t capacity, size_t* count) { return gather(ctx, false, -1, host_out, capacity, count); }
+fdg_status fdg_grads(fdg_ctx* ctx, float* host_out, size_t capacity, size_t* count) { return gather(ctx, true, -1, host_out, capacity, count); }
+fdg_status fdg_params_worker(fdg_ctx* ctx, int32_t worker, float* host_out, size_t capacity, size_t* count) {
+    if (worker < 0) return FDG_ERR_INVALID_ARG;
+    return gather(ctx, false, worker, host_out, capacity, count);
+}
+fdg_status fdg_grads_worker(fdg_ctx* ctx, int32_t worker, float* host_out, size_t capacity, size_t* count) {
+    if (worker < 0) return FDG_ERR_INVALID_ARG;
+    if (ctx && ctx->R == 1) return fail(ctx, FDG_ERR_STATE, "the context keeps one averaged gradient (no mixing matrix was given)");
+    return gather(ctx, true, worker, host_out, capacity, count);
+}
+
+// delta(t) = max over layers l and workers s of || w_{s,l}(t) - (1/N) sum_r w_{r,l}(t) ||_2   (Sec. 5, Eq. max_consensus_error)
+fdg_status fdg_consensus_error(fdg_ctx* ctx, double* delta) {
+    if (!ctx || !delta) return FDG_ERR_INVALID_ARG;
+    if (ctx->R == 1) { *delta = 0.0; return FDG_OK; }       // one copy: the replicas cannot differ
+    int32_t nt = 0;
+    fdg_param_layout(ctx, nullptr, 0, &nt);
+    std::vector<fdg_param_tensor> lay(nt);
+    fdg_param_layout(ctx, lay.data(), nt, &nt);
+    std::vector<std::vector<float>> w(ctx->R, std::vector<float>(ctx->n_params));
+    for (int r = 0; r < ctx->R; ++r) {
+        fdg_status s = gather(ctx, false, r, w[r].data(), ctx->n_params, nullptr);
+        if (s != FDG_OK) return s;
+    }
+    double worst = 0.0;
+    for (size_t i = 0; i < lay.size();) {
+        size_t j = i;                                       // tensors i..j-1 belong to one layer
+        while (j < lay.size() && lay[j].layer == lay[i].layer) ++j;
+        const size_t a = lay[i].offset, b = lay[j - 1].offset + lay[j - 1].count;
+        std::vector<double> mean(b - a, 0.0);
+        for (int r = 0; r < ctx->R; ++r) for (size_t e = a; e < b; ++e) mean[e - a] += w[r][e];
+        for (double& v : mean) v /= ctx->R;
+        for (int r = 0; r < ctx->R; ++r) {
+            double ss = 0.0;
+            for (size_t e = a; e < b; ++e) { const double d = (double)w[r][e] - mean[e - a]; ss += d * d; }
+            worst = std::max(worst, std::sqrt(ss));
+        }
+        i = j;
+    }
+    *delta = worst;
+    return FDG_OK;
+}
 
 fdg_status fdg_trace(fdg_ctx* ctx, int64_t* fwd_batch, int64_t* bwd_batch, int64_t* bwd_weight_version, int32_t K) {
     if (!ctx || !fwd_batch || !bwd_batch || !bwd_weight_version || K != ctx->K) return FDG_ERR_INVALID_ARG;

@@ -357,46 +357,160 @@ void bias_grad(int dt, const void* dy, float* db, float* scratch, long rows, int
 }
 
 // ------------------------------------------------------------------------------------------
-// elementwise layers
+// elementwise layers: 128-bit accesses (8 bf16 or 4 fp32 values per thread and pass), grid-stride loops over a grid of
+// a few CTAs per SM; the last n % V elements are handled one by one by the first threads
 // ------------------------------------------------------------------------------------------
-template <typename T> __global__ void relu_fwd_k(const T* x, T* y, size_t n) {
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; if (i < n) st(y + i, fmaxf(ld(x + i), 0.f)); }
-template <typename T> __global__ void relu_bwd_k(const T* y, const T* dy, T* dx, size_t n, bool accum) {
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n) { float v = ld(y + i) > 0.f ? ld(dy + i) : 0.f; if (accum) v += ld(dx + i); st(dx + i, v); } }
-template <typename T> __global__ void add_k(const T* a, const T* b, T* y, size_t n) {
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; if (i < n) st(y + i, ld(a + i) + ld(b + i)); }
-template <typename T> __global__ void copy_acc_k(const T* src, T* dst, size_t n, bool accum) {
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n) { float v = ld(src + i); if (accum) v += ld(dst + i); st(dst + i, v); } }
+template <typename T> struct Vec;
+template <> struct Vec<float> {
+    static constexpr int V = 4;
+    static __device__ __forceinline__ void load(const float* p, float (&f)[8]) { const float4 v = *(const float4*)p; f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w; }
+    static __device__ __forceinline__ void store(float* p, const float (&f)[8]) { *(float4*)p = make_float4(f[0], f[1], f[2], f[3]); }
+};
+template <> struct Vec<bf16> {
+    static constexpr int V = 8;
+    static __device__ __forceinline__ void load(const bf16* p, float (&f)[8]) {
+        const uint4 v = *(const uint4*)p; const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { f[2 * j] = __uint_as_float(w[j] << 16); f[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u); }
+    }
+    static __device__ __forceinline__ void store(bf16* p, const float (&f)[8]) {
+        uint32_t w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { const __nv_bfloat162 t = __floats2bfloat162_rn(f[2 * j], f[2 * j + 1]); w[j] = *(const uint32_t*)&t; }
+        *(uint4*)p = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+static unsigned ew_grid(size_t nvec) { size_t b = (nvec + 255) / 256; return (unsigned)(b < 1 ? 1 : (b > 148 * 8 ? 148 * 8 : b)); }
+
+// OP 0: y = max(x, 0).  OP 1: dx (+)= dy * (y > 0)   (a = y, b = dy, o = dx).  OP 2: y = a + b.  OP 3: dst (+)= src   (a = src, o = dst).
+template <typename T, int OP>
+__global__ void __launch_bounds__(256) ew_k(const T* __restrict__ a, const T* __restrict__ b, T* o, size_t n, bool accum) {
+    constexpr int V = Vec<T>::V;
+    const size_t nvec = n / V, stride = (size_t)gridDim.x * blockDim.x, t0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (size_t i = t0; i < nvec; i += stride) {
+        float fa[8], fb[8], fo[8];
+        Vec<T>::load(a + i * V, fa);
+        if (OP == 1 || OP == 2) Vec<T>::load(b + i * V, fb);
+        if ((OP == 1 || OP == 3) && accum) Vec<T>::load(o + i * V, fo);
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+            float v;
+            if (OP == 0) v = fmaxf(fa[j], 0.f);
+            else if (OP == 1) v = fa[j] > 0.f ? fb[j] : 0.f;
+            else if (OP == 2) v = fa[j] + fb[j];
+            else v = fa[j];
+            if ((OP == 1 || OP == 3) && accum) v += fo[j];
+            fo[j] = v;
+        }
+        Vec<T>::store(o + i * V, fo);
+    }
+    for (size_t i = nvec * V + t0; i < n; i += stride) {
+        float v;
+        if (OP == 0) v = fmaxf(ld(a + i), 0.f);
+        else if (OP == 1) v = ld(a + i) > 0.f ? ld(b + i) : 0.f;
+        else if (OP == 2) v = ld(a + i) + ld(b + i);
+        else v = ld(a + i);
+        if ((OP == 1 || OP == 3) && accum) v += ld(o + i);
+        st(o + i, v);
+    }
+}
+template <int OP>
+static void ew_launch(int dt, const void* a, const void* b, void* o, size_t n, bool accum, cudaStream_t s) {
+    if (dt) ew_k<bf16, OP><<<ew_grid(n / 8), 256, 0, s>>>((const bf16*)a, (const bf16*)b, (bf16*)o, n, accum);
+    else ew_k<float, OP><<<ew_grid(n / 4), 256, 0, s>>>((const float*)a, (const float*)b, (float*)o, n, accum);
+}
 
 void relu_forward(int dt, const void* x, void* y, size_t n, cudaStream_t s) {
-    const double esz_ = dt ? 2.0 : 4.0; (void)esz_;
-    Scope sc(KC_RELU_FWD, 0.0, 2 * esz_ * n, s);
-    if (dt) relu_fwd_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)x, (bf16*)y, n);
-    else relu_fwd_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)x, (float*)y, n);
-    
+    Scope sc(KC_RELU_FWD, 0.0, 2 * (dt ? 2.0 : 4.0) * n, s);
+    ew_launch<0>(dt, x, nullptr, y, n, false, s);
 }
 void relu_backward(int dt, const void* y, const void* dy, void* dx, size_t n, bool accum, cudaStream_t s) {
-    const double esz_ = dt ? 2.0 : 4.0; (void)esz_;
-    Scope sc(KC_RELU_BWD, 0.0, 3 * esz_ * n, s);
-    if (dt) relu_bwd_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)y, (const bf16*)dy, (bf16*)dx, n, accum);
-    else relu_bwd_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)y, (const float*)dy, (float*)dx, n, accum);
-    
+    Scope sc(KC_RELU_BWD, 0.0, (accum ? 4 : 3) * (dt ? 2.0 : 4.0) * n, s);
+    ew_launch<1>(dt, y, dy, dx, n, accum, s);
 }
 void add_forward(int dt, const void* a, const void* b, void* y, size_t n, cudaStream_t s) {
-    const double esz_ = dt ? 2.0 : 4.0; (void)esz_;
-    Scope sc(KC_ADD_FWD, 0.0, 3 * esz_ * n, s);
-    if (dt) add_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)a, (const bf16*)b, (bf16*)y, n);
-    else add_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)a, (const float*)b, (float*)y, n);
-    
+    Scope sc(KC_ADD_FWD, 0.0, 3 * (dt ? 2.0 : 4.0) * n, s);
+    ew_launch<2>(dt, a, b, y, n, false, s);
 }
 void copy_or_accumulate(int dt, const void* src, void* dst, size_t n, bool accum, cudaStream_t s) {
-    const double esz_ = dt ? 2.0 : 4.0; (void)esz_;
-    Scope sc(KC_COPY_ACC, 0.0, (accum ? 3 : 2) * esz_ * n, s);
-    if (dt) copy_acc_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)src, (bf16*)dst, n, accum);
-    else copy_acc_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)src, (float*)dst, n, accum);
-    
+    Scope sc(KC_COPY_ACC, 0.0, (accum ? 3 : 2) * (dt ? 2.0 : 4.0) * n, s);
+    ew_launch<3>(dt, src, nullptr, dst, n, accum, s);
+}
+
+// ------------------------------------------------------------------------------------------
+// Backward pass through "+ bias, ReLU" of a linear / conv layer in ONE pass over dy:  dy *= (y > 0) in place (if the layer
+// has a ReLU) and db[c] = sum over rows of the masked dy (if it has a bias).  A thread keeps one 128-bit channel group for
+// every row it visits; a CTA owns a contiguous row range; partial sums per CTA, then a fixed-order final sum.
+// Used when C / V is a power of two <= 256 (V = 8 bf16 / 4 fp32 values per access); other widths take the generic kernels.
+// ------------------------------------------------------------------------------------------
+constexpr int RB_MAX_CHUNKS = 592;
+template <typename T>
+__global__ void __launch_bounds__(256) relu_bias_bwd_k(const T* __restrict__ y, T* dy, float* __restrict__ part, long rows, int C, long rows_per_cta) {
+    constexpr int V = Vec<T>::V;
+    const int cgs = C / V, rows_it = 256 / cgs, cg = threadIdx.x % cgs, rl = threadIdx.x / cgs;
+    const long r0 = (long)blockIdx.x * rows_per_cta, r1 = min(rows, r0 + rows_per_cta);
+    float s[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) s[j] = 0.f;
+    for (long r = r0 + rl; r < r1; r += rows_it) {
+        const size_t o = (size_t)r * C + (size_t)cg * V;
+        float g[8];
+        Vec<T>::load(dy + o, g);
+        if (y) {
+            float a[8];
+            Vec<T>::load(y + o, a);
+#pragma unroll
+            for (int j = 0; j < V; ++j) if (!(a[j] > 0.f)) g[j] = 0.f;
+            Vec<T>::store(dy + o, g);
+        }
+#pragma unroll
+        for (int j = 0; j < V; ++j) s[j] += g[j];
+    }
+    if (!part) return;
+    __shared__ float sh[256][9];
+#pragma unroll
+    for (int j = 0; j < V; ++j) sh[threadIdx.x][j] = s[j];
+    __syncthreads();
+    for (int t = threadIdx.x; t < C; t += 256) {
+        const int q = t / V, k = t % V;
+        float acc = 0.f;
+        for (int rr = 0; rr < rows_it; ++rr) acc += sh[rr * cgs + q][k];
+        part[(size_t)blockIdx.x * C + t] = acc;
+    }
+}
+// one warp per channel: lanes take the partials round-robin, then a fixed shuffle tree
+__global__ void colsum_final_warp(const float* __restrict__ part, float* __restrict__ out, int chunks, int C, bool accum) {
+    const int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (c >= C) return;
+    float a = 0.f;
+    for (int k = lane; k < chunks; k += 32) a += part[(size_t)k * C + c];
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
+    if (lane == 0) out[c] = accum ? out[c] + a : a;
+}
+bool relu_bias_backward_supported(int dt, int C) {
+    const int V = dt ? 8 : 4;
+    if (C % V) return false;
+    const int cgs = C / V;
+    return cgs <= 256 && (cgs & (cgs - 1)) == 0;
+}
+size_t relu_bias_backward_scratch_elems(int C) { return (size_t)RB_MAX_CHUNKS * C; }
+void relu_bias_backward(int dt, const void* y_or_null, void* dy, float* db_or_null, float* scratch, long rows, int C, bool accum, cudaStream_t s) {
+    const int V = dt ? 8 : 4, rows_it = 256 / (C / V);
+    long chunks = (rows + (long)rows_it * 8 - 1) / ((long)rows_it * 8);              // at least eight passes per CTA
+    if (chunks > RB_MAX_CHUNKS) chunks = RB_MAX_CHUNKS;
+    if (chunks < 1) chunks = 1;
+    long per = (rows + chunks - 1) / chunks;
+    per = (per + rows_it - 1) / rows_it * rows_it;
+    chunks = (rows + per - 1) / per;
+    const double esz = dt ? 2.0 : 4.0;
+    { Scope sc(db_or_null ? KC_BIAS_GRAD : KC_RELU_BWD, 0.0, esz * rows * C * (y_or_null ? 3 : 1), s);
+      if (dt) relu_bias_bwd_k<bf16><<<(unsigned)chunks, 256, 0, s>>>((const bf16*)y_or_null, (bf16*)dy, db_or_null ? scratch : nullptr, rows, C, per);
+      else relu_bias_bwd_k<float><<<(unsigned)chunks, 256, 0, s>>>((const float*)y_or_null, (float*)dy, db_or_null ? scratch : nullptr, rows, C, per); }
+    if (db_or_null) {
+        Scope sc(KC_BIAS_GRAD, 0.0, 4.0 * chunks * C, s);
+        colsum_final_warp<<<cdiv((size_t)C * 32, 256), 256, 0, s>>>(scratch, db_or_null, (int)chunks, C, accum);
+    }
 }
 
 template <typename T>
@@ -427,21 +541,76 @@ __global__ void maxpool_bwd_k(const T* x, const T* dy, T* dx, int N, int H, int 
 #pragma unroll
     for (int j = 0; j < 4; ++j) { float v = (j == best) ? g : 0.f; if (accum) v += ld(dx + o[j]); st(dx + o[j], v); }
 }
+// the same with one 128-bit channel group per thread (C a multiple of the vector width)
+template <typename T>
+__global__ void __launch_bounds__(256) maxpool_fwd_vk(const T* __restrict__ x, T* __restrict__ y, int N, int H, int W, int C) {
+    constexpr int V = Vec<T>::V;
+    const int Ho = H / 2, Wo = W / 2, cgs = C / V;
+    const size_t total = (size_t)N * Ho * Wo * cgs;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int cg = (int)(i % cgs); size_t p = i / cgs; const int ox = (int)(p % Wo); p /= Wo; const int oy = (int)(p % Ho); const size_t n = p / Ho;
+        const T* b = x + ((n * H + 2 * oy) * W + 2 * ox) * C + (size_t)cg * V;
+        float a0[8], a1[8], a2[8], a3[8];
+        Vec<T>::load(b, a0); Vec<T>::load(b + C, a1); Vec<T>::load(b + (size_t)W * C, a2); Vec<T>::load(b + (size_t)W * C + C, a3);
+#pragma unroll
+        for (int j = 0; j < V; ++j) a0[j] = fmaxf(fmaxf(a0[j], a1[j]), fmaxf(a2[j], a3[j]));
+        Vec<T>::store(y + i * V, a0);
+    }
+}
+template <typename T>
+__global__ void __launch_bounds__(256) maxpool_bwd_vk(const T* __restrict__ x, const T* __restrict__ dy, T* dx, int N, int H, int W, int C, bool accum) {
+    constexpr int V = Vec<T>::V;
+    const int Ho = H / 2, Wo = W / 2, cgs = C / V;
+    const size_t total = (size_t)N * Ho * Wo * cgs;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int cg = (int)(i % cgs); size_t p = i / cgs; const int ox = (int)(p % Wo); p /= Wo; const int oy = (int)(p % Ho); const size_t n = p / Ho;
+        const size_t base = ((n * H + 2 * oy) * W + 2 * ox) * C + (size_t)cg * V;
+        const size_t o[4] = {base, base + (size_t)C, base + (size_t)W * C, base + (size_t)W * C + C};
+        float a[4][8], g[8];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) Vec<T>::load(x + o[q], a[q]);
+        Vec<T>::load(dy + i * V, g);
+        int best[8];
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+            int b = 0; float m = a[0][j];
+#pragma unroll
+            for (int q = 1; q < 4; ++q) if (a[q][j] > m) { m = a[q][j]; b = q; }            // first maximum wins
+            best[j] = b;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            float v[8];
+            if (accum) Vec<T>::load(dx + o[q], v);
+#pragma unroll
+            for (int j = 0; j < V; ++j) { const float t = best[j] == q ? g[j] : 0.f; v[j] = accum ? v[j] + t : t; }
+            Vec<T>::store(dx + o[q], v);
+        }
+    }
+}
 void maxpool_forward(int dt, const void* x, void* y, int N, int H, int W, int C, cudaStream_t s) {
-    const double esz_ = dt ? 2.0 : 4.0; (void)esz_;
+    const double esz_ = dt ? 2.0 : 4.0;
     Scope sc(KC_POOL_FWD, 0.0, 1.25 * esz_ * (double)N * H * W * C, s);
     size_t n = (size_t)N * (H / 2) * (W / 2) * C;
+    if (C % (dt ? 8 : 4) == 0) {
+        if (dt) maxpool_fwd_vk<bf16><<<ew_grid(n / 8), 256, 0, s>>>((const bf16*)x, (bf16*)y, N, H, W, C);
+        else maxpool_fwd_vk<float><<<ew_grid(n / 4), 256, 0, s>>>((const float*)x, (float*)y, N, H, W, C);
+        return;
+    }
     if (dt) maxpool_fwd_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)x, (bf16*)y, N, H, W, C);
     else maxpool_fwd_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)x, (float*)y, N, H, W, C);
-    
 }
 void maxpool_backward(int dt, const void* x, const void* dy, void* dx, int N, int H, int W, int C, bool accum, cudaStream_t s) {
-    const double esz_ = dt ? 2.0 : 4.0; (void)esz_;
+    const double esz_ = dt ? 2.0 : 4.0;
     Scope sc(KC_POOL_BWD, 0.0, 2.25 * esz_ * (double)N * H * W * C, s);
     size_t n = (size_t)N * (H / 2) * (W / 2) * C;
+    if (C % (dt ? 8 : 4) == 0) {
+        if (dt) maxpool_bwd_vk<bf16><<<ew_grid(n / 8), 256, 0, s>>>((const bf16*)x, (const bf16*)dy, (bf16*)dx, N, H, W, C, accum);
+        else maxpool_bwd_vk<float><<<ew_grid(n / 4), 256, 0, s>>>((const float*)x, (const float*)dy, (float*)dx, N, H, W, C, accum);
+        return;
+    }
     if (dt) maxpool_bwd_k<bf16><<<cdiv(n, 256), 256, 0, s>>>((const bf16*)x, (const bf16*)dy, (bf16*)dx, N, H, W, C, accum);
     else maxpool_bwd_k<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)x, (const float*)dy, (float*)dx, N, H, W, C, accum);
-    
 }
 
 template <typename T>
@@ -951,10 +1120,10 @@ void bn_backward(int dt, const void* x, const void* out, const void* dout, const
 // ------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void softmax_ce_k(const float* __restrict__ z, const int32_t* __restrict__ labels, T* __restrict__ dz,
-                             float* __restrict__ loss_out, int M, int C) {
+                             float* __restrict__ loss_out, int M, int C, float scale) {
     __shared__ float sh[256];
     float local = 0.f;
-    float inv_m = 1.f / (float)M;
+    const float inv_m = 1.f / (float)M;
     // exp / log in double: a few thousand values per step, and it keeps the error of (softmax - onehot) at the rounding
     // of the stored result instead of |z| * ulp(expf)
     for (int r = threadIdx.x; r < M; r += blockDim.x) {
@@ -966,17 +1135,17 @@ __global__ void softmax_ce_k(const float* __restrict__ z, const int32_t* __restr
         const double lse = (double)m + log(se);
         int y = labels[r];
         local += (float)(lse - (double)zr[y]);
-        for (int c = 0; c < C; ++c) st(dz + (size_t)r * C + c, (float)((exp((double)zr[c] - lse) - (c == y ? 1.0 : 0.0)) * (double)inv_m));
+        for (int c = 0; c < C; ++c) st(dz + (size_t)r * C + c, (float)((exp((double)zr[c] - lse) - (c == y ? 1.0 : 0.0)) * (double)scale));
     }
     sh[threadIdx.x] = local;
     __syncthreads();
     for (int s = 128; s > 0; s >>= 1) { if ((int)threadIdx.x < s) sh[threadIdx.x] += sh[threadIdx.x + s]; __syncthreads(); }
     if (threadIdx.x == 0) *loss_out = sh[0] * inv_m;
 }
-void softmax_ce(int dt, const float* logits, const int32_t* labels, void* dlogits, float* loss_out, int M, int classes, cudaStream_t s) {
+void softmax_ce(int dt, const float* logits, const int32_t* labels, void* dlogits, float* loss_out, int M, int classes, float scale, cudaStream_t s) {
     Scope sc(KC_SOFTMAX_CE, 0.0, (double)M * classes * (dt ? 6.0 : 8.0) + 4.0 * M, s);
-    if (dt) softmax_ce_k<bf16><<<1, 256, 0, s>>>(logits, labels, (bf16*)dlogits, loss_out, M, classes);
-    else softmax_ce_k<float><<<1, 256, 0, s>>>(logits, labels, (float*)dlogits, loss_out, M, classes);
+    if (dt) softmax_ce_k<bf16><<<1, 256, 0, s>>>(logits, labels, (bf16*)dlogits, loss_out, M, classes, scale);
+    else softmax_ce_k<float><<<1, 256, 0, s>>>(logits, labels, (float*)dlogits, loss_out, M, classes, scale);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1010,6 +1179,65 @@ void sgd_update(int dt, float* master, const float* grad, void* copy_next, size_
     Scope sc(KC_SGD, 0.0, (double)n * ((grad ? 12.0 : 4.0) + (dt ? 2.0 : 4.0)), s);
     if (dt) sgd_k<bf16><<<blocks, 256, 0, s>>>((float4*)master, (const float4*)grad, (bf16*)copy_next, n4, lr);
     else sgd_k<float><<<blocks, 256, 0, s>>>((float4*)master, (const float4*)grad, (float*)copy_next, n4, lr);
+}
+
+// ------------------------------------------------------------------------------------------
+// General mixing matrix (Eq. dl_update (a), (b)): R replicas of a module's parameters, each with its own gradient.
+//   u_r = w_r - lr * g_r ;  w_s(t+1) = sum_r P[s][r] * u_r  (r ascending) ;  copies of w_s(t+1) in the storage dtype.
+// A thread owns 4 consecutive parameters of ALL replicas: it reads the R masters (and gradients) first and writes the R
+// results afterwards, so the update is in place.  master / grad: [R][n_big + n_small]; the copies of replica r start
+// slot_bytes * r after copy0: n_big values in the storage dtype, then n_small floats.
+// ------------------------------------------------------------------------------------------
+constexpr int MIX_MAX_R = 32;
+template <typename T>
+__global__ void __launch_bounds__(256) mix_k(float* master, const float* __restrict__ grad, char* copy0, size_t n_big, size_t n_small, size_t slot_bytes,
+                                              int R, const float* __restrict__ P, float lr) {
+    __shared__ float Ps[MIX_MAX_R * MIX_MAX_R];
+    for (int i = threadIdx.x; i < R * R; i += blockDim.x) Ps[i] = P[i];
+    __syncthreads();
+    const size_t n = n_big + n_small, n4 = n / 4;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        float4 u[MIX_MAX_R];
+        for (int r = 0; r < R; ++r) {
+            float4 w = ((const float4*)(master + (size_t)r * n))[i];
+            if (grad) {
+                const float4 g = ((const float4*)(grad + (size_t)r * n))[i];
+                w.x = fmaf(-lr, g.x, w.x); w.y = fmaf(-lr, g.y, w.y); w.z = fmaf(-lr, g.z, w.z); w.w = fmaf(-lr, g.w, w.w);
+            }
+            u[r] = w;
+        }
+        for (int s = 0; s < R; ++s) {
+            float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int r = 0; r < R; ++r) {
+                const float p = Ps[s * R + r];
+                a.x = fmaf(p, u[r].x, a.x); a.y = fmaf(p, u[r].y, a.y); a.z = fmaf(p, u[r].z, a.z); a.w = fmaf(p, u[r].w, a.w);
+            }
+            ((float4*)(master + (size_t)s * n))[i] = a;
+            char* slot = copy0 + (size_t)s * slot_bytes;
+            const size_t e = i * 4;
+            if (e < n_big) {
+                if (sizeof(T) == 4) ((float4*)slot)[i] = a;
+                else {
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(a.z, a.w);
+                    uint2 pk; pk.x = *(unsigned*)&lo; pk.y = *(unsigned*)&hi;
+                    ((uint2*)slot)[i] = pk;
+                }
+            } else {
+                *(float4*)((float*)(slot + n_big * sizeof(T)) + (e - n_big)) = a;
+            }
+        }
+    }
+}
+int mix_max_replicas() { return MIX_MAX_R; }
+void mix_update(int dt, float* master, const float* grad, void* copy0, size_t n_big, size_t n_small, size_t slot_bytes, int R, const float* P, float lr,
+                cudaStream_t s) {
+    const size_t n4 = (n_big + n_small) / 4;
+    if (n4 == 0) return;
+    unsigned blocks = cdiv(n4, 256);
+    if (blocks > 148 * 4) blocks = 148 * 4;
+    Scope sc(KC_SGD, 0.0, (double)R * (n_big + n_small) * ((grad ? 12.0 : 8.0) + (dt ? 2.0 : 4.0)), s);
+    if (dt) mix_k<bf16><<<blocks, 256, 0, s>>>(master, grad, (char*)copy0, n_big, n_small, slot_bytes, R, P, lr);
+    else mix_k<float><<<blocks, 256, 0, s>>>(master, grad, (char*)copy0, n_big, n_small, slot_bytes, R, P, lr);
 }
 
 // ------------------------------------------------------------------------------------------

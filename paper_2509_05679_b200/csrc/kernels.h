@@ -29,6 +29,13 @@ void conv_wgrad(int dt, const void* x, const void* dy, float* dw, float* workspa
 // db[c] = sum over rows of dy[row][c]; scratch: fp32 [64 * C]
 void bias_grad(int dt, const void* dy, float* db, float* scratch, long rows, int C, bool accum, cudaStream_t st);
 
+// Backward pass through "+ bias, ReLU" of a layer in one pass over dy: dy *= (y > 0) in place (y_or_null == nullptr: no
+// ReLU) and db = column sums of the masked dy (db_or_null == nullptr: no bias).  scratch: relu_bias_backward_scratch_elems(C)
+// floats.  Only for widths relu_bias_backward_supported() accepts.
+bool   relu_bias_backward_supported(int dt, int C);
+size_t relu_bias_backward_scratch_elems(int C);
+void   relu_bias_backward(int dt, const void* y_or_null, void* dy, float* db_or_null, float* scratch, long rows, int C, bool accum, cudaStream_t st);
+
 // First-layer convolution (3x3, stride 1, <= 4 input channels, bf16): dedicated kernels (stem.cu).
 bool   stem_supported(int dt, const ConvGeom& g);
 size_t stem_wgrad_workspace_elems(const ConvGeom& g);
@@ -63,14 +70,21 @@ void bn_backward(int dt, const void* x, const void* out, const void* dout, const
                  float* red, float* scratch, int n_workers, long rows_per_worker, int C, bool relu, bool has_res, bool accum_params,
                  int* err, cudaStream_t st);
 
-// Softmax cross-entropy over fp32 logits [M, classes]: dlogits (storage dtype) = (softmax - onehot) / M,
+// Softmax cross-entropy over fp32 logits [M, classes]: dlogits (storage dtype) = (softmax - onehot) * scale,
 // *loss_out = mean loss.  Deterministic single-block reduction.
 void softmax_ce(int dt, const float* logits, const int32_t* labels, void* dlogits, float* loss_out, int M, int classes,
-                cudaStream_t st);
+                float scale, cudaStream_t st);
 
 // master -= lr * grad (skipped when grad == nullptr: w(t+1) = w(t)); copy_next = storage-dtype copy of
 // the new master (the next weight version).  n must be a multiple of 4; pointers 16-byte aligned.
 void sgd_update(int dt, float* master, const float* grad, void* copy_next, size_t n, float lr, cudaStream_t st);
+
+// General mixing matrix: R replicas [R][n_big + n_small] of master and grad; u_r = w_r - lr g_r (grad == nullptr: u_r = w_r),
+// w_s = sum_r P[s][r] u_r in place, and the storage-dtype copies of the next version (replica r at copy0 + r * slot_bytes:
+// n_big values of the storage dtype, then n_small floats).  R <= mix_max_replicas().
+int  mix_max_replicas();
+void mix_update(int dt, float* master, const float* grad, void* copy0, size_t n_big, size_t n_small, size_t slot_bytes, int R, const float* P, float lr,
+                cudaStream_t st);
 
 // Schedule tags (see fdg_trace).  tags are int64 pairs {batch id, weight version}.
 struct TagOps {

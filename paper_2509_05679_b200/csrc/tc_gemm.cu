@@ -1412,6 +1412,7 @@ cudaError_t run_km(const KmMaps& m, const KmParams& p_in, int n_tile, cudaStream
         }
         for (int i = 0; i < 9; ++i) rows = rows && p.rows_tap[i] >= 0;
     }
+    // three stages: four or five (they fit) change the forward pass by 3 % and the step not at all
     if (rows && n_tile == 64 && p.Cn == 64 && p.kchunks == 1) return launch_km<64, 3, 4, 1, true, 72>(*m.a_rows, *m.b, o, p, s);
     if (rows && n_tile == 128 && p.kchunks >= 2 && m.b_half && even) return launch_km_pair<128, 4, 4, 1, true>(*m.a_rows, *m.b_half, o, p, s);
     // measured on a B200: the narrow tiles run best with two CTAs per SM and short pipelines (3 x 24 KB, 2 x 32 KB stages);
