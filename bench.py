@@ -163,7 +163,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", type=int, default=3, help="0..4 = the five configurations; 3 = ResNet-18-shaped K=4, 8 workers x 128")
+    ap.add_argument("--config", type=int, default=3, help="0..4 = the five configurations; 3 = ResNet-18-shaped K=4, 8 workers x 128; 5 / 6 = the paper's ResNet-20 experiment shape with K = 1 / K = 2")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--worker-groups", type=int, default=0, help="0: chosen by the library; n: every module but the last runs its layers once per n-th of the workers")
     ap.add_argument("--kernel-path", type=int, default=0, help="0: tensor-core kernels where shapes allow (CTA pairs for the 256-column tile), 1: plain FMA kernels only, 2: tensor-core kernels without CTA pairs")

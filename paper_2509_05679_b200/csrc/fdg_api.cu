@@ -60,6 +60,7 @@ struct Op {
     // tensor-core plan (bf16 storage, channel counts that are multiples of 64, power-of-two images)
     bool tc;
     bool stem;                                               // thin first-layer conv: dedicated FMA kernels
+    bool head;                                               // the network's last linear layer: fused with the loss (head_* kernels)
     char shape[40];                                          // "HxW Cin->Cout kR sS", the profiler's detail tag
     int n_tile_f, n_tile_d, n_tile_w, wg_splits;
     tc::KmParams kf;
@@ -95,6 +96,8 @@ struct Module {
     size_t ws_elems, scratch_elems, red_elems;
     char *in_ring, *stash, *gradpool, *d2, *wring, *wtring;
     float *master, *grad, *ws, *scratch, *red, *cstat;
+    bool fused_update;             // one kernel per step updates all parameters and emits the next weight version (both layouts)
+    tc::UpdTable upd;
     size_t cstat_elems;
     int fused_stats_tensor, fused_stats_chunks;   // set by a conv that produced statistics partials for this tensor
     int64_t *tag_in, *tag_stash, *tag_d2, *tag_w, *trace;
@@ -104,6 +107,10 @@ struct Module {
     cudaEvent_t wev, wdone;        // dy ready for the weight-gradient stream / its work of this iteration finished
     cudaEvent_t done, fdone, ev0, ev1;
     float* scratch_f;              // reduction scratch of the forward stream
+    float* fwd_ws;                 // forward stream: partial sums of a forward pass that is split over its contraction
+    size_t fwd_ws_elems;
+    float* head_scratch;           // classifier head: weight-gradient partials, then loss partials
+    size_t head_elems, head_part_elems;
     bool had_bwd;
 };
 
@@ -290,10 +297,16 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
     if (m.ops.empty()) return "a module has no computing layer";
     if (m.ops.back().out != cur) return "internal: dangling tensor";
     h = m.t[cur].h; w = m.t[cur].w; c = m.t[cur].c;
+    m.head_elems = m.head_part_elems = 0;
     if (last) {
-        const Op& o = m.ops.back();
+        Op& o = m.ops.back();
         if (o.type != OP_CONV || o.relu || o.g.Ho * o.g.Wo != 1) return "the network must end with a linear layer";
         m.t[cur].loc = LOC_LOGITS;
+        if (o.g.H * o.g.W == 1 && o.g.R == 1 && head_supported(ctx->dt, o.g.C, o.g.Co)) {
+            o.head = true; o.tc = false; o.stem = false; o.stem_tc = false;
+            m.head_elems = head_scratch_elems(ctx->M, o.g.C, o.g.Co);
+            m.head_part_elems = m.head_elems - (size_t)(ctx->M + 7) / 8;
+        }
     } else {
         m.t[cur].loc = LOC_NEXT;
     }
@@ -308,7 +321,7 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
         if (d.loc == LOC_STASH) { d.off = soff; soff += align_up(d.elems() * ctx->M * ctx->esz, 256); }
         if (d.own_grad) { d.goff = goff; goff += align_up(d.elems() * ctx->M * ctx->esz, 256); }
     }
-    m.ws_elems = 0; m.scratch_elems = 64; m.red_elems = 4;
+    m.ws_elems = 0; m.scratch_elems = 64; m.red_elems = 4; m.fwd_ws_elems = 0;
     for (Op& o : m.ops) {
         if (o.type == OP_BN) {
             o.stats_off = soff; soff += align_up((size_t)ctx->n_workers * o.g.C * 2 * sizeof(float), 256);
@@ -320,6 +333,7 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
             if (o.stem) m.ws_elems = std::max(m.ws_elems, stem_wgrad_workspace_elems(o.g));
             if (o.stem_tc) m.ws_elems = std::max(m.ws_elems, tc::stem_wg_workspace_elems(o.g.Co, (long)o.g.N * o.g.H));
             m.ws_elems = std::max(m.ws_elems, wgrad_workspace_elems(o.g));
+            m.fwd_ws_elems = std::max(m.fwd_ws_elems, forward_workspace_elems(o.g));
             m.scratch_elems = std::max(m.scratch_elems, (size_t)64 * o.g.Co);
             if (relu_bias_backward_supported(ctx->dt, o.g.Co)) m.scratch_elems = std::max(m.scratch_elems, relu_bias_backward_scratch_elems(o.g.Co));
         }
@@ -503,6 +517,14 @@ void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int grou
                 int epi = (o.relu ? EPI_RELU : 0) | (to.loc == LOC_LOGITS ? EPI_OUT_F32 : 0);
                 ConvGeom g = o.g; g.N = wn.n;
                 profile_detail(o.shape);
+                if (o.head && m.groups == 1) {
+                    // logits, loss and dphi/dlogits / M of batch `batch` in one launch (version == the iteration t)
+                    head_forward_loss(dt, T(o.in), wbig(c, m, version, o.w_off), o.bias ? wsmall(c, m, version, o.b_off) : nullptr,
+                                      c->labels + (size_t)(batch % c->label_depth) * c->M, c->logits, c->dlogits, m.head_scratch + m.head_part_elems,
+                                      (unsigned*)(c->tc_err + 16), c->loss_ring + (version % 64), c->M, g.C, g.Co, 1.f / (float)c->M, s);
+                    profile_detail(nullptr);
+                    break;
+                }
                 if (o.tc && tc_forward(c, m, o, P.tensor(o.in), P.tensor(o.out), version, wn, s)) { profile_detail(nullptr); break; }
                 if (o.stem && tc_stem_forward(c, m, o, P.tensor(o.in), P.tensor(o.out), version, wn, s)) { profile_detail(nullptr); break; }
                 if (o.stem) {
@@ -510,7 +532,8 @@ void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int grou
                     profile_detail(nullptr);
                     break;
                 }
-                conv_forward(dt, T(o.in), wbig(c, m, version, o.w_off, rep), o.bias ? wsmall(c, m, version, o.b_off, rep) : nullptr, T(o.out), g, epi, s);
+                conv_forward(dt, T(o.in), wbig(c, m, version, o.w_off, rep), o.bias ? wsmall(c, m, version, o.b_off, rep) : nullptr, T(o.out), g, epi,
+                             m.fwd_ws, m.fwd_ws_elems, s);
                 profile_detail(nullptr);
                 break; }
             case OP_BN: {
@@ -566,6 +589,13 @@ void backward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int64_t
         switch (o.type) {
             case OP_CONV: {
                 ConvGeom g = o.g; g.N = wn.n;
+                if (o.head && m.groups == 1) {
+                    profile_detail(o.shape);
+                    head_backward(dt, T(o.in), wbig(c, m, version, o.w_off), gout, gin, o.acc_in, mgrad + o.w_off, o.bias ? mgrad + m.n_big + o.b_off : nullptr,
+                                  m.head_scratch, c->M, g.C, g.Co, s);
+                    profile_detail(nullptr);
+                    break;
+                }
                 // dZ = dA * (A > 0) in place and the bias gradient, in one pass over dA where the width allows
                 const long orows = (long)g.N * g.Ho * g.Wo;
                 const bool fused_rb = (o.relu || o.bias) && relu_bias_backward_supported(dt, g.Co);
@@ -841,7 +871,9 @@ fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, boo
             float* loss_slot = ctx->loss_ring + (t % 64);
             // one replica: dphi/dlogits / M, the mean over all samples.  One replica per worker: / B, worker s's own
             // gradient scale 1/per_worker_batch of Eq. dl_update (the mixing matrix does the averaging)
-            if (tau_f >= 0) softmax_ce(ctx->dt, ctx->logits, ctx->labels + (size_t)(tau_f % ctx->label_depth) * ctx->M, ctx->dlogits,
+            const bool fused_head = m.ops.back().head && m.groups == 1;     // the forward pass above has computed loss and dlogits
+            if (tau_f >= 0 && fused_head) {}
+            else if (tau_f >= 0) softmax_ce(ctx->dt, ctx->logits, ctx->labels + (size_t)(tau_f % ctx->label_depth) * ctx->M, ctx->dlogits,
                                        loss_slot, ctx->M, ctx->classes, ctx->R > 1 ? 1.f / (float)ctx->B : 1.f / (float)ctx->M, m.stream);
             else fill_f32(loss_slot, NAN, 1, m.stream);
         }
@@ -854,6 +886,9 @@ fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, boo
             // Eq. dl_update (a), (b) with a general P: u_r = w_r - lr g_r, w_s(t+1) = sum_r P_sr u_r, all replicas in one pass
             mix_update(ctx->dt, m.master, tau_b >= 0 ? m.grad : nullptr, wslot(ctx, m, t + 1, 0), m.n_big, m.n_small, m.wslot_bytes, ctx->R, ctx->P_dev,
                        ctx->lr, m.stream);
+        } else if (m.fused_update) {
+            Scope sc(KC_SGD, 0.0, (double)npar(m) * (tau_b >= 0 ? 12.0 : 4.0) + 2.0 * m.n_big + 4.0 * m.n_small + 2.0 * m.n_big, m.stream);
+            CK(tc::run_update_module(m.upd, m.master, m.grad, wslot(ctx, m, t + 1), wtslot(m, t + 1, 0), wsmall(ctx, m, t + 1, 0), ctx->lr, tau_b >= 0, m.stream));
         } else {
             sgd_update(ctx->dt, m.master, tau_b >= 0 ? m.grad : nullptr, wslot(ctx, m, t + 1), m.n_big, ctx->lr, m.stream);
             if (m.n_small)
@@ -1008,6 +1043,8 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
         m.scratch = (float*)get(m.scratch_elems * sizeof(float));
         m.red = (float*)get(m.red_elems * sizeof(float));
         m.scratch_f = (float*)get(m.scratch_elems * sizeof(float));
+        m.fwd_ws = m.fwd_ws_elems ? (float*)get(m.fwd_ws_elems * sizeof(float)) : nullptr;
+        m.head_scratch = m.head_elems ? (float*)get(m.head_elems * sizeof(float)) : nullptr;
         m.cstat = m.cstat_elems ? (float*)get(m.cstat_elems * sizeof(float)) : nullptr;
         if (oom) break;
         m.tag_in = ctx->tags + tpos; tpos += 2 * (size_t)m.in_depth;
@@ -1053,6 +1090,29 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
         const int n = ctx->M / m.groups;
         for (const Op& o : m.ops)
             if (o.tc && (n % o.kf.Nt || (o.kd.Nt && n % o.kd.Nt) || n % o.kw.Nt)) m.groups = 1;
+    }
+    // modules whose update runs as one kernel (instead of two update launches and one transposing launch per tensor-core
+    // layer): bf16, one weight copy, all workers at once, at least one tensor-core layer
+    for (Module& m : ctx->mod) {
+        m.fused_update = false;
+        tc::UpdTable& tb = m.upd; tb = tc::UpdTable{};
+        if (ctx->dt != 1 || ctx->R != 1 || m.groups != 1) continue;
+        size_t pos = 0;                              // everything below pos is covered
+        bool fits = true;
+        auto plain = [&](size_t a, size_t b) { if (b > a) { if (tb.nranges < 14) tb.ranges[tb.nranges++] = tc::UpdRange{a, b - a}; else fits = false; } };
+        for (const Op& o : m.ops) {
+            if (o.type != OP_CONV || !o.tc) continue;
+            if (tb.nops == 12) { fits = false; break; }
+            const int taps = o.g.R * o.g.R;
+            plain(pos, o.w_off);
+            tc::UpdOp u{}; u.w_off = o.w_off; u.Co = o.g.Co; u.taps = taps; u.Ci = o.g.C; u.tile0 = tb.total_tiles;
+            tb.total_tiles += (taps * o.g.C / 32) * (o.g.Co / 32);
+            tb.ops[tb.nops++] = u;
+            pos = o.w_off + (size_t)taps * o.g.C * o.g.Co;
+        }
+        plain(pos, npar(m));
+        tb.n_big = m.n_big;
+        m.fused_update = fits && tb.nops > 0;
     }
     *out = ctx;
     return FDG_OK;

@@ -274,15 +274,54 @@ size_t wgrad_workspace_elems(const ConvGeom& g) {
     return s > 1 ? (size_t)s * g.Co * g.R * g.R * g.C : 0;
 }
 
+// out[m][n] = epilogue(sum_z partial[z][m][n] + bias[n]), z ascending
 template <typename T>
-static void conv_forward_t(const void* x, const void* w, const float* bias, void* y, const ConvGeom& g, int epi, cudaStream_t s) {
+__global__ void splitk_forward_epilogue(const float* __restrict__ partial, void* __restrict__ out, const float* __restrict__ bias, size_t n, int Ng, int splits, int epi) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    float v = 0.f;
+    for (int z = 0; z < splits; ++z) v += partial[(size_t)z * n + i];
+    if (bias) v += bias[i % Ng];
+    if (epi & EPI_RELU) v = fmaxf(v, 0.f);
+    if (epi & EPI_OUT_F32) ((float*)out)[i] = v; else st((T*)out + i, v);
+}
+// A forward pass with few output tiles and a long contraction (a linear layer on a small batch: 8 CTAs walking 3072 terms)
+// is split over the contraction so that it fills the GPU; the partial sums go through `ws`.
+int forward_splits(const ConvGeom& g) {
+    const long Mg = (long)g.N * g.Ho * g.Wo, Ng = g.Co, Kg = (long)g.R * g.R * g.C;
+    const long tiles = (long)cdiv(Ng, BN) * cdiv(Mg, BM);
+    if (tiles >= 74 || Kg < 512 || Mg * Ng > (1 << 18)) return 1;
+    long s = (148 * 2) / tiles, maxs = Kg / 128;
+    if (s > maxs) s = maxs;
+    if (s > 32) s = 32;
+    return (int)(s < 1 ? 1 : s);
+}
+size_t forward_workspace_elems(const ConvGeom& g) {
+    const int s = forward_splits(g);
+    return s > 1 ? (size_t)s * g.N * g.Ho * g.Wo * g.Co : 0;
+}
+template <typename T>
+static void conv_forward_t(const void* x, const void* w, const float* bias, void* y, const ConvGeom& g, int epi, float* ws, size_t ws_elems, cudaStream_t s) {
     int Mg = g.N * g.Ho * g.Wo, Ng = g.Co, Kg = g.R * g.R * g.C;
+    const double flops = 2.0 * Mg * Ng * Kg, bytes = sizeof(T) * ((double)g.N * g.H * g.W * g.C + (double)Ng * Kg + (double)Mg * Ng);
+    int splits = ws ? forward_splits(g) : 1;
+    while (splits > 1 && (size_t)splits * Mg * Ng > ws_elems) --splits;          // a window of the batch: stay inside the workspace sized for the whole batch
+    if (splits > 1) {
+        const int kps = ((Kg + splits - 1) / splits + BK - 1) / BK * BK;
+        splits = (Kg + kps - 1) / kps;
+        dim3 grid(cdiv(Ng, BN), cdiv(Mg, BM), splits);
+        { Scope sc(KC_FMA_FWD, flops, bytes, s);
+          igemm_simt<T, M_FWD><<<grid, 256, 0, s>>>((const T*)x, (const T*)w, nullptr, nullptr, ws, g, Mg, Ng, Kg, kps, 0); }
+        Scope sc(KC_SPLITK, 0.0, 4.0 * (splits + 1) * Mg * Ng, s);
+        splitk_forward_epilogue<T><<<cdiv((size_t)Mg * Ng, 256), 256, 0, s>>>(ws, y, bias, (size_t)Mg * Ng, Ng, splits, epi);
+        return;
+    }
     dim3 grid(cdiv(Ng, BN), cdiv(Mg, BM), 1);
-    Scope sc(KC_FMA_FWD, 2.0 * Mg * Ng * Kg, sizeof(T) * ((double)g.N * g.H * g.W * g.C + (double)Ng * Kg + (double)Mg * Ng), s);
+    Scope sc(KC_FMA_FWD, flops, bytes, s);
     igemm_simt<T, M_FWD><<<grid, 256, 0, s>>>((const T*)x, (const T*)w, y, bias, nullptr, g, Mg, Ng, Kg, Kg, epi);
 }
-void conv_forward(int dt, const void* x, const void* w, const float* bias, void* y, const ConvGeom& g, int epi, cudaStream_t s) {
-    if (dt) conv_forward_t<bf16>(x, w, bias, y, g, epi, s); else conv_forward_t<float>(x, w, bias, y, g, epi, s);
+void conv_forward(int dt, const void* x, const void* w, const float* bias, void* y, const ConvGeom& g, int epi, float* ws, size_t ws_elems, cudaStream_t s) {
+    if (dt) conv_forward_t<bf16>(x, w, bias, y, g, epi, ws, ws_elems, s); else conv_forward_t<float>(x, w, bias, y, g, epi, ws, ws_elems, s);
 }
 
 template <typename T>
@@ -760,17 +799,10 @@ __global__ void bn_bwd_apply_k(const T* __restrict__ x, const T* __restrict__ ou
 constexpr int BNV_THREADS = 256;
 constexpr int BNV_MAX_CHUNKS = 128;
 constexpr int BV = 8;                               // channels per thread (one 128-bit access)
-#ifndef BNS_TILE_BYTES
-#define BNS_TILE_BYTES 16384
-#endif
-constexpr int BNS_TILE = BNS_TILE_BYTES;            // bytes per input tensor and stage
-#ifndef BNS_RING_KB
-#define BNS_RING_KB 96
-#endif
-#ifndef BNS_CTAS
-#define BNS_CTAS 2                                  // CTAs per SM the ring size allows
-#endif
-constexpr int BNS_RING = BNS_RING_KB * 1024;                 // shared memory of the ring (stages = tiles in the ring / input tensors, at most 8)
+// ring geometry: the best of the measured family (rings of 48..192 KB, 1..4 CTAs per SM, tiles of 8..32 KB)
+constexpr int BNS_TILE = 16384;                     // bytes per input tensor and stage
+constexpr int BNS_CTAS = 2;                         // CTAs per SM the ring size allows
+constexpr int BNS_RING = 96 * 1024;                 // shared memory of the ring (stages = tiles in the ring / input tensors, at most 8)
 constexpr int BNS_VPT = BNS_TILE / 16 / 256;        // 16-byte vectors per thread and tile
 constexpr long long BNS_WAIT_CYCLES = 4000000000LL; // ~2 s
 
@@ -1146,6 +1178,179 @@ void softmax_ce(int dt, const float* logits, const int32_t* labels, void* dlogit
     Scope sc(KC_SOFTMAX_CE, 0.0, (double)M * classes * (dt ? 6.0 : 8.0) + 4.0 * M, s);
     if (dt) softmax_ce_k<bf16><<<1, 256, 0, s>>>(logits, labels, (bf16*)dlogits, loss_out, M, classes, scale);
     else softmax_ce_k<float><<<1, 256, 0, s>>>(logits, labels, (float*)dlogits, loss_out, M, classes, scale);
+}
+
+// ------------------------------------------------------------------------------------------
+// Classifier head: the network's last linear layer (c_in -> a few classes) fused with the loss.
+//   head_fwd_loss_k : one warp per sample: logits = x W^T + b (fp32, kept for the caller), softmax cross-entropy,
+//                     dlogits = (softmax - onehot) * scale in the storage dtype, per-CTA loss partials; the CTA that
+//                     finishes last adds the partials in index order (a fixed order) and writes the mean loss.
+//   head_bwd_k      : a CTA owns a range of samples: dx = dlogits W (one warp per sample) and the partial sums of
+//                     dW[c][k] = sum_rows dlogits[row][c] x[row][k] and db[c] = sum_rows dlogits[row][c] (column k = K).
+//   head_reduce_k   : dW / db = partials added in CTA order.
+// Replaces an implicit-GEMM launch on 64 x 64 tiles (8-16 CTAs), a one-CTA loss kernel, two bias-gradient launches, a
+// split weight gradient with its reduction and an input-gradient launch.  classes <= 16, c_in a multiple of the vector width.
+// ------------------------------------------------------------------------------------------
+constexpr int HEAD_MAX_C = 16;
+constexpr int HEAD_ROWS_PER_CTA = 32;       // samples per CTA of head_bwd_k
+template <typename T>
+__global__ void __launch_bounds__(256) head_fwd_loss_k(const T* __restrict__ x, const T* __restrict__ W, const float* __restrict__ bias,
+                                                       const int32_t* __restrict__ labels, float* __restrict__ logits, T* __restrict__ dz,
+                                                       float* __restrict__ loss_part, unsigned* __restrict__ counter, float* __restrict__ loss_out,
+                                                       int M, int K, int C, float scale) {
+    constexpr int V = Vec<T>::V;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = blockIdx.x * 8 + warp;
+    __shared__ float wl[8];
+    __shared__ bool last;
+    float rloss = 0.f;
+    if (row < M) {
+        float acc[HEAD_MAX_C];
+#pragma unroll
+        for (int c = 0; c < HEAD_MAX_C; ++c) acc[c] = 0.f;
+        const T* xr = x + (size_t)row * K;
+        for (int kv = lane; kv < K / V; kv += 32) {
+            float xv[8];
+            Vec<T>::load(xr + (size_t)kv * V, xv);
+#pragma unroll
+            for (int c = 0; c < HEAD_MAX_C; ++c) {
+                if (c < C) {
+                    float wv[8];
+                    Vec<T>::load(W + (size_t)c * K + (size_t)kv * V, wv);
+#pragma unroll
+                    for (int j = 0; j < V; ++j) acc[c] = fmaf(xv[j], wv[j], acc[c]);
+                }
+            }
+        }
+        float z = 0.f;                       // lane c keeps logit c
+#pragma unroll
+        for (int c = 0; c < HEAD_MAX_C; ++c) {
+            float v = acc[c];
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+            if (lane == c) z = v + (bias ? bias[c] : 0.f);
+        }
+        const bool mine = lane < C;
+        if (mine) logits[(size_t)row * C + lane] = z;
+        float m = mine ? z : -INFINITY;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+        // exp / log in double: it keeps the error of (softmax - onehot) at the rounding of the stored result
+        double e = mine ? exp((double)z - (double)m) : 0.0;
+        double se = e;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) se += __shfl_xor_sync(0xffffffffu, se, d);
+        const double lse = (double)m + log(se);
+        const int y = labels[row];
+        const float zy = __shfl_sync(0xffffffffu, z, y);
+        rloss = (float)(lse - (double)zy);
+        if (mine) st(dz + (size_t)row * C + lane, (float)((exp((double)z - lse) - (lane == y ? 1.0 : 0.0)) * (double)scale));
+    }
+    if (lane == 0) wl[warp] = rloss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float s = 0.f;
+        for (int i = 0; i < 8; ++i) s += wl[i];
+        loss_part[blockIdx.x] = s;
+        __threadfence();
+        last = atomicAdd(counter, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (last && threadIdx.x == 0) {
+        __threadfence();
+        float s = 0.f;
+        for (unsigned i = 0; i < gridDim.x; ++i) s += ((volatile float*)loss_part)[i];
+        *loss_out = s / (float)M;
+        *counter = 0u;
+    }
+}
+// grid = ceil(M / HEAD_ROWS_PER_CTA).  part: [CTA][C][K + 1]
+template <typename T>
+__global__ void __launch_bounds__(256) head_bwd_k(const T* __restrict__ x, const T* __restrict__ W, const T* __restrict__ dz, T* dx, float* __restrict__ part,
+                                                  int M, int K, int C, bool accum_dx) {
+    constexpr int V = Vec<T>::V;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r0 = blockIdx.x * HEAD_ROWS_PER_CTA, r1 = min(M, r0 + HEAD_ROWS_PER_CTA);
+    __shared__ float dzs[HEAD_ROWS_PER_CTA][HEAD_MAX_C];
+    for (int i = threadIdx.x; i < (r1 - r0) * C; i += 256) dzs[i / C][i % C] = ld(dz + (size_t)r0 * C + i);
+    __syncthreads();
+    if (dx) {
+        for (int r = r0 + warp; r < r1; r += 8) {
+            for (int kv = lane; kv < K / V; kv += 32) {
+                float a[8];
+#pragma unroll
+                for (int j = 0; j < V; ++j) a[j] = 0.f;
+                for (int c = 0; c < C; ++c) {
+                    float wv[8];
+                    Vec<T>::load(W + (size_t)c * K + (size_t)kv * V, wv);
+                    const float g = dzs[r - r0][c];
+#pragma unroll
+                    for (int j = 0; j < V; ++j) a[j] = fmaf(g, wv[j], a[j]);
+                }
+                T* d = dx + (size_t)r * K + (size_t)kv * V;
+                if (accum_dx) {
+                    float old[8];
+                    Vec<T>::load(d, old);
+#pragma unroll
+                    for (int j = 0; j < V; ++j) a[j] += old[j];
+                }
+                Vec<T>::store(d, a);
+            }
+        }
+    }
+    // partial sums: (class, vector of V columns) pairs round-robin over the threads, rows in ascending order
+    float* out = part + (size_t)blockIdx.x * C * (K + 1);
+    const int nkv = K / V;
+    for (int p = threadIdx.x; p < C * nkv; p += 256) {
+        const int c = p / nkv, kv = p - c * nkv;
+        float a[8];
+#pragma unroll
+        for (int j = 0; j < V; ++j) a[j] = 0.f;
+        for (int r = r0; r < r1; ++r) {
+            float xv[8];
+            Vec<T>::load(x + (size_t)r * K + (size_t)kv * V, xv);
+            const float g = dzs[r - r0][c];
+#pragma unroll
+            for (int j = 0; j < V; ++j) a[j] = fmaf(g, xv[j], a[j]);
+        }
+#pragma unroll
+        for (int j = 0; j < V; ++j) out[(size_t)c * (K + 1) + kv * V + j] = a[j];
+    }
+    if (threadIdx.x < C) {
+        float a = 0.f;
+        for (int r = r0; r < r1; ++r) a += dzs[r - r0][threadIdx.x];
+        out[(size_t)threadIdx.x * (K + 1) + K] = a;
+    }
+}
+__global__ void head_reduce_k(const float* __restrict__ part, float* __restrict__ dW, float* __restrict__ db, int ctas, int K, int C) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= C * (K + 1)) return;
+    float s = 0.f;
+    for (int b = 0; b < ctas; ++b) s += part[(size_t)b * C * (K + 1) + i];
+    const int c = i / (K + 1), k = i - c * (K + 1);
+    if (k < K) dW[(size_t)c * K + k] = s;
+    else if (db) db[c] = s;
+}
+bool head_supported(int dt, int K, int C) { return C >= 2 && C <= HEAD_MAX_C && K % (dt ? 8 : 4) == 0; }
+size_t head_scratch_elems(int M, int K, int C) {
+    const size_t ctas = (M + HEAD_ROWS_PER_CTA - 1) / HEAD_ROWS_PER_CTA;
+    return ctas * C * (K + 1) + (M + 7) / 8;
+}
+void head_forward_loss(int dt, const void* x, const void* W, const float* bias, const int32_t* labels, float* logits, void* dlogits, float* scratch,
+                       unsigned* counter, float* loss_out, int M, int K, int C, float scale, cudaStream_t s) {
+    Scope sc(KC_SOFTMAX_CE, 2.0 * M * K * C, (dt ? 2.0 : 4.0) * ((double)M * K + (double)C * K + (double)M * C) + 4.0 * M * C, s);
+    const unsigned grid = (M + 7) / 8;
+    if (dt) head_fwd_loss_k<bf16><<<grid, 256, 0, s>>>((const bf16*)x, (const bf16*)W, bias, labels, logits, (bf16*)dlogits, scratch, counter, loss_out, M, K, C, scale);
+    else head_fwd_loss_k<float><<<grid, 256, 0, s>>>((const float*)x, (const float*)W, bias, labels, logits, (float*)dlogits, scratch, counter, loss_out, M, K, C, scale);
+}
+void head_backward(int dt, const void* x, const void* W, const void* dlogits, void* dx_or_null, bool accum_dx, float* dW, float* db_or_null, float* scratch,
+                   int M, int K, int C, cudaStream_t s) {
+    const unsigned ctas = (M + HEAD_ROWS_PER_CTA - 1) / HEAD_ROWS_PER_CTA;
+    { Scope sc(KC_FMA_WGRAD, (dx_or_null ? 4.0 : 2.0) * M * K * C, (dt ? 2.0 : 4.0) * ((double)M * K * (dx_or_null ? 2 : 1) + (double)C * K + (double)M * C), s);
+      if (dt) head_bwd_k<bf16><<<ctas, 256, 0, s>>>((const bf16*)x, (const bf16*)W, (const bf16*)dlogits, (bf16*)dx_or_null, scratch, M, K, C, accum_dx);
+      else head_bwd_k<float><<<ctas, 256, 0, s>>>((const float*)x, (const float*)W, (const float*)dlogits, (float*)dx_or_null, scratch, M, K, C, accum_dx); }
+    Scope sc(KC_SPLITK, 0.0, 4.0 * (ctas + 1) * C * (K + 1), s);
+    head_reduce_k<<<cdiv((size_t)C * (K + 1), 256), 256, 0, s>>>(scratch, dW, db_or_null, (int)ctas, K, C);
 }
 
 // ------------------------------------------------------------------------------------------

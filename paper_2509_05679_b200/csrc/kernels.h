@@ -18,8 +18,11 @@ int    wgrad_splits(const ConvGeom& g);
 size_t wgrad_workspace_elems(const ConvGeom& g);
 
 // y = conv(x, W) (+ bias) (relu)            (Eq. forward_step for linear / conv layers)
+// workspace: forward_workspace_elems(g) floats (0: none needed), or nullptr: a forward pass with few output tiles and a
+// long contraction is split over the contraction through it
+size_t forward_workspace_elems(const ConvGeom& g);
 void conv_forward(int dt, const void* x, const void* w, const float* bias, void* y, const ConvGeom& g,
-                  int epi, cudaStream_t st);
+                  int epi, float* workspace, size_t workspace_elems, cudaStream_t st);
 // dx (+)= conv_transpose(dy, W)             (Eq. backward_step, gradient w.r.t. the layer input)
 void conv_dgrad(int dt, const void* dy, const void* w, void* dx, const ConvGeom& g, int epi, cudaStream_t st);
 // dW = sum over all N*Ho*Wo rows of dy^T (x) patches(x), fp32 out; the reduction runs over the
@@ -74,6 +77,17 @@ void bn_backward(int dt, const void* x, const void* out, const void* dout, const
 // *loss_out = mean loss.  Deterministic single-block reduction.
 void softmax_ce(int dt, const float* logits, const int32_t* labels, void* dlogits, float* loss_out, int M, int classes,
                 float scale, cudaStream_t st);
+
+// Classifier head (the last linear layer, c_in = K -> C classes, C <= 16) fused with the loss.  head_forward_loss: logits
+// (fp32), dlogits = (softmax - onehot) * scale (storage dtype) and the mean loss in one launch; `counter` is a device word
+// that is zero between launches.  head_backward: dx (+)= dlogits W (dx_or_null == nullptr: not needed), dW, db.
+// scratch: head_scratch_elems floats, used by both (the loss partials follow the weight-gradient partials).
+bool   head_supported(int dt, int K, int C);
+size_t head_scratch_elems(int M, int K, int C);
+void   head_forward_loss(int dt, const void* x, const void* W, const float* bias, const int32_t* labels, float* logits, void* dlogits, float* scratch,
+                         unsigned* counter, float* loss_out, int M, int K, int C, float scale, cudaStream_t st);
+void   head_backward(int dt, const void* x, const void* W, const void* dlogits, void* dx_or_null, bool accum_dx, float* dW, float* db_or_null, float* scratch,
+                     int M, int K, int C, cudaStream_t st);
 
 // master -= lr * grad (skipped when grad == nullptr: w(t+1) = w(t)); copy_next = storage-dtype copy of
 // the new master (the next weight version).  n must be a multiple of 4; pointers 16-byte aligned.

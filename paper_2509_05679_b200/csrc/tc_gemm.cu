@@ -33,9 +33,7 @@ constexpr int BLOCK_K = 64;       // bf16 elements per 128-byte swizzle row
 constexpr int UMMA_K = 16;
 constexpr int NUM_THREADS = 192;
 constexpr long long WAIT_CYCLES = 4000000000LL;   // ~2 s at 2 GHz
-#ifndef EPI_SLEEP_NS
-#define EPI_SLEEP_NS 200
-#endif
+constexpr unsigned EPI_SLEEP_NS = 200;            // pause between polls of a long wait (epilogue warps)
 
 // ------------------------------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -1248,29 +1246,117 @@ stem_fw_kernel(const __grid_constant__ CUtensorMap tmRaw, const __grid_constant_
     if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 128); }
 }
 
-// dW[co][tap][ci] = sum_z partial[z][(tap, cc)][ci % 64][co], z ascending.  32x32 transposing tiles; a thread owns
-// one (row, column) per pass and keeps eight independent loads in flight along z.
-__global__ void __launch_bounds__(1024) wg_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dw, int splits, int row_blocks, int Co,
-                                                         bool accum) {
+// dW[co][tap][ci] = sum_z partial[z][(tap, cc)][ci % 64][co], z ascending.  32x32 transposing tiles; 256 threads (a CTA of
+// this size fits beside a resident tensor-core CTA of another stream), a thread owns four (row, column) pairs and keeps
+// 32 independent loads in flight (eight along z for each pair).
+__global__ void __launch_bounds__(256) wg_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dw, int splits, int row_blocks, int Co,
+                                                        bool accum) {
     __shared__ float t[32][33];
     const int R = row_blocks * 64;                       // = taps * Cin
     const int r0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
-    const int tx = threadIdx.x, ty = threadIdx.y;        // 32 x 32
-    const size_t o = (size_t)(r0 + ty) * Co + c0 + tx, zs = (size_t)R * Co;
-    float s = 0.f;
+    const int tx = threadIdx.x, ty = threadIdx.y;        // 32 x 8
+    const unsigned zs = (unsigned)R * Co, rs = 8u * Co;                      // one partial matrix (< 2^32 elements); this thread's rows are 8 apart
+    const float* p = partial + (size_t)(r0 + ty) * Co + c0 + tx;
+    float s[4] = {0.f, 0.f, 0.f, 0.f};
     int z = 0;
-    for (; z + 8 <= splits; z += 8) {
-        float v[8];
+    for (; z + 8 <= splits; z += 8, p += (size_t)8 * zs) {
+        float v[4][8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = __ldg(partial + (size_t)(z + j) * zs + o);
+        for (int j = 0; j < 8; ++j)
 #pragma unroll
-        for (int j = 0; j < 8; ++j) s += v[j];
+            for (int i = 0; i < 4; ++i) v[i][j] = __ldg(p + j * zs + i * rs);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) s[i] += v[i][j];
     }
-    for (; z < splits; ++z) s += __ldg(partial + (size_t)z * zs + o);
-    t[ty][tx] = s;
+    for (; z < splits; ++z, p += zs)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) s[i] += __ldg(p + i * rs);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) t[ty + 8 * i][tx] = s[i];
     __syncthreads();
-    float* d = dw + (size_t)(c0 + ty) * R + r0 + tx;
-    *d = accum ? *d + t[tx][ty] : t[tx][ty];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float* d = dw + (size_t)(c0 + ty + 8 * i) * R + r0 + tx;
+        *d = accum ? *d + t[tx][ty + 8 * i] : t[tx][ty + 8 * i];
+    }
+}
+
+// One launch per module and step: the update of Eq. dl_update for ALL of the module's parameters.
+//   * weight matrices of tensor-core layers, in 32 x 32 tiles: w -= lr g on the fp32 master, the bf16 copy W[co][tap][ci] of
+//     the next version and its tap-flipped transpose Wt[ci][taps-1-tap][co] for the input-gradient kernel;
+//   * everything else (matrices of other layers, biases, gamma, beta), 4 values per thread: w -= lr g, the storage copy.
+// has_grad == 0 (no backward batch yet): w(t+1) = w(t), only the copies are written.
+// (Summing the weight-gradient partials here as well was measured slower: that reduction then sits in the module's chain
+// in front of its next forward pass instead of running beside the backward pass on the weight-gradient stream.)
+// 256 threads and few registers per CTA: the CTAs fit beside a resident tensor-core CTA of another module, so the
+// update does not wait for a persistent kernel to drain (with 1024-thread CTAs it did, and the step took 4 % longer).
+__global__ void __launch_bounds__(256) update_module_kernel(UpdTable tb, float* __restrict__ master, const float* __restrict__ grad,
+                                                            bf16* __restrict__ wcopy, bf16* __restrict__ wtcopy, float* __restrict__ small_copy, float lr,
+                                                            int has_grad) {
+    __shared__ bf16 t[32][34];
+    const int tx = threadIdx.x, ty = threadIdx.y;          // 32 x 8
+    int b = blockIdx.x;
+    if (b < tb.total_tiles) {
+        int oi = 0;
+        while (oi + 1 < tb.nops && b >= tb.ops[oi + 1].tile0) ++oi;
+        const UpdOp o = tb.ops[oi];
+        b -= o.tile0;
+        const int R = o.taps * o.Ci, tiles_c = o.Co / 32;
+        const int r0 = (b / tiles_c) * 32, c0 = (b % tiles_c) * 32;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int c = ty + 8 * i;                          // row c0 + c of W, columns r0 + tx
+            const size_t idx = o.w_off + (size_t)(c0 + c) * R + r0 + tx;
+            float w = master[idx];
+            if (has_grad) { w = fmaf(-lr, grad[idx], w); master[idx] = w; }
+            const bf16 wb = __float2bfloat16_rn(w);
+            wcopy[idx] = wb;
+            t[c][tx] = wb;                                     // [c][r]
+        }
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = r0 + ty + 8 * i, tap = r / o.Ci, ci = r - tap * o.Ci;     // a tile's 32 rows share one tap (Ci is a multiple of 64)
+            wtcopy[o.w_off + ((size_t)ci * o.taps + (o.taps - 1 - tap)) * o.Co + c0 + tx] = t[tx][ty + 8 * i];
+        }
+        return;
+    }
+    // the other ranges: float4 number q of their concatenation
+    const size_t q = (size_t)(b - tb.total_tiles) * 256 + ty * 32 + tx;
+    size_t first = 0;
+    for (int j = 0; j < tb.nranges; ++j) {
+        const size_t n4 = tb.ranges[j].count / 4;
+        if (q < first + n4) {
+            const size_t e = tb.ranges[j].start + (q - first) * 4;
+            float4 w = *(const float4*)(master + e);
+            if (has_grad) {
+                const float4 g = *(const float4*)(grad + e);
+                w.x = fmaf(-lr, g.x, w.x); w.y = fmaf(-lr, g.y, w.y); w.z = fmaf(-lr, g.z, w.z); w.w = fmaf(-lr, g.w, w.w);
+                *(float4*)(master + e) = w;
+            }
+            if (e < tb.n_big) {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
+                uint2 pk; pk.x = *(unsigned*)&lo; pk.y = *(unsigned*)&hi;
+                *(uint2*)(wcopy + e) = pk;
+            } else {
+                *(float4*)(small_copy + (e - tb.n_big)) = w;
+            }
+            return;
+        }
+        first += n4;
+    }
+}
+
+cudaError_t run_update_module(const UpdTable& tb, float* master, const float* grad, void* wcopy, void* wtcopy, float* small_copy, float lr,
+                              bool has_grad, cudaStream_t s) {
+    size_t plain4 = 0;
+    for (int j = 0; j < tb.nranges; ++j) plain4 += tb.ranges[j].count / 4;
+    const unsigned blocks = (unsigned)(tb.total_tiles + (plain4 + 255) / 256);
+    if (!blocks) return cudaSuccess;
+    update_module_kernel<<<blocks, dim3(32, 8), 0, s>>>(tb, master, grad, (bf16*)wcopy, (bf16*)wtcopy, small_copy, lr, has_grad ? 1 : 0);
+    return cudaGetLastError();
 }
 
 // Wt[ci][R*R-1-tap][co] = W[co][tap][ci]: the weights of the transposed convolution, K-major for km_kernel.
@@ -1445,7 +1531,7 @@ cudaError_t run_wg(const TensorMap& x, const TensorMap& dy, const WgParams& p, i
     else if (n_tile == 256) e = launch_wg<256, 4>(x, dy, p, grid, s);
     else return cudaErrorInvalidValue;
     if (e != cudaSuccess) return e;
-    dim3 rgrid(p.row_blocks * 2, p.Co / 32), rblk(32, 32);
+    dim3 rgrid(p.row_blocks * 2, p.Co / 32), rblk(32, 8);
     wg_reduce_kernel<<<rgrid, rblk, 0, s>>>(p.partial, dw, splits, p.row_blocks, p.Co, accum);
     return cudaGetLastError();
 }
@@ -1491,7 +1577,7 @@ cudaError_t run_wg_rows(const TensorMap& x_rows, const TensorMap& dy128, const W
     else if (variant == 2) e = launch_wg2<128, 2, 20, 3>(x_rows, dy128, p, dim3(3 * (q.C / 128), q.Co / 128, z), s);
     else return cudaErrorInvalidValue;
     if (e != cudaSuccess) return e;
-    dim3 rgrid(p.row_blocks * 2, p.Co / 32), rblk(32, 32);
+    dim3 rgrid(p.row_blocks * 2, p.Co / 32), rblk(32, 8);
     wg_reduce_kernel<<<rgrid, rblk, 0, s>>>(p.partial, dw, z, p.row_blocks, p.Co, accum);
     return cudaGetLastError();
 }

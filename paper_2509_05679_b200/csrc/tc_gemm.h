@@ -85,6 +85,7 @@ int wg_rows_variant(int H, int W, int C, int Co);
 int wg_rows_splits(int variant, int C, int Co, long steps);
 cudaError_t run_wg_rows(const TensorMap& x_rows, const TensorMap& dy128, const WgRowsParams& p, int variant, int splits, float* dw, bool accum,
                         cudaStream_t s);
+
 // Weight gradient of the first layer (3x3, stride 1, pad 1, 3 input channels) on the tensor cores; the im2col lines are
 // built in shared memory.  x_raw: x as rows of W * 3 elements with a box of (128 / W + 2) rows (make_map_raw_rows);
 // dy128: dy with a box of 64 channels x 128 pixels (make_map_4d).  All N samples; partial: stem_wg_workspace_elems floats.
@@ -99,5 +100,21 @@ cudaError_t run_stem_fw(const TensorMap& x_raw, const TensorMap& out_map, int H,
                         float* stat_part, int* err, cudaStream_t s);
 cudaError_t run_flip_transpose(const void* w, void* wt, int Co, int taps, int Ci, cudaStream_t s);
 
+
+// The whole update of one module in one launch (see update_module_kernel).
+struct UpdOp {                   // weight matrix W[Co][taps][Ci] of a tensor-core layer
+    unsigned long long w_off;    // element offset in the module's matrix segment
+    int Co, taps, Ci;
+    int tile0;                   // first 32 x 32 tile of this matrix in the launch
+};
+struct UpdRange { unsigned long long start, count; };   // elements (multiples of 4) outside those matrices
+struct UpdTable {
+    int nops, nranges, total_tiles;
+    unsigned long long n_big;    // elements of the matrix segment; the vector segment follows it
+    UpdOp ops[12];
+    UpdRange ranges[14];
+};
+cudaError_t run_update_module(const UpdTable& tb, float* master, const float* grad, void* wcopy, void* wtcopy, float* small_copy, float lr,
+                              bool has_grad, cudaStream_t s);
 }  // namespace tc
 }  // namespace fdg

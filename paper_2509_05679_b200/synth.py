@@ -218,8 +218,15 @@ def config(idx: int, *, n_workers: int | None = None, batch: int | None = None,
         else:
             splits = bs[1:]                          # one basic block per module
             net = Net("C5-resnet18-K8-bf16", layers, splits, 32, 32, 3, 10, 16, 256, 0.05, "bf16", steps=50)
+    elif idx in (5, 6):
+        # the paper's experiment shape (Sec. 5) on synthetic data: ResNet-20 (3 stages of 16/32/64 channels, 3 blocks
+        # each), 4 data-groups, mini-batch 194 read as the total (48 samples per worker), step size 0.1;
+        # 5: traditional backpropagation (K = 1), 6: decoupled into K = 2 modules (cut between blocks 4 and 5)
+        layers, bs = resnet_layers(widths=(16, 32, 64), blocks=3)
+        net = Net("resnet20-S4-K1-fp32" if idx == 5 else "resnet20-S4-K2-fp32", layers, [] if idx == 5 else [bs[4]],
+                  32, 32, 3, 10, 4, 48, 0.1, "fp32", steps=50)
     else:
-        raise ValueError("config index 0..4")
+        raise ValueError("config index 0..6")
     if K is not None and K == 1:
         net.splits = []
     if n_workers is not None:
