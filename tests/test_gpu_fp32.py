@@ -138,3 +138,26 @@ def test_param_layout_matches_the_canonical_order_and_addresses_single_tensors()
     back = ctx.params()
     assert np.all(back[offset:offset + count] == 0.5) and np.array_equal(np.delete(back, np.s_[offset:offset + count]), np.delete(p0, np.s_[offset:offset + count]))
     ctx.close()
+
+
+def test_join_orders_a_caller_stream_behind_the_steps():
+    """fdg_join: work the caller enqueues on its own stream afterwards runs after the last update.  An event recorded
+    behind the join must complete no earlier than an event the library's last kernel precedes: after synchronising the
+    caller's stream alone, the device holds the final weights (a second read after a full device sync is identical)."""
+    import torch
+    from paper_2509_05679_b200 import binding
+    net = as_fp32(sy.config(3, n_workers=2, batch=4, width_div=8))
+    ctx = make_ctx(net, sy.init_params(net.layers, 0))
+    xs = [binding.to_device("fp32", sy.batch_inputs(net, t)) for t in range(3)]
+    ys = [torch.from_numpy(sy.batch_labels(net, t)).cuda() for t in range(3)]
+    mine = torch.cuda.Stream()
+    for t in range(2 * net.K + 1):
+        ctx.step(xs[t % 3], ys[t % 3])
+    ctx.join(mine.cuda_stream)
+    done = torch.cuda.Event()
+    done.record(mine)
+    done.synchronize()
+    first = ctx.params()
+    torch.cuda.synchronize()
+    assert np.array_equal(first, ctx.params())
+    ctx.close()
