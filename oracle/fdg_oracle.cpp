@@ -12,7 +12,7 @@
 //    predecessor posted in the previous iteration and back-propagates whatever error gradient
 //    its successor posted in the previous iteration (Algorithm 1's send/receive pairs);
 //  * the backward pass of batch tau in module k uses the weights the forward pass of that batch
-//    used (Sec. 3.2 "Backward": w_l(t-2K+2k) "belonging to itself"), taken from the stash;
+//    used (Sec. 3.2, backward pass: the module's own weights of version t-2K+2k), taken from the stash;
 //  * u_{s,k} = w_{s,k} - eta * g_{s,k};  w_{s,k}(t+1) = sum_r P_{sr} u_{r,k}   (Eq. dl_update),
 //    g = 0 while no error gradient has arrived (tau < 0);
 //  * layers are the textbook definitions written as loops (Eq. forward_step / backward_step).

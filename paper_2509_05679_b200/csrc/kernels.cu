@@ -423,9 +423,9 @@ static unsigned ew_grid(size_t nvec) { size_t b = (nvec + 255) / 256; return (un
 
 // OP 0: y = max(x, 0).  OP 1: dx (+)= dy * (y > 0)   (a = y, b = dy, o = dx).  OP 2: y = a + b.  OP 3: dst (+)= src   (a = src, o = dst).
 template <typename T, int OP>
-__global__ void __launch_bounds__(256) ew_k(const T* __restrict__ a, const T* __restrict__ b, T* o, size_t n, bool accum) {
+__global__ void __launch_bounds__(256) ew_k(const T* __restrict__ a, const T* __restrict__ b, T* o, size_t n, bool accum, bool aligned) {
     constexpr int V = Vec<T>::V;
-    const size_t nvec = n / V, stride = (size_t)gridDim.x * blockDim.x, t0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t nvec = aligned ? n / V : 0, stride = (size_t)gridDim.x * blockDim.x, t0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     for (size_t i = t0; i < nvec; i += stride) {
         float fa[8], fb[8], fo[8];
         Vec<T>::load(a + i * V, fa);
@@ -455,8 +455,11 @@ __global__ void __launch_bounds__(256) ew_k(const T* __restrict__ a, const T* __
 }
 template <int OP>
 static void ew_launch(int dt, const void* a, const void* b, void* o, size_t n, bool accum, cudaStream_t s) {
-    if (dt) ew_k<bf16, OP><<<ew_grid(n / 8), 256, 0, s>>>((const bf16*)a, (const bf16*)b, (bf16*)o, n, accum);
-    else ew_k<float, OP><<<ew_grid(n / 4), 256, 0, s>>>((const float*)a, (const float*)b, (float*)o, n, accum);
+    // a window of a tensor whose rows are no multiple of 16 bytes can start anywhere: such calls go element by element
+    const bool aligned = (((uintptr_t)a | (uintptr_t)b | (uintptr_t)o) & 15) == 0;
+    const size_t work = aligned ? n / (dt ? 8 : 4) : n;
+    if (dt) ew_k<bf16, OP><<<ew_grid(work), 256, 0, s>>>((const bf16*)a, (const bf16*)b, (bf16*)o, n, accum, aligned);
+    else ew_k<float, OP><<<ew_grid(work), 256, 0, s>>>((const float*)a, (const float*)b, (float*)o, n, accum, aligned);
 }
 
 void relu_forward(int dt, const void* x, void* y, size_t n, cudaStream_t s) {

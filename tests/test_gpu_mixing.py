@@ -46,7 +46,8 @@ def nets():
     mlp = sy.Net("mlp-mix", sy.mlp_layers([24, 32, 16, 10]), [2], 1, 1, 24, 10, 4, 6, 0.1, "fp32")
     layers, bs = sy.resnet_layers(widths=(8, 16), blocks=1, in_c=3, classes=10)
     res = sy.without_relu(sy.Net("resnet-mix", layers, [bs[0], bs[1]], 8, 8, 3, 10, 4, 3, 0.05, "fp32"))
-    return {"mlp": mlp, "resnet": res}
+    ragged = sy.Net("mlp-ragged-mix", sy.mlp_layers([22, 33, 17, 10]), [2], 1, 1, 22, 10, 4, 3, 0.1, "fp32")     # windows off 16-byte boundaries
+    return {"mlp": mlp, "resnet": res, "ragged": ragged}
 
 
 def run_pair(orc, net, P, steps, distinct, lr=None):
@@ -89,7 +90,7 @@ def run_pair(orc, net, P, steps, distinct, lr=None):
 
 
 @pytest.mark.parametrize("graph,alpha", [("ring", 0.3), ("line", 0.4)])
-@pytest.mark.parametrize("name", ["mlp", "resnet"])
+@pytest.mark.parametrize("name", ["mlp", "resnet", "ragged"])
 def test_general_mixing_matrix_matches_the_oracle_for_every_worker(orc, name, graph, alpha):
     net = nets()[name]
     P = weight_matrix(graphs(net.n_workers)[graph], net.n_workers, alpha)

@@ -26,6 +26,13 @@ def test_fp32_resnet_grouped_matches_oracle(orc):
     run_parity(orc, net, 3 * net.K, param_tol=1e-5, loss_tol=1e-5, grad_tol=0.2, grad_best_tol=1e-5, worker_groups=2)
 
 
+def test_fp32_ragged_mlp_grouped_windows_that_start_off_a_16_byte_boundary(orc):
+    """Hidden widths 33, 65, 17 and 3 samples per worker: a group's window of an activation starts 6 x 33 x 4 bytes into
+    the tensor, which is no multiple of 16, so the 128-bit elementwise kernels must take their element-wise path."""
+    net = sy.Net("mlp-ragged", sy.mlp_layers([70, 33, 65, 17, 5]), [4], 1, 1, 70, 5, 4, 3, 0.05, "fp32")
+    run_parity(orc, net, 3 * net.K, param_tol=1e-5, loss_tol=1e-5, worker_groups=2)
+
+
 def test_fp32_vgg_with_biases_grouped_matches_oracle(orc):
     layers, starts = sy.vgg_layers(widths=(6, 10, 12, 20), in_c=3, classes=10)
     net = sy.Net("vgg-small", layers, starts[1:], 16, 16, 3, 10, 4, 3, 0.05, "fp32")
