@@ -1246,41 +1246,33 @@ stem_fw_kernel(const __grid_constant__ CUtensorMap tmRaw, const __grid_constant_
     if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 128); }
 }
 
-// dW[co][tap][ci] = sum_z partial[z][(tap, cc)][ci % 64][co], z ascending.  32x32 transposing tiles; 256 threads (a CTA of
-// this size fits beside a resident tensor-core CTA of another stream), a thread owns four (row, column) pairs and keeps
-// 32 independent loads in flight (eight along z for each pair).
+// dW[co][tap][ci] = sum_z partial[z][(tap, cc)][ci % 64][co], z ascending.  A CTA of 256 threads (it fits beside a
+// resident tensor-core CTA of another stream) transposes a tile of 8 rows x 32 columns: many small CTAs, because a layer
+// has few output elements (36 864 for 64 -> 64) and many partial matrices (up to 147), so the kernel lives on the number of
+// loads in flight; a thread owns one element and keeps 16 independent loads in flight along z.
 __global__ void __launch_bounds__(256) wg_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dw, int splits, int row_blocks, int Co,
                                                         bool accum) {
-    __shared__ float t[32][33];
+    __shared__ float t[8][33];
     const int R = row_blocks * 64;                       // = taps * Cin
-    const int r0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+    const int r0 = blockIdx.x * 8, c0 = blockIdx.y * 32;
     const int tx = threadIdx.x, ty = threadIdx.y;        // 32 x 8
-    const unsigned zs = (unsigned)R * Co, rs = 8u * Co;                      // one partial matrix (< 2^32 elements); this thread's rows are 8 apart
+    const unsigned zs = (unsigned)R * Co;                // one partial matrix (< 2^32 elements)
     const float* p = partial + (size_t)(r0 + ty) * Co + c0 + tx;
-    float s[4] = {0.f, 0.f, 0.f, 0.f};
+    float s = 0.f;
     int z = 0;
-    for (; z + 8 <= splits; z += 8, p += (size_t)8 * zs) {
-        float v[4][8];
+    for (; z + 16 <= splits; z += 16, p += (size_t)16 * zs) {
+        float v[16];
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
+        for (int j = 0; j < 16; ++j) v[j] = __ldg(p + j * zs);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) v[i][j] = __ldg(p + j * zs + i * rs);
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int j = 0; j < 8; ++j) s[i] += v[i][j];
+        for (int j = 0; j < 16; ++j) s += v[j];
     }
-    for (; z < splits; ++z, p += zs)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) s[i] += __ldg(p + i * rs);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) t[ty + 8 * i][tx] = s[i];
+    for (; z < splits; ++z, p += zs) s += __ldg(p);
+    t[ty][tx] = s;
     __syncthreads();
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        float* d = dw + (size_t)(c0 + ty + 8 * i) * R + r0 + tx;
-        *d = accum ? *d + t[tx][ty + 8 * i] : t[tx][ty + 8 * i];
-    }
+    const int tid = ty * 32 + tx, c = tid >> 3, r = tid & 7;      // 8 consecutive threads write 8 consecutive elements of a row of dW
+    float* d = dw + (size_t)(c0 + c) * R + r0 + r;
+    *d = accum ? *d + t[r][c] : t[r][c];
 }
 
 // One launch per module and step: the update of Eq. dl_update for ALL of the module's parameters.
@@ -1531,7 +1523,7 @@ cudaError_t run_wg(const TensorMap& x, const TensorMap& dy, const WgParams& p, i
     else if (n_tile == 256) e = launch_wg<256, 4>(x, dy, p, grid, s);
     else return cudaErrorInvalidValue;
     if (e != cudaSuccess) return e;
-    dim3 rgrid(p.row_blocks * 2, p.Co / 32), rblk(32, 8);
+    dim3 rgrid(p.row_blocks * 8, p.Co / 32), rblk(32, 8);
     wg_reduce_kernel<<<rgrid, rblk, 0, s>>>(p.partial, dw, splits, p.row_blocks, p.Co, accum);
     return cudaGetLastError();
 }
@@ -1577,7 +1569,7 @@ cudaError_t run_wg_rows(const TensorMap& x_rows, const TensorMap& dy128, const W
     else if (variant == 2) e = launch_wg2<128, 2, 20, 3>(x_rows, dy128, p, dim3(3 * (q.C / 128), q.Co / 128, z), s);
     else return cudaErrorInvalidValue;
     if (e != cudaSuccess) return e;
-    dim3 rgrid(p.row_blocks * 2, p.Co / 32), rblk(32, 8);
+    dim3 rgrid(p.row_blocks * 8, p.Co / 32), rblk(32, 8);
     wg_reduce_kernel<<<rgrid, rblk, 0, s>>>(p.partial, dw, z, p.row_blocks, p.Co, accum);
     return cudaGetLastError();
 }

@@ -131,3 +131,37 @@ def test_config4_full_size_schedule_invariants_and_mode_equivalence():
     assert worst > 0
     params_serial, _, _ = _run(net, p0, steps, serial=True)
     assert np.array_equal(params, params_serial)
+
+
+def test_config5_full_size_schedule_and_invariants():
+    """ResNet-18-shaped, K = 8, 16 workers x 256 (M = 4096): the whole stash (about 127 GB, store-all) on one GPU.  Until
+    the first module has had its backward pass: the delay schedule on the device equals the closed forms with the maximum
+    delay 2(K-1) = 14, everything stays finite, the classifier's bias gradient sums to zero and the weight gradient of
+    every convolution in front of a batch-norm is orthogonal to its weights channel by channel."""
+    import torch
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    if free < 140 * 2**30:
+        pytest.skip("needs 140 GB of free device memory")
+    net = sy.config(4)
+    p0 = sy.init_params(net.layers, 0, bf16=True)
+    steps = 2 * net.K - 1
+    params, grads, traces = _run(net, p0, steps, serial=False)
+    for t, (f, b, v) in enumerate(traces):
+        fc, bc, vc = closed_form_trace(net.K, t)
+        assert (f == fc).all() and (b == bc).all() and (v == vc).all(), t
+    assert traces[-1][1][0] == 0 and traces[-1][2][0] == 0          # module 1 back-propagates batch 0 with weight version 0 at t = 2K-2
+    assert np.isfinite(params).all() and np.isfinite(grads).all()
+    fc_bias = grads[-net.classes:]
+    assert abs(fc_bias.sum()) <= 1e-3 * np.abs(fc_bias).sum()
+    off = 0
+    shapes = sy.param_shapes(net.layers)
+    for idx, (li, name, shape, _) in enumerate(shapes):
+        n = int(np.prod(shape))
+        if name in ("W", "Wp") and len(shape) == 4 and idx + 1 < len(shapes) and shapes[idx + 1][1].startswith("gamma"):
+            w = params[off:off + n].astype(np.float64).reshape(shape[0], -1)
+            g = grads[off:off + n].astype(np.float64).reshape(shape[0], -1)
+            per_channel = np.abs((w * g).sum(1)) / (np.linalg.norm(w, axis=1) * np.linalg.norm(g, axis=1) + 1e-300)
+            assert np.median(per_channel) <= 2e-2, (li, name, float(np.median(per_channel)))
+        off += n
+    torch.cuda.empty_cache()
