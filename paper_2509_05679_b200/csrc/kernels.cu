@@ -847,6 +847,9 @@ struct BnsArgs {
     bf16* y;                    // mode 2: output; mode 3: dx
     bf16* dres;                 // mode 3: gradient of the residual input, or nullptr
     long rpw; int C; int relu; int mask_from_x; int accum_dx; int accum_dres;
+    int reverse;                // walk the CTA's tiles from the last to the first: a kernel that re-reads what the kernel before it
+                                // has just streamed in ascending order (backward apply after backward sums) starts with the part
+                                // that is still in L2
     int* err;
 };
 
@@ -875,7 +878,7 @@ __global__ void __launch_bounds__(BNV_THREADS, BNS_CTAS) bns_kernel(const BnsArg
     const size_t wbase = (size_t)w * a.rpw * C;           // first element of this worker
     auto issue = [&](int i) {                             // thread 0: fill stage i % stages with tile i
         const int st = i % stages;
-        const long row = r0 + (long)i * tile_rows;
+        const long row = r0 + (long)(a.reverse ? ntiles - 1 - i : i) * tile_rows;
         const long rows = r1 - row < tile_rows ? r1 - row : tile_rows;
         const uint32_t bytes = (uint32_t)(rows * C * 2), bar = full0 + 8 * st;
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes * n_in) : "memory");
@@ -903,7 +906,7 @@ __global__ void __launch_bounds__(BNV_THREADS, BNS_CTAS) bns_kernel(const BnsArg
         const int st = i % stages;
         if (ok && !bns_wait(full0 + 8 * st, (uint32_t)(i / stages) & 1u, a.err)) ok = false;
         const uint8_t* sx = bns_sm + (size_t)(st * n_in) * BNS_TILE;
-        const long trow = r0 + (long)i * tile_rows;
+        const long trow = r0 + (long)(a.reverse ? ntiles - 1 - i : i) * tile_rows;
 #pragma unroll
         for (int k = 0; k < BNS_VPT; ++k) {
             const int lr = rl + k * rows_it;                 // row inside the tile
@@ -1093,6 +1096,7 @@ void bn_forward(int dt, const void* x, const float* gamma, const float* beta, co
         Scope sc(KC_BN_FWD_APPLY, 0.0, 2.0 * total * (res ? 3 : 2), s);
         a.y = (bf16*)y; a.res = (const bf16*)res;
         if (res) { a.in[1] = (const bf16*)res; a.n_in = 2; }
+        a.reverse = conv_part ? 0 : 1;       // after a statistics pass of its own: x was just read front to back
         bns_launch<2>(a, chunks, nw, s);
         return;
     }
@@ -1131,6 +1135,7 @@ void bn_backward(int dt, const void* x, const void* out, const void* dout, const
           else bn_bwd_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C, accum_params); }
         Scope sc(KC_BN_BWD_APPLY, 0.0, 2.0 * total * (reads + 1 + (accum_dx ? 1 : 0) + (dres ? (accum_dres ? 2 : 1) : 0)), s);
         a.y = (bf16*)dx; a.accum_dx = accum_dx; a.dres = (bf16*)dres; a.accum_dres = accum_dres;
+        a.reverse = 1;                       // the sums kernel above has just read the same tensors front to back
         bns_launch<3>(a, chunks, nw, s);
         return;
     }
