@@ -170,6 +170,7 @@ def main():
     ap.add_argument("--batch", type=int, default=None, help="per-worker batch override (testing only; changes the workload name)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-kernel-pass", action="store_true", help="skip the extra one-stream pass that times every kernel class (roofline becomes null)")
+    ap.add_argument("--grid-sms", type=int, default=0, help="SMs the persistent kernels size their grids for (0: the library's choice, half of the device with concurrent module streams)")
     ap.add_argument("--serial", action="store_true", help="diagnosis: all modules on one stream (uncontended per-kernel times)")
     args = ap.parse_args()
 
@@ -196,8 +197,9 @@ def main():
     timing_stream = torch.cuda.Stream()       # carries only the two timing events; the library runs on its own streams
     ctx = binding.Context(net.layers, net.splits, net.n_workers, net.batch, net.lr, dtype=net.dtype,
                           in_shape=(net.in_h, net.in_w, net.in_c), num_classes=net.classes, device=local,
-                          kernel_path=args.kernel_path, serial=args.serial, worker_groups=args.worker_groups)
+                          kernel_path=args.kernel_path, serial=args.serial, worker_groups=args.worker_groups, grid_sms=args.grid_sms)
     ctx.set_params(sy.init_params(net.layers, 0, bf16=net.dtype == "bf16"))
+    grid_sms = ctx.grid_sms
 
     # a pool of distinct batches, resident in HBM (device arm) and in pinned host memory (e2e arm)
     pool = 4
@@ -258,13 +260,16 @@ def main():
 
     # ---- kernel pass: the same workload with every module on ONE stream and CUDA events around every launch, so that
     # an event pair brackets one kernel running alone (with the module streams running side by side a pair would also
-    # contain whatever the other modules had on the GPU).  Not part of `value`.
-    kstats, kshapes, kernel_steps = None, None, 3
+    # contain whatever the other modules had on the GPU).  With one stream the library sizes every grid for the whole
+    # device (nothing runs beside a kernel), so these are the kernels' own times; the timed steps above launch the same
+    # kernels on `grid_sms` SMs, two of them side by side.  Not part of `value`.
+    kstats, kshapes, kernel_steps, kernel_grid_sms = None, None, 3, None
     if not args.no_kernel_pass:
         ctx.close()
         ctx = binding.Context(net.layers, net.splits, net.n_workers, net.batch, net.lr, dtype=net.dtype,
                               in_shape=(net.in_h, net.in_w, net.in_c), num_classes=net.classes, device=local,
                               kernel_path=args.kernel_path, serial=True, worker_groups=args.worker_groups)
+        kernel_grid_sms = ctx.grid_sms
         ctx.set_params(sy.init_params(net.layers, 0, bf16=net.dtype == "bf16"))
         for i in range(fill + 3):
             ctx.step(dev_x[i % pool], dev_y[i % pool])
@@ -328,7 +333,8 @@ def main():
             "config": {"workload": net.name + ("" if args.batch is None else f"-B{args.batch}"), "K": net.K, "n_workers": net.n_workers,
                        "per_worker_batch": net.batch, "M": net.M, "lr": net.lr, "pipeline_fill_steps": fill,
                        "l2": "inputs rotate over 4 batches; each step streams the multi-GB activation stash, far larger than L2",
-                       "multi_gpu": "independent replicas (no exchange between GPUs)", "kernel_path": args.kernel_path, "serial": bool(args.serial), "worker_groups": args.worker_groups},
+                       "multi_gpu": "independent replicas (no exchange between GPUs)", "kernel_path": args.kernel_path, "serial": bool(args.serial), "worker_groups": args.worker_groups,
+                       "grid_sms": grid_sms, "kernel_pass_grid_sms": kernel_grid_sms},
             "clocks": clocks,
             "roofline": roof,
             "kernels": {k: {"launches_per_step": v["launches"] / kernel_steps, "ms_per_step": round(v["ms"] / kernel_steps, 4),

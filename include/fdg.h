@@ -114,6 +114,13 @@ typedef struct {
                                   worker's own gradient with scale 1/per_worker_batch, and updates
                                   u_{s,k} = w^_{s,k} - lr g_{s,k},  w^_{s,k}(t+1) = sum_r P_sr u_{r,k}  (Eq. "dl_update").
                                   At most 32 workers.  The matrix is copied.                                     */
+    int32_t grid_sms;          /* SMs the persistent kernels (tensor-core convolutions / GEMMs, streamed batch-norm) size
+                                  their grids for.  0: half of the device's SMs when the modules run on streams of their
+                                  own (the concurrency of Sec. 3.2: a tensor-core kernel of one module then runs beside a
+                                  memory-bound kernel of another instead of after it), all of them with serial = 1.
+                                  n > 0: n SMs (clamped to the device).  Results depend on it only through fp32 summation
+                                  order (contraction splits, batch-norm row chunks): two contexts with the same value are
+                                  bit-identical whatever their streams                                              */
 } fdg_options;
 
 /* Stash policy.  Every activation a module's backward pass needs is kept from the module's forward pass of
@@ -134,6 +141,9 @@ FDG_API fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers,
                       const int32_t* split_points, int32_t K,
                       int32_t n_workers, int32_t per_worker_batch, float lr,
                       const fdg_options* opt, const fdg_allocator* alloc, fdg_ctx** out);
+
+/* The SM count the context's persistent kernels are sized for (fdg_options.grid_sms after the automatic choice). */
+FDG_API fdg_status fdg_grid_sms(const fdg_ctx* ctx, int32_t* sms);
 
 /* Number of parameters (length of the canonical parameter vector). */
 FDG_API fdg_status fdg_param_count(const fdg_ctx* ctx, size_t* count);

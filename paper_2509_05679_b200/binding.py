@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libfdg.so")
 STATUS = {0: "FDG_OK", 1: "FDG_ERR_INVALID_ARG", 2: "FDG_ERR_BAD_SPLIT", 3: "FDG_ERR_UNSUPPORTED",
           4: "FDG_ERR_ARCH", 5: "FDG_ERR_OOM", 6: "FDG_ERR_CUDA", 7: "FDG_ERR_TIMEOUT", 8: "FDG_ERR_STATE"}
 
-EXPORTS = ["fdg_create", "fdg_param_count", "fdg_param_layout", "fdg_set_params", "fdg_set_params_worker", "fdg_params_worker",
+EXPORTS = ["fdg_create", "fdg_grid_sms", "fdg_param_count", "fdg_param_layout", "fdg_set_params", "fdg_set_params_worker", "fdg_params_worker",
            "fdg_grads_worker", "fdg_consensus_error", "fdg_step", "fdg_step_host", "fdg_wait_ingest", "fdg_join", "fdg_params",
            "fdg_grads", "fdg_trace", "fdg_set_lr", "fdg_stats", "fdg_module_times", "fdg_profile", "fdg_profile_read",
            "fdg_bias_grad_static", "fdg_static_last_error",
@@ -59,7 +59,8 @@ PARAM_ROLES = ["W", "b", "gamma", "beta", "Wp", "gamma_p", "beta_p"]     # fdg_p
 class fdg_options(C.Structure):
     _fields_ = [("dtype", C.c_int32), ("in_h", C.c_int32), ("in_w", C.c_int32), ("in_c", C.c_int32),
                 ("num_classes", C.c_int32), ("serial", C.c_int32), ("kernel_path", C.c_int32),
-                ("worker_groups", C.c_int32), ("streams", C.POINTER(C.c_void_p)), ("mixing", C.POINTER(C.c_double))]
+                ("worker_groups", C.c_int32), ("streams", C.POINTER(C.c_void_p)), ("mixing", C.POINTER(C.c_double)),
+                ("grid_sms", C.c_int32)]
 
 
 _lib = None
@@ -76,6 +77,8 @@ def lib():
         L.fdg_create.restype = C.c_int
         L.fdg_create.argtypes = [C.POINTER(fdg_layer), C.c_int32, C.POINTER(C.c_int32), C.c_int32, C.c_int32, C.c_int32,
                                  C.c_float, C.POINTER(fdg_options), C.POINTER(fdg_allocator), C.POINTER(vp)]
+        L.fdg_grid_sms.restype = C.c_int
+        L.fdg_grid_sms.argtypes = [vp, C.POINTER(C.c_int32)]
         L.fdg_param_count.restype = C.c_int
         L.fdg_param_count.argtypes = [vp, C.POINTER(C.c_size_t)]
         L.fdg_param_layout.restype = C.c_int
@@ -163,7 +166,7 @@ class Context:
     def __init__(self, layers: Sequence[Sequence[int]], split_points: Sequence[int], n_workers: int,
                  per_worker_batch: int, lr: float, *, dtype: str = "bf16", in_shape=(32, 32, 3), num_classes: int = 10,
                  serial: bool = False, kernel_path: int = 0, device: int = 0, use_torch_allocator: bool = True,
-                 streams: Optional[Sequence[int]] = None, worker_groups: int = 0, mixing=None):
+                 streams: Optional[Sequence[int]] = None, worker_groups: int = 0, mixing=None, grid_sms: int = 0):
         import torch
         L = lib()
         if not torch.cuda.is_available():
@@ -186,7 +189,7 @@ class Context:
         opt = fdg_options({"fp32": 0, "bf16": 1}[dtype], int(in_shape[0]), int(in_shape[1]), int(in_shape[2]),
                           int(num_classes), int(serial), int(kernel_path), int(worker_groups),
                           C.cast(self._streams, C.POINTER(C.c_void_p)) if self._streams is not None else None,
-                          self._mixing.ctypes.data_as(C.POINTER(C.c_double)) if self._mixing is not None else None)
+                          self._mixing.ctypes.data_as(C.POINTER(C.c_double)) if self._mixing is not None else None, int(grid_sms))
         self._alloc = _TorchAllocator(torch.device("cuda", device)) if use_torch_allocator else None
         h = C.c_void_p()
         st = L.fdg_create(arr, len(layers), sp, self.K, n_workers, per_worker_batch, float(lr), C.byref(opt),
@@ -197,6 +200,9 @@ class Context:
         n = C.c_size_t()
         self._ck(L.fdg_param_count(self.h, C.byref(n)))
         self.n_params = n.value
+        g = C.c_int32()
+        self._ck(L.fdg_grid_sms(self.h, C.byref(g)))
+        self.grid_sms = g.value          # SMs the persistent kernels are sized for (fdg_options.grid_sms, resolved)
 
     def _ck(self, st):
         if st != 0:

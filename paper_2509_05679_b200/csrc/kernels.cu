@@ -809,21 +809,28 @@ constexpr int BNS_RING = 96 * 1024;                 // shared memory of the ring
 constexpr int BNS_VPT = BNS_TILE / 16 / 256;        // 16-byte vectors per thread and tile
 constexpr long long BNS_WAIT_CYCLES = 4000000000LL; // ~2 s
 
-__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[BV]) {
+constexpr int BP = BV / 2;                          // channel pairs per thread
+__device__ __forceinline__ void unpack8(const uint4& v, float2 (&f)[BP]) {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-    for (int j = 0; j < 4; ++j) { f[2 * j] = __uint_as_float(w[j] << 16); f[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u); }
+    for (int j = 0; j < BP; ++j) f[j] = make_float2(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xffff0000u));
 }
-__device__ __forceinline__ uint4 pack8(const float (&f)[BV]) {
-    uint32_t w[4];
+// round to nearest even; RELU: negative values become zero in the same conversion
+template <bool RELU>
+__device__ __forceinline__ uint4 pack8(const float2 (&f)[BP]) {
+    uint32_t w[BP];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) { const __nv_bfloat162 t = __floats2bfloat162_rn(f[2 * j], f[2 * j + 1]); w[j] = *(const uint32_t*)&t; }
+    for (int j = 0; j < BP; ++j) {
+        if (RELU) asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(w[j]) : "f"(f[j].y), "f"(f[j].x));
+        else asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[j]) : "f"(f[j].y), "f"(f[j].x));
+    }
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
-// the one expression both passes use for the normalised value, so that the backward pass can
-// recompute the sign of the forward output from x alone
-__device__ __forceinline__ float bn_value(float x, float mean, float istd, float g, float b) {
-    return __fmaf_rn(g, (x - mean) * istd, b);
+// the one expression both passes use for the normalised value, so that the backward pass can recompute the sign of
+// the forward output from x alone: gamma * ((x - mean) * invstd) + beta, the product rounded before the fused last
+// step, two channels per instruction
+__device__ __forceinline__ float2 bn_pair(float2 x, float2 neg_mean, float2 invstd, float2 gamma, float2 beta) {
+    return __ffma2_rn(gamma, __fmul2_rn(__fadd2_rn(x, neg_mean), invstd), beta);
 }
 
 __device__ __forceinline__ uint32_t bns_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -855,7 +862,7 @@ struct BnsArgs {
 
 // MODE 0: (sum x, sum x^2).  MODE 1: (sum dy, sum dy * xhat) with dy = dout * [forward output > 0] if relu.
 // MODE 2: y = bn(x) (+ res) (relu).  MODE 3: dx (+)= BN backward of dy, dres (+)= dy.
-// mask_from_x: the forward output had no residual, so its sign is the sign of bn_value(x).
+// mask_from_x: the forward output had no residual, so its sign is the sign of bn_pair(x).
 template <int MODE>
 __global__ void __launch_bounds__(BNV_THREADS, BNS_CTAS) bns_kernel(const BnsArgs a) {
     extern __shared__ __align__(128) uint8_t bns_sm[];
@@ -888,83 +895,94 @@ __global__ void __launch_bounds__(BNV_THREADS, BNS_CTAS) bns_kernel(const BnsArg
     };
     if (tid == 0) for (int i = 0; i < stages - 1 && i < ntiles; ++i) issue(i);
 
-    float s1[BV], s2[BV], mean[BV], istd[BV], g[BV], b[BV], c1[BV], c2[BV];
+    // Per-channel coefficients, two channels per register pair (the arithmetic below is packed fp32: one instruction per
+    // channel pair).  With d = x - mean and scale = gamma * invstd the input gradient gamma * invstd * (dy - c1 - xhat * c2)
+    // is scale * dy + (d * ka + kb), ka = -scale * invstd * c2, kb = -scale * c1; sum dy * xhat = invstd * sum dy * d.
+    float2 s1[BP], s2[BP], nmean[BP], is[BP], ga[BP], be[BP], sc[BP], ka[BP], kb[BP];
     const float inv_n = 1.f / (float)a.rpw;
 #pragma unroll
-    for (int j = 0; j < BV; ++j) {
-        const int c = cg * BV + j;
-        const size_t so = ((size_t)w * C + c) * 2;
-        s1[j] = 0.f; s2[j] = 0.f;
-        if (MODE != 0) { mean[j] = a.stats[so]; istd[j] = a.stats[so + 1]; g[j] = a.gamma[c]; b[j] = a.beta[c]; }
-        if (MODE == 3) { c1[j] = a.red[so] * inv_n; c2[j] = a.red[so + 1] * inv_n; }
+    for (int j = 0; j < BP; ++j) {
+        float* const f1 = &s1[j].x; float* const f2 = &s2[j].x; float* const fnm = &nmean[j].x; float* const fis = &is[j].x;
+        float* const fga = &ga[j].x; float* const fbe = &be[j].x; float* const fsc = &sc[j].x; float* const fka = &ka[j].x; float* const fkb = &kb[j].x;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int c = cg * BV + 2 * j + h;
+            const size_t so = ((size_t)w * C + c) * 2;
+            f1[h] = 0.f; f2[h] = 0.f;
+            if (MODE != 0) { fnm[h] = -a.stats[so]; fis[h] = a.stats[so + 1]; fga[h] = a.gamma[c]; fbe[h] = a.beta[c]; }
+            if (MODE == 3) {
+                const float c1 = a.red[so] * inv_n, c2 = a.red[so + 1] * inv_n;
+                fsc[h] = fga[h] * fis[h]; fka[h] = -fsc[h] * fis[h] * c2; fkb[h] = -fsc[h] * c1;
+            }
+        }
     }
     const bool need_out = (MODE == 1 || MODE == 3) && a.relu && !a.mask_from_x;
+    const bool res_in_ring = MODE == 2 && a.res && n_in > 1;
     bool ok = true;
     for (int i = 0; i < ntiles; ++i) {
         // every thread left tile i - 1 at the barrier below, so its stage can take tile i + stages - 1
         if (tid == 0 && i + stages - 1 < ntiles) issue(i + stages - 1);
         const int st = i % stages;
         if (ok && !bns_wait(full0 + 8 * st, (uint32_t)(i / stages) & 1u, a.err)) ok = false;
-        const uint8_t* sx = bns_sm + (size_t)(st * n_in) * BNS_TILE;
+        const uint8_t* sx = bns_sm + (size_t)(st * n_in) * BNS_TILE + tid * 16;      // row lr, channel group cg: vector lr * cgs + cg = tid + k * 256
         const long trow = r0 + (long)(a.reverse ? ntiles - 1 - i : i) * tile_rows;
+        const size_t o0 = wbase + (size_t)trow * C + (size_t)tid * BV;
+        const int vec_rows = ok ? (int)min((long)tile_rows, r1 - trow) : 0;            // rows of this tile that exist
 #pragma unroll
         for (int k = 0; k < BNS_VPT; ++k) {
-            const int lr = rl + k * rows_it;                 // row inside the tile
-            const long row = trow + lr;
-            if (row >= r1 || !ok) continue;
-            const int so = (lr * cgs + cg) * 16;
-            float xv[BV];
-            unpack8(*(const uint4*)(sx + so), xv);
+            if (rl + k * rows_it >= vec_rows) break;
+            const uint4 xw = *(const uint4*)(sx + k * (BNV_THREADS * 16));
+            const size_t o = o0 + (size_t)k * (BNV_THREADS * BV);
+            float2 xv[BP];
+            unpack8(xw, xv);
             if (MODE == 0) {
 #pragma unroll
-                for (int j = 0; j < BV; ++j) { s1[j] += xv[j]; s2[j] = fmaf(xv[j], xv[j], s2[j]); }
+                for (int j = 0; j < BP; ++j) { s1[j] = __fadd2_rn(s1[j], xv[j]); s2[j] = __ffma2_rn(xv[j], xv[j], s2[j]); }
             } else if (MODE == 2) {
-                float rv[BV];
-                const size_t o = wbase + (size_t)row * C + (size_t)cg * BV;
-                if (a.res) { if (n_in > 1) unpack8(*(const uint4*)(sx + BNS_TILE + so), rv); else unpack8(__ldg((const uint4*)(a.res + o)), rv); }
 #pragma unroll
-                for (int j = 0; j < BV; ++j) {
-                    float v = bn_value(xv[j], mean[j], istd[j], g[j], b[j]);
-                    if (a.res) v += rv[j];
-                    if (a.relu) v = fmaxf(v, 0.f);
-                    xv[j] = v;
+                for (int j = 0; j < BP; ++j) xv[j] = bn_pair(xv[j], nmean[j], is[j], ga[j], be[j]);
+                if (a.res) {
+                    float2 rv[BP];
+                    unpack8(res_in_ring ? *(const uint4*)(sx + BNS_TILE + k * (BNV_THREADS * 16)) : __ldg((const uint4*)(a.res + o)), rv);
+#pragma unroll
+                    for (int j = 0; j < BP; ++j) xv[j] = __fadd2_rn(xv[j], rv[j]);
                 }
-                *(uint4*)(a.y + o) = pack8(xv);
+                *(uint4*)(a.y + o) = a.relu ? pack8<true>(xv) : pack8<false>(xv);
             } else {
-                float dv[BV], ov[BV];
-                unpack8(*(const uint4*)(sx + BNS_TILE + so), dv);
-                if (need_out) unpack8(*(const uint4*)(sx + 2 * BNS_TILE + so), ov);
-                if (a.relu) {
+                float2 dv[BP];
+                unpack8(*(const uint4*)(sx + BNS_TILE + k * (BNV_THREADS * 16)), dv);
 #pragma unroll
-                    for (int j = 0; j < BV; ++j) {
-                        const float f = a.mask_from_x ? bn_value(xv[j], mean[j], istd[j], g[j], b[j]) : ov[j];
-                        if (!(f > 0.f)) dv[j] = 0.f;
+                for (int j = 0; j < BP; ++j) xv[j] = __fadd2_rn(xv[j], nmean[j]);          // d = x - mean from here on
+                if (a.relu) {
+                    float2 f[BP];
+                    if (need_out) unpack8(*(const uint4*)(sx + 2 * BNS_TILE + k * (BNV_THREADS * 16)), f);
+                    else {
+#pragma unroll
+                        for (int j = 0; j < BP; ++j) f[j] = __ffma2_rn(ga[j], __fmul2_rn(xv[j], is[j]), be[j]);   // bn_pair after its first step
                     }
+#pragma unroll
+                    for (int j = 0; j < BP; ++j) { if (!(f[j].x > 0.f)) dv[j].x = 0.f; if (!(f[j].y > 0.f)) dv[j].y = 0.f; }
                 }
                 if (MODE == 1) {
 #pragma unroll
-                    for (int j = 0; j < BV; ++j) { s1[j] += dv[j]; s2[j] = fmaf(dv[j], (xv[j] - mean[j]) * istd[j], s2[j]); }
+                    for (int j = 0; j < BP; ++j) { s1[j] = __fadd2_rn(s1[j], dv[j]); s2[j] = __ffma2_rn(dv[j], xv[j], s2[j]); }
                 } else {
-                    const size_t o = wbase + (size_t)row * C + (size_t)cg * BV;
-                    float t[BV];
+                    float2 t[BP];
 #pragma unroll
-                    for (int j = 0; j < BV; ++j) {
-                        const float xh = (xv[j] - mean[j]) * istd[j];
-                        t[j] = g[j] * istd[j] * (dv[j] - c1[j] - xh * c2[j]);
-                    }
+                    for (int j = 0; j < BP; ++j) t[j] = __ffma2_rn(sc[j], dv[j], __ffma2_rn(xv[j], ka[j], kb[j]));
                     if (a.accum_dx) {
-                        float old[BV]; unpack8(*(const uint4*)(a.y + o), old);
+                        float2 old[BP]; unpack8(*(const uint4*)(a.y + o), old);
 #pragma unroll
-                        for (int j = 0; j < BV; ++j) t[j] += old[j];
+                        for (int j = 0; j < BP; ++j) t[j] = __fadd2_rn(t[j], old[j]);
                     }
-                    *(uint4*)(a.y + o) = pack8(t);
+                    *(uint4*)(a.y + o) = pack8<false>(t);
                     if (a.dres) {
                         if (a.accum_dres) {
-                            float old[BV]; unpack8(*(const uint4*)(a.dres + o), old);
+                            float2 old[BP]; unpack8(*(const uint4*)(a.dres + o), old);
 #pragma unroll
-                            for (int j = 0; j < BV; ++j) dv[j] += old[j];
+                            for (int j = 0; j < BP; ++j) dv[j] = __fadd2_rn(dv[j], old[j]);
                         }
-                        *(uint4*)(a.dres + o) = pack8(dv);
+                        *(uint4*)(a.dres + o) = pack8<false>(dv);
                     }
                 }
             }
@@ -973,15 +991,18 @@ __global__ void __launch_bounds__(BNV_THREADS, BNS_CTAS) bns_kernel(const BnsArg
     }
     if (MODE == 0 || MODE == 1) {
         // the ring is idle now (every issued tile was waited for): reuse it for the reduction over the row lanes
-        float (*sh)[2 * BV + 1] = (float (*)[2 * BV + 1])bns_sm;
+        float (*red_sh)[2 * BV + 1] = (float (*)[2 * BV + 1])bns_sm;
 #pragma unroll
-        for (int j = 0; j < BV; ++j) { sh[tid][j] = s1[j]; sh[tid][BV + j] = s2[j]; }
+        for (int j = 0; j < BP; ++j) {
+            if (MODE == 1) s2[j] = __fmul2_rn(s2[j], is[j]);            // sum dy * d -> sum dy * xhat
+            red_sh[tid][2 * j] = s1[j].x; red_sh[tid][2 * j + 1] = s1[j].y; red_sh[tid][BV + 2 * j] = s2[j].x; red_sh[tid][BV + 2 * j + 1] = s2[j].y;
+        }
         __syncthreads();
         // thread t < 2*BV*cgs sums one (channel group, value) column over the rows_it row lanes, in a fixed order
         for (int t = tid; t < cgs * 2 * BV; t += BNV_THREADS) {
             const int q = t / (2 * BV), k = t % (2 * BV);
             float acc = 0.f;
-            for (int rr = 0; rr < rows_it; ++rr) acc += sh[rr * cgs + q][k];
+            for (int rr = 0; rr < rows_it; ++rr) acc += red_sh[rr * cgs + q][k];
             const int c = q * BV + (k % BV);
             a.part[(((size_t)blockIdx.x * nw + w) * C + c) * 2 + (k / BV)] = acc;
         }
@@ -1057,10 +1078,16 @@ __global__ void bnv_bwd_final(const float* __restrict__ part, float* __restrict_
 
 static bool bnv_ok(int dt, int C) { int cgs = C / BV; return dt == 1 && C % BV == 0 && cgs <= BNV_THREADS && (cgs & (cgs - 1)) == 0; }
 constexpr int BNS_SMEM = BNS_RING + 8 * 8;
-// Row chunks per worker such that chunks * nw CTAs fill the GPU once (two CTAs per SM), each with at least four tiles.
-static int bns_chunks(int nw, long rpw, int C) {
+// Row chunks per worker such that chunks * nw CTAs fill the SM budget once (two CTAs per SM), each with at least four tiles.
+static int g_bn_sm_budget = 0;
+static int bn_device_sms() {
     static int sms = 0;
     if (!sms) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); if (sms <= 0) sms = 148; }
+    return sms;
+}
+void bn_set_sm_budget(int sms) { g_bn_sm_budget = sms > 0 && sms < bn_device_sms() ? sms : 0; }
+static int bns_chunks(int nw, long rpw, int C) {
+    const int sms = g_bn_sm_budget ? g_bn_sm_budget : bn_device_sms();
     const long tile_rows = BNS_TILE / (C * 2);
     long want = ((long)sms * BNS_CTAS) / nw, maxc = (rpw + tile_rows * 4 - 1) / (tile_rows * 4);
     long c = want < maxc ? want : maxc;

@@ -56,6 +56,9 @@ void maxpool_backward(int dt, const void* x, const void* dy, void* dx, int N, in
 void gap_forward(int dt, const void* x, void* y, int N, int HW, int C, cudaStream_t st);
 void gap_backward(int dt, const void* dy, void* dx, int N, int HW, int C, bool accum, cudaStream_t st);
 
+// SMs the streamed batch-norm kernels size their grids for (0 or >= the device's count: all).  Process-wide, set by the
+// context like tc::set_sm_budget; the partial sums depend on it through the number of row chunks (fp32 summation order).
+void bn_set_sm_budget(int sms);
 // Batch-norm with per-worker statistics.  x: [n_workers * rows_per_worker, C].
 // err: device word that a kernel sets non-zero if a bounded wait on an asynchronous copy gave up (nullptr: the
 // kernels that stream through shared memory are not used).

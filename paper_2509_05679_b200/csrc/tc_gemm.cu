@@ -1417,11 +1417,16 @@ bool pixel_tile(int H, int W, int pixels, int* Wt, int* Ht, int* Nt) {
     return true;
 }
 
-static int sm_count() {
+static int device_sms() {
     static int n = 0;
     if (!n) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev); if (n <= 0) n = 148; }
     return n;
 }
+// SMs the persistent kernels size their grids (and contraction splits) for.  Fewer than the device has: kernels of
+// different module streams then run side by side, a tensor-core kernel next to a memory-bound one.
+static int g_sm_budget = 0;
+void set_sm_budget(int sms) { g_sm_budget = sms > 0 && sms < device_sms() ? sms : 0; }
+static int sm_count() { return g_sm_budget ? g_sm_budget : device_sms(); }
 
 template <int N_TILE, int STAGES, int EPI_WARPS, int KSUB, bool ROWS, int RES_KB>
 static cudaError_t launch_km(const TensorMap& a, const TensorMap& b, const TensorMap& o, const KmParams& p, cudaStream_t s) {
@@ -1458,15 +1463,16 @@ static cudaError_t launch_km_pair(const TensorMap& a, const TensorMap& b, const 
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.blockDim = dim3(64 + 32 * EPI_WARPS); cfg.dynamicSmemBytes = smem; cfg.stream = s; cfg.attrs = at; cfg.numAttrs = 1;
-    static int max_pairs = 0;                   // pairs that can be resident at once
-    if (!max_pairs) {
+    static int resident_pairs = 0;              // pairs that can be resident at once on the whole device
+    if (!resident_pairs) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
-        cfg.gridDim = dim3(sm_count());
+        cfg.gridDim = dim3(device_sms());
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n <= 0) { cudaGetLastError(); n = sm_count() / 2; }
-        max_pairs = n < sm_count() / 2 ? n : sm_count() / 2;
+        if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n <= 0) { cudaGetLastError(); n = device_sms() / 2; }
+        resident_pairs = n;
     }
+    const int max_pairs = resident_pairs < sm_count() / 2 ? resident_pairs : sm_count() / 2;
     const int total = (p.tiles_w * p.tiles_h * p.tiles_n / 2) * (p.Cn / N_TILE) * p.ncls;
     cfg.gridDim = dim3(2 * (total < max_pairs ? total : max_pairs));
     return cudaLaunchKernelEx(&cfg, kernel, *(const CUtensorMap*)&a, *(const CUtensorMap*)&b, *(const CUtensorMap*)&o, p);

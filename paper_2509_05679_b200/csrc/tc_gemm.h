@@ -47,6 +47,10 @@ struct WgParams {
 };
 
 bool init();     // resolves the driver's tensor-map encoder; false if unavailable
+// SMs the persistent kernels below size their grids for, and the contraction splits of the weight gradients their CTA
+// counts (0 or >= the device's count: all of them).  Process-wide; the context sets it before it sizes workspaces and
+// before every step it enqueues.  The results depend on it only through fp32 summation order (split counts).
+void set_sm_budget(int sms);
 // NHWC bf16 tensor [N,H,W,C]; box = boxC channels x (boxW x boxH x boxN) pixels; stride 2 samples every other pixel
 bool make_map_4d(TensorMap* out, const void* base, int C, int W, int H, int N, int boxC, int boxW, int boxH, int boxN, int stride);
 bool make_map_2d(TensorMap* out, const void* base, long inner, long outer, int box_inner, int box_outer);

@@ -53,9 +53,10 @@ def test_serial_and_concurrent_modes_are_bit_identical():
     from paper_2509_05679_b200 import binding
     net = as_fp32(sy.config(3, n_workers=2, batch=4, width_div=8))
     p0 = sy.perturb_params(sy.init_params(net.layers, 0), net.layers, 7, 0.1)
-    outs = []
+    outs, sms = [], 0
     for serial in (False, True):
-        ctx = make_ctx(net, p0, serial=serial)
+        ctx = make_ctx(net, p0, serial=serial, grid_sms=sms)
+        sms = ctx.grid_sms                 # the one-stream run sizes its grids like the concurrent one: same summation order
         for t in range(3 * net.K):
             x, y = binding.to_device("fp32", sy.batch_inputs(net, t)), torch.from_numpy(sy.batch_labels(net, t)).cuda()
             ctx.step(x, y)                 # asynchronous: steps of different modules overlap
