@@ -170,7 +170,8 @@ def main():
     ap.add_argument("--batch", type=int, default=None, help="per-worker batch override (testing only; changes the workload name)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-kernel-pass", action="store_true", help="skip the extra one-stream pass that times every kernel class (roofline becomes null)")
-    ap.add_argument("--grid-sms", type=int, default=0, help="SMs the persistent kernels size their grids for (0: the library's choice, half of the device with concurrent module streams)")
+    ap.add_argument("--grid-sms", type=int, default=0, help="SMs the persistent kernels size their grids for (0: the library's choice, a third of the device with concurrent module streams)")
+    ap.add_argument("--kernel-pass-grid-sms", type=int, default=0, help="grid size of the one-stream kernel pass (0: all SMs, a kernel alone; diagnosis: the timed steps' grid_sms shows what each kernel does on its share)")
     ap.add_argument("--serial", action="store_true", help="diagnosis: all modules on one stream (uncontended per-kernel times)")
     args = ap.parse_args()
 
@@ -268,7 +269,7 @@ def main():
         ctx.close()
         ctx = binding.Context(net.layers, net.splits, net.n_workers, net.batch, net.lr, dtype=net.dtype,
                               in_shape=(net.in_h, net.in_w, net.in_c), num_classes=net.classes, device=local,
-                              kernel_path=args.kernel_path, serial=True, worker_groups=args.worker_groups)
+                              kernel_path=args.kernel_path, serial=True, worker_groups=args.worker_groups, grid_sms=args.kernel_pass_grid_sms)
         kernel_grid_sms = ctx.grid_sms
         ctx.set_params(sy.init_params(net.layers, 0, bf16=net.dtype == "bf16"))
         for i in range(fill + 3):

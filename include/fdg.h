@@ -115,7 +115,7 @@ typedef struct {
                                   u_{s,k} = w^_{s,k} - lr g_{s,k},  w^_{s,k}(t+1) = sum_r P_sr u_{r,k}  (Eq. "dl_update").
                                   At most 32 workers.  The matrix is copied.                                     */
     int32_t grid_sms;          /* SMs the persistent kernels (tensor-core convolutions / GEMMs, streamed batch-norm) size
-                                  their grids for.  0: half of the device's SMs when the modules run on streams of their
+                                  their grids for.  0: a third of the device's SMs when the modules run on streams of their
                                   own (the concurrency of Sec. 3.2: a tensor-core kernel of one module then runs beside a
                                   memory-bound kernel of another instead of after it), all of them with serial = 1.
                                   n > 0: n SMs (clamped to the device).  Results depend on it only through fp32 summation

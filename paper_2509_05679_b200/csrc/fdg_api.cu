@@ -964,11 +964,13 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
     ctx->K = K; ctx->n_workers = n_workers; ctx->B = per_worker_batch; ctx->M = n_workers * per_worker_batch;
     ctx->dt = opt->dtype; ctx->esz = opt->dtype ? 2 : 4; ctx->classes = opt->num_classes; ctx->serial = opt->serial;
     ctx->kernel_path = opt->kernel_path;
-    // modules on streams of their own: grids for half of the SMs, so that a tensor-core kernel of one module and a
-    // memory-bound kernel of another run side by side (measured on a B200, ResNet-18-shaped, 4 modules: 5.0 against 5.3 ms
-    // per step; 60..88 SMs are within 1 % of each other).  One stream: nothing runs beside a kernel, all SMs.
+    // modules on streams of their own: grids for a third of the SMs, so that tensor-core kernels and memory-bound kernels
+    // of different modules run side by side instead of one after the other (a streamed batch-norm kernel keeps 92 % of
+    // its bandwidth on half of the SMs, a tensor-core kernel takes 1.6 times as long there, not twice).  Measured on a
+    // B200, ResNet-18-shaped, 4 modules, 30 steps under the power cap: 5.05-5.12 ms per step for 37..74 SMs against
+    // 5.3-5.5 for all 148; VGG-shaped 0.77 against 0.90.  One stream: nothing runs beside a kernel, all SMs.
     ctx->grid_sms = opt->grid_sms > 0 ? (opt->grid_sms < prop.multiProcessorCount ? opt->grid_sms : prop.multiProcessorCount)
-                                      : (opt->serial ? prop.multiProcessorCount : prop.multiProcessorCount / 2);
+                                      : (opt->serial ? prop.multiProcessorCount : (prop.multiProcessorCount + 2) / 3);
     apply_sm_budget(ctx);
     ctx->R = 1; ctx->P_dev = nullptr;
     if (opt->mixing) {

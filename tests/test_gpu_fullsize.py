@@ -90,9 +90,9 @@ def test_config3_full_width_50_step_loss_trajectory(orc):
 def _run(net, p0, steps, serial):
     import torch
     from paper_2509_05679_b200 import binding
-    # the one-stream run sizes its grids like the concurrent one (half of the SMs): same contraction splits and batch-norm
-    # row chunks, hence the same fp32 summation order
-    ctx = make_ctx(net, p0, serial=serial, grid_sms=torch.cuda.get_device_properties(0).multi_processor_count // 2 if serial else 0)
+    # the one-stream run sizes its grids like the concurrent one (a third of the SMs): same contraction splits and
+    # batch-norm row chunks, hence the same fp32 summation order
+    ctx = make_ctx(net, p0, serial=serial, grid_sms=(torch.cuda.get_device_properties(0).multi_processor_count + 2) // 3 if serial else 0)
     xs = [binding.to_device(net.dtype, sy.batch_inputs(net, t)) for t in range(2)]
     ys = [torch.from_numpy(sy.batch_labels(net, t)).cuda() for t in range(2)]
     traces = []
