@@ -849,8 +849,9 @@ __device__ __forceinline__ bool bns_wait(uint32_t bar, uint32_t parity, int* err
 struct BnsArgs {
     const bf16* in[3];          // input tensors streamed through the ring: x, then dout, then the forward output (as the mode needs)
     int n_in;
-    const float* gamma; const float* beta; const float* stats; const float* red; const bf16* res;
-    float* part;                // modes 0, 1: partial sums [chunk][worker][C][2]
+    const float* gamma; const float* beta; const float* stats; const bf16* res;
+    float* part;                // modes 0, 1: partial sums [chunk][worker][C][2], written; mode 3: the same, read (gridDim.x chunks)
+    float* dgamma; float* dbeta; int accum_params;   // mode 3: parameter gradients, written by one CTA
     bf16* y;                    // mode 2: output; mode 3: dx
     bf16* dres;                 // mode 3: gradient of the residual input, or nullptr
     long rpw; int C; int relu; int mask_from_x; int accum_dx; int accum_dres;
@@ -895,6 +896,31 @@ __global__ void __launch_bounds__(BNV_THREADS, BNS_CTAS) bns_kernel(const BnsArg
     };
     if (tid == 0) for (int i = 0; i < stages - 1 && i < ntiles; ++i) issue(i);
 
+    // MODE 3: (sum dy, sum dy xhat) of this worker from the chunk partials of the sums kernel (same grid), chunks in
+    // ascending order, while the first tiles are on their way; CTA (0, 0) also adds the workers in ascending order
+    // into dgamma / dbeta.  Every CTA of a worker computes the same sums in the same order.
+    float2* const red_s = (float2*)(bns_sm + BNS_RING + 64);
+    if (MODE == 3) {
+        const int chunks = gridDim.x;
+        const float2* const part = (const float2*)a.part;
+        for (int c = tid; c < C; c += BNV_THREADS) {
+            float2 acc = make_float2(0.f, 0.f);
+            for (int k = 0; k < chunks; ++k) { const float2 v = part[((size_t)k * nw + w) * C + c]; acc.x += v.x; acc.y += v.y; }
+            red_s[c] = acc;
+        }
+        if (blockIdx.x == 0 && w == 0) {
+            for (int c = tid; c < C; c += BNV_THREADS) {
+                float g = 0.f, b = 0.f;
+                for (int ww = 0; ww < nw; ++ww) {
+                    float2 acc = make_float2(0.f, 0.f);
+                    for (int k = 0; k < chunks; ++k) { const float2 v = part[((size_t)k * nw + ww) * C + c]; acc.x += v.x; acc.y += v.y; }
+                    b += acc.x; g += acc.y;
+                }
+                a.dgamma[c] = a.accum_params ? a.dgamma[c] + g : g; a.dbeta[c] = a.accum_params ? a.dbeta[c] + b : b;
+            }
+        }
+        __syncthreads();
+    }
     // Per-channel coefficients, two channels per register pair (the arithmetic below is packed fp32: one instruction per
     // channel pair).  With d = x - mean and scale = gamma * invstd the input gradient gamma * invstd * (dy - c1 - xhat * c2)
     // is scale * dy + (d * ka + kb), ka = -scale * invstd * c2, kb = -scale * c1; sum dy * xhat = invstd * sum dy * d.
@@ -911,7 +937,7 @@ __global__ void __launch_bounds__(BNV_THREADS, BNS_CTAS) bns_kernel(const BnsArg
             f1[h] = 0.f; f2[h] = 0.f;
             if (MODE != 0) { fnm[h] = -a.stats[so]; fis[h] = a.stats[so + 1]; fga[h] = a.gamma[c]; fbe[h] = a.beta[c]; }
             if (MODE == 3) {
-                const float c1 = a.red[so] * inv_n, c2 = a.red[so + 1] * inv_n;
+                const float c1 = red_s[c].x * inv_n, c2 = red_s[c].y * inv_n;
                 fsc[h] = fga[h] * fis[h]; fka[h] = -fsc[h] * fis[h] * c2; fkb[h] = -fsc[h] * c1;
             }
         }
@@ -1058,26 +1084,9 @@ __global__ void __launch_bounds__(256) bnv_stats_final_tiles(const float* __rest
         *(float2*)(stats + ((size_t)w * C + c) * 2) = make_float2((float)mean, (float)(1.0 / sqrt(var + 1e-5)));
     }
 }
-// block = one channel, one warp per worker (nw <= 32): red[w][c] = (sum dy, sum dy xhat); warp 0 then adds the
-// workers in ascending order into dgamma / dbeta
-__global__ void bnv_bwd_final(const float* __restrict__ part, float* __restrict__ red, float* __restrict__ dgamma,
-                              float* __restrict__ dbeta, int chunks, int nw, int C, bool accum) {
-    __shared__ float2 sh[32];
-    const int c = blockIdx.x, w = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    float2 a = make_float2(0.f, 0.f);
-    for (int k = lane; k < chunks; k += 32) { const float2 v = *(const float2*)(part + (((size_t)k * nw + w) * C + c) * 2); a.x += v.x; a.y += v.y; }
-    a = warp_sum2(a);
-    if (lane == 0) { *(float2*)(red + ((size_t)w * C + c) * 2) = a; sh[w] = a; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        float g = 0.f, b = 0.f;
-        for (int i = 0; i < nw; ++i) { b += sh[i].x; g += sh[i].y; }
-        dgamma[c] = accum ? dgamma[c] + g : g; dbeta[c] = accum ? dbeta[c] + b : b;
-    }
-}
-
 static bool bnv_ok(int dt, int C) { int cgs = C / BV; return dt == 1 && C % BV == 0 && cgs <= BNV_THREADS && (cgs & (cgs - 1)) == 0; }
 constexpr int BNS_SMEM = BNS_RING + 8 * 8;
+constexpr int BNS_RED_BYTES = BNV_THREADS * BV * 8;   // backward apply: (sum dy, sum dy xhat) per channel, up to 256 * 8 channels
 // Row chunks per worker such that chunks * nw CTAs fill the SM budget once (two CTAs per SM), each with at least four tiles.
 static int g_bn_sm_budget = 0;
 static int bn_device_sms() {
@@ -1097,8 +1106,9 @@ static int bns_chunks(int nw, long rpw, int C) {
 template <int MODE>
 static void bns_launch(const BnsArgs& a, int chunks, int nw, cudaStream_t s) {
     static bool attr = false;
-    if (!attr) { cudaFuncSetAttribute(bns_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, BNS_SMEM); attr = true; }
-    bns_kernel<MODE><<<dim3(chunks, nw), BNV_THREADS, BNS_SMEM, s>>>(a);
+    constexpr int smem = BNS_SMEM + (MODE == 3 ? BNS_RED_BYTES : 0);
+    if (!attr) { cudaFuncSetAttribute(bns_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem); attr = true; }
+    bns_kernel<MODE><<<dim3(chunks, nw), BNV_THREADS, smem, s>>>(a);
 }
 
 bool bn_accepts_conv_partials(int dt, int C) { return bnv_ok(dt, C); }
@@ -1153,15 +1163,13 @@ void bn_backward(int dt, const void* x, const void* out, const void* dout, const
         const int reads = 2 + (need_out ? 1 : 0);
         BnsArgs a{};
         a.in[0] = (const bf16*)x; a.in[1] = (const bf16*)dout; a.in[2] = (const bf16*)out; a.n_in = reads;
-        a.gamma = gamma; a.beta = beta; a.stats = stats; a.red = red; a.rpw = rpw; a.C = C; a.relu = relu; a.mask_from_x = mask_from_x; a.err = err;
+        a.gamma = gamma; a.beta = beta; a.stats = stats; a.rpw = rpw; a.C = C; a.relu = relu; a.mask_from_x = mask_from_x; a.err = err;
         { Scope sc(KC_BN_BWD_REDUCE, 0.0, 2.0 * total * reads, s);
           BnsArgs r = a; r.part = scratch;
           bns_launch<1>(r, chunks, nw, s); }
-        { Scope sc(KC_BN_BWD_REDUCE, 0.0, 8.0 * chunks * nw * C, s);
-          if (nw <= 32) bnv_bwd_final<<<C, 32 * nw, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C, accum_params);
-          else bn_bwd_final<<<cdiv(C, 128), 128, 0, s>>>(scratch, red, dgamma, dbeta, chunks, nw, C, accum_params); }
         Scope sc(KC_BN_BWD_APPLY, 0.0, 2.0 * total * (reads + 1 + (accum_dx ? 1 : 0) + (dres ? (accum_dres ? 2 : 1) : 0)), s);
         a.y = (bf16*)dx; a.accum_dx = accum_dx; a.dres = (bf16*)dres; a.accum_dres = accum_dres;
+        a.part = scratch; a.dgamma = dgamma; a.dbeta = dbeta; a.accum_params = accum_params;   // the apply kernel finishes the sums itself
         a.reverse = 1;                       // the sums kernel above has just read the same tensors front to back
         bns_launch<3>(a, chunks, nw, s);
         return;
