@@ -259,29 +259,39 @@ def main():
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
-    # ---- kernel pass: the same workload with every module on ONE stream and CUDA events around every launch, so that
+    # ---- kernel passes: the same workload with every module on ONE stream and CUDA events around every launch, so that
     # an event pair brackets one kernel running alone (with the module streams running side by side a pair would also
-    # contain whatever the other modules had on the GPU).  With one stream the library sizes every grid for the whole
-    # device (nothing runs beside a kernel), so these are the kernels' own times; the timed steps above launch the same
-    # kernels on `grid_sms` SMs, two of them side by side.  Not part of `value`.
-    kstats, kshapes, kernel_steps, kernel_grid_sms = None, None, 3, None
+    # contain whatever the other modules had on the GPU).  First with the grids of the timed steps (`grid_sms` SMs per
+    # persistent kernel: the launch configuration that was timed, and the one an ncu launch list of this command shows),
+    # then with grids for the whole device (what the same kernels do when nothing is meant to run beside them).
+    # Not part of `value`.
+    kernel_steps = 3
+    device_sms = torch.cuda.get_device_properties(local).multi_processor_count
+
+    def kernel_pass(sms):
+        c = binding.Context(net.layers, net.splits, net.n_workers, net.batch, net.lr, dtype=net.dtype,
+                            in_shape=(net.in_h, net.in_w, net.in_c), num_classes=net.classes, device=local,
+                            kernel_path=args.kernel_path, serial=True, worker_groups=args.worker_groups, grid_sms=sms)
+        c.set_params(sy.init_params(net.layers, 0, bf16=net.dtype == "bf16"))
+        for i in range(fill + 3):
+            c.step(dev_x[i % pool], dev_y[i % pool])
+        torch.cuda.synchronize()
+        c.profile(True)
+        for i in range(kernel_steps):
+            c.step(dev_x[i % pool], dev_y[i % pool])
+        c.profile(False)
+        kall = c.profile_read()
+        sms = c.grid_sms
+        c.close()
+        return {k: v for k, v in kall.items() if "[" not in k}, {k: v for k, v in kall.items() if "[" in k}, sms
+
+    kstats, kshapes, kernel_grid_sms, kstats_all = None, None, None, None
     if not args.no_kernel_pass:
         ctx.close()
-        ctx = binding.Context(net.layers, net.splits, net.n_workers, net.batch, net.lr, dtype=net.dtype,
-                              in_shape=(net.in_h, net.in_w, net.in_c), num_classes=net.classes, device=local,
-                              kernel_path=args.kernel_path, serial=True, worker_groups=args.worker_groups, grid_sms=args.kernel_pass_grid_sms)
-        kernel_grid_sms = ctx.grid_sms
-        ctx.set_params(sy.init_params(net.layers, 0, bf16=net.dtype == "bf16"))
-        for i in range(fill + 3):
-            ctx.step(dev_x[i % pool], dev_y[i % pool])
-        torch.cuda.synchronize()
-        ctx.profile(True)
-        for i in range(kernel_steps):
-            ctx.step(dev_x[i % pool], dev_y[i % pool])
-        ctx.profile(False)
-        kall = ctx.profile_read()
-        kstats = {k: v for k, v in kall.items() if "[" not in k}
-        kshapes = {k: v for k, v in kall.items() if "[" in k}
+        ctx = None
+        kstats, kshapes, kernel_grid_sms = kernel_pass(args.kernel_pass_grid_sms or grid_sms)
+        if kernel_grid_sms != device_sms:
+            kstats_all, _, _ = kernel_pass(device_sms)
 
     ms, e2e_s = max_over_ranks([ms, e2e_s], dist, "cuda")
 
@@ -305,7 +315,8 @@ def main():
             name, st = max(stats.items(), key=lambda kv: kv[1]["ms"])
             total_ms = sum(v["ms"] for v in stats.values())
             per_step = st["launches"] / kernel_steps
-            base = {"kernel": name, "launches_per_step": per_step, "avg_launch_ms": st["ms"] / st["launches"],
+            base = {"kernel": name, "grid_sms": kernel_grid_sms, "device_sms": device_sms,
+                    "launches_per_step": per_step, "avg_launch_ms": st["ms"] / st["launches"],
                     "class_ms_per_step": st["ms"] / kernel_steps, "share_of_kernel_time": st["ms"] / total_ms,
                     "kernel_ms_per_step_all_classes": total_ms / kernel_steps, "traffic": traffic_per_launch(name),
                     "timing": f"CUDA events around every launch, separate pass of {kernel_steps} steps with all modules on one stream "
@@ -315,6 +326,9 @@ def main():
                 ach = st["flops"] / (st["ms"] * 1e-3) / 1e12
                 peak = pk["tensor_burst"] if tensor else FMA_PEAK_TFLOPS
                 base.update({"bound": "tensor" if tensor else "alu", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
+                             # the launch is sized for grid_sms of the device's SMs (others run kernels of other modules
+                             # meanwhile): its fraction of what those SMs can do
+                             "frac_of_sm_share": ach / (peak * kernel_grid_sms / device_sms),
                              "peak_source": (pk["source"] + ", burst bf16 GEMM (a kernel timed alone)") if tensor
                              else "derived: 148 SMs x 128 FMA x 2 x 1.965 GHz"})
             else:
@@ -324,6 +338,14 @@ def main():
 
         roof = roofline_of(kstats)
         if roof:
+            if kstats_all and roof["kernel"] in kstats_all:
+                # the same kernel class with every grid sized for the whole device, each launch alone
+                sa = kstats_all[roof["kernel"]]
+                work, peak = (sa["bytes"] / 1e9, roof["peak"]) if roof["bound"] == "hbm" else (sa["flops"] / 1e12, roof["peak"])
+                ach = work / (sa["ms"] * 1e-3)
+                roof["all_sms"] = {"grid_sms": device_sms, "avg_launch_ms": sa["ms"] / sa["launches"], "class_ms_per_step": sa["ms"] / kernel_steps,
+                                   "achieved": ach, "frac": ach / peak,
+                                   "kernel_ms_per_step_all_classes": sum(v["ms"] for v in kstats_all.values()) / kernel_steps}
             roof["step"] = step_entry
         else:
             roof = {"kernel": None, "step": step_entry}
@@ -342,6 +364,10 @@ def main():
                             "tflops": round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 2) if v["ms"] > 0 else None,
                             "gbs": round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1) if v["ms"] > 0 else None}
                         for k, v in sorted((kstats or {}).items(), key=lambda kv: -kv[1]["ms"])},
+            "kernels_all_sms": {k: {"ms_per_step": round(v["ms"] / kernel_steps, 4),
+                                    "tflops": round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 2) if v["ms"] > 0 else None,
+                                    "gbs": round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1) if v["ms"] > 0 else None}
+                                for k, v in sorted((kstats_all or {}).items(), key=lambda kv: -kv[1]["ms"])},
             "kernel_shapes": {k: {"launches_per_step": v["launches"] / kernel_steps, "ms_per_step": round(v["ms"] / kernel_steps, 4),
                                   "tflops": round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 1) if v["ms"] > 0 else None,
                                   "gbs": round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1) if v["ms"] > 0 else None}
@@ -356,7 +382,8 @@ def main():
             v, cores, desc, _ = oracle_sample(net, 3, 0)
             out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
         print(json.dumps(out))
-    ctx.close()
+    if ctx is not None:
+        ctx.close()
     if dist:
         dist.destroy_process_group()
 

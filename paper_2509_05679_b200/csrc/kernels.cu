@@ -846,6 +846,13 @@ __device__ __forceinline__ bool bns_wait(uint32_t bar, uint32_t parity, int* err
     }
 }
 
+// a fixed shuffle tree: the summation order never changes
+__device__ __forceinline__ float2 warp_sum2(float2 v) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) { v.x += __shfl_xor_sync(0xffffffffu, v.x, d); v.y += __shfl_xor_sync(0xffffffffu, v.y, d); }
+    return v;
+}
+
 struct BnsArgs {
     const bf16* in[3];          // input tensors streamed through the ring: x, then dout, then the forward output (as the mode needs)
     int n_in;
@@ -896,27 +903,44 @@ __global__ void __launch_bounds__(BNV_THREADS, BNS_CTAS) bns_kernel(const BnsArg
     };
     if (tid == 0) for (int i = 0; i < stages - 1 && i < ntiles; ++i) issue(i);
 
-    // MODE 3: (sum dy, sum dy xhat) of this worker from the chunk partials of the sums kernel (same grid), chunks in
-    // ascending order, while the first tiles are on their way; CTA (0, 0) also adds the workers in ascending order
-    // into dgamma / dbeta.  Every CTA of a worker computes the same sums in the same order.
+    // MODE 3: (sum dy, sum dy xhat) of this worker from the chunk partials of the sums kernel (same grid), while the first
+    // tiles are on their way: all threads take part (up to 256 / C interleaved chunk subsets per channel, then a
+    // fixed-order sum of the subsets), so every CTA of a worker gets the same sums in the same order.  The CTAs of
+    // worker 0 also write dgamma / dbeta: CTA x takes the channels c = x (mod chunks), one warp per channel, lanes over
+    // the (worker, chunk) partials and a fixed shuffle tree.
     float2* const red_s = (float2*)(bns_sm + BNS_RING + 64);
     if (MODE == 3) {
         const int chunks = gridDim.x;
         const float2* const part = (const float2*)a.part;
-        for (int c = tid; c < C; c += BNV_THREADS) {
+        if (C <= BNV_THREADS) {
+            float2* const tmp = red_s + C;                  // [256 / C][C]
+            const int nparts = BNV_THREADS / C, c = tid % C, pt = tid / C;
             float2 acc = make_float2(0.f, 0.f);
-            for (int k = 0; k < chunks; ++k) { const float2 v = part[((size_t)k * nw + w) * C + c]; acc.x += v.x; acc.y += v.y; }
-            red_s[c] = acc;
-        }
-        if (blockIdx.x == 0 && w == 0) {
+            for (int k = pt; k < chunks; k += nparts) { const float2 v = part[((size_t)k * nw + w) * C + c]; acc.x += v.x; acc.y += v.y; }
+            tmp[pt * C + c] = acc;
+            __syncthreads();
+            if (tid < C) {
+                float2 t = make_float2(0.f, 0.f);
+                for (int q = 0; q < nparts; ++q) { t.x += tmp[q * C + tid].x; t.y += tmp[q * C + tid].y; }
+                red_s[tid] = t;
+            }
+        } else {
             for (int c = tid; c < C; c += BNV_THREADS) {
-                float g = 0.f, b = 0.f;
-                for (int ww = 0; ww < nw; ++ww) {
-                    float2 acc = make_float2(0.f, 0.f);
-                    for (int k = 0; k < chunks; ++k) { const float2 v = part[((size_t)k * nw + ww) * C + c]; acc.x += v.x; acc.y += v.y; }
-                    b += acc.x; g += acc.y;
+                float2 acc = make_float2(0.f, 0.f);
+                for (int k = 0; k < chunks; ++k) { const float2 v = part[((size_t)k * nw + w) * C + c]; acc.x += v.x; acc.y += v.y; }
+                red_s[c] = acc;
+            }
+        }
+        if (w == 0) {
+            const int warp = tid >> 5, lane = tid & 31, rows = nw * chunks;
+            for (int c = blockIdx.x + warp * chunks; c < C; c += (BNV_THREADS / 32) * chunks) {
+                float2 acc = make_float2(0.f, 0.f);
+                for (int r = lane; r < rows; r += 32) {
+                    const float2 v = part[((size_t)(r % chunks) * nw + r / chunks) * C + c];
+                    acc.x += v.x; acc.y += v.y;
                 }
-                a.dgamma[c] = a.accum_params ? a.dgamma[c] + g : g; a.dbeta[c] = a.accum_params ? a.dbeta[c] + b : b;
+                acc = warp_sum2(acc);
+                if (lane == 0) { a.dbeta[c] = a.accum_params ? a.dbeta[c] + acc.x : acc.x; a.dgamma[c] = a.accum_params ? a.dgamma[c] + acc.y : acc.y; }
             }
         }
         __syncthreads();
@@ -1037,11 +1061,6 @@ __global__ void __launch_bounds__(BNV_THREADS, BNS_CTAS) bns_kernel(const BnsArg
 
 // One warp per (worker, channel): lanes take the chunk partials round-robin, then a fixed shuffle tree adds the
 // lanes, so the summation order never changes.  stats[w][c] = (mean, invstd).
-__device__ __forceinline__ float2 warp_sum2(float2 v) {
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) { v.x += __shfl_xor_sync(0xffffffffu, v.x, d); v.y += __shfl_xor_sync(0xffffffffu, v.y, d); }
-    return v;
-}
 __global__ void bnv_stats_final(const float* __restrict__ part, float* __restrict__ stats, int chunks, int nwC, long rpw) {
     const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (i >= nwC) return;
@@ -1086,7 +1105,7 @@ __global__ void __launch_bounds__(256) bnv_stats_final_tiles(const float* __rest
 }
 static bool bnv_ok(int dt, int C) { int cgs = C / BV; return dt == 1 && C % BV == 0 && cgs <= BNV_THREADS && (cgs & (cgs - 1)) == 0; }
 constexpr int BNS_SMEM = BNS_RING + 8 * 8;
-constexpr int BNS_RED_BYTES = BNV_THREADS * BV * 8;   // backward apply: (sum dy, sum dy xhat) per channel, up to 256 * 8 channels
+constexpr int BNS_RED_BYTES = BNV_THREADS * BV * 8;   // backward apply: (sum dy, sum dy xhat) per channel, up to 256 * 8 channels (C <= 256: + 256 subset sums)
 // Row chunks per worker such that chunks * nw CTAs fill the SM budget once (two CTAs per SM), each with at least four tiles.
 static int g_bn_sm_budget = 0;
 static int bn_device_sms() {
