@@ -846,6 +846,20 @@ __device__ __forceinline__ bool bns_wait(uint32_t bar, uint32_t parity, int* err
     }
 }
 
+// p[0] + p[stride] + ... (n terms, in that order), eight loads in flight
+__device__ __forceinline__ float2 sum_strided(const float2* p, size_t stride, int n) {
+    float2 acc = make_float2(0.f, 0.f);
+    int i = 0;
+    for (; i + 8 <= n; i += 8) {
+        float2 v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = p[(size_t)(i + j) * stride];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { acc.x += v[j].x; acc.y += v[j].y; }
+    }
+    for (; i < n; ++i) { const float2 v = p[(size_t)i * stride]; acc.x += v.x; acc.y += v.y; }
+    return acc;
+}
 // a fixed shuffle tree: the summation order never changes
 __device__ __forceinline__ float2 warp_sum2(float2 v) {
 #pragma unroll
@@ -915,9 +929,7 @@ __global__ void __launch_bounds__(BNV_THREADS, BNS_CTAS) bns_kernel(const BnsArg
         if (C <= BNV_THREADS) {
             float2* const tmp = red_s + C;                  // [256 / C][C]
             const int nparts = BNV_THREADS / C, c = tid % C, pt = tid / C;
-            float2 acc = make_float2(0.f, 0.f);
-            for (int k = pt; k < chunks; k += nparts) { const float2 v = part[((size_t)k * nw + w) * C + c]; acc.x += v.x; acc.y += v.y; }
-            tmp[pt * C + c] = acc;
+            tmp[pt * C + c] = sum_strided(part + ((size_t)pt * nw + w) * C + c, (size_t)nparts * nw * C, (chunks - pt + nparts - 1) / nparts);
             __syncthreads();
             if (tid < C) {
                 float2 t = make_float2(0.f, 0.f);
@@ -925,19 +937,21 @@ __global__ void __launch_bounds__(BNV_THREADS, BNS_CTAS) bns_kernel(const BnsArg
                 red_s[tid] = t;
             }
         } else {
-            for (int c = tid; c < C; c += BNV_THREADS) {
-                float2 acc = make_float2(0.f, 0.f);
-                for (int k = 0; k < chunks; ++k) { const float2 v = part[((size_t)k * nw + w) * C + c]; acc.x += v.x; acc.y += v.y; }
-                red_s[c] = acc;
-            }
+            for (int c = tid; c < C; c += BNV_THREADS) red_s[c] = sum_strided(part + (size_t)w * C + c, (size_t)nw * C, chunks);
         }
         if (w == 0) {
             const int warp = tid >> 5, lane = tid & 31, rows = nw * chunks;
             for (int c = blockIdx.x + warp * chunks; c < C; c += (BNV_THREADS / 32) * chunks) {
                 float2 acc = make_float2(0.f, 0.f);
-                for (int r = lane; r < rows; r += 32) {
-                    const float2 v = part[((size_t)(r % chunks) * nw + r / chunks) * C + c];
-                    acc.x += v.x; acc.y += v.y;
+                for (int r0w = lane; r0w < rows; r0w += 32 * 4) {              // four loads in flight
+                    float2 v[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int r = r0w + 32 * j;
+                        v[j] = r < rows ? part[((size_t)(r % chunks) * nw + r / chunks) * C + c] : make_float2(0.f, 0.f);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) { acc.x += v[j].x; acc.y += v[j].y; }
                 }
                 acc = warp_sum2(acc);
                 if (lane == 0) { a.dbeta[c] = a.accum_params ? a.dbeta[c] + acc.x : acc.x; a.dgamma[c] = a.accum_params ? a.dgamma[c] + acc.y : acc.y; }
