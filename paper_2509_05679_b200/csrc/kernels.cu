@@ -919,9 +919,9 @@ __global__ void __launch_bounds__(BNV_THREADS, BNS_CTAS) bns_kernel(const BnsArg
 
     // MODE 3: (sum dy, sum dy xhat) of this worker from the chunk partials of the sums kernel (same grid), while the first
     // tiles are on their way: all threads take part (up to 256 / C interleaved chunk subsets per channel, then a
-    // fixed-order sum of the subsets), so every CTA of a worker gets the same sums in the same order.  The CTAs of
-    // worker 0 also write dgamma / dbeta: CTA x takes the channels c = x (mod chunks), one warp per channel, lanes over
-    // the (worker, chunk) partials and a fixed shuffle tree.
+    // fixed-order sum of the subsets), so every CTA of a worker gets the same sums in the same order.  dgamma / dbeta:
+    // CTA i of the launch takes the channels c = i (mod number of CTAs), one warp per channel, lanes over the
+    // (worker, chunk) partials and a fixed shuffle tree.
     float2* const red_s = (float2*)(bns_sm + BNS_RING + 64);
     if (MODE == 3) {
         const int chunks = gridDim.x;
@@ -939,9 +939,9 @@ __global__ void __launch_bounds__(BNV_THREADS, BNS_CTAS) bns_kernel(const BnsArg
         } else {
             for (int c = tid; c < C; c += BNV_THREADS) red_s[c] = sum_strided(part + (size_t)w * C + c, (size_t)nw * C, chunks);
         }
-        if (w == 0) {
-            const int warp = tid >> 5, lane = tid & 31, rows = nw * chunks;
-            for (int c = blockIdx.x + warp * chunks; c < C; c += (BNV_THREADS / 32) * chunks) {
+        {
+            const int warp = tid >> 5, lane = tid & 31, rows = nw * chunks, me = w * chunks + blockIdx.x;      // rows = CTAs of the launch
+            for (int c = me + warp * rows; c < C; c += (BNV_THREADS / 32) * rows) {
                 float2 acc = make_float2(0.f, 0.f);
                 for (int r0w = lane; r0w < rows; r0w += 32 * 4) {              // four loads in flight
                     float2 v[4];
