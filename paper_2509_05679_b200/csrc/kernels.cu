@@ -992,9 +992,8 @@ __global__ void __launch_bounds__(BNV_THREADS, BNS_CTAS) bns_kernel(const BnsArg
         const long trow = r0 + (long)(a.reverse ? ntiles - 1 - i : i) * tile_rows;
         const size_t o0 = wbase + (size_t)trow * C + (size_t)tid * BV;
         const int vec_rows = ok ? (int)min((long)tile_rows, r1 - trow) : 0;            // rows of this tile that exist
-#pragma unroll
-        for (int k = 0; k < BNS_VPT; ++k) {
-            if (rl + k * rows_it >= vec_rows) break;
+        // one 16-byte vector (row rl + k * rows_it of the tile, channel group cg) per call
+        auto vec = [&](const int k) {
             const uint4 xw = *(const uint4*)(sx + k * (BNV_THREADS * 16));
             const size_t o = o0 + (size_t)k * (BNV_THREADS * BV);
             float2 xv[BP];
@@ -1050,6 +1049,14 @@ __global__ void __launch_bounds__(BNV_THREADS, BNS_CTAS) bns_kernel(const BnsArg
                     }
                 }
             }
+        };
+        if (vec_rows == tile_rows) {
+            // a whole tile: no per-vector test, so that the four vectors of a thread are independent instruction streams
+#pragma unroll
+            for (int k = 0; k < BNS_VPT; ++k) vec(k);
+        } else {
+#pragma unroll
+            for (int k = 0; k < BNS_VPT; ++k) if (rl + k * rows_it < vec_rows) vec(k);
         }
         __syncthreads();
     }
