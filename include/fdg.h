@@ -28,9 +28,8 @@
  *     conv W[c_out][kh][kw][c_in]); batch-norm gamma then beta; a projecting FDG_RES_ADD
  *     carries Wp[c_out][c_in], gamma_p, beta_p.
  *   - The library needs an sm_100 device; there is no CPU path.
- *   - Threads: calls on one context must not overlap in time, and neither must fdg_create / fdg_step / fdg_step_host
- *     calls on different contexts (they set the process-wide grid sizing from the context's grid_sms before
- *     they enqueue).  Everything a call enqueues runs asynchronously on the context's streams.
+ *   - Threads: calls on one context must not overlap in time; different contexts are independent.  Everything a
+ *     call enqueues runs asynchronously on the context's streams.
  */
 #ifndef FDG_H
 #define FDG_H

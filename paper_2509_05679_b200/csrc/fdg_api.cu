@@ -218,7 +218,7 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
             o.wgr_variant = (g.R == 3 && g.stride == 1) ? tc::wg_rows_variant(g.H, g.W, g.C, g.Co) : 0;
             if (o.wgr_variant) {
                 tc::pixel_tile(g.Ho, g.Wo, 128, &wt, &ht, &nt);
-                o.wgr_splits = tc::wg_rows_splits(o.wgr_variant, g.C, g.Co, (long)(g.Ho / ht) * ((g.N + nt - 1) / nt));
+                o.wgr_splits = tc::wg_rows_splits(o.wgr_variant, g.C, g.Co, (long)(g.Ho / ht) * ((g.N + nt - 1) / nt), ctx->grid_sms);
             }
         }
         m.ops.push_back(o);
@@ -332,7 +332,7 @@ std::string compile_module(fdg_ctx* ctx, Module& m, int& h, int& w, int& c, bool
         if (o.type == OP_CONV) {
             if (o.tc) m.ws_elems = std::max(m.ws_elems, (size_t)std::max(o.wg_splits, o.wgr_variant ? o.wgr_splits : 0) * o.g.R * o.g.R * o.g.C * o.g.Co);
             if (o.stem) m.ws_elems = std::max(m.ws_elems, stem_wgrad_workspace_elems(o.g));
-            if (o.stem_tc) m.ws_elems = std::max(m.ws_elems, tc::stem_wg_workspace_elems(o.g.Co, (long)o.g.N * o.g.H));
+            if (o.stem_tc) m.ws_elems = std::max(m.ws_elems, tc::stem_wg_workspace_elems(o.g.Co, (long)o.g.N * o.g.H, ctx->grid_sms));
             m.ws_elems = std::max(m.ws_elems, wgrad_workspace_elems(o.g));
             m.fwd_ws_elems = std::max(m.fwd_ws_elems, forward_workspace_elems(o.g));
             m.scratch_elems = std::max(m.scratch_elems, (size_t)64 * o.g.Co);
@@ -412,7 +412,7 @@ bool tc_forward(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* y_base, 
     if (ia < 0) return false;
     tc::KmParams p = o.kf;
     p.bias = o.bias ? wsmall(c, m, version, o.b_off) : nullptr;
-    p.out = y_base; p.epi = o.relu ? EPI_RELU : 0; p.err = c->tc_err;
+    p.out = y_base; p.epi = o.relu ? EPI_RELU : 0; p.err = c->tc_err; p.sms = c->grid_sms;
     p.stat_part = o.stat_chunks ? m.cstat : nullptr;
     p.n_base = wn.n0; p.N = wn.n0 + wn.n; p.tiles_n = (wn.n + p.Nt - 1) / p.Nt;
     const ConvGeom& g = o.g;
@@ -435,7 +435,7 @@ bool tc_dgrad(fdg_ctx* c, Module& m, const Op& o, char* dy_base, char* dx_base, 
         cudaMemsetAsync(dx_base + (size_t)wn.n0 * g.H * g.W * g.C * 2, 0, (size_t)rows * g.C * 2, s);
     }
     tc::KmParams p = o.kd;
-    p.bias = nullptr; p.out = dx_base; p.epi = accum ? EPI_ACCUM : 0; p.err = c->tc_err; p.stat_part = nullptr;
+    p.bias = nullptr; p.out = dx_base; p.epi = accum ? EPI_ACCUM : 0; p.err = c->tc_err; p.stat_part = nullptr; p.sms = c->grid_sms;
     p.n_base = wn.n0; p.N = wn.n0 + wn.n; p.tiles_n = (wn.n + p.Nt - 1) / p.Nt;
     const double crows = (double)wn.n * p.Hd * p.Wd;         // pixels of one class; every tap belongs to exactly one class
     Scope sc(KC_TC_DGRAD, 2.0 * crows * g.C * p.ntaps * g.Co,
@@ -479,7 +479,7 @@ bool tc_stem_forward(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* y_b
     const double pix = (double)g.N * g.H * g.W;
     Scope sc(KC_FMA_FWD, 2.0 * pix * g.Co * 9 * g.C, 2.0 * pix * (g.C + g.Co), s);
     const bool ok = tc::run_stem_fw(o.sxr[ix], o.fo[io], g.H, g.W, g.N, g.Co, wbig(c, m, version, o.w_off), o.bias ? wsmall(c, m, version, o.b_off) : nullptr,
-                                    o.relu, o.stat_chunks ? m.cstat : nullptr, c->tc_err, s) == cudaSuccess;
+                                    o.relu, o.stat_chunks ? m.cstat : nullptr, c->tc_err, c->grid_sms, s) == cudaSuccess;
     if (ok && o.stat_chunks) { m.fused_stats_tensor = o.out; m.fused_stats_chunks = o.stat_chunks; }
     return ok;
 }
@@ -492,7 +492,7 @@ bool tc_stem_wgrad(fdg_ctx* c, Module& m, const Op& o, char* x_base, char* dy_ba
     const ConvGeom& g = o.g;
     const double pix = (double)g.N * g.H * g.W;
     Scope sc(KC_FMA_WGRAD, 2.0 * pix * g.Co * 9 * g.C, 2.0 * pix * (g.C + g.Co), s);
-    return tc::run_stem_wg(o.sxr[ix], o.sdy[id], g.H, g.W, g.N, g.Co, m.ws, dw, false, c->tc_err, s) == cudaSuccess;
+    return tc::run_stem_wg(o.sxr[ix], o.sdy[id], g.H, g.W, g.N, g.Co, m.ws, dw, false, c->tc_err, c->grid_sms, s) == cudaSuccess;
 }
 
 // byte offset of the group's first sample inside a tensor of the module
@@ -545,7 +545,7 @@ void forward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int grou
                 const float* part = fused ? m.cstat + (size_t)wn.w0 * m.fused_stats_chunks * ti.c * 2 : nullptr;
                 bn_forward(dt, T(o.in), wsmall(c, m, version, o.gamma_off, rep), wsmall(c, m, version, o.beta_off, rep),
                            o.has_res ? T(o.in2) : nullptr, T(o.out), P.stats(o) + (size_t)wn.w0 * ti.c * 2, m.scratch_f, wn.nw,
-                           (long)c->B * ti.h * ti.w, ti.c, o.relu, part, fused ? m.fused_stats_chunks : 0, c->tc_err, s);
+                           (long)c->B * ti.h * ti.w, ti.c, o.relu, part, fused ? m.fused_stats_chunks : 0, c->grid_sms, c->tc_err, s);
                 profile_detail(nullptr);
                 m.fused_stats_tensor = -1;
                 break; }
@@ -622,7 +622,7 @@ void backward_module(fdg_ctx* c, int kk, int64_t batch, int64_t version, int64_t
                 char* gres = o.has_res ? G(o.in2) : nullptr;
                 bn_backward(dt, T(o.in), T(o.out), gout, wsmall(c, m, version, o.gamma_off, rep), wsmall(c, m, version, o.beta_off, rep),
                             P.stats(o) + (size_t)wn.w0 * ti.c * 2, gin, o.acc_in, gres, o.acc_in2, mgrad + m.n_big + o.gamma_off,
-                            mgrad + m.n_big + o.beta_off, m.red, m.scratch, wn.nw, (long)c->B * ti.h * ti.w, ti.c, o.relu, o.has_res, acc_p, c->tc_err, s);
+                            mgrad + m.n_big + o.beta_off, m.red, m.scratch, wn.nw, (long)c->B * ti.h * ti.w, ti.c, o.relu, o.has_res, acc_p, c->grid_sms, c->tc_err, s);
                 profile_detail(nullptr);
                 break; }
             case OP_RELU: if (gin) relu_backward(dt, T(o.out), gout, gin, n_out, o.acc_in, s); break;
@@ -937,10 +937,6 @@ void fdg_destroy(fdg_ctx* ctx) {
     delete ctx;
 }
 
-// The launchers' grid sizing is process-wide state: every entry point that sizes workspaces or enqueues kernels sets it
-// from its own context first.
-static void apply_sm_budget(const fdg_ctx* ctx) { tc::set_sm_budget(ctx->grid_sms); bn_set_sm_budget(ctx->grid_sms); }
-
 fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* split_points, int32_t K,
                       int32_t n_workers, int32_t per_worker_batch, float lr, const fdg_options* opt,
                       const fdg_allocator* alloc, fdg_ctx** out) {
@@ -971,7 +967,6 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
     // 5.3-5.5 for all 148; VGG-shaped 0.77 against 0.90.  One stream: nothing runs beside a kernel, all SMs.
     ctx->grid_sms = opt->grid_sms > 0 ? (opt->grid_sms < prop.multiProcessorCount ? opt->grid_sms : prop.multiProcessorCount)
                                       : (opt->serial ? prop.multiProcessorCount : (prop.multiProcessorCount + 2) / 3);
-    apply_sm_budget(ctx);
     ctx->R = 1; ctx->P_dev = nullptr;
     if (opt->mixing) {
         // general mixing matrix: one weight replica per worker, every layer runs once per worker on the plain FMA kernels
@@ -1250,7 +1245,6 @@ fdg_status fdg_set_params_worker(fdg_ctx* ctx, int32_t worker, const float* host
 // A CUDA error in the middle of a step leaves some of its kernels enqueued and the iteration counter where it was:
 // the context then refuses further steps until fdg_set_params resets the FIFOs.
 static fdg_status guarded_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, bool host_src, float* host_loss) {
-    if (ctx) apply_sm_budget(ctx);
     const fdg_status s = run_step(ctx, inputs, labels, host_src, host_loss);
     if (ctx && (s == FDG_ERR_CUDA || s == FDG_ERR_TIMEOUT)) ctx->broken = true;
     return s;

@@ -1127,16 +1127,15 @@ __global__ void __launch_bounds__(256) bnv_stats_final_tiles(const float* __rest
 static bool bnv_ok(int dt, int C) { int cgs = C / BV; return dt == 1 && C % BV == 0 && cgs <= BNV_THREADS && (cgs & (cgs - 1)) == 0; }
 constexpr int BNS_SMEM = BNS_RING + 8 * 8;
 constexpr int BNS_RED_BYTES = BNV_THREADS * BV * 8;   // backward apply: (sum dy, sum dy xhat) per channel, up to 256 * 8 channels (C <= 256: + 256 subset sums)
-// Row chunks per worker such that chunks * nw CTAs fill the SM budget once (two CTAs per SM), each with at least four tiles.
-static int g_bn_sm_budget = 0;
+// Row chunks per worker such that chunks * nw CTAs fill the SMs the caller sizes for once (two CTAs per SM; 0: all SMs),
+// each with at least four tiles.
 static int bn_device_sms() {
     static int sms = 0;
     if (!sms) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); if (sms <= 0) sms = 148; }
     return sms;
 }
-void bn_set_sm_budget(int sms) { g_bn_sm_budget = sms > 0 && sms < bn_device_sms() ? sms : 0; }
-static int bns_chunks(int nw, long rpw, int C) {
-    const int sms = g_bn_sm_budget ? g_bn_sm_budget : bn_device_sms();
+static int bns_chunks(int nw, long rpw, int C, int sms_wanted) {
+    const int sms = sms_wanted > 0 && sms_wanted < bn_device_sms() ? sms_wanted : bn_device_sms();
     const long tile_rows = BNS_TILE / (C * 2);
     long want = ((long)sms * BNS_CTAS) / nw, maxc = (rpw + tile_rows * 4 - 1) / (tile_rows * 4);
     long c = want < maxc ? want : maxc;
@@ -1154,9 +1153,9 @@ static void bns_launch(const BnsArgs& a, int chunks, int nw, cudaStream_t s) {
 bool bn_accepts_conv_partials(int dt, int C) { return bnv_ok(dt, C); }
 
 void bn_forward(int dt, const void* x, const float* gamma, const float* beta, const void* res, void* y, float* stats,
-                float* scratch, int nw, long rpw, int C, bool relu, const float* conv_part, int conv_chunks, int* err, cudaStream_t s) {
+                float* scratch, int nw, long rpw, int C, bool relu, const float* conv_part, int conv_chunks, int sms, int* err, cudaStream_t s) {
     if (bnv_ok(dt, C) && err) {
-        const int chunks = bns_chunks(nw, rpw, C);
+        const int chunks = bns_chunks(nw, rpw, C, sms);
         const double total = (double)nw * rpw * C;
         BnsArgs a{};
         a.in[0] = (const bf16*)x; a.n_in = 1; a.gamma = gamma; a.beta = beta; a.stats = stats; a.rpw = rpw; a.C = C; a.relu = relu; a.err = err;
@@ -1194,9 +1193,9 @@ void bn_forward(int dt, const void* x, const float* gamma, const float* beta, co
 
 void bn_backward(int dt, const void* x, const void* out, const void* dout, const float* gamma, const float* beta,
                  const float* stats, void* dx, bool accum_dx, void* dres, bool accum_dres, float* dgamma, float* dbeta, float* red,
-                 float* scratch, int nw, long rpw, int C, bool relu, bool has_res, bool accum_params, int* err, cudaStream_t s) {
+                 float* scratch, int nw, long rpw, int C, bool relu, bool has_res, bool accum_params, int sms, int* err, cudaStream_t s) {
     if (bnv_ok(dt, C) && err) {
-        const int chunks = bns_chunks(nw, rpw, C);
+        const int chunks = bns_chunks(nw, rpw, C, sms);
         const double total = (double)nw * rpw * C;
         const int mask_from_x = relu && !has_res;
         const bool need_out = relu && !mask_from_x;

@@ -56,25 +56,24 @@ void maxpool_backward(int dt, const void* x, const void* dy, void* dx, int N, in
 void gap_forward(int dt, const void* x, void* y, int N, int HW, int C, cudaStream_t st);
 void gap_backward(int dt, const void* dy, void* dx, int N, int HW, int C, bool accum, cudaStream_t st);
 
-// SMs the streamed batch-norm kernels size their grids for (0 or >= the device's count: all).  Process-wide, set by the
-// context like tc::set_sm_budget; the partial sums depend on it through the number of row chunks (fp32 summation order).
-void bn_set_sm_budget(int sms);
 // Batch-norm with per-worker statistics.  x: [n_workers * rows_per_worker, C].
 // err: device word that a kernel sets non-zero if a bounded wait on an asynchronous copy gave up (nullptr: the
 // kernels that stream through shared memory are not used).
 // stats: fp32 [n_workers][C][2] = (mean, invstd).  scratch: fp32 [128 * n_workers * C * 2].
 // conv_part / conv_chunks: if non-null, the producing convolution already left per-tile (sum, sum of squares)
 // partials [n_workers * conv_chunks][C][2] (worker-major); the statistics pass over x is skipped.
+// sms: the SMs the streamed kernels size their grids for (0 or >= the device's count: all); the partial sums depend on it
+// through the number of row chunks (fp32 summation order).
 void bn_forward(int dt, const void* x, const float* gamma, const float* beta, const void* residual_or_null,
                 void* y, float* stats, float* scratch, int n_workers, long rows_per_worker, int C, bool relu,
-                const float* conv_part, int conv_chunks, int* err, cudaStream_t st);
+                const float* conv_part, int conv_chunks, int sms, int* err, cudaStream_t st);
 bool bn_accepts_conv_partials(int dt, int C);
 // dy_eff = dout * (out > 0 if relu).  dx (+)= BN backward of dy_eff; dres (+)= dy_eff;
 // dgamma, dbeta (fp32) = sums over all workers.  red: fp32 [n_workers][C][2] scratch for (sum dy, sum dy xhat).
 void bn_backward(int dt, const void* x, const void* out, const void* dout, const float* gamma, const float* beta,
                  const float* stats, void* dx, bool accum_dx, void* dres_or_null, bool accum_dres, float* dgamma, float* dbeta,
                  float* red, float* scratch, int n_workers, long rows_per_worker, int C, bool relu, bool has_res, bool accum_params,
-                 int* err, cudaStream_t st);
+                 int sms, int* err, cudaStream_t st);
 
 // Softmax cross-entropy over fp32 logits [M, classes]: dlogits (storage dtype) = (softmax - onehot) * scale,
 // *loss_out = mean loss.  Deterministic single-block reduction.

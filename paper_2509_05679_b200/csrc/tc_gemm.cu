@@ -1422,11 +1422,10 @@ static int device_sms() {
     if (!n) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev); if (n <= 0) n = 148; }
     return n;
 }
-// SMs the persistent kernels size their grids (and contraction splits) for.  Fewer than the device has: kernels of
-// different module streams then run side by side, a tensor-core kernel next to a memory-bound one.
-static int g_sm_budget = 0;
-void set_sm_budget(int sms) { g_sm_budget = sms > 0 && sms < device_sms() ? sms : 0; }
-static int sm_count() { return g_sm_budget ? g_sm_budget : device_sms(); }
+// SMs a launcher sizes its grid (or its contraction splits) for: `sms` of the caller, clamped to the device; 0 = all.
+// Fewer than the device has: kernels of different module streams then run side by side, a tensor-core kernel next to
+// a memory-bound one.
+static int sm_count(int sms) { return sms > 0 && sms < device_sms() ? sms : device_sms(); }
 
 template <int N_TILE, int STAGES, int EPI_WARPS, int KSUB, bool ROWS, int RES_KB>
 static cudaError_t launch_km(const TensorMap& a, const TensorMap& b, const TensorMap& o, const KmParams& p, cudaStream_t s) {
@@ -1445,7 +1444,7 @@ static cudaError_t launch_km(const TensorMap& a, const TensorMap& b, const Tenso
         attr = true;
     }
     const int total = p.tiles_w * p.tiles_h * p.tiles_n * (p.Cn / N_TILE) * p.ncls;
-    const int slots = sm_count() * per_sm;
+    const int slots = sm_count(p.sms) * per_sm;
     const int grid = total < slots ? total : slots;
     kernel<<<grid, 64 + 32 * EPI_WARPS, smem, s>>>(*(const CUtensorMap*)&a, *(const CUtensorMap*)&b, *(const CUtensorMap*)&o, p);
     return cudaGetLastError();
@@ -1472,7 +1471,7 @@ static cudaError_t launch_km_pair(const TensorMap& a, const TensorMap& b, const 
         if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n <= 0) { cudaGetLastError(); n = device_sms() / 2; }
         resident_pairs = n;
     }
-    const int max_pairs = resident_pairs < sm_count() / 2 ? resident_pairs : sm_count() / 2;
+    const int max_pairs = resident_pairs < sm_count(p.sms) / 2 ? resident_pairs : sm_count(p.sms) / 2;
     const int total = (p.tiles_w * p.tiles_h * p.tiles_n / 2) * (p.Cn / N_TILE) * p.ncls;
     cfg.gridDim = dim3(2 * (total < max_pairs ? total : max_pairs));
     return cudaLaunchKernelEx(&cfg, kernel, *(const CUtensorMap*)&a, *(const CUtensorMap*)&b, *(const CUtensorMap*)&o, p);
@@ -1554,9 +1553,9 @@ int wg_rows_variant(int H, int W, int C, int Co) {
     return 0;
 }
 
-int wg_rows_splits(int variant, int C, int Co, long steps) {
+int wg_rows_splits(int variant, int C, int Co, long steps, int sms) {
     const int tiles = variant == 1 ? Co / 64 : 3 * (C / 128) * (Co / 128);
-    long s = sm_count() / tiles;
+    long s = sm_count(sms) / tiles;
     if (s < 1) s = 1;
     if (s > steps) s = steps;
     const long per = (steps + s - 1) / s;
@@ -1595,11 +1594,11 @@ bool make_map_raw_rows(TensorMap* out, const void* base, int C, int W, int H, in
 bool stem_wg_supported(int H, int W, int C, int Co) {
     return C == 3 && Co % 64 == 0 && (W == 32 || W == 16) && H % (128 / W) == 0 && (W * C * 2) % 16 == 0 && (128 / W + 2) * W * 6 <= STEM_RAW_BYTES;
 }
-int stem_wg_ctas(long steps) { const long n = sm_count(); return (int)(steps < n ? steps : n); }
-size_t stem_wg_workspace_elems(int Co, long steps) { return (size_t)(Co / 64) * stem_wg_ctas(steps) * 64 * 64; }
+int stem_wg_ctas(long steps, int sms) { const long n = sm_count(sms); return (int)(steps < n ? steps : n); }
+size_t stem_wg_workspace_elems(int Co, long steps, int sms) { return (size_t)(Co / 64) * stem_wg_ctas(steps, sms) * 64 * 64; }
 
 cudaError_t run_stem_wg(const TensorMap& x_raw, const TensorMap& dy128, int H, int W, int N, int Co, float* partial, float* dw, bool accum, int* err,
-                        cudaStream_t s) {
+                        int sms, cudaStream_t s) {
     constexpr int STAGES = 4;
     constexpr int smem = STAGES * (2 * 128 * 128 + STEM_RAW_BYTES) + 1024 + 256;
     static bool attr = false;
@@ -1610,7 +1609,7 @@ cudaError_t run_stem_wg(const TensorMap& x_raw, const TensorMap& dy128, int H, i
     }
     StemWgParams p{};
     p.W = W; p.Ht = 128 / W; p.tiles_h = H / p.Ht; p.steps = N * p.tiles_h;
-    const int ctas = stem_wg_ctas(p.steps);
+    const int ctas = stem_wg_ctas(p.steps, sms);
     p.steps_per_cta = (p.steps + ctas - 1) / ctas;
     p.partial = partial; p.err = err;
     stem_wg_kernel<STAGES><<<dim3(ctas, Co / 64), NUM_THREADS, smem, s>>>(*(const CUtensorMap*)&x_raw, *(const CUtensorMap*)&dy128, p);
@@ -1621,7 +1620,7 @@ cudaError_t run_stem_wg(const TensorMap& x_raw, const TensorMap& dy128, int H, i
 }
 
 cudaError_t run_stem_fw(const TensorMap& x_raw, const TensorMap& out_map, int H, int W, int N, int Co, const void* w, const float* bias, bool relu,
-                        float* stat_part, int* err, cudaStream_t s) {
+                        float* stat_part, int* err, int sms, cudaStream_t s) {
     constexpr int STAGES = 3;
     constexpr int smem = STAGES * (128 * 128 + STEM_RAW_BYTES) + 64 * 128 + 4 * 2 * EPI_BUF_BYTES + 1024 + 256;
     static bool attr = false;
@@ -1633,7 +1632,7 @@ cudaError_t run_stem_fw(const TensorMap& x_raw, const TensorMap& out_map, int H,
     StemFwParams p{};
     p.W = W; p.Ht = 128 / W; p.tiles_h = H / p.Ht; p.tiles = N * p.tiles_h; p.Co = Co; p.epi = relu ? EPI_RELU : 0;
     p.w = (const bf16*)w; p.bias = bias; p.stat_part = stat_part; p.err = err;
-    const int slots = 2 * sm_count();
+    const int slots = 2 * sm_count(sms);
     stem_fw_kernel<STAGES><<<dim3(p.tiles < slots ? p.tiles : slots, Co / 64), 320, smem, s>>>(*(const CUtensorMap*)&x_raw, *(const CUtensorMap*)&out_map, p);
     return cudaGetLastError();
 }

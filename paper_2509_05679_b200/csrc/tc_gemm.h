@@ -28,6 +28,7 @@ struct KmParams {
     int Ho, Wo, Co, os;                          // output tensor [N,Ho,Wo,Co] and the output stride of a domain pixel
     int Cn;                                      // output channels computed (multiple of the column tile)
     int epi;                                     // EPI_RELU | EPI_ACCUM
+    int sms;                                     // SMs the grid is sized for (0: all)
     const float* bias;                           // or nullptr
     void* out;
     float* stat_part;                            // or nullptr: [tile_m * 4 + warp][Cn][2] = (sum, sum of squares) over the
@@ -47,10 +48,9 @@ struct WgParams {
 };
 
 bool init();     // resolves the driver's tensor-map encoder; false if unavailable
-// SMs the persistent kernels below size their grids for, and the contraction splits of the weight gradients their CTA
-// counts (0 or >= the device's count: all of them).  Process-wide; the context sets it before it sizes workspaces and
-// before every step it enqueues.  The results depend on it only through fp32 summation order (split counts).
-void set_sm_budget(int sms);
+// `sms` below (KmParams::sms, the last integer of the other launchers): the SMs a persistent kernel sizes its grid for and
+// a weight gradient its contraction splits (0 or >= the device's count: all of them).  Results depend on it only
+// through fp32 summation order (split counts).
 // NHWC bf16 tensor [N,H,W,C]; box = boxC channels x (boxW x boxH x boxN) pixels; stride 2 samples every other pixel
 bool make_map_4d(TensorMap* out, const void* base, int C, int W, int H, int N, int boxC, int boxW, int boxH, int boxN, int stride);
 bool make_map_2d(TensorMap* out, const void* base, long inner, long outer, int box_inner, int box_outer);
@@ -86,7 +86,7 @@ struct WgRowsParams {
     int* err;
 };
 int wg_rows_variant(int H, int W, int C, int Co);
-int wg_rows_splits(int variant, int C, int Co, long steps);
+int wg_rows_splits(int variant, int C, int Co, long steps, int sms);
 cudaError_t run_wg_rows(const TensorMap& x_rows, const TensorMap& dy128, const WgRowsParams& p, int variant, int splits, float* dw, bool accum,
                         cudaStream_t s);
 
@@ -95,13 +95,13 @@ cudaError_t run_wg_rows(const TensorMap& x_rows, const TensorMap& dy128, const W
 // dy128: dy with a box of 64 channels x 128 pixels (make_map_4d).  All N samples; partial: stem_wg_workspace_elems floats.
 bool make_map_raw_rows(TensorMap* out, const void* base, int C, int W, int H, int N, int box_rows);
 bool stem_wg_supported(int H, int W, int C, int Co);
-size_t stem_wg_workspace_elems(int Co, long steps);
+size_t stem_wg_workspace_elems(int Co, long steps, int sms);
 cudaError_t run_stem_wg(const TensorMap& x_raw, const TensorMap& dy128, int H, int W, int N, int Co, float* partial, float* dw, bool accum, int* err,
-                        cudaStream_t s);
+                        int sms, cudaStream_t s);
 // Forward pass of the first layer on the tensor cores (same geometry as run_stem_wg).  out_map: the output's map from
 // make_map_out with the tile geometry W x (128 / W) x 1.  w: [Co][27] bf16.  stat_part as in KmParams.
 cudaError_t run_stem_fw(const TensorMap& x_raw, const TensorMap& out_map, int H, int W, int N, int Co, const void* w, const float* bias, bool relu,
-                        float* stat_part, int* err, cudaStream_t s);
+                        float* stat_part, int* err, int sms, cudaStream_t s);
 cudaError_t run_flip_transpose(const void* w, void* wt, int Co, int taps, int Ci, cudaStream_t s);
 
 
