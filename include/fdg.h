@@ -90,7 +90,8 @@ typedef struct {
     int32_t in_h, in_w, in_c;  /* sample shape; 1,1,3072 for an MLP on flattened 32x32x3 inputs */
     int32_t num_classes;       /* must equal the last layer's c_out                             */
     int32_t serial;            /* 1: run every module on one stream (results are bit-identical
-                                  to the concurrent mode; used to test the event wiring)        */
+                                  to the concurrent mode when both contexts have the same
+                                  grid_sms; used to test the event wiring)                      */
     int32_t kernel_path;       /* 0: tensor-core kernels where shapes allow (bf16 only), the 256-column
                                      tile (and the 128-column tile of 3x3 stride-1 layers on 16x16 images) as
                                      pairs of CTAs on two SMs (tcgen05 cta_group::2);
