@@ -183,9 +183,10 @@ FDG_API fdg_status fdg_set_params_worker(fdg_ctx* ctx, int32_t worker, const flo
  *                that copy is enqueued on module 1's stream; fdg_wait_ingest() blocks until it
  *                is done.  The library does not keep the pointer.
  *   dev_labels : device, int32 [M].
- *   host_loss_or_null : if non-NULL the call waits for the last module and stores the mean
- *                loss of the batch it processed in this iteration (tau = t-K+1; NaN while
- *                tau < 0).  If NULL the call only enqueues work and returns. */
+ *   host_loss_or_null : if non-NULL the call waits until the last module has computed the loss
+ *                of the batch it forwards in this iteration (tau = t-K+1; NaN while tau < 0) and
+ *                stores its mean; the rest of the iteration (backward passes, updates) is still
+ *                in flight when the call returns.  If NULL the call only enqueues work. */
 FDG_API fdg_status fdg_step(fdg_ctx* ctx, const void* dev_inputs, const int32_t* dev_labels,
                     float* host_loss_or_null);
 

@@ -143,6 +143,7 @@ struct fdg_ctx {
     int* tc_err;                   // device word: set by a tensor-core kernel whose bounded wait gave up
     bool any_tc;
     cudaEvent_t ingested;
+    cudaEvent_t loss_ready;        // recorded behind the kernel that writes the step's loss
     std::string err;
 };
 
@@ -873,10 +874,11 @@ fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, boo
             // one replica: dphi/dlogits / M, the mean over all samples.  One replica per worker: / B, worker s's own
             // gradient scale 1/per_worker_batch of Eq. dl_update (the mixing matrix does the averaging)
             const bool fused_head = m.ops.back().head && m.groups == 1;     // the forward pass above has computed loss and dlogits
-            if (tau_f >= 0 && fused_head) {}
+            if (tau_f >= 0 && fused_head) CK(cudaEventRecord(ctx->loss_ready, m.fstream));
             else if (tau_f >= 0) softmax_ce(ctx->dt, ctx->logits, ctx->labels + (size_t)(tau_f % ctx->label_depth) * ctx->M, ctx->dlogits,
                                        loss_slot, ctx->M, ctx->classes, ctx->R > 1 ? 1.f / (float)ctx->B : 1.f / (float)ctx->M, m.stream);
             else fill_f32(loss_slot, NAN, 1, m.stream);
+            if (!(tau_f >= 0 && fused_head)) CK(cudaEventRecord(ctx->loss_ready, m.stream));
         }
         if (tau_b >= 0) for (int g = 0; g < m.groups; ++g) backward_module(ctx, kk, tau_b, v_b, t, g);
         // Eq. dl_update with P = 11^T/N: w(t+1) = w(t) - lr * averaged gradient; also emits version t+1
@@ -904,7 +906,7 @@ fdg_status run_step(fdg_ctx* ctx, const void* inputs, const int32_t* labels, boo
     CK(cudaGetLastError());
     ctx->t = t + 1;
     if (host_loss) {
-        CK(cudaStreamSynchronize(ctx->mod[K - 1].stream));
+        CK(cudaEventSynchronize(ctx->loss_ready));          // the loss only: the last module's backward pass and update go on
         float l = 0.f;
         CK(cudaMemcpy(&l, ctx->loss_ring + (t % 64), sizeof(float), cudaMemcpyDeviceToHost));
         fdg_status es = check_device_error(ctx);
@@ -932,6 +934,7 @@ void fdg_destroy(fdg_ctx* ctx) {
         if (m.ev1) cudaEventDestroy(m.ev1);
     }
     if (ctx->ingested) cudaEventDestroy(ctx->ingested);
+    if (ctx->loss_ready) cudaEventDestroy(ctx->loss_ready);
     for (cudaStream_t s : ctx->owned) cudaStreamDestroy(s);
     for (void* p : ctx->blocks) ctx->alloc.free(p, ctx->alloc.user);
     delete ctx;
@@ -985,6 +988,7 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
     ctx->own_streams = opt->streams == nullptr;
     ctx->device_bytes = 0;
     ctx->ingested = nullptr;
+    ctx->loss_ready = nullptr;
     ctx->mod.resize(K);
     auto bail = [&](fdg_status s, const std::string& msg) { g_create_error = msg; fdg_destroy(ctx); return s; };
 
@@ -1086,6 +1090,7 @@ fdg_status fdg_create(const fdg_layer* layers, int32_t n_layers, const int32_t* 
         if (e != cudaSuccess) return bail(FDG_ERR_CUDA, cudaGetErrorString(e));
     }
     if (cudaEventCreateWithFlags(&ctx->ingested, cudaEventDisableTiming) != cudaSuccess) return bail(FDG_ERR_CUDA, "cudaEventCreate failed");
+    if (cudaEventCreateWithFlags(&ctx->loss_ready, cudaEventDisableTiming) != cudaSuccess) return bail(FDG_ERR_CUDA, "cudaEventCreate failed");
     if (cudaMemset(ctx->tc_err, 0, 256) != cudaSuccess) return bail(FDG_ERR_CUDA, "cudaMemset failed");
     if (ctx->R > 1) {
         std::vector<float> pf(ctx->P.begin(), ctx->P.end());
